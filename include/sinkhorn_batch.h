@@ -1,0 +1,165 @@
+/*
+ * sinkhorn_batch.h — C ABI of the shrinking-active-set batched log-domain
+ * Sinkhorn library for NVIDIA B200 (sm_100a).
+ *
+ * W independent entropic optimal-transport problems ("lanes") are solved side by
+ * side.  Problem statement (paper Eq. 1): positive unit-mass marginals
+ * a in R^n, b in R^m, cost C_ij = |x_i - y_j|^2 recomputed from the point clouds,
+ * regularisation eps.  One cycle is the pair of scaling updates of Eq. 3 in log
+ * form,
+ *      f_i <- eps (log a_i - LSE_j((g_j - C_ij)/eps)),
+ *      g_j <- eps (log b_j - LSE_i((f_i - C_ij)/eps)),
+ * and the plan is pi_ij = exp((f_i + g_j - C_ij)/eps); it is never stored.
+ * After each audited cycle a lane's row residual is screened, screen-positive
+ * lanes get the two-sided check of Eq. 5, and lanes that pass are retired at
+ * completion depth l_t (Section "Screen, verify, and compact").  What happens to
+ * a retired lane is the execution mode (Section "Execution modes and fallback").
+ *
+ * Conventions
+ *   - Every data pointer is DEVICE memory owned by the caller unless it says
+ *     "host".  Inputs are const and never modified.  The library allocates no
+ *     device memory: all of its state lives in the caller's workspace.
+ *   - All work is enqueued on the stream given at creation.
+ *   - Every call returns an skb_status; nothing throws or aborts.  The text of
+ *     the last error is available from sinkhorn_batch_last_error().
+ *   - There is no CPU path: every step runs in CUDA kernels.
+ */
+#ifndef SINKHORN_BATCH_H
+#define SINKHORN_BATCH_H
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct skb_batch skb_batch; /* opaque host object */
+
+typedef enum {
+    SKB_OK = 0,
+    SKB_ERR_NULL = 1,      /* a required pointer is null */
+    SKB_ERR_SHAPE = 2,     /* W, n, m, d < 1 or an unsupported combination */
+    SKB_ERR_VALUE = 3,     /* tol <= 0, max_iter < 1, bad enum, non-finite or non-positive input */
+    SKB_ERR_WORKSPACE = 4, /* workspace missing, misaligned (256 B) or too small */
+    SKB_ERR_STATE = 5,     /* call not valid in the batch's current state */
+    SKB_ERR_CUDA = 6       /* a CUDA call or a kernel reported an error */
+} skb_status;
+
+/* What is done with a lane that passed the two-sided check. */
+typedef enum {
+    SKB_ACTIVE = 0, /* retire and physically compact: later kernels run at survivor width A_k */
+    SKB_MASKED = 1, /* freeze its potentials, keep it in place: kernels stay at width W        */
+    SKB_STATIC = 2  /* keep updating every lane until the deepest lane passes (l_max)          */
+} skb_mode;
+
+typedef enum { SKB_F32 = 0, SKB_BF16 = 1 } skb_dtype;           /* storage type of x and y only */
+typedef enum { SKB_COMPUTE_F32 = 0, SKB_COMPUTE_F64 = 1 } skb_compute; /* pair-term arithmetic */
+
+typedef enum {
+    SKB_LANE_RUNNING = 0,
+    SKB_LANE_DONE = 1,       /* passed the two-sided check at its depth                    */
+    SKB_LANE_ITER_LIMIT = 2, /* did not pass within max_iter cycles; depth = max_iter      */
+    SKB_LANE_NONFINITE = 3   /* a potential or residual became non-finite; output invalid  */
+} skb_lane_status;
+
+typedef struct {
+    int W, n, m, d;        /* lanes, source points, target points, dimension               */
+    int xy_dtype;          /* skb_dtype                                                    */
+    int mode;              /* skb_mode                                                     */
+    int compute;           /* skb_compute; F64 is the slow validation arithmetic           */
+    int max_iter;          /* cycle cap per lane, >= 1                                     */
+    int audit_every;       /* audit after every k-th cycle, >= 1                           */
+    float tol_screen;      /* row-screen threshold; <= 0 means "same as tol"               */
+    int column_split;      /* 0 = automatic; 1, 8 or 32 forces how many lanes of a warp     */
+                           /* share one row's columns in the update kernel (tuning knob)  */
+    void *stream;          /* cudaStream_t (0 = legacy default stream)                     */
+    void *workspace;       /* device, 256-byte aligned                                     */
+    size_t workspace_bytes;
+} skb_config;
+
+/* Bytes of device workspace a batch with this shape, dtype, mode and compute type
+ * needs.  Returns 0 if the configuration is invalid. */
+size_t sinkhorn_batch_workspace_bytes(const skb_config *cfg);
+
+/*
+ * Create a batch (Eq. 1 inputs) and enqueue its set-up kernels.
+ *   x   [W, n, d] row-major, fp32 or bf16 per cfg->xy_dtype      (device)
+ *   y   [W, m, d]                                                (device)
+ *   a   [W, n] fp32, > 0, each lane sums to 1                    (device)
+ *   b   [W, m] fp32, > 0, each lane sums to 1                    (device)
+ *   eps [W]    fp32, > 0, per-lane regularisation                (device)
+ *   tol        two-sided stopping tolerance tau_stop of Eq. 5    (> 0)
+ * Potentials start cold, f = g = 0.  Inputs are copied into the workspace in the
+ * kernels' own layout; they may be freed once the stream has passed this call.
+ * Non-positive weights or eps and non-finite coordinates are detected on the
+ * device and reported by the first step/drain as SKB_ERR_VALUE.
+ * On success *out holds the handle; the caller releases it with
+ * sinkhorn_batch_destroy (the workspace stays the caller's).
+ */
+skb_status sinkhorn_batch_create(const void *x, const void *y, const float *a, const float *b,
+                                 const float *eps, float tol, const skb_config *cfg,
+                                 skb_batch **out);
+
+/* Enqueue `cycles` full cycles (both legs of Eq. 3 plus screen, two-sided check and
+ * retirement after every audited one).  Never synchronises.  Cycles past the point
+ * where every lane is finished are no-ops. */
+skb_status sinkhorn_batch_step(skb_batch *h, int cycles);
+
+/* Run until every lane is retired (passed, hit max_iter, or went non-finite), then
+ * synchronise the stream.  *cycles_run (host, may be null) receives the number of
+ * complete cycles executed, i.e. the largest depth. */
+skb_status sinkhorn_batch_drain(skb_batch *h, int *cycles_run);
+
+/* Number of lanes still running (host out).  Synchronises the stream. */
+skb_status sinkhorn_batch_active(skb_batch *h, int *n_active);
+
+/* Potentials in the paper's convention pi = exp((f + g - C)/eps), original lane order.
+ * f [W, n], g [W, m] device out, either may be null.  Retired lanes give their state at
+ * the completion depth (STATIC: at l_max); running lanes give their current state. */
+skb_status sinkhorn_batch_potentials(skb_batch *h, float *f, float *g);
+skb_status sinkhorn_batch_potentials_f64(skb_batch *h, double *f, double *g);
+
+/* Completion depth l_t (first audited cycle at which the lane passed; Eq. 6) and
+ * skb_lane_status per lane, device out [W], original lane order; either may be null. */
+skb_status sinkhorn_batch_depths(skb_batch *h, int *depth, int *lane_status);
+
+/* Residuals of Eq. 5 measured at the state that was emitted: r_row = |pi 1 - a|_1,
+ * r_col = |pi^T 1 - b|_1, device out [W] fp32.  r_col is NaN for a lane that was never
+ * sent to the two-sided check (iteration limit without a screen pass). */
+skb_status sinkhorn_batch_residuals(skb_batch *h, float *r_row, float *r_col);
+
+/*
+ * Work accounting (Eq. 6-8), host outs, any may be null.  Synchronises.
+ *   slots      lane-cycles physically executed: sum_k A_k in ACTIVE mode, W*l_max otherwise
+ *   cycles     complete cycles executed (l_max)
+ *   widths     widths[k-1] = physical width of cycle k, for k = 1..min(cycles, widths_cap)
+ *   pair_terms exp-terms evaluated by the update kernel, all passes (legs, look-ahead
+ *              screen, column check)
+ */
+skb_status sinkhorn_batch_stats(skb_batch *h, long long *slots, int *cycles, int *widths,
+                                int widths_cap, long long *pair_terms);
+
+/*
+ * Whole solve from HOST buffers in one call: copies x, y, a, b, eps to the device,
+ * creates the batch, drains it, and copies the results back.  Every data pointer here is
+ * HOST memory (pinned memory makes the copies asynchronous); outputs may be null.
+ * cfg->workspace is still device memory and must hold
+ * sinkhorn_batch_host_workspace_bytes(cfg) bytes: the batch's own workspace followed by
+ * staging for the inputs and outputs.  Returns after the stream has been synchronised.
+ */
+size_t sinkhorn_batch_host_workspace_bytes(const skb_config *cfg);
+skb_status sinkhorn_batch_solve_host(const void *x, const void *y, const float *a, const float *b,
+                                     const float *eps, float tol, const skb_config *cfg,
+                                     float *f, float *g, int *depth, int *lane_status,
+                                     float *r_row, float *r_col, long long *slots, int *cycles);
+
+void sinkhorn_batch_destroy(skb_batch *h);
+
+/* Host string describing the last error on this handle (or of the last failed create
+ * when h is null).  Valid until the next call on the same handle. */
+const char *sinkhorn_batch_last_error(const skb_batch *h);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SINKHORN_BATCH_H */

@@ -1,0 +1,219 @@
+"""ctypes binding of libsinkhorn_batch.so — argument marshalling only.
+
+Every step of the solve runs in the library's CUDA kernels; PyTorch supplies
+device memory and the stream.  There is no fallback: if the shared library is
+missing or fails to load, importing this module raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libsinkhorn_batch.so")
+
+SKB_OK = 0
+STATUS_NAMES = {0: "SKB_OK", 1: "SKB_ERR_NULL", 2: "SKB_ERR_SHAPE", 3: "SKB_ERR_VALUE",
+                4: "SKB_ERR_WORKSPACE", 5: "SKB_ERR_STATE", 6: "SKB_ERR_CUDA"}
+MODES = {"active": 0, "masked": 1, "static": 2}
+COMPUTE = {"f32": 0, "f64": 1}
+LANE_RUNNING, LANE_DONE, LANE_ITER_LIMIT, LANE_NONFINITE = 0, 1, 2, 3
+
+EXPORTS = (
+    "sinkhorn_batch_workspace_bytes", "sinkhorn_batch_create", "sinkhorn_batch_step",
+    "sinkhorn_batch_drain", "sinkhorn_batch_active", "sinkhorn_batch_potentials",
+    "sinkhorn_batch_potentials_f64", "sinkhorn_batch_depths", "sinkhorn_batch_residuals",
+    "sinkhorn_batch_stats", "sinkhorn_batch_destroy", "sinkhorn_batch_last_error",
+    "sinkhorn_batch_host_workspace_bytes", "sinkhorn_batch_solve_host",
+)
+
+
+class SkbConfig(ctypes.Structure):
+    _fields_ = [("W", ctypes.c_int), ("n", ctypes.c_int), ("m", ctypes.c_int), ("d", ctypes.c_int),
+                ("xy_dtype", ctypes.c_int), ("mode", ctypes.c_int), ("compute", ctypes.c_int),
+                ("max_iter", ctypes.c_int), ("audit_every", ctypes.c_int),
+                ("tol_screen", ctypes.c_float), ("column_split", ctypes.c_int),
+                ("stream", ctypes.c_void_p), ("workspace", ctypes.c_void_p),
+                ("workspace_bytes", ctypes.c_size_t)]
+
+
+class SkbError(RuntimeError):
+    def __init__(self, code, msg):
+        super().__init__(f"{STATUS_NAMES.get(code, code)}: {msg}")
+        self.code = code
+
+
+def _load():
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2607_24741_b200.build` "
+                          "(there is no CPU or PyTorch fallback)")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, cfgp = ctypes.c_void_p, ctypes.POINTER(SkbConfig)
+    lib.sinkhorn_batch_workspace_bytes.restype = ctypes.c_size_t
+    lib.sinkhorn_batch_workspace_bytes.argtypes = [cfgp]
+    lib.sinkhorn_batch_host_workspace_bytes.restype = ctypes.c_size_t
+    lib.sinkhorn_batch_host_workspace_bytes.argtypes = [cfgp]
+    lib.sinkhorn_batch_create.argtypes = [vp, vp, vp, vp, vp, ctypes.c_float, cfgp, ctypes.POINTER(vp)]
+    lib.sinkhorn_batch_step.argtypes = [vp, ctypes.c_int]
+    lib.sinkhorn_batch_drain.argtypes = [vp, ctypes.POINTER(ctypes.c_int)]
+    lib.sinkhorn_batch_active.argtypes = [vp, ctypes.POINTER(ctypes.c_int)]
+    lib.sinkhorn_batch_potentials.argtypes = [vp, vp, vp]
+    lib.sinkhorn_batch_potentials_f64.argtypes = [vp, vp, vp]
+    lib.sinkhorn_batch_depths.argtypes = [vp, vp, vp]
+    lib.sinkhorn_batch_residuals.argtypes = [vp, vp, vp]
+    lib.sinkhorn_batch_stats.argtypes = [vp, ctypes.POINTER(ctypes.c_longlong), ctypes.POINTER(ctypes.c_int),
+                                         vp, ctypes.c_int, ctypes.POINTER(ctypes.c_longlong)]
+    lib.sinkhorn_batch_destroy.argtypes = [vp]
+    lib.sinkhorn_batch_destroy.restype = None
+    lib.sinkhorn_batch_last_error.argtypes = [vp]
+    lib.sinkhorn_batch_last_error.restype = ctypes.c_char_p
+    lib.sinkhorn_batch_solve_host.argtypes = [vp, vp, vp, vp, vp, ctypes.c_float, cfgp, vp, vp, vp, vp, vp, vp,
+                                              ctypes.POINTER(ctypes.c_longlong), ctypes.POINTER(ctypes.c_int)]
+    for name in EXPORTS:
+        if name not in ("sinkhorn_batch_workspace_bytes", "sinkhorn_batch_host_workspace_bytes",
+                        "sinkhorn_batch_destroy", "sinkhorn_batch_last_error"):
+            getattr(lib, name).restype = ctypes.c_int
+    return lib
+
+
+lib = _load()
+
+
+def _check(code, handle=None):
+    if code != SKB_OK:
+        msg = lib.sinkhorn_batch_last_error(handle)
+        raise SkbError(code, msg.decode() if msg else "")
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def make_config(W, n, m, d, *, bf16=False, mode="active", compute="f32", max_iter=5000,
+                audit_every=1, tol_screen=0.0, column_split=0, stream=0) -> SkbConfig:
+    return SkbConfig(W, n, m, d, 1 if bf16 else 0, MODES[mode] if isinstance(mode, str) else mode,
+                     COMPUTE[compute] if isinstance(compute, str) else compute, max_iter, audit_every,
+                     tol_screen, column_split, stream, None, 0)
+
+
+# ---- functions with the C names ------------------------------------------------------
+
+def sinkhorn_batch_workspace_bytes(cfg: SkbConfig) -> int:
+    return lib.sinkhorn_batch_workspace_bytes(ctypes.byref(cfg))
+
+
+def sinkhorn_batch_host_workspace_bytes(cfg: SkbConfig) -> int:
+    return lib.sinkhorn_batch_host_workspace_bytes(ctypes.byref(cfg))
+
+
+def sinkhorn_batch_create(x, y, a, b, eps, tol, cfg: SkbConfig):
+    h = ctypes.c_void_p()
+    _check(lib.sinkhorn_batch_create(_ptr(x), _ptr(y), _ptr(a), _ptr(b), _ptr(eps), tol, ctypes.byref(cfg),
+                                     ctypes.byref(h)))
+    return h
+
+
+def sinkhorn_batch_step(h, cycles):
+    _check(lib.sinkhorn_batch_step(h, cycles), h)
+
+
+def sinkhorn_batch_drain(h) -> int:
+    c = ctypes.c_int(0)
+    _check(lib.sinkhorn_batch_drain(h, ctypes.byref(c)), h)
+    return c.value
+
+
+def sinkhorn_batch_active(h) -> int:
+    c = ctypes.c_int(0)
+    _check(lib.sinkhorn_batch_active(h, ctypes.byref(c)), h)
+    return c.value
+
+
+def sinkhorn_batch_destroy(h):
+    lib.sinkhorn_batch_destroy(h)
+
+
+class SinkhornBatch:
+    """One batch of W lanes on the current CUDA device (thin wrapper over the C calls)."""
+
+    def __init__(self, x, y, a, b, eps, tol, *, mode="active", compute="f32", max_iter=5000,
+                 audit_every=1, tol_screen=0.0, column_split=0, stream=None):
+        if not (x.is_cuda and y.is_cuda and a.is_cuda and b.is_cuda and eps.is_cuda):
+            raise ValueError("x, y, a, b, eps must be CUDA tensors")
+        if x.dtype not in (torch.float32, torch.bfloat16) or y.dtype != x.dtype:
+            raise ValueError("x and y must both be float32 or both be bfloat16")
+        for t in (a, b, eps):
+            if t.dtype != torch.float32:
+                raise ValueError("a, b, eps must be float32")
+        x, y, a, b, eps = (t.contiguous() for t in (x, y, a, b, eps))
+        W, n, d = x.shape
+        m = y.shape[1]
+        if y.shape != (W, m, d) or a.shape != (W, n) or b.shape != (W, m) or eps.shape != (W,):
+            raise ValueError("shapes must be x[W,n,d] y[W,m,d] a[W,n] b[W,m] eps[W]")
+        self.W, self.n, self.m, self.d = W, n, m, d
+        self.device = x.device
+        self.stream = stream if stream is not None else torch.cuda.current_stream(x.device)
+        self.cfg = make_config(W, n, m, d, bf16=x.dtype == torch.bfloat16, mode=mode, compute=compute,
+                               max_iter=max_iter, audit_every=audit_every, tol_screen=tol_screen,
+                               column_split=column_split, stream=self.stream.cuda_stream)
+        need = sinkhorn_batch_workspace_bytes(self.cfg)
+        if need == 0:
+            raise SkbError(2, "configuration rejected (unsupported shape or bad option)")
+        self.workspace = torch.empty(need, dtype=torch.uint8, device=x.device)
+        self.cfg.workspace = self.workspace.data_ptr()
+        self.cfg.workspace_bytes = need
+        self._keep = (x, y, a, b, eps)
+        self.h = None
+        with torch.cuda.device(x.device):
+            self.h = sinkhorn_batch_create(x, y, a, b, eps, float(tol), self.cfg)
+
+    def step(self, cycles=1):
+        sinkhorn_batch_step(self.h, cycles)
+
+    def drain(self) -> int:
+        return sinkhorn_batch_drain(self.h)
+
+    def active(self) -> int:
+        return sinkhorn_batch_active(self.h)
+
+    def potentials(self, f64=False):
+        dt = torch.float64 if f64 else torch.float32
+        f = torch.zeros(self.W, self.n, dtype=dt, device=self.device)
+        g = torch.zeros(self.W, self.m, dtype=dt, device=self.device)
+        fn = lib.sinkhorn_batch_potentials_f64 if f64 else lib.sinkhorn_batch_potentials
+        _check(fn(self.h, _ptr(f), _ptr(g)), self.h)
+        return f, g
+
+    def depths(self):
+        depth = torch.zeros(self.W, dtype=torch.int32, device=self.device)
+        status = torch.zeros(self.W, dtype=torch.int32, device=self.device)
+        _check(lib.sinkhorn_batch_depths(self.h, _ptr(depth), _ptr(status)), self.h)
+        return depth, status
+
+    def residuals(self):
+        rr = torch.zeros(self.W, dtype=torch.float32, device=self.device)
+        rc = torch.zeros(self.W, dtype=torch.float32, device=self.device)
+        _check(lib.sinkhorn_batch_residuals(self.h, _ptr(rr), _ptr(rc)), self.h)
+        return rr, rc
+
+    def stats(self, widths_cap=0):
+        slots, terms, cycles = ctypes.c_longlong(0), ctypes.c_longlong(0), ctypes.c_int(0)
+        buf = (ctypes.c_int * max(widths_cap, 1))()
+        _check(lib.sinkhorn_batch_stats(self.h, ctypes.byref(slots), ctypes.byref(cycles),
+                                        ctypes.cast(buf, ctypes.c_void_p), widths_cap, ctypes.byref(terms)), self.h)
+        k = min(cycles.value, widths_cap)
+        return {"slots": slots.value, "cycles": cycles.value, "pair_terms": terms.value,
+                "widths": list(buf[:k])}
+
+    def close(self):
+        if self.h is not None:
+            sinkhorn_batch_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -1,0 +1,396 @@
+// Host side of the C ABI: validation, workspace carving, the cycle enqueue loop and the
+// asynchronous width read-back.  No device memory is allocated here; the only CUDA
+// objects the handle owns are two events and a small pinned host block.
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+
+#include "../../include/sinkhorn_batch.h"
+#include "skb_host.h"
+
+using namespace skb;
+
+struct skb_batch {
+    Dev dev;
+    skb_config cfg;
+    const Variant *var;
+    cudaStream_t stream;
+    Ctl *h_ctl;            // pinned, 2 snapshots
+    cudaEvent_t ev[2];
+    int known_width;       // last physical width the host has seen
+    bool finished;
+    long long enqueued;    // cycles enqueued so far
+    std::string err;
+};
+
+static std::string g_create_err;
+
+static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+static bool config_ok(const skb_config *c, std::string &why)
+{
+    if (!c) { why = "config is null"; return false; }
+    if (c->W < 1 || c->n < 1 || c->m < 1 || c->d < 1) { why = "W, n, m, d must be >= 1"; return false; }
+    if (c->xy_dtype != SKB_F32 && c->xy_dtype != SKB_BF16) { why = "bad xy_dtype"; return false; }
+    if (c->mode < SKB_ACTIVE || c->mode > SKB_STATIC) { why = "bad mode"; return false; }
+    if (c->compute != SKB_COMPUTE_F32 && c->compute != SKB_COMPUTE_F64) { why = "bad compute type"; return false; }
+    if (c->max_iter < 1 || c->audit_every < 1) { why = "max_iter and audit_every must be >= 1"; return false; }
+    if (c->column_split != 0 && c->column_split != 1 && c->column_split != 8 && c->column_split != 32) {
+        why = "column_split must be 0, 1, 8 or 32"; return false;
+    }
+    return true;
+}
+
+// Lays the batch's arrays out in the workspace (base may be null: size query only).
+static size_t carve(const skb_config *c, const Variant *var, char *base, Dev *D, size_t *zero_end_out = nullptr)
+{
+    size_t off = 0;
+    auto take = [&](size_t bytes) -> void * {
+        void *p = base ? base + off : nullptr;
+        off += align_up(bytes, 256);
+        return p;
+    };
+    const size_t W = c->W, n = c->n, m = c->m;
+    const size_t np = align_up(n, 4), mp = align_up(m, 4), DP = var->DP;
+    const size_t ts = var->f64 ? 8 : 4;
+    Dev d;
+    memset(&d, 0, sizeof(d));
+    d.W = c->W; d.n = c->n; d.m = c->m; d.d = c->d; d.np = (int)np; d.mp = (int)mp; d.DP = (int)DP;
+    d.mode = c->mode; d.max_iter = c->max_iter; d.audit_every = c->audit_every;
+    d.xy_bf16 = c->xy_dtype == SKB_BF16; d.compute_f64 = var->f64;
+    // control block first, then everything that must start at zero, in one contiguous range
+    d.ctl = (Ctl *)take(sizeof(Ctl));
+    d.state = (int *)take(W * 4); d.flag = (int *)take(W * 4); d.verdict = (int *)take(W * 4);
+    d.nonfinite = (int *)take(W * 4);
+    d.cnt_row = (unsigned *)take(W * 4); d.cnt_col = (unsigned *)take(W * 4);
+    d.depth = (int *)take(W * 4); d.status = (int *)take(W * 4); d.emitted = (int *)take(W * 4);
+    d.res_row = (double *)take(W * 8); d.res_col = (double *)take(W * 8);
+    d.rrow = (double *)take(W * 8); d.rcol = (double *)take(W * 8);
+    d.widths = (int *)take(((size_t)c->max_iter + 2) * 4);
+    const size_t zero_end = off;
+    d.scale = (double *)take(W * 8); d.lane_id = (int *)take(W * 4);
+    d.ret_slot = (int *)take(W * 4); d.ret_lane = (int *)take(W * 4); d.ret_src = (int *)take(W * 4);
+    d.ret_scale = (double *)take(W * 8);
+    d.hole_list = (int *)take(W * 4); d.fill_list = (int *)take(W * 4);
+    d.part_row = (double *)take(W * MAX_PARTS * 8); d.part_col = (double *)take(W * MAX_PARTS * 8);
+    d.xs = take(W * DP * np * ts); d.ys = take(W * DP * mp * ts);
+    d.ft[0] = take(W * np * ts); d.ft[1] = take(W * np * ts); d.gt = take(W * mp * ts);
+    d.sqx = (double *)take(W * np * 8); d.sqy = (double *)take(W * mp * 8);
+    d.la2 = (double *)take(W * np * 8); d.lb2 = (double *)take(W * mp * 8);
+    d.phi[0] = (double *)take(W * np * 8); d.phi[1] = (double *)take(W * np * 8);
+    d.gam = (double *)take(W * mp * 8);
+    d.f_out = (double *)take(W * n * 8); d.g_out = (double *)take(W * m * 8);
+    if (D) { *D = d; D->tol_screen = 0; D->tol_stop = 0; }
+    if (zero_end_out) *zero_end_out = zero_end;
+    return off;
+}
+
+extern "C" size_t sinkhorn_batch_workspace_bytes(const skb_config *cfg)
+{
+    std::string why;
+    if (!config_ok(cfg, why)) return 0;
+    const Variant *v = choose_variant(cfg->W, cfg->n, cfg->m, cfg->d, cfg->compute == SKB_COMPUTE_F64, cfg->column_split);
+    if (!v) return 0;
+    return carve(cfg, v, nullptr, nullptr);
+}
+
+static skb_status fail(skb_batch *h, skb_status st, const std::string &msg)
+{
+    if (h) h->err = msg; else g_create_err = msg;
+    return st;
+}
+
+static skb_status cuda_fail(skb_batch *h, cudaError_t e, const char *where)
+{
+    return fail(h, SKB_ERR_CUDA, std::string(where) + ": " + cudaGetErrorString(e));
+}
+
+extern "C" skb_status sinkhorn_batch_create(const void *x, const void *y, const float *a, const float *b,
+                                            const float *eps, float tol, const skb_config *cfg, skb_batch **out)
+{
+    if (!out) return fail(nullptr, SKB_ERR_NULL, "out is null");
+    *out = nullptr;
+    if (!x || !y || !a || !b || !eps || !cfg) return fail(nullptr, SKB_ERR_NULL, "x, y, a, b, eps and cfg are required");
+    std::string why;
+    if (!config_ok(cfg, why)) {
+        const bool shape = cfg->W < 1 || cfg->n < 1 || cfg->m < 1 || cfg->d < 1;
+        return fail(nullptr, shape ? SKB_ERR_SHAPE : SKB_ERR_VALUE, why);
+    }
+    if (!(tol > 0.0f) || !std::isfinite(tol)) return fail(nullptr, SKB_ERR_VALUE, "tol must be positive and finite");
+    const Variant *var = choose_variant(cfg->W, cfg->n, cfg->m, cfg->d, cfg->compute == SKB_COMPUTE_F64, cfg->column_split);
+    if (!var) return fail(nullptr, SKB_ERR_SHAPE, "dimension d is not supported by any update kernel");
+    const int mx = cfg->n > cfg->m ? cfg->n : cfg->m;
+    if ((mx + var->rows_per_cta - 1) / var->rows_per_cta > MAX_PARTS)
+        return fail(nullptr, SKB_ERR_SHAPE, "n or m too large for the residual scratch");
+    if (cfg->W > 65535) return fail(nullptr, SKB_ERR_SHAPE, "W must be <= 65535");
+    size_t zero_end = 0;
+    const size_t need = carve(cfg, var, nullptr, nullptr, &zero_end);
+    if (!cfg->workspace) return fail(nullptr, SKB_ERR_WORKSPACE, "workspace is null");
+    if (((uintptr_t)cfg->workspace & 255u) != 0) return fail(nullptr, SKB_ERR_WORKSPACE, "workspace must be 256-byte aligned");
+    if (cfg->workspace_bytes < need) {
+        char buf[128];
+        snprintf(buf, sizeof(buf), "workspace too small: %zu bytes given, %zu needed", cfg->workspace_bytes, need);
+        return fail(nullptr, SKB_ERR_WORKSPACE, buf);
+    }
+    skb_batch *h = new (std::nothrow) skb_batch();
+    if (!h) return fail(nullptr, SKB_ERR_CUDA, "host allocation failed");
+    h->cfg = *cfg; h->var = var; h->stream = (cudaStream_t)cfg->stream;
+    h->known_width = cfg->W; h->finished = false; h->enqueued = 0; h->h_ctl = nullptr;
+    h->ev[0] = h->ev[1] = nullptr;
+    carve(cfg, var, (char *)cfg->workspace, &h->dev);
+    h->dev.tol_stop = (double)tol;
+    h->dev.tol_screen = cfg->tol_screen > 0.0f ? (double)cfg->tol_screen : (double)tol;
+    cudaError_t e;
+    if ((e = cudaHostAlloc((void **)&h->h_ctl, 2 * sizeof(Ctl), cudaHostAllocDefault)) != cudaSuccess ||
+        (e = cudaEventCreateWithFlags(&h->ev[0], cudaEventDisableTiming)) != cudaSuccess ||
+        (e = cudaEventCreateWithFlags(&h->ev[1], cudaEventDisableTiming)) != cudaSuccess) {
+        skb_status st = cuda_fail(nullptr, e, "create");
+        sinkhorn_batch_destroy(h);
+        return st;
+    }
+    memset(h->h_ctl, 0, 2 * sizeof(Ctl));
+    Ctl init;
+    memset(&init, 0, sizeof(init));
+    init.n_phys = cfg->W; init.n_running = cfg->W;
+    h->h_ctl[0] = init;
+    if ((e = cudaMemsetAsync(cfg->workspace, 0, zero_end, h->stream)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(h->dev.ctl, &h->h_ctl[0], sizeof(Ctl), cudaMemcpyHostToDevice, h->stream)) != cudaSuccess) {
+        skb_status st = cuda_fail(nullptr, e, "create");
+        sinkhorn_batch_destroy(h);
+        return st;
+    }
+    launch_prep(h->dev, x, y, a, b, eps, h->stream);
+    // the pinned block is reused for snapshots: wait until the initial copy has been consumed
+    if ((e = cudaEventRecord(h->ev[0], h->stream)) != cudaSuccess || (e = cudaGetLastError()) != cudaSuccess) {
+        skb_status st = cuda_fail(nullptr, e, "create");
+        sinkhorn_batch_destroy(h);
+        return st;
+    }
+    cudaEventSynchronize(h->ev[0]);
+    *out = h;
+    return SKB_OK;
+}
+
+// one full cycle: f-leg (+ row screen of the previous state), column check of screen-positive
+// lanes, plan, emit/compact, g-leg
+static void enqueue_cycle(skb_batch *h)
+{
+    const int w = h->known_width;
+    h->var->launch(h->dev, LEG_F, w, h->stream);
+    h->var->launch(h->dev, LEG_V, w, h->stream);
+    launch_plan(h->dev, h->stream);
+    launch_emit_move(h->dev, w, h->stream);
+    h->var->launch(h->dev, LEG_G, w, h->stream);
+    h->enqueued++;
+}
+
+static skb_status absorb(skb_batch *h, const Ctl &c)
+{
+    if (c.error & ERR_VALUE) return fail(h, SKB_ERR_VALUE, "inputs rejected on the device: weights and eps must be positive, coordinates finite");
+    if (c.error) return fail(h, SKB_ERR_CUDA, "a kernel reported an internal error");
+    if (h->cfg.mode == SKB_ACTIVE && c.n_phys >= 0 && c.n_phys < h->known_width) h->known_width = c.n_phys;
+    if (c.done) h->finished = true;
+    return SKB_OK;
+}
+
+extern "C" skb_status sinkhorn_batch_step(skb_batch *h, int cycles)
+{
+    if (!h) return SKB_ERR_NULL;
+    if (cycles < 0) return fail(h, SKB_ERR_VALUE, "cycles must be >= 0");
+    for (int i = 0; i < cycles && !h->finished; ++i) enqueue_cycle(h);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(h, e, "step");
+    return SKB_OK;
+}
+
+extern "C" skb_status sinkhorn_batch_drain(skb_batch *h, int *cycles_run)
+{
+    if (!h) return SKB_ERR_NULL;
+    cudaError_t e;
+    int chunk = 2, snap = 0;
+    bool have_prev = false;
+    // every lane is retired by the audit that follows cycle max_iter; STATIC needs one more pass
+    const long long hard_cap = (long long)h->cfg.max_iter + 4;
+    while (!h->finished) {
+        for (int i = 0; i < chunk; ++i) enqueue_cycle(h);
+        if ((e = cudaMemcpyAsync(&h->h_ctl[snap], h->dev.ctl, sizeof(Ctl), cudaMemcpyDeviceToHost, h->stream)) != cudaSuccess)
+            return cuda_fail(h, e, "drain");
+        if ((e = cudaEventRecord(h->ev[snap], h->stream)) != cudaSuccess) return cuda_fail(h, e, "drain");
+        if (have_prev) {
+            if ((e = cudaEventSynchronize(h->ev[snap ^ 1])) != cudaSuccess) return cuda_fail(h, e, "drain");
+            skb_status st = absorb(h, h->h_ctl[snap ^ 1]);
+            if (st != SKB_OK) { cudaStreamSynchronize(h->stream); return st; }
+        }
+        have_prev = true;
+        snap ^= 1;
+        if (chunk < 16) chunk *= 2;
+        if (h->enqueued > hard_cap + 64) break;
+    }
+    if ((e = cudaStreamSynchronize(h->stream)) != cudaSuccess) return cuda_fail(h, e, "drain");
+    if ((e = cudaMemcpy(&h->h_ctl[0], h->dev.ctl, sizeof(Ctl), cudaMemcpyDeviceToHost)) != cudaSuccess)
+        return cuda_fail(h, e, "drain");
+    skb_status st = absorb(h, h->h_ctl[0]);
+    if (st != SKB_OK) return st;
+    if (!h->finished) return fail(h, SKB_ERR_STATE, "drain ended with lanes still running");
+    if (cycles_run) *cycles_run = h->h_ctl[0].cycle;
+    return SKB_OK;
+}
+
+static skb_status read_ctl(skb_batch *h, Ctl *c)
+{
+    cudaError_t e;
+    if ((e = cudaStreamSynchronize(h->stream)) != cudaSuccess) return cuda_fail(h, e, "sync");
+    if ((e = cudaMemcpy(&h->h_ctl[0], h->dev.ctl, sizeof(Ctl), cudaMemcpyDeviceToHost)) != cudaSuccess)
+        return cuda_fail(h, e, "read control block");
+    *c = h->h_ctl[0];
+    return absorb(h, *c);
+}
+
+extern "C" skb_status sinkhorn_batch_active(skb_batch *h, int *n_active)
+{
+    if (!h || !n_active) return SKB_ERR_NULL;
+    Ctl c;
+    skb_status st = read_ctl(h, &c);
+    if (st != SKB_OK) return st;
+    *n_active = c.done ? 0 : (h->cfg.mode == SKB_STATIC ? h->cfg.W : c.n_running);
+    return SKB_OK;
+}
+
+extern "C" skb_status sinkhorn_batch_potentials(skb_batch *h, float *f, float *g)
+{
+    if (!h) return SKB_ERR_NULL;
+    launch_gather(h->dev, f, g, false, h->stream);
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? SKB_OK : cuda_fail(h, e, "potentials");
+}
+
+extern "C" skb_status sinkhorn_batch_potentials_f64(skb_batch *h, double *f, double *g)
+{
+    if (!h) return SKB_ERR_NULL;
+    launch_gather(h->dev, f, g, true, h->stream);
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? SKB_OK : cuda_fail(h, e, "potentials");
+}
+
+extern "C" skb_status sinkhorn_batch_depths(skb_batch *h, int *depth, int *lane_status)
+{
+    if (!h) return SKB_ERR_NULL;
+    launch_gather_small(h->dev, depth, lane_status, nullptr, nullptr, h->stream);
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? SKB_OK : cuda_fail(h, e, "depths");
+}
+
+extern "C" skb_status sinkhorn_batch_residuals(skb_batch *h, float *r_row, float *r_col)
+{
+    if (!h) return SKB_ERR_NULL;
+    launch_gather_small(h->dev, nullptr, nullptr, r_row, r_col, h->stream);
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? SKB_OK : cuda_fail(h, e, "residuals");
+}
+
+extern "C" skb_status sinkhorn_batch_stats(skb_batch *h, long long *slots, int *cycles, int *widths,
+                                           int widths_cap, long long *pair_terms)
+{
+    if (!h) return SKB_ERR_NULL;
+    Ctl c;
+    skb_status st = read_ctl(h, &c);
+    if (st != SKB_OK) return st;
+    if (slots) *slots = c.slots;
+    if (cycles) *cycles = c.cycle;
+    if (pair_terms) *pair_terms = c.pair_terms;
+    if (widths && widths_cap > 0) {
+        int k = c.cycle < widths_cap ? c.cycle : widths_cap;
+        if (k > h->cfg.max_iter + 2) k = h->cfg.max_iter + 2;
+        cudaError_t e = cudaMemcpy(widths, h->dev.widths, (size_t)k * sizeof(int), cudaMemcpyDeviceToHost);
+        if (e != cudaSuccess) return cuda_fail(h, e, "stats");
+    }
+    return SKB_OK;
+}
+
+struct HostStage { size_t x, y, a, b, eps, f, g, depth, status, rrow, rcol, end; };
+
+static HostStage host_stage(const skb_config *c, size_t base)
+{
+    HostStage s;
+    size_t off = align_up(base, 256);
+    auto take = [&](size_t b) { size_t o = off; off += align_up(b, 256); return o; };
+    const size_t W = c->W, n = c->n, m = c->m, d = c->d, es = c->xy_dtype == SKB_BF16 ? 2 : 4;
+    s.x = take(W * n * d * es); s.y = take(W * m * d * es);
+    s.a = take(W * n * 4); s.b = take(W * m * 4); s.eps = take(W * 4);
+    s.f = take(W * n * 4); s.g = take(W * m * 4);
+    s.depth = take(W * 4); s.status = take(W * 4); s.rrow = take(W * 4); s.rcol = take(W * 4);
+    s.end = off;
+    return s;
+}
+
+extern "C" size_t sinkhorn_batch_host_workspace_bytes(const skb_config *cfg)
+{
+    const size_t core = sinkhorn_batch_workspace_bytes(cfg);
+    if (core == 0) return 0;
+    return host_stage(cfg, core).end;
+}
+
+extern "C" skb_status sinkhorn_batch_solve_host(const void *x, const void *y, const float *a, const float *b,
+                                                const float *eps, float tol, const skb_config *cfg,
+                                                float *f, float *g, int *depth, int *lane_status,
+                                                float *r_row, float *r_col, long long *slots, int *cycles)
+{
+    if (!x || !y || !a || !b || !eps || !cfg) return fail(nullptr, SKB_ERR_NULL, "x, y, a, b, eps and cfg are required");
+    const size_t core = sinkhorn_batch_workspace_bytes(cfg);
+    if (core == 0) return fail(nullptr, SKB_ERR_SHAPE, "configuration rejected");
+    const HostStage s = host_stage(cfg, core);
+    if (!cfg->workspace || cfg->workspace_bytes < s.end) return fail(nullptr, SKB_ERR_WORKSPACE, "workspace too small for the host-buffer call");
+    char *base = (char *)cfg->workspace;
+    cudaStream_t st = (cudaStream_t)cfg->stream;
+    const size_t W = cfg->W, n = cfg->n, m = cfg->m, d = cfg->d, es = cfg->xy_dtype == SKB_BF16 ? 2 : 4;
+    cudaError_t e;
+    if ((e = cudaMemcpyAsync(base + s.x, x, W * n * d * es, cudaMemcpyHostToDevice, st)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(base + s.y, y, W * m * d * es, cudaMemcpyHostToDevice, st)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(base + s.a, a, W * n * 4, cudaMemcpyHostToDevice, st)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(base + s.b, b, W * m * 4, cudaMemcpyHostToDevice, st)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(base + s.eps, eps, W * 4, cudaMemcpyHostToDevice, st)) != cudaSuccess)
+        return cuda_fail(nullptr, e, "solve_host (copy in)");
+    skb_config inner = *cfg;
+    inner.workspace_bytes = core;
+    skb_batch *h = nullptr;
+    skb_status rc = sinkhorn_batch_create(base + s.x, base + s.y, (const float *)(base + s.a), (const float *)(base + s.b),
+                                          (const float *)(base + s.eps), tol, &inner, &h);
+    if (rc != SKB_OK) return rc;
+    int cyc = 0;
+    rc = sinkhorn_batch_drain(h, &cyc);
+    if (rc == SKB_OK) rc = sinkhorn_batch_potentials(h, f ? (float *)(base + s.f) : nullptr, g ? (float *)(base + s.g) : nullptr);
+    if (rc == SKB_OK) rc = sinkhorn_batch_depths(h, (int *)(base + s.depth), (int *)(base + s.status));
+    if (rc == SKB_OK) rc = sinkhorn_batch_residuals(h, (float *)(base + s.rrow), (float *)(base + s.rcol));
+    if (rc == SKB_OK) {
+        e = cudaSuccess;
+        if (f) e = cudaMemcpyAsync(f, base + s.f, W * n * 4, cudaMemcpyDeviceToHost, st);
+        if (g && e == cudaSuccess) e = cudaMemcpyAsync(g, base + s.g, W * m * 4, cudaMemcpyDeviceToHost, st);
+        if (depth && e == cudaSuccess) e = cudaMemcpyAsync(depth, base + s.depth, W * 4, cudaMemcpyDeviceToHost, st);
+        if (lane_status && e == cudaSuccess) e = cudaMemcpyAsync(lane_status, base + s.status, W * 4, cudaMemcpyDeviceToHost, st);
+        if (r_row && e == cudaSuccess) e = cudaMemcpyAsync(r_row, base + s.rrow, W * 4, cudaMemcpyDeviceToHost, st);
+        if (r_col && e == cudaSuccess) e = cudaMemcpyAsync(r_col, base + s.rcol, W * 4, cudaMemcpyDeviceToHost, st);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+        if (e != cudaSuccess) rc = cuda_fail(nullptr, e, "solve_host (copy out)");
+    }
+    if (rc == SKB_OK && (slots || cycles)) rc = sinkhorn_batch_stats(h, slots, cycles, nullptr, 0, nullptr);
+    if (rc != SKB_OK && h) g_create_err = h->err;
+    sinkhorn_batch_destroy(h);
+    return rc;
+}
+
+extern "C" void sinkhorn_batch_destroy(skb_batch *h)
+{
+    if (!h) return;
+    if (h->stream || h->h_ctl) cudaStreamSynchronize(h->stream);
+    if (h->ev[0]) cudaEventDestroy(h->ev[0]);
+    if (h->ev[1]) cudaEventDestroy(h->ev[1]);
+    if (h->h_ctl) cudaFreeHost(h->h_ctl);
+    delete h;
+}
+
+extern "C" const char *sinkhorn_batch_last_error(const skb_batch *h)
+{
+    return h ? h->err.c_str() : g_create_err.c_str();
+}

@@ -1,0 +1,329 @@
+// Set-up, audit planning, retirement/compaction and read-back kernels.
+//
+//  prep       inputs -> the kernels' layout (scaled dimension-major coordinates, squared
+//             norms, log2 weights, cold potentials f = g = 0); validates values.
+//  plan       one CTA per audit: turns the per-lane flags into the retire list by a warp
+//             ballot / prefix-sum scan, records depth, status and residuals of retirees
+//             (completion depth l_t, Eq. 6), pairs every hole left below the new width
+//             with a survivor from above it, and advances the counters of Eq. 7.
+//  emit_move  writes retirees' potentials to the result buffers in the caller's units and
+//             copies each paired survivor's state into its hole ("physically compacts all
+//             candidate-indexed state", Section "Screen, verify, and compact").  Holes and
+//             sources are disjoint slot sets, so the in-place copies cannot race.
+//  gather     potentials in original lane order (retired lanes from the result buffers,
+//             running lanes from their slots).
+#include "skb_device.cuh"
+#include "skb_host.h"
+
+namespace skb {
+
+// ---------------------------------------------------------------- prep
+template <typename T>
+__global__ void prep_kernel(const Dev P, const void *xin, const void *yin, const float *a,
+                            const float *b, const float *eps)
+{
+    const int slot = blockIdx.y;
+    const int side = blockIdx.z;                     // 0: x / a, 1: y / b
+    const int npts = side ? P.m : P.n, pp = side ? P.mp : P.np;
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= pp) return;
+    const double e = (double)eps[slot];
+    const bool eps_ok = (e > 0.0) && isfinite(e);
+    const double s = eps_ok ? 1.4426950408889634 / e : 1.0;
+    if (i == 0 && side == 0) {
+        P.scale[slot] = s;
+        P.lane_id[slot] = slot;
+        if (!eps_ok) atomicOr(&P.ctl->error, ERR_VALUE);
+    }
+    T *crd = reinterpret_cast<T *>(side ? P.ys : P.xs) + (size_t)slot * P.DP * pp;
+    const size_t o = (size_t)slot * pp + i;
+    T *ctm = side ? reinterpret_cast<T *>(P.gt) : reinterpret_cast<T *>(P.ft[0]);
+    double *sq = side ? P.sqy : P.sqx, *lw = side ? P.lb2 : P.la2;
+    if (i >= npts) {                                  // padding points
+        for (int k = 0; k < P.DP; ++k) crd[(size_t)k * pp + i] = T(0);
+        ctm[o] = T(NEG_BIG);
+        if (!side) { reinterpret_cast<T *>(P.ft[1])[o] = T(NEG_BIG); P.phi[0][o] = 0.0; P.phi[1][o] = 0.0; }
+        else P.gam[o] = 0.0;
+        sq[o] = 0.0; lw[o] = 0.0;
+        return;
+    }
+    const double sc = sqrt(2.0 * s);
+    const size_t ibase = ((size_t)slot * npts + i) * P.d;
+    double nrm = 0.0;
+    bool ok = true;
+    for (int k = 0; k < P.DP; ++k) {
+        T v = T(0);
+        if (k < P.d) {
+            float raw;
+            if (P.xy_bf16) {
+                const unsigned short bits = reinterpret_cast<const unsigned short *>(side ? yin : xin)[ibase + k];
+                raw = __uint_as_float(((unsigned)bits) << 16);
+            } else {
+                raw = reinterpret_cast<const float *>(side ? yin : xin)[ibase + k];
+            }
+            ok = ok && isfinite(raw);
+            v = (T)(sc * (double)raw);
+        }
+        crd[(size_t)k * pp + i] = v;
+        nrm += (double)v * (double)v;
+    }
+    nrm *= 0.5;
+    const float w = (side ? b : a)[(size_t)slot * npts + i];
+    ok = ok && (w > 0.0f) && isfinite(w);
+    if (!ok) atomicOr(&P.ctl->error, ERR_VALUE);
+    sq[o] = nrm;
+    lw[o] = ok ? log2((double)w) : 0.0;
+    ctm[o] = (T)(-nrm);                                // cold start: phi = gam = 0
+    if (!side) { reinterpret_cast<T *>(P.ft[1])[o] = (T)(-nrm); P.phi[0][o] = 0.0; P.phi[1][o] = 0.0; }
+    else P.gam[o] = 0.0;
+}
+
+// ---------------------------------------------------------------- plan
+constexpr int PLAN_THREADS = 1024;
+
+// exclusive prefix sums of up to three 0/1 flags over the block, by warp ballot + popc
+__device__ __forceinline__ void block_scan3(int f0, int f1, int f2, int (&ex)[3], int (&tot)[3], int (*wsum)[3])
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const unsigned lt = (1u << lane) - 1u;
+    const unsigned b0 = __ballot_sync(0xffffffffu, f0), b1 = __ballot_sync(0xffffffffu, f1),
+                   b2 = __ballot_sync(0xffffffffu, f2);
+    ex[0] = __popc(b0 & lt); ex[1] = __popc(b1 & lt); ex[2] = __popc(b2 & lt);
+    __syncthreads();
+    if (lane == 0) { wsum[warp][0] = __popc(b0); wsum[warp][1] = __popc(b1); wsum[warp][2] = __popc(b2); }
+    __syncthreads();
+    int run[3] = {0, 0, 0};
+    for (int w = 0; w < PLAN_THREADS / 32; ++w) {
+        if (w == warp) { ex[0] += run[0]; ex[1] += run[1]; ex[2] += run[2]; }
+        run[0] += wsum[w][0]; run[1] += wsum[w][1]; run[2] += wsum[w][2];
+    }
+    tot[0] = run[0]; tot[1] = run[1]; tot[2] = run[2];
+}
+
+__global__ void __launch_bounds__(PLAN_THREADS) plan_kernel(const Dev P)
+{
+    __shared__ int wsum[PLAN_THREADS / 32][3];
+    Ctl c = *P.ctl;
+    const int tid = threadIdx.x;
+    if (c.done) { if (tid == 0) P.ctl->n_retire = 0; return; }
+    const int k = c.cycle;                           // cycles completed by the audited state
+    const int A = c.n_phys;
+    const bool limit = k >= P.max_iter;
+
+    if (P.mode == MODE_STATIC && c.static_final) {   // emit every lane at the common boundary
+        for (int s = tid; s < P.W; s += PLAN_THREADS) {
+            P.ret_slot[s] = s; P.ret_lane[s] = s; P.ret_src[s] = -1; P.ret_scale[s] = P.scale[s];
+            P.res_row[s] = P.rrow[s]; P.res_col[s] = P.rcol[s];
+            if (P.nonfinite[s]) P.status[s] = LANE_NONFINITE;
+        }
+        if (tid == 0) {
+            Ctl *g = P.ctl;
+            g->n_retire = P.W; g->emit_parity = c.parity; g->n_running = 0; g->done = 1;
+            g->pair_terms += (long long)P.W * P.n * P.m;      // the final column check
+        }
+        return;
+    }
+
+    // which running lanes leave at this audit
+    auto decide = [&](int s, int &ret, int &st) {
+        ret = 0; st = LANE_RUNNING;
+        if (s >= A) return;
+        const bool held = (P.mode != MODE_ACTIVE) && P.state[s] != 0;   // frozen / already passed
+        if (held) return;
+        if (P.nonfinite[s]) { ret = 1; st = LANE_NONFINITE; }
+        else if (P.flag[s] && P.verdict[s]) { ret = 1; st = LANE_DONE; }
+        else if (limit) { ret = 1; st = LANE_ITER_LIMIT; }
+    };
+
+    // pass 1: count retirees and screen-positive lanes
+    int cnt = 0, nflag = 0;
+    for (int s = tid; s < A; s += PLAN_THREADS) {
+        int r, st; decide(s, r, st); cnt += r;
+        nflag += (P.flag[s] != 0);
+    }
+    for (int off = 16; off > 0; off >>= 1) {
+        cnt += __shfl_down_sync(0xffffffffu, cnt, off);
+        nflag += __shfl_down_sync(0xffffffffu, nflag, off);
+    }
+    if ((tid & 31) == 0) { wsum[tid >> 5][0] = cnt; wsum[tid >> 5][1] = nflag; }
+    __syncthreads();
+    int nret = 0, nflagged = 0;
+    for (int w = 0; w < PLAN_THREADS / 32; ++w) { nret += wsum[w][0]; nflagged += wsum[w][1]; }
+    __syncthreads();
+    const int Anew = (P.mode == MODE_ACTIVE) ? A - nret : A;
+
+    // pass 2: ordered lists (retirees, holes below Anew, survivors at or above Anew)
+    int base[3] = {0, 0, 0};
+    for (int s0 = 0; s0 < A; s0 += PLAN_THREADS) {
+        const int s = s0 + tid;
+        int r, st; decide(s, r, st);
+        const int hole = (P.mode == MODE_ACTIVE) && r && s < Anew;
+        const int fill = (P.mode == MODE_ACTIVE) && !r && s >= Anew && s < A;
+        int ex[3], tot[3];
+        block_scan3(r, hole, fill, ex, tot, wsum);
+        if (r) {
+            const int idx = base[0] + ex[0];
+            const int lane = P.lane_id[s];
+            P.ret_slot[idx] = s; P.ret_lane[idx] = lane; P.ret_scale[idx] = P.scale[s];
+            P.ret_src[idx] = hole ? -(base[1] + ex[1]) - 2 : -1;      // hole ordinal, resolved below
+            if (P.mode != MODE_STATIC || st != LANE_DONE) {            // STATIC keeps residuals for the end
+                P.res_row[lane] = P.rrow[s];
+                P.res_col[lane] = P.flag[s] ? P.rcol[s] : __longlong_as_double(0x7ff8000000000000LL);
+            }
+            P.depth[lane] = limit && st != LANE_DONE ? P.max_iter : k;
+            P.status[lane] = st;
+            if (P.mode != MODE_ACTIVE) P.state[s] = 1;
+        }
+        if (hole) P.hole_list[base[1] + ex[1]] = s;
+        if (fill) P.fill_list[base[2] + ex[2]] = s;
+        base[0] += tot[0]; base[1] += tot[1]; base[2] += tot[2];
+        __syncthreads();
+    }
+    __threadfence_block();
+    __syncthreads();
+    const int nholes = base[1];
+    // resolve each hole's source, then move the per-slot scalars
+    for (int r = tid; r < nret; r += PLAN_THREADS) {
+        const int code = P.ret_src[r];
+        if (code <= -2) P.ret_src[r] = P.fill_list[-(code + 2)];
+    }
+    __syncthreads();
+    for (int h = tid; h < nholes; h += PLAN_THREADS) {
+        const int dst = P.hole_list[h], src = P.fill_list[h];
+        P.lane_id[dst] = P.lane_id[src];
+        P.scale[dst] = P.scale[src];
+        P.nonfinite[dst] = 0;
+    }
+    if (tid == 0) {
+        Ctl *g = P.ctl;
+        g->n_retire = (P.mode == MODE_STATIC) ? 0 : nret;
+        g->emit_parity = c.parity;
+        g->pair_terms += (long long)A * P.n * P.m              // the f-leg that produced this screen
+                         + (long long)nflagged * P.n * P.m;    // column checks
+        bool go_on;
+        if (P.mode == MODE_ACTIVE) {
+            g->n_phys = Anew; g->n_running = Anew; go_on = Anew > 0;
+        } else if (P.mode == MODE_MASKED) {
+            g->n_running = c.n_running - nret; go_on = g->n_running > 0;
+        } else {
+            g->n_passed = c.n_passed + nret;
+            go_on = g->n_passed < P.W;
+            if (!go_on) g->static_final = 1;
+        }
+        if (go_on) {
+            const int width = (P.mode == MODE_ACTIVE) ? Anew : P.W;
+            g->cycle = k + 1;
+            g->parity = c.parity ^ 1;
+            g->slots += width;
+            g->pair_terms += (long long)width * P.n * P.m;     // the g-leg that completes cycle k+1
+            if (k < P.max_iter + 1) P.widths[k] = width;
+        } else if (P.mode != MODE_STATIC) {
+            g->done = 1;
+        }
+    }
+}
+
+// ---------------------------------------------------------------- emit + move
+template <typename T>
+__global__ void __launch_bounds__(256) emit_move_kernel(const Dev P)
+{
+    const Ctl c = *P.ctl;
+    const int r = blockIdx.y;
+    if (r >= c.n_retire) return;
+    const int slot = P.ret_slot[r], lane = P.ret_lane[r], src = P.ret_src[r];
+    const double inv_s = 1.0 / P.ret_scale[r];
+    const int tid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
+    const int ep = c.emit_parity;
+    // emit: potentials of the audited state in the caller's units (f = phi / s)
+    for (int i = tid; i < P.n; i += nth)
+        P.f_out[(size_t)lane * P.n + i] = P.phi[ep][(size_t)slot * P.np + i] * inv_s;
+    for (int j = tid; j < P.m; j += nth)
+        P.g_out[(size_t)lane * P.m + j] = P.gam[(size_t)slot * P.mp + j] * inv_s;
+    if (tid == 0) P.emitted[lane] = 1;
+    if (src < 0) return;
+    // move the survivor in slot `src` into the hole `slot` (16-byte vector copies)
+    auto copy = [&](void *base, size_t bytes_per_lane) {
+        const uint4 *s4 = reinterpret_cast<const uint4 *>((const char *)base + (size_t)src * bytes_per_lane);
+        uint4 *d4 = reinterpret_cast<uint4 *>((char *)base + (size_t)slot * bytes_per_lane);
+        const size_t nv = bytes_per_lane / 16;
+        for (size_t v = tid; v < nv; v += nth) d4[v] = s4[v];
+    };
+    const int np_ = ep ^ 1;   // buffer that holds the survivors' current row potentials
+    copy(P.xs, (size_t)P.DP * P.np * sizeof(T));
+    copy(P.ys, (size_t)P.DP * P.mp * sizeof(T));
+    copy(P.sqx, (size_t)P.np * 8); copy(P.sqy, (size_t)P.mp * 8);
+    copy(P.la2, (size_t)P.np * 8); copy(P.lb2, (size_t)P.mp * 8);
+    copy(P.phi[np_], (size_t)P.np * 8);
+    copy(P.ft[np_], (size_t)P.np * sizeof(T));
+}
+
+// ---------------------------------------------------------------- gather (read-back)
+template <typename O>
+__global__ void gather_kernel(const Dev P, O *f, O *g)
+{
+    const Ctl c = *P.ctl;
+    const int y = blockIdx.y;
+    const int tid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
+    if (y < P.W) {                                    // emitted lanes, by lane id
+        const int lane = y;
+        if (!P.emitted[lane]) return;
+        if (f) for (int i = tid; i < P.n; i += nth) f[(size_t)lane * P.n + i] = (O)P.f_out[(size_t)lane * P.n + i];
+        if (g) for (int j = tid; j < P.m; j += nth) g[(size_t)lane * P.m + j] = (O)P.g_out[(size_t)lane * P.m + j];
+    } else {                                          // lanes still held in a slot
+        const int slot = y - P.W;
+        if (c.done || slot >= c.n_phys) return;
+        if (P.mode == MODE_MASKED && P.state[slot]) return;
+        const int lane = P.lane_id[slot];
+        if (P.emitted[lane]) return;
+        const double inv_s = 1.0 / P.scale[slot];
+        if (f) for (int i = tid; i < P.n; i += nth)
+            f[(size_t)lane * P.n + i] = (O)(P.phi[c.parity][(size_t)slot * P.np + i] * inv_s);
+        if (g) for (int j = tid; j < P.m; j += nth)
+            g[(size_t)lane * P.m + j] = (O)(P.gam[(size_t)slot * P.mp + j] * inv_s);
+    }
+}
+
+__global__ void gather_small_kernel(const Dev P, int *depth, int *status, float *rrow, float *rcol)
+{
+    const int t = blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= P.W) return;
+    if (depth) depth[t] = P.depth[t];
+    if (status) status[t] = P.status[t];
+    if (rrow) rrow[t] = (float)P.res_row[t];
+    if (rcol) rcol[t] = (float)P.res_col[t];
+}
+
+// ---------------------------------------------------------------- launchers
+void launch_prep(const Dev &P, const void *x, const void *y, const float *a, const float *b,
+                 const float *eps, cudaStream_t st)
+{
+    const int pp = P.np > P.mp ? P.np : P.mp;
+    dim3 grid((pp + 127) / 128, P.W, 2);
+    if (P.compute_f64) prep_kernel<double><<<grid, 128, 0, st>>>(P, x, y, a, b, eps);
+    else prep_kernel<float><<<grid, 128, 0, st>>>(P, x, y, a, b, eps);
+}
+void launch_plan(const Dev &P, cudaStream_t st) { plan_kernel<<<1, PLAN_THREADS, 0, st>>>(P); }
+void launch_emit_move(const Dev &P, int width, cudaStream_t st)
+{
+    if (width < 1) width = 1;
+    const size_t bytes = (size_t)P.DP * (P.np + P.mp) * (P.compute_f64 ? 8 : 4);
+    int gx = (int)(bytes / (256 * 16 * 4)) + 1;
+    if (gx > 64) gx = 64;
+    dim3 grid(gx, width);
+    if (P.compute_f64) emit_move_kernel<double><<<grid, 256, 0, st>>>(P);
+    else emit_move_kernel<float><<<grid, 256, 0, st>>>(P);
+}
+void launch_gather(const Dev &P, void *f, void *g, bool f64, cudaStream_t st)
+{
+    const int mx = P.n > P.m ? P.n : P.m;
+    int gx = (mx + 1023) / 1024; if (gx > 16) gx = 16;
+    dim3 grid(gx, 2 * P.W);
+    if (f64) gather_kernel<double><<<grid, 256, 0, st>>>(P, (double *)f, (double *)g);
+    else gather_kernel<float><<<grid, 256, 0, st>>>(P, (float *)f, (float *)g);
+}
+void launch_gather_small(const Dev &P, int *depth, int *status, float *rrow, float *rcol, cudaStream_t st)
+{
+    gather_small_kernel<<<(P.W + 255) / 256, 256, 0, st>>>(P, depth, status, rrow, rcol);
+}
+
+}  // namespace skb

@@ -1,0 +1,95 @@
+// Device-side state of a Sinkhorn batch and small numeric helpers shared by the kernels.
+//
+// Internal representation (all lane-indexed arrays are indexed by PHYSICAL SLOT; the
+// slot -> original lane map is lane_id[]):
+//   s        = log2(e)/eps                      per-lane scale, log2 domain
+//   phi, gam = s*f, s*g                          potentials, float64
+//   xs, ys   = sqrt(2s)*x, sqrt(2s)*y            coordinates, dimension-major [DP][npad]
+//   sqx, sqy = |xs_i|^2/2, |ys_j|^2/2            float64
+//   ft, gt   = phi - sqx, gam - sqy              per-point terms streamed by the opposite leg
+// so that log2 pi_ij = ft_i + gt_j + xs_i.ys_j  (plan of Eq. 3 with f = eps log u).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace skb {
+
+enum Leg : int { LEG_F = 0, LEG_G = 1, LEG_V = 2 };
+enum Mode : int { MODE_ACTIVE = 0, MODE_MASKED = 1, MODE_STATIC = 2 };
+enum LaneStatus : int { LANE_RUNNING = 0, LANE_DONE = 1, LANE_ITER_LIMIT = 2, LANE_NONFINITE = 3 };
+enum ErrBits : int { ERR_VALUE = 1, ERR_WAIT = 2 };
+
+constexpr float NEG_BIG = -1.0e30f;   // "minus infinity" for padded columns (finite: no NaNs)
+constexpr int UPD_THREADS = 128;
+constexpr int MAX_PARTS = 1024;       // upper bound on row blocks per lane (residual partials)
+
+// Device-resident control block.  Written by the plan kernel (one CTA), read by all.
+struct Ctl {
+    int n_phys;        // physical width of the next update launch (ACTIVE: survivors; else W)
+    int n_running;     // lanes not yet retired
+    int cycle;         // completed cycles; the state being audited is the one after `cycle` cycles
+    int parity;        // phi[parity] / ft[parity] hold the current row potentials
+    int n_retire;      // entries of the retire list written by the last plan
+    int emit_parity;   // buffer the retirees' f is emitted from
+    int done;          // nothing left to do
+    int static_final;  // STATIC: every lane has passed, next audit emits all lanes
+    int error;         // sticky ErrBits
+    int n_passed;      // STATIC: lanes that have recorded a depth
+    int pad0, pad1;
+    long long slots;       // lane-cycles physically executed
+    long long pair_terms;  // exp terms evaluated by update launches
+};
+
+struct Dev {
+    int W, n, m, d, np, mp, DP;
+    int mode, max_iter, audit_every, xy_bf16, compute_f64;
+    double tol_screen, tol_stop;
+    // slabs by slot
+    void *xs, *ys;            // [W][DP][np|mp]   T
+    void *ft[2];              // [W][np]          T
+    void *gt;                 // [W][mp]          T
+    double *sqx, *sqy;        // [W][np], [W][mp]
+    double *la2, *lb2;        // log2 a, log2 b
+    double *phi[2];           // [W][np]
+    double *gam;              // [W][mp]
+    // per-slot scalars
+    double *scale;            // s
+    int *lane_id;
+    int *state;               // MASKED: frozen; STATIC: passed
+    int *flag;                // screen-positive at this audit
+    int *verdict;             // two-sided check passed
+    int *nonfinite;
+    double *rrow, *rcol;      // residuals of the audited state
+    unsigned *cnt_row, *cnt_col;
+    double *part_row, *part_col;   // [W][MAX_PARTS] per-CTA partial sums (scratch)
+    // retire / move lists (plan -> emit_move)
+    int *ret_slot, *ret_lane, *ret_src;
+    double *ret_scale;
+    int *hole_list, *fill_list;
+    // results by original lane
+    double *f_out, *g_out;    // [W][n], [W][m]  potentials in the caller's units
+    int *depth, *status, *emitted;
+    double *res_row, *res_col;
+    int *widths;              // [max_iter + 2]
+    Ctl *ctl;
+};
+
+__device__ __forceinline__ float ex2_fast(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float ex2_t(float x) { return ex2_fast(x); }
+__device__ __forceinline__ double ex2_t(double x) { return exp2(x); }
+
+__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src)
+{
+    unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+}  // namespace skb

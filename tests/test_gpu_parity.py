@@ -1,0 +1,207 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the float64 CPU oracle on the
+same seeded inputs.  Bar: completion depths equal (F64 arithmetic: always; F32 arithmetic: a
+lane may sit one audit away only when the oracle's residual at the disputed audit is within
+the fp32 evaluation noise of tol, and every such lane is reported), potentials within 1e-4
+relative (fp32 pair arithmetic) of the oracle state at the same depth, achieved two-sided
+residual <= tol, slot counts exactly those of Eq. 6-8."""
+import ctypes
+
+import numpy as np
+import pytest
+
+from helpers import check_accounting, check_against_oracle, pot_err, run_gpu
+from paper_2607_24741_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+POT_TOL_F32 = 1e-4      # acceptance bar for fp32 pair arithmetic
+POT_TOL_F64 = 1e-9      # float64 pair arithmetic: differences are summation order only
+MARGIN_F32 = 2e-2       # a +-1 lane must have |r - tol|/tol below this at the disputed audit
+
+CASES = {
+    "tiny": dict(name="tiny"),
+    "sensor_ragged": dict(name="sensor", W=16, n=200, m=264),
+    "registration_small": dict(name="registration", W=4, n=1000),
+    "sweep_small": dict(name="sweep", W=48, n=100, m=77, max_iter=3000),
+}
+
+
+def _make(case):
+    kw = dict(CASES[case]); name = kw.pop("name")
+    return wl.make(name, **kw)
+
+
+@pytest.mark.parametrize("case", list(CASES))
+@pytest.mark.parametrize("mode", ["active", "masked"])
+def test_f64_arithmetic_reproduces_oracle_exactly(oracle, case, mode):
+    w = _make(case)
+    W = w.shape[0]
+    r = run_gpu(w, mode=mode, compute="f64")
+    misses = check_against_oracle(oracle, w, r, range(W), pot_tol=POT_TOL_F64, exact_depth=True)
+    assert misses == []
+    check_accounting(oracle, r, W, mode)
+
+
+@pytest.mark.parametrize("case", list(CASES))
+def test_f32_arithmetic_meets_the_bar(oracle, case):
+    w = _make(case)
+    W = w.shape[0]
+    r = run_gpu(w, mode="active", compute="f32")
+    misses = check_against_oracle(oracle, w, r, range(W), pot_tol=POT_TOL_F32, exact_depth=False)
+    for t, dg, do, margin in misses:
+        print(f"[depth miss] {case} lane {t}: gpu {dg} oracle {do} oracle margin {margin:.2e}")
+        assert margin <= MARGIN_F32
+    assert len(misses) <= max(1, W // 8)
+    check_accounting(oracle, r, W, "active")
+    # the float getter is the float64 one rounded
+    np.testing.assert_array_equal(r["f32"], r["f"].astype(np.float32))
+
+
+@pytest.mark.parametrize("case", ["tiny", "sweep_small"])
+@pytest.mark.parametrize("compute", ["f32", "f64"])
+def test_masked_equals_active_bitwise_and_static_matches_fixed_depth(oracle, case, compute):
+    w = _make(case)
+    W = w.shape[0]
+    ra = run_gpu(w, mode="active", compute=compute)
+    rm = run_gpu(w, mode="masked", compute=compute)
+    rs = run_gpu(w, mode="static", compute=compute)
+    # same update, screen, check, tolerance and completion times (logical-mask control)
+    np.testing.assert_array_equal(ra["depth"], rm["depth"])
+    np.testing.assert_array_equal(ra["f"], rm["f"]); np.testing.assert_array_equal(ra["g"], rm["g"])
+    np.testing.assert_array_equal(ra["r_row"], rm["r_row"])
+    # fixed-width control: same first-pass depths, every lane carried to l_max
+    np.testing.assert_array_equal(ra["depth"], rs["depth"])
+    lmax = int(ra["depth"].max())
+    check_accounting(oracle, rs, W, "static"); check_accounting(oracle, rm, W, "masked")
+    ref = oracle.solve_batch(w.x, w.y, w.a, w.b, w.eps, w.tol, max_iter=w.max_iter, fixed_cycles=lmax)
+    done = ra["status"] == 1
+    e = pot_err(rs["f"], rs["g"], ref.f, ref.g, w.eps.astype(np.float64))
+    assert e[done].max() <= (POT_TOL_F32 if compute == "f32" else POT_TOL_F64)
+    assert np.all(rs["r_row"][done] <= w.tol)
+    # removable slots R = W*l_max - sum l_t (Eq. 8)
+    assert rs["stats"]["slots"] - ra["stats"]["slots"] == W * lmax - int(ra["depth"].sum())
+
+
+def test_packing_commutes_with_the_per_lane_map(oracle):
+    # Eq. 2: a W-lane batch gives each lane what a one-lane batch gives it, bit for bit
+    w = wl.make("sweep", W=6, n=96, m=80, max_iter=2000)
+    r = run_gpu(w, mode="active", column_split=8)
+    for t in (0, 3, 5):
+        one = wl.Workload(w.name, w.x[t:t + 1], w.y[t:t + 1], w.a[t:t + 1], w.b[t:t + 1],
+                          w.eps[t:t + 1], w.tol, w.max_iter)
+        r1 = run_gpu(one, mode="active", column_split=8)
+        assert r1["depth"][0] == r["depth"][t]
+        np.testing.assert_array_equal(r1["f"][0], r["f"][t]); np.testing.assert_array_equal(r1["g"][0], r["g"][t])
+    r2 = run_gpu(w, mode="active", column_split=8)              # run-to-run determinism
+    np.testing.assert_array_equal(r2["f"], r["f"]); np.testing.assert_array_equal(r2["depth"], r["depth"])
+
+
+@pytest.mark.parametrize("cs", [1, 8, 32])
+def test_every_column_split_agrees_with_the_oracle(oracle, cs):
+    w = wl.make("sensor", W=5, n=150, m=333)
+    r = run_gpu(w, mode="active", compute="f64", column_split=cs)
+    assert check_against_oracle(oracle, w, r, range(5), pot_tol=POT_TOL_F64, exact_depth=True) == []
+    w3 = wl.make("registration", W=3, n=700)
+    r3 = run_gpu(w3, mode="active", compute="f32", column_split=cs)
+    check_against_oracle(oracle, w3, r3, range(3), pot_tol=POT_TOL_F32, exact_depth=False)
+
+
+def test_audit_grid_screen_threshold_and_iteration_limit(oracle):
+    w = wl.make("tiny")
+    r4 = run_gpu(w, compute="f64", audit_every=4)
+    assert np.all(r4["depth"] % 4 == 0)
+    assert check_against_oracle(oracle, w, r4, range(8), pot_tol=POT_TOL_F64, exact_depth=True, audit_every=4) == []
+    rs = run_gpu(w, compute="f64", tol_screen=5e-4)
+    assert check_against_oracle(oracle, w, rs, range(8), pot_tol=POT_TOL_F64, exact_depth=True, tol_screen=5e-4) == []
+    assert np.all(rs["r_row"] <= 5e-4)
+    cap = int(np.median(r4["depth"]))
+    rl = run_gpu(w, compute="f64", max_iter=cap)
+    assert check_against_oracle(oracle, w, rl, range(8), pot_tol=POT_TOL_F64, exact_depth=True, max_iter=cap) == []
+    assert set(rl["status"]) == {1, 2} and rl["depth"].max() == cap
+    assert np.all(np.isnan(rl["r_col"][rl["status"] == 2]))
+    check_accounting(oracle, rl, 8, "active")
+
+
+def test_degenerate_shapes(oracle):
+    one = wl.Workload("one", np.array([[[1.0, 2.0]]], np.float32), np.array([[[4.0, 6.0]]], np.float32),
+                      np.ones((1, 1), np.float32), np.ones((1, 1), np.float32),
+                      np.array([0.3], np.float32), 1e-6, 50)
+    r = run_gpu(one, compute="f64")
+    assert r["depth"][0] == 1 and r["f"][0, 0] + r["g"][0, 0] == pytest.approx(25.0, rel=1e-12)
+    w = wl.make("sensor", W=1, n=3, m=5)                          # far below one tile
+    r = run_gpu(w, compute="f64")
+    assert check_against_oracle(oracle, w, r, [0], pot_tol=POT_TOL_F64, exact_depth=True) == []
+    w = wl.make("sweep", W=300, n=8, m=9, max_iter=400)            # W beyond one scan block... of lanes
+    r = run_gpu(w, compute="f64")
+    assert check_against_oracle(oracle, w, r, [0, 17, 255, 299], pot_tol=POT_TOL_F64, exact_depth=True,
+                                max_iter=400) == []
+    check_accounting(oracle, r, 300, "active")
+
+
+def test_step_runs_fixed_cycles_and_running_lanes_are_readable(oracle):
+    import torch
+    from paper_2607_24741_b200 import binding as B
+    w = wl.make("tiny")
+    dev = torch.device("cuda:0")
+    t = lambda v: torch.from_numpy(v).to(dev)
+    sb = B.SinkhornBatch(t(w.x), t(w.y), t(w.a), t(w.b), t(w.eps), w.tol, mode="static", compute="f64")
+    sb.step(7)
+    f, g = sb.potentials(f64=True)
+    assert sb.active() == 8
+    ref = oracle.solve_batch(w.x, w.y, w.a, w.b, w.eps, w.tol, fixed_cycles=7)
+    # after 7 enqueued cycles the g-leg of cycle 7 has run: state (f7, g7)
+    assert pot_err(f.cpu().numpy(), g.cpu().numpy(), ref.f, ref.g, w.eps.astype(np.float64)).max() <= POT_TOL_F64
+    sb.drain(); assert sb.active() == 0
+    sb.close()
+
+
+def test_bad_inputs_are_reported_not_trapped():
+    import torch
+    from paper_2607_24741_b200 import binding as B
+    w = wl.make("tiny")
+    dev = torch.device("cuda:0")
+    t = lambda v: torch.from_numpy(v).to(dev)
+    a = w.a.copy(); a[2, 5] = 0.0
+    sb = B.SinkhornBatch(t(w.x), t(w.y), t(a), t(w.b), t(w.eps), w.tol)
+    with pytest.raises(B.SkbError) as e:
+        sb.drain()
+    assert e.value.code == 3
+    sb.close()
+    eps = w.eps.copy(); eps[1] = -1.0
+    sb = B.SinkhornBatch(t(w.x), t(w.y), t(w.a), t(w.b), t(eps), w.tol)
+    with pytest.raises(B.SkbError):
+        sb.drain()
+    sb.close()
+    with pytest.raises(B.SkbError):
+        B.SinkhornBatch(t(w.x), t(w.y), t(w.a), t(w.b), t(w.eps), -1.0)
+    cfg = B.make_config(8, 64, 64, 2)
+    cfg.workspace_bytes = 16
+    h = ctypes.c_void_p()
+    ws = torch.empty(1024, dtype=torch.uint8, device=dev)
+    cfg.workspace = ws.data_ptr()
+    rc = B.lib.sinkhorn_batch_create(t(w.x).data_ptr(), t(w.y).data_ptr(), t(w.a).data_ptr(), t(w.b).data_ptr(),
+                                     t(w.eps).data_ptr(), 1e-3, ctypes.byref(cfg), ctypes.byref(h))
+    assert rc == 4 and b"workspace too small" in B.lib.sinkhorn_batch_last_error(None)
+
+
+def test_host_buffer_call_matches_device_call(oracle):
+    import torch
+    from paper_2607_24741_b200 import binding as B
+    w = wl.make("sensor", W=8, n=128)
+    r = run_gpu(w)
+    W, n, m, d = w.shape
+    cfg = B.make_config(W, n, m, d, max_iter=w.max_iter)
+    need = B.sinkhorn_batch_host_workspace_bytes(cfg)
+    ws = torch.empty(need, dtype=torch.uint8, device="cuda:0")
+    cfg.workspace = ws.data_ptr(); cfg.workspace_bytes = need
+    f = np.empty((W, n), np.float32); g = np.empty((W, m), np.float32)
+    depth = np.empty(W, np.int32); status = np.empty(W, np.int32)
+    rr = np.empty(W, np.float32); rc = np.empty(W, np.float32)
+    slots = ctypes.c_longlong(0); cycles = ctypes.c_int(0)
+    p = lambda v: v.ctypes.data_as(ctypes.c_void_p)
+    code = B.lib.sinkhorn_batch_solve_host(p(w.x), p(w.y), p(w.a), p(w.b), p(w.eps), w.tol, ctypes.byref(cfg),
+                                           p(f), p(g), p(depth), p(status), p(rr), p(rc),
+                                           ctypes.byref(slots), ctypes.byref(cycles))
+    assert code == 0
+    np.testing.assert_array_equal(depth, r["depth"]); np.testing.assert_array_equal(f, r["f32"])
+    np.testing.assert_array_equal(g, r["g32"]); assert slots.value == r["stats"]["slots"]
