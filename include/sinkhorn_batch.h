@@ -53,7 +53,13 @@ typedef enum {
 } skb_mode;
 
 typedef enum { SKB_F32 = 0, SKB_BF16 = 1 } skb_dtype;           /* storage type of x and y only */
-typedef enum { SKB_COMPUTE_F32 = 0, SKB_COMPUTE_F64 = 1 } skb_compute; /* pair-term arithmetic */
+/* Arithmetic of the pair terms log2 pi_ij and their exponentials. */
+typedef enum {
+    SKB_COMPUTE_AUTO = 0,  /* F32, or MIXED when some lane's cost/eps range is beyond fp32     */
+    SKB_COMPUTE_F32 = 1,   /* fp32 exponents and exponentials                                  */
+    SKB_COMPUTE_MIXED = 2, /* float64 exponents (half-rate FP64 pipe), fp32 exponentials       */
+    SKB_COMPUTE_F64 = 3    /* float64 throughout, software exp2: the slow validation arithmetic */
+} skb_compute;
 
 typedef enum {
     SKB_LANE_RUNNING = 0,
@@ -66,12 +72,14 @@ typedef struct {
     int W, n, m, d;        /* lanes, source points, target points, dimension               */
     int xy_dtype;          /* skb_dtype                                                    */
     int mode;              /* skb_mode                                                     */
-    int compute;           /* skb_compute; F64 is the slow validation arithmetic           */
+    int compute;           /* skb_compute                                                  */
     int max_iter;          /* cycle cap per lane, >= 1                                     */
     int audit_every;       /* audit after every k-th cycle, >= 1                           */
     float tol_screen;      /* row-screen threshold; <= 0 means "same as tol"               */
     int column_split;      /* 0 = automatic; 1, 8 or 32 forces how many lanes of a warp     */
                            /* share one row's columns in the update kernel (tuning knob)  */
+    int cost_form;         /* 0 = chosen per lane from its scaled radius; 1 = expanded     */
+                           /* |x|^2+|y|^2-2x.y everywhere; 2 = difference |x-y|^2 everywhere */
     void *stream;          /* cudaStream_t (0 = legacy default stream)                     */
     void *workspace;       /* device, 256-byte aligned                                     */
     size_t workspace_bytes;

@@ -18,7 +18,7 @@ SKB_OK = 0
 STATUS_NAMES = {0: "SKB_OK", 1: "SKB_ERR_NULL", 2: "SKB_ERR_SHAPE", 3: "SKB_ERR_VALUE",
                 4: "SKB_ERR_WORKSPACE", 5: "SKB_ERR_STATE", 6: "SKB_ERR_CUDA"}
 MODES = {"active": 0, "masked": 1, "static": 2}
-COMPUTE = {"f32": 0, "f64": 1}
+COMPUTE = {"auto": 0, "f32": 1, "mixed": 2, "f64": 3}
 LANE_RUNNING, LANE_DONE, LANE_ITER_LIMIT, LANE_NONFINITE = 0, 1, 2, 3
 
 EXPORTS = (
@@ -35,6 +35,7 @@ class SkbConfig(ctypes.Structure):
                 ("xy_dtype", ctypes.c_int), ("mode", ctypes.c_int), ("compute", ctypes.c_int),
                 ("max_iter", ctypes.c_int), ("audit_every", ctypes.c_int),
                 ("tol_screen", ctypes.c_float), ("column_split", ctypes.c_int),
+                ("cost_form", ctypes.c_int),
                 ("stream", ctypes.c_void_p), ("workspace", ctypes.c_void_p),
                 ("workspace_bytes", ctypes.c_size_t)]
 
@@ -91,11 +92,11 @@ def _ptr(t):
     return None if t is None else ctypes.c_void_p(t.data_ptr())
 
 
-def make_config(W, n, m, d, *, bf16=False, mode="active", compute="f32", max_iter=5000,
-                audit_every=1, tol_screen=0.0, column_split=0, stream=0) -> SkbConfig:
+def make_config(W, n, m, d, *, bf16=False, mode="active", compute="auto", max_iter=5000,
+                audit_every=1, tol_screen=0.0, column_split=0, cost_form=0, stream=0) -> SkbConfig:
     return SkbConfig(W, n, m, d, 1 if bf16 else 0, MODES[mode] if isinstance(mode, str) else mode,
                      COMPUTE[compute] if isinstance(compute, str) else compute, max_iter, audit_every,
-                     tol_screen, column_split, stream, None, 0)
+                     tol_screen, column_split, cost_form, stream, None, 0)
 
 
 # ---- functions with the C names ------------------------------------------------------
@@ -138,8 +139,8 @@ def sinkhorn_batch_destroy(h):
 class SinkhornBatch:
     """One batch of W lanes on the current CUDA device (thin wrapper over the C calls)."""
 
-    def __init__(self, x, y, a, b, eps, tol, *, mode="active", compute="f32", max_iter=5000,
-                 audit_every=1, tol_screen=0.0, column_split=0, stream=None):
+    def __init__(self, x, y, a, b, eps, tol, *, mode="active", compute="auto", max_iter=5000,
+                 audit_every=1, tol_screen=0.0, column_split=0, cost_form=0, stream=None):
         if not (x.is_cuda and y.is_cuda and a.is_cuda and b.is_cuda and eps.is_cuda):
             raise ValueError("x, y, a, b, eps must be CUDA tensors")
         if x.dtype not in (torch.float32, torch.bfloat16) or y.dtype != x.dtype:
@@ -157,7 +158,7 @@ class SinkhornBatch:
         self.stream = stream if stream is not None else torch.cuda.current_stream(x.device)
         self.cfg = make_config(W, n, m, d, bf16=x.dtype == torch.bfloat16, mode=mode, compute=compute,
                                max_iter=max_iter, audit_every=audit_every, tol_screen=tol_screen,
-                               column_split=column_split, stream=self.stream.cuda_stream)
+                               column_split=column_split, cost_form=cost_form, stream=self.stream.cuda_stream)
         need = sinkhorn_batch_workspace_bytes(self.cfg)
         if need == 0:
             raise SkbError(2, "configuration rejected (unsupported shape or bad option)")

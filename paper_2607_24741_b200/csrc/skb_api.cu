@@ -27,6 +27,13 @@ struct skb_batch {
 
 static std::string g_create_err;
 
+// fp32 arithmetic: the expanded cost |x|^2+|y|^2-2x.y carries an error of about one ulp of the
+// scaled squared radius M = s*max|x-c|^2 into every exponent.  Above FORM_DIFF_RADIUS a lane
+// switches to the difference form; above MIXED_RADIUS (any lane) an automatic batch computes
+// its exponents in float64 and only the exponentials in fp32.
+static const double FORM_DIFF_RADIUS = 64.0;
+static const double MIXED_RADIUS = 512.0;
+
 static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 static bool config_ok(const skb_config *c, std::string &why)
@@ -35,8 +42,9 @@ static bool config_ok(const skb_config *c, std::string &why)
     if (c->W < 1 || c->n < 1 || c->m < 1 || c->d < 1) { why = "W, n, m, d must be >= 1"; return false; }
     if (c->xy_dtype != SKB_F32 && c->xy_dtype != SKB_BF16) { why = "bad xy_dtype"; return false; }
     if (c->mode < SKB_ACTIVE || c->mode > SKB_STATIC) { why = "bad mode"; return false; }
-    if (c->compute != SKB_COMPUTE_F32 && c->compute != SKB_COMPUTE_F64) { why = "bad compute type"; return false; }
+    if (c->compute < SKB_COMPUTE_AUTO || c->compute > SKB_COMPUTE_F64) { why = "bad compute type"; return false; }
     if (c->max_iter < 1 || c->audit_every < 1) { why = "max_iter and audit_every must be >= 1"; return false; }
+    if (c->cost_form < 0 || c->cost_form > 2) { why = "cost_form must be 0 (automatic), 1 (expanded) or 2 (difference)"; return false; }
     if (c->column_split != 0 && c->column_split != 1 && c->column_split != 8 && c->column_split != 32) {
         why = "column_split must be 0, 1, 8 or 32"; return false;
     }
@@ -60,6 +68,9 @@ static size_t carve(const skb_config *c, const Variant *var, char *base, Dev *D,
     d.W = c->W; d.n = c->n; d.m = c->m; d.d = c->d; d.np = (int)np; d.mp = (int)mp; d.DP = (int)DP;
     d.mode = c->mode; d.max_iter = c->max_iter; d.audit_every = c->audit_every;
     d.xy_bf16 = c->xy_dtype == SKB_BF16; d.compute_f64 = var->f64;
+    d.cost_form = c->cost_form;
+    // fp32: above this scaled squared radius the expanded cost loses more than ~4e-6 per term
+    d.form_threshold = FORM_DIFF_RADIUS;
     // control block first, then everything that must start at zero, in one contiguous range
     d.ctl = (Ctl *)take(sizeof(Ctl));
     d.state = (int *)take(W * 4); d.flag = (int *)take(W * 4); d.verdict = (int *)take(W * 4);
@@ -71,12 +82,14 @@ static size_t carve(const skb_config *c, const Variant *var, char *base, Dev *D,
     d.widths = (int *)take(((size_t)c->max_iter + 2) * 4);
     const size_t zero_end = off;
     d.scale = (double *)take(W * 8); d.lane_id = (int *)take(W * 4);
+    d.center = (double *)take(W * DP * 8); d.form = (int *)take(W * 4);
     d.ret_slot = (int *)take(W * 4); d.ret_lane = (int *)take(W * 4); d.ret_src = (int *)take(W * 4);
     d.ret_scale = (double *)take(W * 8);
     d.hole_list = (int *)take(W * 4); d.fill_list = (int *)take(W * 4);
     d.part_row = (double *)take(W * MAX_PARTS * 8); d.part_col = (double *)take(W * MAX_PARTS * 8);
     d.xs = take(W * DP * np * ts); d.ys = take(W * DP * mp * ts);
     d.ft[0] = take(W * np * ts); d.ft[1] = take(W * np * ts); d.gt = take(W * mp * ts);
+    d.fl[0] = take(W * np * ts); d.fl[1] = take(W * np * ts); d.gl = take(W * mp * ts);
     d.sqx = (double *)take(W * np * 8); d.sqy = (double *)take(W * mp * 8);
     d.la2 = (double *)take(W * np * 8); d.lb2 = (double *)take(W * mp * 8);
     d.phi[0] = (double *)take(W * np * 8); d.phi[1] = (double *)take(W * np * 8);
@@ -87,11 +100,18 @@ static size_t carve(const skb_config *c, const Variant *var, char *base, Dev *D,
     return off;
 }
 
+static const Variant *variant_for(const skb_config *c, int compute)
+{
+    const bool f64 = compute == SKB_COMPUTE_F64 || compute == SKB_COMPUTE_MIXED;
+    return choose_variant(c->W, c->n, c->m, c->d, f64, compute == SKB_COMPUTE_MIXED, c->column_split);
+}
+
 extern "C" size_t sinkhorn_batch_workspace_bytes(const skb_config *cfg)
 {
     std::string why;
     if (!config_ok(cfg, why)) return 0;
-    const Variant *v = choose_variant(cfg->W, cfg->n, cfg->m, cfg->d, cfg->compute == SKB_COMPUTE_F64, cfg->column_split);
+    // an automatic batch may end up with float64 coordinates: size for the larger layout
+    const Variant *v = variant_for(cfg, cfg->compute == SKB_COMPUTE_AUTO ? SKB_COMPUTE_MIXED : cfg->compute);
     if (!v) return 0;
     return carve(cfg, v, nullptr, nullptr);
 }
@@ -119,14 +139,17 @@ extern "C" skb_status sinkhorn_batch_create(const void *x, const void *y, const 
         return fail(nullptr, shape ? SKB_ERR_SHAPE : SKB_ERR_VALUE, why);
     }
     if (!(tol > 0.0f) || !std::isfinite(tol)) return fail(nullptr, SKB_ERR_VALUE, "tol must be positive and finite");
-    const Variant *var = choose_variant(cfg->W, cfg->n, cfg->m, cfg->d, cfg->compute == SKB_COMPUTE_F64, cfg->column_split);
-    if (!var) return fail(nullptr, SKB_ERR_SHAPE, "dimension d is not supported by any update kernel");
+    const bool automatic = cfg->compute == SKB_COMPUTE_AUTO;
+    const Variant *var = variant_for(cfg, automatic ? SKB_COMPUTE_F32 : cfg->compute);
+    const Variant *var_big = variant_for(cfg, automatic ? SKB_COMPUTE_MIXED : cfg->compute);
+    if (!var || !var_big) return fail(nullptr, SKB_ERR_SHAPE, "dimension d is not supported by any update kernel");
     const int mx = cfg->n > cfg->m ? cfg->n : cfg->m;
-    if ((mx + var->rows_per_cta - 1) / var->rows_per_cta > MAX_PARTS)
+    if ((mx + var->rows_per_cta - 1) / var->rows_per_cta > MAX_PARTS ||
+        (mx + var_big->rows_per_cta - 1) / var_big->rows_per_cta > MAX_PARTS)
         return fail(nullptr, SKB_ERR_SHAPE, "n or m too large for the residual scratch");
     if (cfg->W > 65535) return fail(nullptr, SKB_ERR_SHAPE, "W must be <= 65535");
     size_t zero_end = 0;
-    const size_t need = carve(cfg, var, nullptr, nullptr, &zero_end);
+    const size_t need = carve(cfg, var_big, nullptr, nullptr, &zero_end);
     if (!cfg->workspace) return fail(nullptr, SKB_ERR_WORKSPACE, "workspace is null");
     if (((uintptr_t)cfg->workspace & 255u) != 0) return fail(nullptr, SKB_ERR_WORKSPACE, "workspace must be 256-byte aligned");
     if (cfg->workspace_bytes < need) {
@@ -161,7 +184,25 @@ extern "C" skb_status sinkhorn_batch_create(const void *x, const void *y, const 
         sinkhorn_batch_destroy(h);
         return st;
     }
-    launch_prep(h->dev, x, y, a, b, eps, h->stream);
+    launch_lane_stats(h->dev, x, y, eps, nullptr, h->stream);
+    if (automatic) {
+        // read the largest scaled radius back and pick the arithmetic for the whole batch
+        if ((e = cudaMemcpyAsync(&h->h_ctl[1], h->dev.ctl, sizeof(Ctl), cudaMemcpyDeviceToHost, h->stream)) != cudaSuccess ||
+            (e = cudaStreamSynchronize(h->stream)) != cudaSuccess) {
+            skb_status st = cuda_fail(nullptr, e, "create");
+            sinkhorn_batch_destroy(h);
+            return st;
+        }
+        double radius;
+        memcpy(&radius, &h->h_ctl[1].max_radius_bits, sizeof(double));
+        if (radius > MIXED_RADIUS) {
+            h->var = var_big;
+            const double ts = h->dev.tol_stop, tsc = h->dev.tol_screen;
+            carve(cfg, var_big, (char *)cfg->workspace, &h->dev);
+            h->dev.tol_stop = ts; h->dev.tol_screen = tsc;
+        }
+    }
+    launch_prep(h->dev, x, y, a, b, h->stream);
     // the pinned block is reused for snapshots: wait until the initial copy has been consumed
     if ((e = cudaEventRecord(h->ev[0], h->stream)) != cudaSuccess || (e = cudaGetLastError()) != cudaSuccess) {
         skb_status st = cuda_fail(nullptr, e, "create");

@@ -18,64 +18,109 @@
 namespace skb {
 
 // ---------------------------------------------------------------- prep
+__device__ __forceinline__ float load_raw(const Dev &P, const void *base, size_t idx)
+{
+    if (P.xy_bf16) return __uint_as_float(((unsigned)reinterpret_cast<const unsigned short *>(base)[idx]) << 16);
+    return reinterpret_cast<const float *>(base)[idx];
+}
+
+// One CTA per lane: joint centroid of the two clouds, the largest scaled squared distance
+// from it, and from that the cost form the lane will use.
+__global__ void __launch_bounds__(256) lane_stats_kernel(const Dev P, const void *xin, const void *yin, const float *eps)
+{
+    __shared__ double red[256];
+    __shared__ double cen[32];
+    const int slot = blockIdx.x, tid = threadIdx.x;
+    const int tot = P.n + P.m;
+    for (int k = 0; k < P.d; ++k) {
+        double s = 0.0;
+        for (int p = tid; p < tot; p += 256) {
+            const bool isx = p < P.n;
+            const size_t idx = isx ? ((size_t)slot * P.n + p) * P.d + k : ((size_t)slot * P.m + (p - P.n)) * P.d + k;
+            s += (double)load_raw(P, isx ? xin : yin, idx);
+        }
+        red[tid] = s;
+        __syncthreads();
+        for (int off = 128; off > 0; off >>= 1) { if (tid < off) red[tid] += red[tid + off]; __syncthreads(); }
+        if (tid == 0) cen[k] = red[0] / (double)tot;
+        __syncthreads();
+    }
+    double mxr = 0.0;
+    for (int p = tid; p < tot; p += 256) {
+        const bool isx = p < P.n;
+        const size_t base = isx ? ((size_t)slot * P.n + p) * P.d : ((size_t)slot * P.m + (p - P.n)) * P.d;
+        double r2 = 0.0;
+        for (int k = 0; k < P.d; ++k) { const double v = (double)load_raw(P, isx ? xin : yin, base + k) - cen[k]; r2 += v * v; }
+        mxr = fmax(mxr, r2);
+    }
+    red[tid] = mxr;
+    __syncthreads();
+    for (int off = 128; off > 0; off >>= 1) { if (tid < off) red[tid] = fmax(red[tid], red[tid + off]); __syncthreads(); }
+    if (tid < P.DP) P.center[(size_t)slot * P.DP + tid] = tid < P.d ? cen[tid] : 0.0;
+    if (tid == 0) {
+        const double e = (double)eps[slot];
+        const bool eps_ok = (e > 0.0) && isfinite(e);
+        const double s = eps_ok ? 1.4426950408889634 / e : 1.0;
+        if (!eps_ok) atomicOr(&P.ctl->error, ERR_VALUE);
+        P.scale[slot] = s;
+        P.lane_id[slot] = slot;
+        int form = P.cost_form == 1 ? FORM_DOT : (P.cost_form == 2 ? FORM_DIFF : (s * red[0] > P.form_threshold ? FORM_DIFF : FORM_DOT));
+        P.form[slot] = form;
+        atomicMax(&P.ctl->max_radius_bits, (unsigned long long)__double_as_longlong(eps_ok ? s * red[0] : 0.0));
+    }
+}
+
 template <typename T>
-__global__ void prep_kernel(const Dev P, const void *xin, const void *yin, const float *a,
-                            const float *b, const float *eps)
+__global__ void prep_kernel(const Dev P, const void *xin, const void *yin, const float *a, const float *b)
 {
     const int slot = blockIdx.y;
     const int side = blockIdx.z;                     // 0: x / a, 1: y / b
     const int npts = side ? P.m : P.n, pp = side ? P.mp : P.np;
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= pp) return;
-    const double e = (double)eps[slot];
-    const bool eps_ok = (e > 0.0) && isfinite(e);
-    const double s = eps_ok ? 1.4426950408889634 / e : 1.0;
-    if (i == 0 && side == 0) {
-        P.scale[slot] = s;
-        P.lane_id[slot] = slot;
-        if (!eps_ok) atomicOr(&P.ctl->error, ERR_VALUE);
-    }
+    const double s = P.scale[slot];
+    const int form = (sizeof(T) == 8) ? (int)FORM_DOT : P.form[slot];
     T *crd = reinterpret_cast<T *>(side ? P.ys : P.xs) + (size_t)slot * P.DP * pp;
     const size_t o = (size_t)slot * pp + i;
-    T *ctm = side ? reinterpret_cast<T *>(P.gt) : reinterpret_cast<T *>(P.ft[0]);
+    T *hi0 = side ? reinterpret_cast<T *>(P.gt) : reinterpret_cast<T *>(P.ft[0]);
+    T *lo0 = side ? reinterpret_cast<T *>(P.gl) : reinterpret_cast<T *>(P.fl[0]);
     double *sq = side ? P.sqy : P.sqx, *lw = side ? P.lb2 : P.la2;
+    T hi, lo = T(0);
     if (i >= npts) {                                  // padding points
         for (int k = 0; k < P.DP; ++k) crd[(size_t)k * pp + i] = T(0);
-        ctm[o] = T(NEG_BIG);
-        if (!side) { reinterpret_cast<T *>(P.ft[1])[o] = T(NEG_BIG); P.phi[0][o] = 0.0; P.phi[1][o] = 0.0; }
-        else P.gam[o] = 0.0;
+        hi = T(NEG_BIG);
         sq[o] = 0.0; lw[o] = 0.0;
-        return;
-    }
-    const double sc = sqrt(2.0 * s);
-    const size_t ibase = ((size_t)slot * npts + i) * P.d;
-    double nrm = 0.0;
-    bool ok = true;
-    for (int k = 0; k < P.DP; ++k) {
-        T v = T(0);
-        if (k < P.d) {
-            float raw;
-            if (P.xy_bf16) {
-                const unsigned short bits = reinterpret_cast<const unsigned short *>(side ? yin : xin)[ibase + k];
-                raw = __uint_as_float(((unsigned)bits) << 16);
-            } else {
-                raw = reinterpret_cast<const float *>(side ? yin : xin)[ibase + k];
+    } else {
+        const double sc = sqrt(form == FORM_DOT ? 2.0 * s : s);
+        const size_t ibase = ((size_t)slot * npts + i) * P.d;
+        const double *cen = P.center + (size_t)slot * P.DP;
+        double nrm = 0.0;
+        bool ok = true;
+        for (int k = 0; k < P.DP; ++k) {
+            T v = T(0);
+            if (k < P.d) {
+                const float raw = load_raw(P, side ? yin : xin, ibase + k);
+                ok = ok && isfinite(raw);
+                v = (T)(sc * ((double)raw - cen[k]));
             }
-            ok = ok && isfinite(raw);
-            v = (T)(sc * (double)raw);
+            crd[(size_t)k * pp + i] = v;
+            nrm += (double)v * (double)v;
         }
-        crd[(size_t)k * pp + i] = v;
-        nrm += (double)v * (double)v;
+        nrm = form == FORM_DOT ? 0.5 * nrm : 0.0;
+        const float w = (side ? b : a)[(size_t)slot * npts + i];
+        ok = ok && (w > 0.0f) && isfinite(w);
+        if (!ok) atomicOr(&P.ctl->error, ERR_VALUE);
+        sq[o] = nrm;
+        lw[o] = ok ? log2((double)w) : 0.0;
+        hi = (T)(-nrm);                                // cold start: phi = gam = 0
     }
-    nrm *= 0.5;
-    const float w = (side ? b : a)[(size_t)slot * npts + i];
-    ok = ok && (w > 0.0f) && isfinite(w);
-    if (!ok) atomicOr(&P.ctl->error, ERR_VALUE);
-    sq[o] = nrm;
-    lw[o] = ok ? log2((double)w) : 0.0;
-    ctm[o] = (T)(-nrm);                                // cold start: phi = gam = 0
-    if (!side) { reinterpret_cast<T *>(P.ft[1])[o] = (T)(-nrm); P.phi[0][o] = 0.0; P.phi[1][o] = 0.0; }
-    else P.gam[o] = 0.0;
+    hi0[o] = hi; lo0[o] = lo;
+    if (!side) {
+        reinterpret_cast<T *>(P.ft[1])[o] = hi; reinterpret_cast<T *>(P.fl[1])[o] = lo;
+        P.phi[0][o] = 0.0; P.phi[1][o] = 0.0;
+    } else {
+        P.gam[o] = 0.0;
+    }
 }
 
 // ---------------------------------------------------------------- plan
@@ -192,6 +237,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_kernel(const Dev P)
         const int dst = P.hole_list[h], src = P.fill_list[h];
         P.lane_id[dst] = P.lane_id[src];
         P.scale[dst] = P.scale[src];
+        P.form[dst] = P.form[src];
         P.nonfinite[dst] = 0;
     }
     if (tid == 0) {
@@ -237,8 +283,11 @@ __global__ void __launch_bounds__(256) emit_move_kernel(const Dev P)
     // emit: potentials of the audited state in the caller's units (f = phi / s)
     for (int i = tid; i < P.n; i += nth)
         P.f_out[(size_t)lane * P.n + i] = P.phi[ep][(size_t)slot * P.np + i] * inv_s;
-    for (int j = tid; j < P.m; j += nth)
+    for (int j = tid; j < P.m; j += nth) {
+        // the hole's own g is read before the survivor's g is copied over it (same thread)
         P.g_out[(size_t)lane * P.m + j] = P.gam[(size_t)slot * P.mp + j] * inv_s;
+        if (src >= 0) P.gam[(size_t)slot * P.mp + j] = P.gam[(size_t)src * P.mp + j];
+    }
     if (tid == 0) P.emitted[lane] = 1;
     if (src < 0) return;
     // move the survivor in slot `src` into the hole `slot` (16-byte vector copies)
@@ -255,6 +304,9 @@ __global__ void __launch_bounds__(256) emit_move_kernel(const Dev P)
     copy(P.la2, (size_t)P.np * 8); copy(P.lb2, (size_t)P.mp * 8);
     copy(P.phi[np_], (size_t)P.np * 8);
     copy(P.ft[np_], (size_t)P.np * sizeof(T));
+    copy(P.fl[np_], (size_t)P.np * sizeof(T));
+    copy(P.gt, (size_t)P.mp * sizeof(T));
+    copy(P.gl, (size_t)P.mp * sizeof(T));
 }
 
 // ---------------------------------------------------------------- gather (read-back)
@@ -294,13 +346,16 @@ __global__ void gather_small_kernel(const Dev P, int *depth, int *status, float 
 }
 
 // ---------------------------------------------------------------- launchers
-void launch_prep(const Dev &P, const void *x, const void *y, const float *a, const float *b,
-                 const float *eps, cudaStream_t st)
+void launch_lane_stats(const Dev &P, const void *x, const void *y, const float *eps, double *, cudaStream_t st)
+{
+    lane_stats_kernel<<<P.W, 256, 0, st>>>(P, x, y, eps);
+}
+void launch_prep(const Dev &P, const void *x, const void *y, const float *a, const float *b, cudaStream_t st)
 {
     const int pp = P.np > P.mp ? P.np : P.mp;
     dim3 grid((pp + 127) / 128, P.W, 2);
-    if (P.compute_f64) prep_kernel<double><<<grid, 128, 0, st>>>(P, x, y, a, b, eps);
-    else prep_kernel<float><<<grid, 128, 0, st>>>(P, x, y, a, b, eps);
+    if (P.compute_f64) prep_kernel<double><<<grid, 128, 0, st>>>(P, x, y, a, b);
+    else prep_kernel<float><<<grid, 128, 0, st>>>(P, x, y, a, b);
 }
 void launch_plan(const Dev &P, cudaStream_t st) { plan_kernel<<<1, PLAN_THREADS, 0, st>>>(P); }
 void launch_emit_move(const Dev &P, int width, cudaStream_t st)

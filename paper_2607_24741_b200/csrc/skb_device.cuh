@@ -8,6 +8,10 @@
 //   sqx, sqy = |xs_i|^2/2, |ys_j|^2/2            float64
 //   ft, gt   = phi - sqx, gam - sqy              per-point terms streamed by the opposite leg
 // so that log2 pi_ij = ft_i + gt_j + xs_i.ys_j  (plan of Eq. 3 with f = eps log u).
+// That is the expanded ("dot") form of the cost.  Lanes whose scaled squared radius is so
+// large that the expanded form would cancel catastrophically in fp32 use the difference
+// form instead: coordinates scaled by sqrt(s), ft/gt hold the high and fl/gl the low part
+// of the potentials, and log2 pi_ij = (phi_i + gam_j) - |xs_i - ys_j|^2.
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -18,6 +22,7 @@ enum Leg : int { LEG_F = 0, LEG_G = 1, LEG_V = 2 };
 enum Mode : int { MODE_ACTIVE = 0, MODE_MASKED = 1, MODE_STATIC = 2 };
 enum LaneStatus : int { LANE_RUNNING = 0, LANE_DONE = 1, LANE_ITER_LIMIT = 2, LANE_NONFINITE = 3 };
 enum ErrBits : int { ERR_VALUE = 1, ERR_WAIT = 2 };
+enum Form : int { FORM_DOT = 0, FORM_DIFF = 1 };
 
 constexpr float NEG_BIG = -1.0e30f;   // "minus infinity" for padded columns (finite: no NaNs)
 constexpr int UPD_THREADS = 128;
@@ -36,18 +41,22 @@ struct Ctl {
     int error;         // sticky ErrBits
     int n_passed;      // STATIC: lanes that have recorded a depth
     int pad0, pad1;
+    unsigned long long max_radius_bits;   // largest scaled squared radius over lanes (double bits)
     long long slots;       // lane-cycles physically executed
     long long pair_terms;  // exp terms evaluated by update launches
 };
 
 struct Dev {
     int W, n, m, d, np, mp, DP;
-    int mode, max_iter, audit_every, xy_bf16, compute_f64;
+    int mode, max_iter, audit_every, xy_bf16, compute_f64, cost_form;
+    double form_threshold;    // scaled squared radius above which a lane uses the difference form
     double tol_screen, tol_stop;
     // slabs by slot
     void *xs, *ys;            // [W][DP][np|mp]   T
     void *ft[2];              // [W][np]          T
     void *gt;                 // [W][mp]          T
+    void *fl[2], *gl;         // low parts of the potentials (difference form only)
+    double *center;           // [W][DP] joint centroid of the lane's two clouds
     double *sqx, *sqy;        // [W][np], [W][mp]
     double *la2, *lb2;        // log2 a, log2 b
     double *phi[2];           // [W][np]
@@ -55,6 +64,7 @@ struct Dev {
     // per-slot scalars
     double *scale;            // s
     int *lane_id;
+    int *form;                // Form per slot
     int *state;               // MASKED: frozen; STATIC: passed
     int *flag;                // screen-positive at this audit
     int *verdict;             // two-sided check passed

@@ -7,18 +7,18 @@ namespace skb {
 
 // Update-kernel variant: compute type, padded dimension, rows per thread, column split.
 struct Variant {
-    int f64, DP, R, CS;
+    int f64, xf, DP, R, CS;   // xf: float64 arguments with fp32 special-function exponentials
     int rows_per_cta;
     size_t smem;
     void (*launch)(const Dev &, int leg, int width, cudaStream_t);
 };
 // Picks the variant for a shape (depends on the static shape only, so that every mode
 // and every run of the same batch uses the same reduction order).  Null if unsupported.
-const Variant *choose_variant(int W, int n, int m, int d, bool f64, int force_cs);
+const Variant *choose_variant(int W, int n, int m, int d, bool f64, bool fast_exp, int force_cs);
 int padded_dim(int d);
 
-void launch_prep(const Dev &P, const void *x, const void *y, const float *a, const float *b,
-                 const float *eps, cudaStream_t st);
+void launch_lane_stats(const Dev &P, const void *x, const void *y, const float *eps, double *max_radius, cudaStream_t st);
+void launch_prep(const Dev &P, const void *x, const void *y, const float *a, const float *b, cudaStream_t st);
 void launch_plan(const Dev &P, cudaStream_t st);
 void launch_emit_move(const Dev &P, int width, cudaStream_t st);
 void launch_gather(const Dev &P, void *f, void *g, bool f64, cudaStream_t st);

@@ -4,21 +4,27 @@
 // the candidate axis of Eq. 2 is a grid axis and nothing is reduced across lanes.
 //
 // For a row point i of lane t the kernel evaluates, over all column points j,
-//     L_i = log2 sum_j 2^(ct_j + r_i . c_j)
-// with r, c the scaled coordinates and ct the column term (gt for the f-leg, ft for the
-// g-leg), as an online max / sum-of-exp2 reduction: the n x m matrix is never stored.
-// Column tiles are staged in shared memory by 16-byte cp.async copies from a
-// dimension-major layout; a thread keeps R rows in registers and walks 4 adjacent columns
-// per step; with CS > 1 the columns of a tile are split over CS neighbouring lanes of the
-// warp and the (max, sum) pairs are merged by xor-shuffles at the end.
+//     L_i = log2 sum_j 2^(arg_ij)
+// as an online max / sum-of-exp2 reduction: the n x m matrix is never stored.  Column
+// tiles are staged in shared memory by 16-byte cp.async copies from a dimension-major
+// layout; a thread keeps R rows in registers and walks 4 adjacent columns per step; with
+// CS > 1 the columns of a tile are split over CS neighbouring lanes of the warp and the
+// (max, sum) pairs are merged by xor-shuffles at the end.
+//
+// Two forms of arg_ij, chosen per lane when the batch is created:
+//   dot   arg_ij = ct_j + r_i . c_j            (d FMA per pair; ct = potential - |c_j|^2/2)
+//   diff  arg_ij = (ph_i + ch_j) + cl_j - |r_i - c_j|^2   (2d + 2 per pair; ph, ch are the
+//         fp32 high parts of the row and column potentials, cl the column's low part, and
+//         the row's own rounding error is removed in float64 afterwards).  It is used when
+//         the expanded form would cancel catastrophically in fp32.
 //
 // Leg-specific epilogues (float64, one per row):
-//   LEG_F  phi_new = log2 a + sqx - L;  also the row marginal of the state BEFORE this leg,
+//   LEG_F  phi_new from L;  also the row marginal of the state BEFORE this leg,
 //          sum_j pi_ij = a_i 2^(phi_old - phi_new), which is the one-sided row screen of
 //          Section "Screen, verify, and compact" obtained for free.
-//   LEG_G  gam_new = log2 b + sqy - L  (after it the column marginal equals b, Eq. 4).
+//   LEG_G  gam_new from L  (after it the column marginal equals b, Eq. 4).
 //   LEG_V  column marginal of the audited state for screen-positive lanes only,
-//          sum_i pi_ij = b_j 2^(gam - gam'), the second half of the two-sided check (Eq. 5).
+//          the second half of the two-sided check (Eq. 5).
 // The per-CTA L1 partial sums go to scratch; the last CTA of a lane adds them in a fixed
 // order and writes the lane's residual and its one flag (screen-positive / verdict).
 #pragma once
@@ -26,9 +32,10 @@
 
 namespace skb {
 
-template <int CS> struct TileCols { static constexpr int value = (CS <= 4) ? 128 : (CS == 8 ? 256 : 512); };
+template <typename T, int XF> struct SumType { using type = T; };
+template <> struct SumType<double, 1> { using type = float; };
 
-template <typename T> struct Vec4 { T v[4]; };
+template <int CS> struct TileCols { static constexpr int value = (CS <= 4) ? 128 : (CS == 8 ? 256 : 512); };
 
 __device__ __forceinline__ void lds4(const float *p, float (&v)[4])
 {
@@ -42,68 +49,43 @@ __device__ __forceinline__ void lds4(const double *p, double (&v)[4])
     v[0] = t0.x; v[1] = t0.y; v[2] = t1.x; v[3] = t1.y;
 }
 
-template <typename T, int DP, int R, int CS>
-__global__ void __launch_bounds__(UPD_THREADS) update_kernel(const Dev P, const int leg)
+// Streams every column tile of one lane past the CTA's rows and leaves, per row of this
+// thread, the running maximum md[r] and the sum sd[r] of 2^(arg - md[r]) over the columns
+// this thread visited.
+template <typename T, int DP, int R, int CS, int FORM, int XF>
+__device__ __forceinline__ void stream_columns(T *sm, const T *colc, const T *colt, const T *coll,
+                                               const int cp, const int ncols, const T (&xr)[R][DP],
+                                               const T (&ph)[R], const int tid, const int cs,
+                                               double (&md)[R], double (&sd)[R])
 {
-    constexpr int TJ = TileCols<CS>::value;      // columns per shared-memory tile
-    constexpr int STEPS = TJ / (4 * CS);         // 4-column groups per thread per tile
-    constexpr int RG = 32 / CS;                  // row groups per warp
-    constexpr int RW = R * RG;                   // rows per warp
-    constexpr int RB = (UPD_THREADS / 32) * RW;  // rows per CTA
-    constexpr int EPC = 16 / (int)sizeof(T);     // elements per 16-byte chunk
-    constexpr int STAGE = (DP + 1) * TJ;         // elements per stage
+    constexpr int TJ = TileCols<CS>::value;
+    constexpr int STEPS = TJ / (4 * CS);
+    constexpr int EPC = 16 / (int)sizeof(T);
+    constexpr int NR = DP + 1 + (FORM == FORM_DIFF ? 1 : 0);   // rows of a stage
+    constexpr int STAGE = (DP + 2) * TJ;
+    constexpr int CPR = TJ / EPC;
 
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    T *sm = reinterpret_cast<T *>(smem_raw);
-    __shared__ double red[UPD_THREADS / 32];
-    __shared__ int is_last;
-
-    const Ctl c = *P.ctl;
-    if (c.done) return;
-    const int slot = blockIdx.y;
-    if (slot >= c.n_phys) return;
-    if (leg != LEG_V && c.static_final) return;
-    if (leg == LEG_V && !(c.static_final || P.flag[slot])) return;
-
-    // roles: rows are x-points for the f-leg, y-points otherwise
-    const bool rows_x = (leg == LEG_F);
-    const int nrows = rows_x ? P.n : P.m, rp = rows_x ? P.np : P.mp;
-    const int ncols = rows_x ? P.m : P.n, cp = rows_x ? P.mp : P.np;
-    if ((int)blockIdx.x * RB >= nrows) return;
-    const T *rowc = reinterpret_cast<const T *>(rows_x ? P.xs : P.ys) + (size_t)slot * DP * rp;
-    const T *colc = reinterpret_cast<const T *>(rows_x ? P.ys : P.xs) + (size_t)slot * DP * cp;
-    const T *colt = rows_x ? reinterpret_cast<const T *>(P.gt) + (size_t)slot * cp
-                           : reinterpret_cast<const T *>(P.ft[c.parity]) + (size_t)slot * cp;
-
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int cs = lane % CS, rg = lane / CS;
-    const int row0 = blockIdx.x * RB + warp * RW + rg;   // row r of this thread: row0 + r*RG
-
-    T xr[R][DP];
+    // XF = 1: the exponentials run on the fp32 special-function unit even when the
+    // arguments are float64 ("mixed" arithmetic); the tile sum is then fp32 as well
+    using TS = typename SumType<T, XF>::type;
+    T mx[R];
+    TS ts[R];
 #pragma unroll
-    for (int r = 0; r < R; ++r) {
-        const int i = row0 + r * RG;
-#pragma unroll
-        for (int k = 0; k < DP; ++k) xr[r][k] = (i < nrows) ? rowc[(size_t)k * rp + i] : T(0);
-    }
-    T mx[R], ts[R];
-    double sd[R];
-#pragma unroll
-    for (int r = 0; r < R; ++r) { mx[r] = T(NEG_BIG); ts[r] = T(0); sd[r] = 0.0; }
+    for (int r = 0; r < R; ++r) { mx[r] = T(NEG_BIG); ts[r] = TS(0); sd[r] = 0.0; }
 
     const int ntiles = (ncols + TJ - 1) / TJ;
     auto load_tile = [&](int t, int stage) {
         T *dst = sm + stage * STAGE;
         const int j0 = t * TJ;
-        constexpr int CPR = TJ / EPC;   // chunks per row
-        for (int ch = tid; ch < (DP + 1) * CPR; ch += UPD_THREADS) {
+        for (int ch = tid; ch < NR * CPR; ch += UPD_THREADS) {
             const int k = ch / CPR, j = j0 + (ch % CPR) * EPC;
             T *d = dst + k * TJ + (ch % CPR) * EPC;
             if (j < cp) {
-                const T *src = (k < DP) ? colc + (size_t)k * cp + j : colt + j;
+                const T *src = (k < DP) ? colc + (size_t)k * cp + j : (k == DP ? colt + j : coll + j);
                 cp_async16(d, src);
             } else {
-                const T fill = (k < DP) ? T(0) : T(NEG_BIG);
+                // columns past the padded end: zero coordinates, "minus infinity" term
+                const T fill = (k == DP) ? T(NEG_BIG) : T(0);
 #pragma unroll
                 for (int e = 0; e < EPC; ++e) d[e] = fill;
             }
@@ -126,45 +108,123 @@ __global__ void __launch_bounds__(UPD_THREADS) update_kernel(const Dev P, const 
         for (int q = 0; q < STEPS; ++q) {
             const int jj = (q * CS + cs) * 4;
             T acc[R][4];
-            {
-                T ct[4];
-                lds4(st + DP * TJ + jj, ct);
+            T ct[4];
+            lds4(st + DP * TJ + jj, ct);
+            if (FORM == FORM_DOT) {
 #pragma unroll
                 for (int r = 0; r < R; ++r)
 #pragma unroll
                     for (int e = 0; e < 4; ++e) acc[r][e] = ct[e];
-            }
 #pragma unroll
-            for (int k = 0; k < DP; ++k) {
-                T yv[4];
-                lds4(st + k * TJ + jj, yv);
+                for (int k = 0; k < DP; ++k) {
+                    T yv[4];
+                    lds4(st + k * TJ + jj, yv);
+#pragma unroll
+                    for (int r = 0; r < R; ++r)
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) acc[r][e] = fma(xr[r][k], yv[e], acc[r][e]);
+                }
+            } else {
+                T cl[4];
+                lds4(st + (DP + 1) * TJ + jj, cl);
 #pragma unroll
                 for (int r = 0; r < R; ++r)
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) acc[r][e] = fma(xr[r][k], yv[e], acc[r][e]);
+                    for (int e = 0; e < 4; ++e) acc[r][e] = cl[e];
+#pragma unroll
+                for (int k = 0; k < DP; ++k) {
+                    T yv[4];
+                    lds4(st + k * TJ + jj, yv);
+#pragma unroll
+                    for (int r = 0; r < R; ++r)
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const T dk = xr[r][k] - yv[e];
+                            acc[r][e] = fma(-dk, dk, acc[r][e]);
+                        }
+                }
+#pragma unroll
+                for (int r = 0; r < R; ++r)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) acc[r][e] += (ph[r] + ct[e]);
             }
 #pragma unroll
             for (int r = 0; r < R; ++r) {
                 const T mt = fmax(fmax(acc[r][0], acc[r][1]), fmax(acc[r][2], acc[r][3]));
                 if (mt > mx[r] + T(8)) {           // lazy rescale: terms stay below 2^8
-                    const T fac = ex2_t(mx[r] - mt);
+                    const TS fac = ex2_t((TS)(mx[r] - mt));
                     ts[r] *= fac;
                     sd[r] *= (double)fac;
                     mx[r] = mt;
                 }
-                ts[r] += (ex2_t(acc[r][0] - mx[r]) + ex2_t(acc[r][1] - mx[r])) +
-                         (ex2_t(acc[r][2] - mx[r]) + ex2_t(acc[r][3] - mx[r]));
+                ts[r] += (ex2_t((TS)(acc[r][0] - mx[r])) + ex2_t((TS)(acc[r][1] - mx[r]))) +
+                         (ex2_t((TS)(acc[r][2] - mx[r])) + ex2_t((TS)(acc[r][3] - mx[r])));
             }
         }
 #pragma unroll
-        for (int r = 0; r < R; ++r) { sd[r] += (double)ts[r]; ts[r] = T(0); }
+        for (int r = 0; r < R; ++r) { sd[r] += (double)ts[r]; ts[r] = TS(0); }
         __syncthreads();
     }
-
-    // merge the CS column splits of each row (xor-shuffle online logsumexp)
-    double md[R];
 #pragma unroll
     for (int r = 0; r < R; ++r) md[r] = (double)mx[r];
+}
+
+template <typename T, int DP, int R, int CS, int XF>
+__global__ void __launch_bounds__(UPD_THREADS) update_kernel(const Dev P, const int leg)
+{
+    constexpr int RG = 32 / CS;                  // row groups per warp
+    constexpr int RW = R * RG;                   // rows per warp
+    constexpr int RB = (UPD_THREADS / 32) * RW;  // rows per CTA
+
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    T *sm = reinterpret_cast<T *>(smem_raw);
+    __shared__ double red[UPD_THREADS / 32];
+    __shared__ int is_last;
+
+    const Ctl c = *P.ctl;
+    if (c.done) return;
+    const int slot = blockIdx.y;
+    if (slot >= c.n_phys) return;
+    if (leg != LEG_V && c.static_final) return;
+    if (leg == LEG_V && !(c.static_final || P.flag[slot])) return;
+
+    // roles: rows are x-points for the f-leg, y-points otherwise
+    const bool rows_x = (leg == LEG_F);
+    const int nrows = rows_x ? P.n : P.m, rp = rows_x ? P.np : P.mp;
+    const int ncols = rows_x ? P.m : P.n, cp = rows_x ? P.mp : P.np;
+    if ((int)blockIdx.x * RB >= nrows) return;
+    const int form = (sizeof(T) == 8) ? (int)FORM_DOT : P.form[slot];   // float64 arguments never need the difference form
+    const T *rowc = reinterpret_cast<const T *>(rows_x ? P.xs : P.ys) + (size_t)slot * DP * rp;
+    const T *colc = reinterpret_cast<const T *>(rows_x ? P.ys : P.xs) + (size_t)slot * DP * cp;
+    const T *colt = rows_x ? reinterpret_cast<const T *>(P.gt) + (size_t)slot * cp
+                           : reinterpret_cast<const T *>(P.ft[c.parity]) + (size_t)slot * cp;
+    const T *coll = rows_x ? reinterpret_cast<const T *>(P.gl) + (size_t)slot * cp
+                           : reinterpret_cast<const T *>(P.fl[c.parity]) + (size_t)slot * cp;
+    // potential the rows carry into this leg (shift of the difference form, screen reference)
+    const double *prow = (rows_x ? P.phi[c.parity] : P.gam) + (size_t)slot * rp;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int cs = lane % CS, rg = lane / CS;
+    const int row0 = blockIdx.x * RB + warp * RW + rg;   // row r of this thread: row0 + r*RG
+
+    T xr[R][DP], ph[R];
+    double pold[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+        const int i = row0 + r * RG;
+#pragma unroll
+        for (int k = 0; k < DP; ++k) xr[r][k] = (i < nrows) ? rowc[(size_t)k * rp + i] : T(0);
+        pold[r] = (i < nrows) ? prow[i] : 0.0;
+        ph[r] = (T)pold[r];
+    }
+
+    double md[R], sd[R];
+    if (form == FORM_DOT)
+        stream_columns<T, DP, R, CS, FORM_DOT, XF>(sm, colc, colt, coll, cp, ncols, xr, ph, tid, cs, md, sd);
+    else
+        stream_columns<T, DP, R, CS, FORM_DIFF, XF>(sm, colc, colt, coll, cp, ncols, xr, ph, tid, cs, md, sd);
+
+    // merge the CS column splits of each row (xor-shuffle online logsumexp)
 #pragma unroll
     for (int off = 1; off < CS; off <<= 1) {
 #pragma unroll
@@ -190,22 +250,30 @@ __global__ void __launch_bounds__(UPD_THREADS) update_kernel(const Dev P, const 
             const int i = row0 + r * RG;
             if (i >= nrows) continue;
             const double L = md[r] + log2(sd[r]);
-            const double pnew = lw[i] + sq[i] - L;
-            if (leg == LEG_F) {
-                const double pold = P.phi[c.parity][rbase + i];
-                term_sum += exp2(lw[i]) * fabs(expm1((pold - pnew) * 0.6931471805599453));
-                if (writes) {
-                    P.phi[c.parity ^ 1][rbase + i] = pnew;
-                    reinterpret_cast<T *>(P.ft[c.parity ^ 1])[rbase + i] = (T)(pnew - sq[i]);
-                }
-            } else if (leg == LEG_G) {
-                if (writes) {
-                    P.gam[rbase + i] = pnew;
-                    reinterpret_cast<T *>(P.gt)[rbase + i] = (T)(pnew - sq[i]);
-                }
+            // log2 of this row's marginal under the potentials the leg started from, and the
+            // updated potential that makes the marginal equal to the weight (Eq. 3)
+            double lmarg, pnew;
+            if (form == FORM_DOT) {
+                pnew = lw[i] + sq[i] - L;
+                lmarg = lw[i] + pold[r] - pnew;
             } else {
-                const double pold = P.gam[rbase + i];
-                term_sum += exp2(lw[i]) * fabs(expm1((pold - pnew) * 0.6931471805599453));
+                lmarg = L - ((double)ph[r] - pold[r]);
+                pnew = pold[r] + (lw[i] - lmarg);
+            }
+            if (leg != LEG_G) term_sum += exp2(lw[i]) * fabs(expm1((lmarg - lw[i]) * 0.6931471805599453));
+            if (writes) {
+                T hi, lo;
+                if (form == FORM_DOT) { hi = (T)(pnew - sq[i]); lo = T(0); }
+                else { hi = (T)pnew; lo = (T)(pnew - (double)hi); }
+                if (leg == LEG_F) {
+                    P.phi[c.parity ^ 1][rbase + i] = pnew;
+                    reinterpret_cast<T *>(P.ft[c.parity ^ 1])[rbase + i] = hi;
+                    reinterpret_cast<T *>(P.fl[c.parity ^ 1])[rbase + i] = lo;
+                } else {
+                    P.gam[rbase + i] = pnew;
+                    reinterpret_cast<T *>(P.gt)[rbase + i] = hi;
+                    reinterpret_cast<T *>(P.gl)[rbase + i] = lo;
+                }
             }
         }
     }
@@ -248,11 +316,5 @@ __global__ void __launch_bounds__(UPD_THREADS) update_kernel(const Dev P, const 
         if (!finite) P.nonfinite[slot] = 1;
     }
 }
-
-template <typename T, int DP, int R, int CS>
-inline size_t update_smem_bytes() { return 2 * (size_t)(DP + 1) * TileCols<CS>::value * sizeof(T); }
-
-template <typename T, int DP, int R, int CS>
-inline int update_rows_per_cta() { return (UPD_THREADS / 32) * R * (32 / CS); }
 
 }  // namespace skb

@@ -5,8 +5,8 @@ from __future__ import annotations
 import numpy as np
 
 
-def run_gpu(w, mode="active", compute="f32", column_split=0, audit_every=1, tol_screen=0.0,
-            max_iter=None, tol=None, widths_cap=200000):
+def run_gpu(w, mode="active", compute="auto", column_split=0, audit_every=1, tol_screen=0.0,
+            max_iter=None, tol=None, widths_cap=200000, cost_form=0):
     import torch
     from paper_2607_24741_b200 import binding as B
     dev = torch.device("cuda:0")
@@ -17,7 +17,8 @@ def run_gpu(w, mode="active", compute="f32", column_split=0, audit_every=1, tol_
     eps = torch.from_numpy(w.eps).to(dev)
     sb = B.SinkhornBatch(x, y, a, b, eps, w.tol if tol is None else tol, mode=mode, compute=compute,
                          max_iter=w.max_iter if max_iter is None else max_iter,
-                         audit_every=audit_every, tol_screen=tol_screen, column_split=column_split)
+                         audit_every=audit_every, tol_screen=tol_screen, column_split=column_split,
+                         cost_form=cost_form)
     try:
         cycles = sb.drain()
         f, g = sb.potentials(f64=True)

@@ -1,9 +1,11 @@
 """GPU parity: the CUDA path, called through the C ABI, against the float64 CPU oracle on the
-same seeded inputs.  Bar: completion depths equal (F64 arithmetic: always; F32 arithmetic: a
-lane may sit one audit away only when the oracle's residual at the disputed audit is within
-the fp32 evaluation noise of tol, and every such lane is reported), potentials within 1e-4
-relative (fp32 pair arithmetic) of the oracle state at the same depth, achieved two-sided
-residual <= tol, slot counts exactly those of Eq. 6-8."""
+same seeded inputs.  Bar: completion depths equal; potentials within 1e-4 relative of the
+oracle state at the same depth; achieved two-sided residual <= tol; slot counts exactly those
+of Eq. 6-8.  Float64 arithmetic must meet it with no exception.  The default arithmetic
+(fp32, or float64 exponents with fp32 exponentials when a lane's cost/eps range is beyond
+fp32) may sit one audit away only when the oracle's own residual at the disputed audit is
+within 1e-5 relative of tol; every such lane is printed.  Pure fp32 arithmetic is held to the
+same bar where its error model says it can meet it, and to its documented limits elsewhere."""
 import ctypes
 
 import numpy as np
@@ -16,7 +18,8 @@ pytestmark = pytest.mark.gpu
 
 POT_TOL_F32 = 1e-4      # acceptance bar for fp32 pair arithmetic
 POT_TOL_F64 = 1e-9      # float64 pair arithmetic: differences are summation order only
-MARGIN_F32 = 2e-2       # a +-1 lane must have |r - tol|/tol below this at the disputed audit
+MARGIN_F32 = 2e-2       # pure fp32: a +-1 lane must have |r - tol|/tol below this at the disputed audit
+MARGIN_AUTO = 1e-5      # default arithmetic: fp32 exponential error (2^-22) over a ~1%/cycle decay
 
 CASES = {
     "tiny": dict(name="tiny"),
@@ -43,22 +46,53 @@ def test_f64_arithmetic_reproduces_oracle_exactly(oracle, case, mode):
 
 
 @pytest.mark.parametrize("case", list(CASES))
-def test_f32_arithmetic_meets_the_bar(oracle, case):
+def test_default_arithmetic_meets_the_bar(oracle, case):
     w = _make(case)
     W = w.shape[0]
-    r = run_gpu(w, mode="active", compute="f32")
+    r = run_gpu(w, mode="active")
     misses = check_against_oracle(oracle, w, r, range(W), pot_tol=POT_TOL_F32, exact_depth=False)
     for t, dg, do, margin in misses:
         print(f"[depth miss] {case} lane {t}: gpu {dg} oracle {do} oracle margin {margin:.2e}")
-        assert margin <= MARGIN_F32
-    assert len(misses) <= max(1, W // 8)
+        assert margin <= MARGIN_AUTO
     check_accounting(oracle, r, W, "active")
     # the float getter is the float64 one rounded
     np.testing.assert_array_equal(r["f32"], r["f"].astype(np.float32))
 
 
+@pytest.mark.parametrize("case", ["tiny", "sensor_ragged", "registration_small"])
+@pytest.mark.parametrize("cost_form", [0, 1, 2])
+def test_pure_fp32_arithmetic_where_it_suffices(oracle, case, cost_form):
+    # scaled squared radius up to a few hundred: fp32 exponents are good to ~1e-5
+    w = _make(case)
+    W = w.shape[0]
+    r = run_gpu(w, mode="active", compute="f32", cost_form=cost_form)
+    misses = check_against_oracle(oracle, w, r, range(W), pot_tol=POT_TOL_F32, exact_depth=False)
+    for t, dg, do, margin in misses:
+        print(f"[depth miss] {case} form {cost_form} lane {t}: gpu {dg} oracle {do} margin {margin:.2e}")
+        assert margin <= MARGIN_F32
+    assert len(misses) <= max(1, W // 8)
+
+
+def test_pure_fp32_limits_on_small_eps_lanes(oracle):
+    # eps down to 0.01 on unit-variance 8-d clouds: cost/eps ~ 10^3 even for the closest pair, so
+    # an fp32 exponent carries ~1e-4 and slow lanes amplify it.  This is why the default
+    # arithmetic leaves fp32 for such batches; the pure fp32 numbers are recorded, not hidden.
+    w = _make("sweep_small")
+    W = w.shape[0]
+    o = oracle.solve_batch(w.x, w.y, w.a, w.b, w.eps, w.tol, max_iter=w.max_iter)
+    r = run_gpu(w, mode="active", compute="f32")
+    dd = r["depth"].astype(np.int64) - o.depth
+    e = pot_err(r["f"], r["g"], o.f, o.g, w.eps.astype(np.float64))
+    print(f"[fp32 limits] lanes off: {np.count_nonzero(dd)}/{W}, max |depth diff| {np.abs(dd).max()}, "
+          f"max potential error on equal-depth lanes {e[dd == 0].max():.2e}")
+    assert np.abs(dd).max() <= 4 and e[dd == 0].max() <= 1e-3
+    np.testing.assert_array_equal(r["status"], o.status)
+    ra = run_gpu(w, mode="active")
+    assert np.array_equal(ra["depth"], o.depth)
+
+
 @pytest.mark.parametrize("case", ["tiny", "sweep_small"])
-@pytest.mark.parametrize("compute", ["f32", "f64"])
+@pytest.mark.parametrize("compute", ["f32", "auto", "f64"])
 def test_masked_equals_active_bitwise_and_static_matches_fixed_depth(oracle, case, compute):
     w = _make(case)
     W = w.shape[0]
@@ -76,7 +110,7 @@ def test_masked_equals_active_bitwise_and_static_matches_fixed_depth(oracle, cas
     ref = oracle.solve_batch(w.x, w.y, w.a, w.b, w.eps, w.tol, max_iter=w.max_iter, fixed_cycles=lmax)
     done = ra["status"] == 1
     e = pot_err(rs["f"], rs["g"], ref.f, ref.g, w.eps.astype(np.float64))
-    assert e[done].max() <= (POT_TOL_F32 if compute == "f32" else POT_TOL_F64)
+    assert e[done].max() <= {"f32": 1e-3, "auto": POT_TOL_F32, "f64": POT_TOL_F64}[compute]
     assert np.all(rs["r_row"][done] <= w.tol)
     # removable slots R = W*l_max - sum l_t (Eq. 8)
     assert rs["stats"]["slots"] - ra["stats"]["slots"] == W * lmax - int(ra["depth"].sum())
@@ -84,16 +118,18 @@ def test_masked_equals_active_bitwise_and_static_matches_fixed_depth(oracle, cas
 
 def test_packing_commutes_with_the_per_lane_map(oracle):
     # Eq. 2: a W-lane batch gives each lane what a one-lane batch gives it, bit for bit
+    # (the arithmetic is fixed here: the automatic choice looks at the whole batch)
     w = wl.make("sweep", W=6, n=96, m=80, max_iter=2000)
-    r = run_gpu(w, mode="active", column_split=8)
-    for t in (0, 3, 5):
-        one = wl.Workload(w.name, w.x[t:t + 1], w.y[t:t + 1], w.a[t:t + 1], w.b[t:t + 1],
-                          w.eps[t:t + 1], w.tol, w.max_iter)
-        r1 = run_gpu(one, mode="active", column_split=8)
-        assert r1["depth"][0] == r["depth"][t]
-        np.testing.assert_array_equal(r1["f"][0], r["f"][t]); np.testing.assert_array_equal(r1["g"][0], r["g"][t])
-    r2 = run_gpu(w, mode="active", column_split=8)              # run-to-run determinism
-    np.testing.assert_array_equal(r2["f"], r["f"]); np.testing.assert_array_equal(r2["depth"], r["depth"])
+    for compute in ("mixed", "f32"):
+        r = run_gpu(w, mode="active", column_split=8, compute=compute)
+        for t in (0, 3, 5):
+            one = wl.Workload(w.name, w.x[t:t + 1], w.y[t:t + 1], w.a[t:t + 1], w.b[t:t + 1],
+                              w.eps[t:t + 1], w.tol, w.max_iter)
+            r1 = run_gpu(one, mode="active", column_split=8, compute=compute)
+            assert r1["depth"][0] == r["depth"][t]
+            np.testing.assert_array_equal(r1["f"][0], r["f"][t]); np.testing.assert_array_equal(r1["g"][0], r["g"][t])
+        r2 = run_gpu(w, mode="active", column_split=8, compute=compute)      # run-to-run determinism
+        np.testing.assert_array_equal(r2["f"], r["f"]); np.testing.assert_array_equal(r2["depth"], r["depth"])
 
 
 @pytest.mark.parametrize("cs", [1, 8, 32])
@@ -102,7 +138,7 @@ def test_every_column_split_agrees_with_the_oracle(oracle, cs):
     r = run_gpu(w, mode="active", compute="f64", column_split=cs)
     assert check_against_oracle(oracle, w, r, range(5), pot_tol=POT_TOL_F64, exact_depth=True) == []
     w3 = wl.make("registration", W=3, n=700)
-    r3 = run_gpu(w3, mode="active", compute="f32", column_split=cs)
+    r3 = run_gpu(w3, mode="active", column_split=cs)
     check_against_oracle(oracle, w3, r3, range(3), pot_tol=POT_TOL_F32, exact_depth=False)
 
 
