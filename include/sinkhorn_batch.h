@@ -76,7 +76,7 @@ typedef struct {
     int max_iter;          /* cycle cap per lane, >= 1                                     */
     int audit_every;       /* audit after every k-th cycle, >= 1                           */
     float tol_screen;      /* row-screen threshold; <= 0 means "same as tol"               */
-    int column_split;      /* 0 = automatic; 1, 8 or 32 forces how many lanes of a warp     */
+    int column_split;      /* 0 = automatic; 1, 4 or 32 forces how many lanes of a warp     */
                            /* share one row's columns in the update kernel (tuning knob)  */
     int cost_form;         /* 0 = chosen per lane from its scaled radius; 1 = expanded     */
                            /* |x|^2+|y|^2-2x.y everywhere; 2 = difference |x-y|^2 everywhere */
@@ -146,6 +146,22 @@ skb_status sinkhorn_batch_residuals(skb_batch *h, float *r_row, float *r_col);
  */
 skb_status sinkhorn_batch_stats(skb_batch *h, long long *slots, int *cycles, int *widths,
                                 int widths_cap, long long *pair_terms);
+
+/* The arithmetic the batch actually runs (skb_compute, never AUTO): what an automatic
+ * batch resolved to from its data.  Host out. */
+skb_status sinkhorn_batch_arithmetic(skb_batch *h, int *compute);
+
+/* Number of kernels this handle has launched so far (host out). */
+skb_status sinkhorn_batch_launch_count(skb_batch *h, long long *launches);
+
+/*
+ * Measurement aid: launches the update kernel for one leg (0 = f-leg, 1 = g-leg) `reps`
+ * times at the batch's current width, bracketed by CUDA events on the batch's stream, and
+ * returns the mean duration per launch in milliseconds (host out).  The f-leg only reads
+ * the current state and rewrites the look-ahead buffers, so the solve is not disturbed;
+ * the g-leg recomputes g from the current f.  Synchronises.
+ */
+skb_status sinkhorn_batch_profile_update(skb_batch *h, int leg, int reps, float *ms_per_launch);
 
 /*
  * Whole solve from HOST buffers in one call: copies x, y, a, b, eps to the device,

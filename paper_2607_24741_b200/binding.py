@@ -27,6 +27,7 @@ EXPORTS = (
     "sinkhorn_batch_potentials_f64", "sinkhorn_batch_depths", "sinkhorn_batch_residuals",
     "sinkhorn_batch_stats", "sinkhorn_batch_destroy", "sinkhorn_batch_last_error",
     "sinkhorn_batch_host_workspace_bytes", "sinkhorn_batch_solve_host",
+    "sinkhorn_batch_launch_count", "sinkhorn_batch_profile_update", "sinkhorn_batch_arithmetic",
 )
 
 
@@ -66,6 +67,9 @@ def _load():
     lib.sinkhorn_batch_residuals.argtypes = [vp, vp, vp]
     lib.sinkhorn_batch_stats.argtypes = [vp, ctypes.POINTER(ctypes.c_longlong), ctypes.POINTER(ctypes.c_int),
                                          vp, ctypes.c_int, ctypes.POINTER(ctypes.c_longlong)]
+    lib.sinkhorn_batch_arithmetic.argtypes = [vp, ctypes.POINTER(ctypes.c_int)]
+    lib.sinkhorn_batch_launch_count.argtypes = [vp, ctypes.POINTER(ctypes.c_longlong)]
+    lib.sinkhorn_batch_profile_update.argtypes = [vp, ctypes.c_int, ctypes.c_int, ctypes.POINTER(ctypes.c_float)]
     lib.sinkhorn_batch_destroy.argtypes = [vp]
     lib.sinkhorn_batch_destroy.restype = None
     lib.sinkhorn_batch_last_error.argtypes = [vp]
@@ -207,6 +211,21 @@ class SinkhornBatch:
         k = min(cycles.value, widths_cap)
         return {"slots": slots.value, "cycles": cycles.value, "pair_terms": terms.value,
                 "widths": list(buf[:k])}
+
+    def arithmetic(self) -> str:
+        c = ctypes.c_int(0)
+        _check(lib.sinkhorn_batch_arithmetic(self.h, ctypes.byref(c)), self.h)
+        return {v: k for k, v in COMPUTE.items()}[c.value]
+
+    def launch_count(self) -> int:
+        c = ctypes.c_longlong(0)
+        _check(lib.sinkhorn_batch_launch_count(self.h, ctypes.byref(c)), self.h)
+        return c.value
+
+    def profile_update(self, leg=0, reps=10) -> float:
+        ms = ctypes.c_float(0)
+        _check(lib.sinkhorn_batch_profile_update(self.h, leg, reps, ctypes.byref(ms)), self.h)
+        return ms.value
 
     def close(self):
         if self.h is not None:

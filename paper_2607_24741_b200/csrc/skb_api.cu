@@ -22,6 +22,7 @@ struct skb_batch {
     int known_width;       // last physical width the host has seen
     bool finished;
     long long enqueued;    // cycles enqueued so far
+    long long launches;    // kernels launched so far
     std::string err;
 };
 
@@ -45,8 +46,8 @@ static bool config_ok(const skb_config *c, std::string &why)
     if (c->compute < SKB_COMPUTE_AUTO || c->compute > SKB_COMPUTE_F64) { why = "bad compute type"; return false; }
     if (c->max_iter < 1 || c->audit_every < 1) { why = "max_iter and audit_every must be >= 1"; return false; }
     if (c->cost_form < 0 || c->cost_form > 2) { why = "cost_form must be 0 (automatic), 1 (expanded) or 2 (difference)"; return false; }
-    if (c->column_split != 0 && c->column_split != 1 && c->column_split != 8 && c->column_split != 32) {
-        why = "column_split must be 0, 1, 8 or 32"; return false;
+    if (c->column_split != 0 && c->column_split != 1 && c->column_split != 4 && c->column_split != 32) {
+        why = "column_split must be 0, 1, 4 or 32"; return false;
     }
     return true;
 }
@@ -92,6 +93,7 @@ static size_t carve(const skb_config *c, const Variant *var, char *base, Dev *D,
     d.fl[0] = take(W * np * ts); d.fl[1] = take(W * np * ts); d.gl = take(W * mp * ts);
     d.sqx = (double *)take(W * np * 8); d.sqy = (double *)take(W * mp * 8);
     d.la2 = (double *)take(W * np * 8); d.lb2 = (double *)take(W * mp * 8);
+    d.wa = (double *)take(W * np * 8); d.wb = (double *)take(W * mp * 8);
     d.phi[0] = (double *)take(W * np * 8); d.phi[1] = (double *)take(W * np * 8);
     d.gam = (double *)take(W * mp * 8);
     d.f_out = (double *)take(W * n * 8); d.g_out = (double *)take(W * m * 8);
@@ -160,7 +162,7 @@ extern "C" skb_status sinkhorn_batch_create(const void *x, const void *y, const 
     skb_batch *h = new (std::nothrow) skb_batch();
     if (!h) return fail(nullptr, SKB_ERR_CUDA, "host allocation failed");
     h->cfg = *cfg; h->var = var; h->stream = (cudaStream_t)cfg->stream;
-    h->known_width = cfg->W; h->finished = false; h->enqueued = 0; h->h_ctl = nullptr;
+    h->known_width = cfg->W; h->finished = false; h->enqueued = 0; h->launches = 0; h->h_ctl = nullptr;
     h->ev[0] = h->ev[1] = nullptr;
     carve(cfg, var, (char *)cfg->workspace, &h->dev);
     h->dev.tol_stop = (double)tol;
@@ -185,6 +187,7 @@ extern "C" skb_status sinkhorn_batch_create(const void *x, const void *y, const 
         return st;
     }
     launch_lane_stats(h->dev, x, y, eps, nullptr, h->stream);
+    h->launches += 2;   // lane statistics + layout kernel
     if (automatic) {
         // read the largest scaled radius back and pick the arithmetic for the whole batch
         if ((e = cudaMemcpyAsync(&h->h_ctl[1], h->dev.ctl, sizeof(Ctl), cudaMemcpyDeviceToHost, h->stream)) != cudaSuccess ||
@@ -225,6 +228,7 @@ static void enqueue_cycle(skb_batch *h)
     launch_emit_move(h->dev, w, h->stream);
     h->var->launch(h->dev, LEG_G, w, h->stream);
     h->enqueued++;
+    h->launches += 5;
 }
 
 static skb_status absorb(skb_batch *h, const Ctl &c)
@@ -347,6 +351,42 @@ extern "C" skb_status sinkhorn_batch_stats(skb_batch *h, long long *slots, int *
         cudaError_t e = cudaMemcpy(widths, h->dev.widths, (size_t)k * sizeof(int), cudaMemcpyDeviceToHost);
         if (e != cudaSuccess) return cuda_fail(h, e, "stats");
     }
+    return SKB_OK;
+}
+
+extern "C" skb_status sinkhorn_batch_arithmetic(skb_batch *h, int *compute)
+{
+    if (!h || !compute) return SKB_ERR_NULL;
+    *compute = !h->var->f64 ? SKB_COMPUTE_F32 : (h->var->xf ? SKB_COMPUTE_MIXED : SKB_COMPUTE_F64);
+    return SKB_OK;
+}
+
+extern "C" skb_status sinkhorn_batch_launch_count(skb_batch *h, long long *launches)
+{
+    if (!h || !launches) return SKB_ERR_NULL;
+    *launches = h->launches;
+    return SKB_OK;
+}
+
+extern "C" skb_status sinkhorn_batch_profile_update(skb_batch *h, int leg, int reps, float *ms_per_launch)
+{
+    if (!h || !ms_per_launch) return SKB_ERR_NULL;
+    if ((leg != LEG_F && leg != LEG_G) || reps < 1) return fail(h, SKB_ERR_VALUE, "leg must be 0 or 1 and reps >= 1");
+    cudaEvent_t a, b;
+    cudaError_t e;
+    if ((e = cudaEventCreate(&a)) != cudaSuccess) return cuda_fail(h, e, "profile");
+    if ((e = cudaEventCreate(&b)) != cudaSuccess) { cudaEventDestroy(a); return cuda_fail(h, e, "profile"); }
+    h->var->launch(h->dev, leg, h->known_width, h->stream);          // warm-up
+    cudaEventRecord(a, h->stream);
+    for (int i = 0; i < reps; ++i) h->var->launch(h->dev, leg, h->known_width, h->stream);
+    cudaEventRecord(b, h->stream);
+    e = cudaEventSynchronize(b);
+    float ms = 0.f;
+    if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, a, b);
+    cudaEventDestroy(a); cudaEventDestroy(b);
+    h->launches += reps + 1;
+    if (e != cudaSuccess) return cuda_fail(h, e, "profile");
+    *ms_per_launch = ms / (float)reps;
     return SKB_OK;
 }
 

@@ -84,12 +84,12 @@ __global__ void prep_kernel(const Dev P, const void *xin, const void *yin, const
     const size_t o = (size_t)slot * pp + i;
     T *hi0 = side ? reinterpret_cast<T *>(P.gt) : reinterpret_cast<T *>(P.ft[0]);
     T *lo0 = side ? reinterpret_cast<T *>(P.gl) : reinterpret_cast<T *>(P.fl[0]);
-    double *sq = side ? P.sqy : P.sqx, *lw = side ? P.lb2 : P.la2;
+    double *sq = side ? P.sqy : P.sqx, *lw = side ? P.lb2 : P.la2, *wt = side ? P.wb : P.wa;
     T hi, lo = T(0);
     if (i >= npts) {                                  // padding points
         for (int k = 0; k < P.DP; ++k) crd[(size_t)k * pp + i] = T(0);
         hi = T(NEG_BIG);
-        sq[o] = 0.0; lw[o] = 0.0;
+        sq[o] = 0.0; lw[o] = 0.0; wt[o] = 0.0;
     } else {
         const double sc = sqrt(form == FORM_DOT ? 2.0 * s : s);
         const size_t ibase = ((size_t)slot * npts + i) * P.d;
@@ -112,6 +112,7 @@ __global__ void prep_kernel(const Dev P, const void *xin, const void *yin, const
         if (!ok) atomicOr(&P.ctl->error, ERR_VALUE);
         sq[o] = nrm;
         lw[o] = ok ? log2((double)w) : 0.0;
+        wt[o] = ok ? (double)w : 0.0;
         hi = (T)(-nrm);                                // cold start: phi = gam = 0
     }
     hi0[o] = hi; lo0[o] = lo;
@@ -302,6 +303,7 @@ __global__ void __launch_bounds__(256) emit_move_kernel(const Dev P)
     copy(P.ys, (size_t)P.DP * P.mp * sizeof(T));
     copy(P.sqx, (size_t)P.np * 8); copy(P.sqy, (size_t)P.mp * 8);
     copy(P.la2, (size_t)P.np * 8); copy(P.lb2, (size_t)P.mp * 8);
+    copy(P.wa, (size_t)P.np * 8); copy(P.wb, (size_t)P.mp * 8);
     copy(P.phi[np_], (size_t)P.np * 8);
     copy(P.ft[np_], (size_t)P.np * sizeof(T));
     copy(P.fl[np_], (size_t)P.np * sizeof(T));

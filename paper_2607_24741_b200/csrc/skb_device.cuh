@@ -59,6 +59,7 @@ struct Dev {
     double *center;           // [W][DP] joint centroid of the lane's two clouds
     double *sqx, *sqy;        // [W][np], [W][mp]
     double *la2, *lb2;        // log2 a, log2 b
+    double *wa, *wb;          // a, b
     double *phi[2];           // [W][np]
     double *gam;              // [W][mp]
     // per-slot scalars

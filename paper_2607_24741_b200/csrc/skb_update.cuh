@@ -7,18 +7,22 @@
 //     L_i = log2 sum_j 2^(arg_ij)
 // as an online max / sum-of-exp2 reduction: the n x m matrix is never stored.  Column
 // tiles are staged in shared memory by 16-byte cp.async copies from a dimension-major
-// layout; a thread keeps R rows in registers and walks 4 adjacent columns per step; with
-// CS > 1 the columns of a tile are split over CS neighbouring lanes of the warp and the
-// (max, sum) pairs are merged by xor-shuffles at the end.
+// layout; a thread keeps R rows in registers and walks a group of adjacent columns per
+// step; with CS > 1 the column groups of a tile are dealt round-robin to CS neighbouring
+// lanes of the warp and the (max, sum) pairs are merged by xor-shuffles at the end.
+// The running maximum is kept integer-valued, so every rescale is an exact power of two.
 //
-// Two forms of arg_ij, chosen per lane when the batch is created:
-//   dot   arg_ij = ct_j + r_i . c_j            (d FMA per pair; ct = potential - |c_j|^2/2)
-//   diff  arg_ij = (ph_i + ch_j) + cl_j - |r_i - c_j|^2   (2d + 2 per pair; ph, ch are the
-//         fp32 high parts of the row and column potentials, cl the column's low part, and
-//         the row's own rounding error is removed in float64 afterwards).  It is used when
-//         the expanded form would cancel catastrophically in fp32.
+// Arithmetic of arg_ij:
+//   fp32, dot form   arg = ct_j + r_i . c_j, packed two columns at a time (fma.rn.f32x2);
+//   fp32, diff form  arg = (ph_i + ch_j) + (cl_j - |r_i - c_j|^2), for lanes whose scaled
+//                    radius makes the expanded form cancel catastrophically in fp32
+//                    (ph, ch: fp32 high parts of the potentials, cl: the column's low part;
+//                    the row's own rounding error is removed in float64 afterwards);
+//   float64          arg = ct_j + r_i . c_j on the FP64 pipe, with the exponentials either
+//                    on the fp32 special-function unit ("mixed") or in software (validation).
 //
-// Leg-specific epilogues (float64, one per row):
+// Leg-specific epilogues (float64, one thread per row, rows handed over through shared
+// memory so that no lane repeats another's work):
 //   LEG_F  phi_new from L;  also the row marginal of the state BEFORE this leg,
 //          sum_j pi_ij = a_i 2^(phi_old - phi_new), which is the one-sided row screen of
 //          Section "Screen, verify, and compact" obtained for free.
@@ -32,153 +36,290 @@
 
 namespace skb {
 
-template <typename T, int XF> struct SumType { using type = T; };
-template <> struct SumType<double, 1> { using type = float; };
+typedef unsigned long long u64;
 
-template <int CS> struct TileCols { static constexpr int value = (CS <= 4) ? 128 : (CS == 8 ? 256 : 512); };
+template <typename T> struct Tune;
+template <> struct Tune<float> { static constexpr int R = 2, CW = 8; };    // rows per thread, columns per step
+template <> struct Tune<double> { static constexpr int R = 2, CW = 4; };
 
-__device__ __forceinline__ void lds4(const float *p, float (&v)[4])
+template <typename T, int CS> struct TileCols {
+    static constexpr int value = (Tune<T>::CW * CS * 2 > 128) ? Tune<T>::CW * CS * 2 : 128;   // >= 2 steps per tile
+};
+
+__device__ __forceinline__ u64 pack2(float lo, float hi)
 {
-    float4 t = *reinterpret_cast<const float4 *>(p);
-    v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+    u64 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
 }
-__device__ __forceinline__ void lds4(const double *p, double (&v)[4])
+__device__ __forceinline__ void unpack2(u64 v, float &lo, float &hi)
 {
-    double2 t0 = *reinterpret_cast<const double2 *>(p);
-    double2 t1 = *reinterpret_cast<const double2 *>(p + 2);
-    v[0] = t0.x; v[1] = t0.y; v[2] = t1.x; v[3] = t1.y;
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ u64 fma2(u64 a, u64 b, u64 c)
+{
+    u64 d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ u64 add2(u64 a, u64 b)
+{
+    u64 d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ u64 sub2(u64 a, u64 b)
+{
+    u64 d;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+// 2^k for an integer-valued k <= 0 (exact; flushes to 0 below the normal range)
+__device__ __forceinline__ float pow2i(float k)
+{
+    const int e = (int)fmaxf(k, -127.0f) + 127;
+    return __int_as_float(e << 23);
 }
 
-// Streams every column tile of one lane past the CTA's rows and leaves, per row of this
-// thread, the running maximum md[r] and the sum sd[r] of 2^(arg - md[r]) over the columns
-// this thread visited.
-template <typename T, int DP, int R, int CS, int FORM, int XF>
-__device__ __forceinline__ void stream_columns(T *sm, const T *colc, const T *colt, const T *coll,
-                                               const int cp, const int ncols, const T (&xr)[R][DP],
-                                               const T (&ph)[R], const int tid, const int cs,
-                                               double (&md)[R], double (&sd)[R])
+// Column-tile loader shared by all arithmetic flavours: NR rows of TJ elements per stage.
+template <typename T, int DP, int TJ, int NR>
+__device__ __forceinline__ void load_tile(T *dst, const T *colc, const T *colt, const T *coll,
+                                          const int cp, const int j0, const int tid)
 {
-    constexpr int TJ = TileCols<CS>::value;
-    constexpr int STEPS = TJ / (4 * CS);
     constexpr int EPC = 16 / (int)sizeof(T);
-    constexpr int NR = DP + 1 + (FORM == FORM_DIFF ? 1 : 0);   // rows of a stage
-    constexpr int STAGE = (DP + 2) * TJ;
     constexpr int CPR = TJ / EPC;
-
-    // XF = 1: the exponentials run on the fp32 special-function unit even when the
-    // arguments are float64 ("mixed" arithmetic); the tile sum is then fp32 as well
-    using TS = typename SumType<T, XF>::type;
-    T mx[R];
-    TS ts[R];
+    for (int ch = tid; ch < NR * CPR; ch += UPD_THREADS) {
+        const int k = ch / CPR, j = j0 + (ch % CPR) * EPC;
+        T *d = dst + k * TJ + (ch % CPR) * EPC;
+        if (j < cp) {
+            const T *src = (k < DP) ? colc + (size_t)k * cp + j : (k == DP ? colt + j : coll + j);
+            cp_async16(d, src);
+        } else {
+            // columns past the padded end: zero coordinates, "minus infinity" term
+            const T fill = (k == DP) ? T(NEG_BIG) : T(0);
 #pragma unroll
-    for (int r = 0; r < R; ++r) { mx[r] = T(NEG_BIG); ts[r] = TS(0); sd[r] = 0.0; }
+            for (int e = 0; e < EPC; ++e) d[e] = fill;
+        }
+    }
+}
+
+// ------------------------------------------------------------------ fp32, packed pairs
+// Leaves per row the integer-valued maximum mx[r] and sd[r] = sum 2^(arg - mx[r]) over the
+// columns this thread visited.
+template <int DP, int CS, int FORM>
+__device__ __forceinline__ void stream_f32(float *sm, const float *colc, const float *colt, const float *coll,
+                                           const int cp, const int ncols, const float (&xrow)[2][DP],
+                                           const float (&ph)[2], const int tid, const int cs,
+                                           float (&mx)[2], double (&sd)[2])
+{
+    constexpr int R = 2, CW = 8;
+    constexpr int TJ = TileCols<float, CS>::value;
+    constexpr int STEPS = TJ / (CW * CS);
+    constexpr int NR = DP + 1 + (FORM == FORM_DIFF ? 1 : 0);
+    constexpr int STAGE = (DP + 2) * TJ;
+
+    u64 xd[R][DP];                       // each row coordinate duplicated into both halves
+    u64 phd[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+#pragma unroll
+        for (int k = 0; k < DP; ++k) xd[r][k] = pack2(xrow[r][k], xrow[r][k]);
+        phd[r] = pack2(ph[r], ph[r]);
+    }
+    u64 ts[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) { mx[r] = NEG_BIG; ts[r] = 0ull; sd[r] = 0.0; }
 
     const int ntiles = (ncols + TJ - 1) / TJ;
-    auto load_tile = [&](int t, int stage) {
-        T *dst = sm + stage * STAGE;
-        const int j0 = t * TJ;
-        for (int ch = tid; ch < NR * CPR; ch += UPD_THREADS) {
-            const int k = ch / CPR, j = j0 + (ch % CPR) * EPC;
-            T *d = dst + k * TJ + (ch % CPR) * EPC;
-            if (j < cp) {
-                const T *src = (k < DP) ? colc + (size_t)k * cp + j : (k == DP ? colt + j : coll + j);
-                cp_async16(d, src);
-            } else {
-                // columns past the padded end: zero coordinates, "minus infinity" term
-                const T fill = (k == DP) ? T(NEG_BIG) : T(0);
-#pragma unroll
-                for (int e = 0; e < EPC; ++e) d[e] = fill;
-            }
-        }
-    };
-
-    load_tile(0, 0);
+    load_tile<float, DP, TJ, NR>(sm, colc, colt, coll, cp, 0, tid);
     cp_async_commit();
     for (int t = 0; t < ntiles; ++t) {
         if (t + 1 < ntiles) {
-            load_tile(t + 1, (t + 1) & 1);
+            load_tile<float, DP, TJ, NR>(sm + ((t + 1) & 1) * STAGE, colc, colt, coll, cp, (t + 1) * TJ, tid);
             cp_async_commit();
             cp_async_wait<1>();
         } else {
             cp_async_wait<0>();
         }
         __syncthreads();
-        const T *st = sm + (t & 1) * STAGE;
-#pragma unroll 2
+        const float *st = sm + (t & 1) * STAGE;
+#pragma unroll 1
         for (int q = 0; q < STEPS; ++q) {
-            const int jj = (q * CS + cs) * 4;
-            T acc[R][4];
-            T ct[4];
-            lds4(st + DP * TJ + jj, ct);
+            const int jj = (q * CS + cs) * CW;
+            u64 acc[R][4];
+            const ulonglong2 c0 = *reinterpret_cast<const ulonglong2 *>(st + DP * TJ + jj);
+            const ulonglong2 c1 = *reinterpret_cast<const ulonglong2 *>(st + DP * TJ + jj + 4);
             if (FORM == FORM_DOT) {
 #pragma unroll
-                for (int r = 0; r < R; ++r)
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) acc[r][e] = ct[e];
+                for (int r = 0; r < R; ++r) { acc[r][0] = c0.x; acc[r][1] = c0.y; acc[r][2] = c1.x; acc[r][3] = c1.y; }
 #pragma unroll
                 for (int k = 0; k < DP; ++k) {
-                    T yv[4];
-                    lds4(st + k * TJ + jj, yv);
+                    const ulonglong2 y0 = *reinterpret_cast<const ulonglong2 *>(st + k * TJ + jj);
+                    const ulonglong2 y1 = *reinterpret_cast<const ulonglong2 *>(st + k * TJ + jj + 4);
 #pragma unroll
-                    for (int r = 0; r < R; ++r)
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) acc[r][e] = fma(xr[r][k], yv[e], acc[r][e]);
+                    for (int r = 0; r < R; ++r) {
+                        acc[r][0] = fma2(xd[r][k], y0.x, acc[r][0]);
+                        acc[r][1] = fma2(xd[r][k], y0.y, acc[r][1]);
+                        acc[r][2] = fma2(xd[r][k], y1.x, acc[r][2]);
+                        acc[r][3] = fma2(xd[r][k], y1.y, acc[r][3]);
+                    }
                 }
             } else {
-                T cl[4];
-                lds4(st + (DP + 1) * TJ + jj, cl);
+                u64 sq[R][4];
 #pragma unroll
-                for (int r = 0; r < R; ++r)
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) acc[r][e] = cl[e];
+                for (int r = 0; r < R; ++r) { sq[r][0] = 0ull; sq[r][1] = 0ull; sq[r][2] = 0ull; sq[r][3] = 0ull; }
 #pragma unroll
                 for (int k = 0; k < DP; ++k) {
-                    T yv[4];
-                    lds4(st + k * TJ + jj, yv);
+                    const ulonglong2 y0 = *reinterpret_cast<const ulonglong2 *>(st + k * TJ + jj);
+                    const ulonglong2 y1 = *reinterpret_cast<const ulonglong2 *>(st + k * TJ + jj + 4);
 #pragma unroll
-                    for (int r = 0; r < R; ++r)
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const T dk = xr[r][k] - yv[e];
-                            acc[r][e] = fma(-dk, dk, acc[r][e]);
-                        }
+                    for (int r = 0; r < R; ++r) {
+                        u64 dk;
+                        dk = sub2(xd[r][k], y0.x); sq[r][0] = fma2(dk, dk, sq[r][0]);
+                        dk = sub2(xd[r][k], y0.y); sq[r][1] = fma2(dk, dk, sq[r][1]);
+                        dk = sub2(xd[r][k], y1.x); sq[r][2] = fma2(dk, dk, sq[r][2]);
+                        dk = sub2(xd[r][k], y1.y); sq[r][3] = fma2(dk, dk, sq[r][3]);
+                    }
                 }
+                const ulonglong2 l0 = *reinterpret_cast<const ulonglong2 *>(st + (DP + 1) * TJ + jj);
+                const ulonglong2 l1 = *reinterpret_cast<const ulonglong2 *>(st + (DP + 1) * TJ + jj + 4);
 #pragma unroll
-                for (int r = 0; r < R; ++r)
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) acc[r][e] += (ph[r] + ct[e]);
+                for (int r = 0; r < R; ++r) {
+                    acc[r][0] = add2(add2(phd[r], c0.x), sub2(l0.x, sq[r][0]));
+                    acc[r][1] = add2(add2(phd[r], c0.y), sub2(l0.y, sq[r][1]));
+                    acc[r][2] = add2(add2(phd[r], c1.x), sub2(l1.x, sq[r][2]));
+                    acc[r][3] = add2(add2(phd[r], c1.y), sub2(l1.y, sq[r][3]));
+                }
             }
 #pragma unroll
             for (int r = 0; r < R; ++r) {
-                const T mt = fmax(fmax(acc[r][0], acc[r][1]), fmax(acc[r][2], acc[r][3]));
-                if (mt > mx[r] + T(8)) {           // lazy rescale: terms stay below 2^8
-                    const TS fac = ex2_t((TS)(mx[r] - mt));
-                    ts[r] *= fac;
+                float a0, a1, a2, a3, a4, a5, a6, a7;
+                unpack2(acc[r][0], a0, a1); unpack2(acc[r][1], a2, a3);
+                unpack2(acc[r][2], a4, a5); unpack2(acc[r][3], a6, a7);
+                const float mt = fmaxf(fmaxf(fmaxf(a0, a1), fmaxf(a2, a3)), fmaxf(fmaxf(a4, a5), fmaxf(a6, a7)));
+                if (mt > mx[r] + 8.0f) {                       // lazy rescale: terms stay below 2^9
+                    const float mn = ceilf(mt);
+                    const float fac = pow2i(mx[r] - mn);
+                    float t0, t1;
+                    unpack2(ts[r], t0, t1);
+                    ts[r] = pack2(t0 * fac, t1 * fac);
                     sd[r] *= (double)fac;
-                    mx[r] = mt;
+                    mx[r] = mn;
                 }
-                ts[r] += (ex2_t((TS)(acc[r][0] - mx[r])) + ex2_t((TS)(acc[r][1] - mx[r]))) +
-                         (ex2_t((TS)(acc[r][2] - mx[r])) + ex2_t((TS)(acc[r][3] - mx[r])));
+                const u64 mm = pack2(mx[r], mx[r]);
+                unpack2(sub2(acc[r][0], mm), a0, a1); unpack2(sub2(acc[r][1], mm), a2, a3);
+                unpack2(sub2(acc[r][2], mm), a4, a5); unpack2(sub2(acc[r][3], mm), a6, a7);
+                const u64 e0 = pack2(ex2_fast(a0), ex2_fast(a1)), e1 = pack2(ex2_fast(a2), ex2_fast(a3));
+                const u64 e2 = pack2(ex2_fast(a4), ex2_fast(a5)), e3 = pack2(ex2_fast(a6), ex2_fast(a7));
+                ts[r] = add2(ts[r], add2(add2(e0, e1), add2(e2, e3)));
             }
         }
 #pragma unroll
-        for (int r = 0; r < R; ++r) { sd[r] += (double)ts[r]; ts[r] = TS(0); }
+        for (int r = 0; r < R; ++r) {
+            float t0, t1;
+            unpack2(ts[r], t0, t1);
+            sd[r] += (double)(t0 + t1);
+            ts[r] = 0ull;
+        }
         __syncthreads();
     }
-#pragma unroll
-    for (int r = 0; r < R; ++r) md[r] = (double)mx[r];
 }
 
-template <typename T, int DP, int R, int CS, int XF>
+// ------------------------------------------------------------------ float64 arguments
+// XF = 1: exponentials on the fp32 special-function unit; XF = 0: software exp2 in float64.
+template <int DP, int CS, int XF>
+__device__ __forceinline__ void stream_f64(double *sm, const double *colc, const double *colt,
+                                           const int cp, const int ncols, const double (&xr)[2][DP],
+                                           const int tid, const int cs, float (&mx)[2], double (&sd)[2])
+{
+    constexpr int R = 2, CW = 4;
+    constexpr int TJ = TileCols<double, CS>::value;
+    constexpr int STEPS = TJ / (CW * CS);
+    constexpr int NR = DP + 1;
+    constexpr int STAGE = (DP + 2) * TJ;
+
+    float ts[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) { mx[r] = NEG_BIG; ts[r] = 0.f; sd[r] = 0.0; }
+
+    const int ntiles = (ncols + TJ - 1) / TJ;
+    load_tile<double, DP, TJ, NR>(sm, colc, colt, colt, cp, 0, tid);
+    cp_async_commit();
+    for (int t = 0; t < ntiles; ++t) {
+        if (t + 1 < ntiles) {
+            load_tile<double, DP, TJ, NR>(sm + ((t + 1) & 1) * STAGE, colc, colt, colt, cp, (t + 1) * TJ, tid);
+            cp_async_commit();
+            cp_async_wait<1>();
+        } else {
+            cp_async_wait<0>();
+        }
+        __syncthreads();
+        const double *st = sm + (t & 1) * STAGE;
+#pragma unroll 1
+        for (int q = 0; q < STEPS; ++q) {
+            const int jj = (q * CS + cs) * CW;
+            double acc[R][4];
+            {
+                const double2 c0 = *reinterpret_cast<const double2 *>(st + DP * TJ + jj);
+                const double2 c1 = *reinterpret_cast<const double2 *>(st + DP * TJ + jj + 2);
+#pragma unroll
+                for (int r = 0; r < R; ++r) { acc[r][0] = c0.x; acc[r][1] = c0.y; acc[r][2] = c1.x; acc[r][3] = c1.y; }
+            }
+#pragma unroll
+            for (int k = 0; k < DP; ++k) {
+                const double2 y0 = *reinterpret_cast<const double2 *>(st + k * TJ + jj);
+                const double2 y1 = *reinterpret_cast<const double2 *>(st + k * TJ + jj + 2);
+#pragma unroll
+                for (int r = 0; r < R; ++r) {
+                    acc[r][0] = fma(xr[r][k], y0.x, acc[r][0]);
+                    acc[r][1] = fma(xr[r][k], y0.y, acc[r][1]);
+                    acc[r][2] = fma(xr[r][k], y1.x, acc[r][2]);
+                    acc[r][3] = fma(xr[r][k], y1.y, acc[r][3]);
+                }
+            }
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                // the maximum only has to be near the true one: track it on fp32 copies
+                const float mt = fmaxf(fmaxf((float)acc[r][0], (float)acc[r][1]), fmaxf((float)acc[r][2], (float)acc[r][3]));
+                if (mt > mx[r] + 8.0f) {
+                    const float mn = ceilf(mt);
+                    const float fac = pow2i(mx[r] - mn);
+                    ts[r] *= fac;
+                    sd[r] *= (double)fac;
+                    mx[r] = mn;
+                }
+                const double md = (double)mx[r];
+                if (XF) {
+                    ts[r] += (ex2_fast((float)(acc[r][0] - md)) + ex2_fast((float)(acc[r][1] - md))) +
+                             (ex2_fast((float)(acc[r][2] - md)) + ex2_fast((float)(acc[r][3] - md)));
+                } else {
+                    sd[r] += (exp2(acc[r][0] - md) + exp2(acc[r][1] - md)) + (exp2(acc[r][2] - md) + exp2(acc[r][3] - md));
+                }
+            }
+        }
+        if (XF) {
+#pragma unroll
+            for (int r = 0; r < R; ++r) { sd[r] += (double)ts[r]; ts[r] = 0.f; }
+        }
+        __syncthreads();
+    }
+}
+
+template <typename T, int DP, int CS, int XF>
 __global__ void __launch_bounds__(UPD_THREADS) update_kernel(const Dev P, const int leg)
 {
+    constexpr int R = Tune<T>::R;
     constexpr int RG = 32 / CS;                  // row groups per warp
     constexpr int RW = R * RG;                   // rows per warp
-    constexpr int RB = (UPD_THREADS / 32) * RW;  // rows per CTA
+    constexpr int NWARP = UPD_THREADS / 32;
+    constexpr int RB = NWARP * RW;               // rows per CTA
 
     extern __shared__ __align__(16) unsigned char smem_raw[];
     T *sm = reinterpret_cast<T *>(smem_raw);
-    __shared__ double red[UPD_THREADS / 32];
+    __shared__ double row_s[RB];
+    __shared__ float row_m[RB];
+    __shared__ float row_h[RB];
+    __shared__ double red[NWARP];
     __shared__ int is_last;
 
     const Ctl c = *P.ctl;
@@ -205,75 +346,85 @@ __global__ void __launch_bounds__(UPD_THREADS) update_kernel(const Dev P, const 
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int cs = lane % CS, rg = lane / CS;
-    const int row0 = blockIdx.x * RB + warp * RW + rg;   // row r of this thread: row0 + r*RG
+    const int lrow0 = warp * RW + rg;                    // CTA-local row of r = 0; row r: + r*RG
+    const int row0 = blockIdx.x * RB + lrow0;
 
-    T xr[R][DP], ph[R];
-    double pold[R];
+    T xr[R][DP];
+    T ph[R];
 #pragma unroll
     for (int r = 0; r < R; ++r) {
         const int i = row0 + r * RG;
 #pragma unroll
         for (int k = 0; k < DP; ++k) xr[r][k] = (i < nrows) ? rowc[(size_t)k * rp + i] : T(0);
-        pold[r] = (i < nrows) ? prow[i] : 0.0;
-        ph[r] = (T)pold[r];
+        ph[r] = (i < nrows && form == FORM_DIFF) ? (T)prow[i] : T(0);
     }
 
-    double md[R], sd[R];
-    if (form == FORM_DOT)
-        stream_columns<T, DP, R, CS, FORM_DOT, XF>(sm, colc, colt, coll, cp, ncols, xr, ph, tid, cs, md, sd);
-    else
-        stream_columns<T, DP, R, CS, FORM_DIFF, XF>(sm, colc, colt, coll, cp, ncols, xr, ph, tid, cs, md, sd);
+    float mx[R];
+    double sd[R];
+    if constexpr (sizeof(T) == 4) {
+        if (form == FORM_DOT) stream_f32<DP, CS, FORM_DOT>(sm, colc, colt, coll, cp, ncols, xr, ph, tid, cs, mx, sd);
+        else stream_f32<DP, CS, FORM_DIFF>(sm, colc, colt, coll, cp, ncols, xr, ph, tid, cs, mx, sd);
+    } else {
+        stream_f64<DP, CS, XF>(sm, colc, colt, cp, ncols, xr, tid, cs, mx, sd);
+    }
 
-    // merge the CS column splits of each row (xor-shuffle online logsumexp)
+    // merge the CS column splits of each row: maxima are integers, so the scalings are exact
 #pragma unroll
     for (int off = 1; off < CS; off <<= 1) {
 #pragma unroll
         for (int r = 0; r < R; ++r) {
-            const double mo = __shfl_xor_sync(0xffffffffu, md[r], off);
+            const float mo = __shfl_xor_sync(0xffffffffu, mx[r], off);
             const double so = __shfl_xor_sync(0xffffffffu, sd[r], off);
-            const double mn = fmax(md[r], mo);
-            sd[r] = sd[r] * exp2(md[r] - mn) + so * exp2(mo - mn);
-            md[r] = mn;
+            const float mn = fmaxf(mx[r], mo);
+            sd[r] = sd[r] * (double)pow2i(mx[r] - mn) + so * (double)pow2i(mo - mn);
+            mx[r] = mn;
         }
     }
+    if (cs == 0) {
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            row_m[lrow0 + r * RG] = mx[r];
+            row_s[lrow0 + r * RG] = sd[r];
+            row_h[lrow0 + r * RG] = (float)ph[r];
+        }
+    }
+    __syncthreads();
 
-    // epilogue (float64 per row)
+    // epilogue: one thread per row of the CTA (float64)
     const bool frozen = (P.mode == MODE_MASKED) && P.state[slot] != 0;
     const bool writes = !frozen && leg != LEG_V;
     double term_sum = 0.0;
-    if (cs == 0) {
-        const size_t rbase = (size_t)slot * rp;
-        const double *sq = (rows_x ? P.sqx : P.sqy) + rbase;
-        const double *lw = (rows_x ? P.la2 : P.lb2) + rbase;
-#pragma unroll
-        for (int r = 0; r < R; ++r) {
-            const int i = row0 + r * RG;
-            if (i >= nrows) continue;
-            const double L = md[r] + log2(sd[r]);
-            // log2 of this row's marginal under the potentials the leg started from, and the
-            // updated potential that makes the marginal equal to the weight (Eq. 3)
-            double lmarg, pnew;
-            if (form == FORM_DOT) {
-                pnew = lw[i] + sq[i] - L;
-                lmarg = lw[i] + pold[r] - pnew;
+    for (int lr = tid; lr < RB; lr += UPD_THREADS) {
+        const int i = blockIdx.x * RB + lr;
+        if (i >= nrows) continue;
+        const size_t o = (size_t)slot * rp + i;
+        const double lw = (rows_x ? P.la2 : P.lb2)[o];
+        const double sq = (rows_x ? P.sqx : P.sqy)[o];
+        const double pold = prow[i];
+        const double L = (double)row_m[lr] + log2(row_s[lr]);
+        // log2 of this row's marginal under the potentials the leg started from, and the
+        // updated potential that makes the marginal equal to the weight (Eq. 3)
+        double lmarg, pnew;
+        if (form == FORM_DOT) {
+            pnew = lw + sq - L;
+            lmarg = lw + pold - pnew;
+        } else {
+            lmarg = L - ((double)row_h[lr] - pold);
+            pnew = pold + (lw - lmarg);
+        }
+        if (leg != LEG_G) term_sum += (rows_x ? P.wa : P.wb)[o] * fabs(expm1((lmarg - lw) * 0.6931471805599453));
+        if (writes) {
+            T hi, lo;
+            if (form == FORM_DOT) { hi = (T)(pnew - sq); lo = T(0); }
+            else { hi = (T)pnew; lo = (T)(pnew - (double)hi); }
+            if (leg == LEG_F) {
+                P.phi[c.parity ^ 1][o] = pnew;
+                reinterpret_cast<T *>(P.ft[c.parity ^ 1])[o] = hi;
+                reinterpret_cast<T *>(P.fl[c.parity ^ 1])[o] = lo;
             } else {
-                lmarg = L - ((double)ph[r] - pold[r]);
-                pnew = pold[r] + (lw[i] - lmarg);
-            }
-            if (leg != LEG_G) term_sum += exp2(lw[i]) * fabs(expm1((lmarg - lw[i]) * 0.6931471805599453));
-            if (writes) {
-                T hi, lo;
-                if (form == FORM_DOT) { hi = (T)(pnew - sq[i]); lo = T(0); }
-                else { hi = (T)pnew; lo = (T)(pnew - (double)hi); }
-                if (leg == LEG_F) {
-                    P.phi[c.parity ^ 1][rbase + i] = pnew;
-                    reinterpret_cast<T *>(P.ft[c.parity ^ 1])[rbase + i] = hi;
-                    reinterpret_cast<T *>(P.fl[c.parity ^ 1])[rbase + i] = lo;
-                } else {
-                    P.gam[rbase + i] = pnew;
-                    reinterpret_cast<T *>(P.gt)[rbase + i] = hi;
-                    reinterpret_cast<T *>(P.gl)[rbase + i] = lo;
-                }
+                P.gam[o] = pnew;
+                reinterpret_cast<T *>(P.gt)[o] = hi;
+                reinterpret_cast<T *>(P.gl)[o] = lo;
             }
         }
     }
@@ -290,7 +441,7 @@ __global__ void __launch_bounds__(UPD_THREADS) update_kernel(const Dev P, const 
     if (tid == 0) {
         double s = 0.0;
 #pragma unroll
-        for (int w = 0; w < UPD_THREADS / 32; ++w) s += red[w];
+        for (int w = 0; w < NWARP; ++w) s += red[w];
         parts[blockIdx.x] = s;
         __threadfence();
         const unsigned ticket = atomicAdd(cnt, 1u);
