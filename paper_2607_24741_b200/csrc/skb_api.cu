@@ -32,7 +32,7 @@ static std::string g_create_err;
 // scaled squared radius M = s*max|x-c|^2 into every exponent.  Above FORM_DIFF_RADIUS a lane
 // switches to the difference form; above MIXED_RADIUS (any lane) an automatic batch computes
 // its exponents in float64 and only the exponentials in fp32.
-static const double FORM_DIFF_RADIUS = 64.0;
+static const double FORM_DIFF_RADIUS = 512.0;
 static const double MIXED_RADIUS = 512.0;
 
 static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }

@@ -9,20 +9,20 @@ template <typename T, int DP, int CS, int XF>
 static void launch_update(const Dev &P, int leg, int width, cudaStream_t st)
 {
     static bool attr_set = false;
-    const size_t smem = 2 * (size_t)(DP + 2) * TileCols<T, CS>::value * sizeof(T);
+    const size_t smem = 2 * (size_t)(DP + 2) * TileCols<T, DP, CS>::value * sizeof(T);
     if (!attr_set) {
         cudaFuncSetAttribute(update_kernel<T, DP, CS, XF>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         attr_set = true;
     }
-    const int rb = (UPD_THREADS / 32) * Tune<T>::R * (32 / CS);
+    const int rb = (UPD_THREADS / 32) * Tune<T, DP>::R * (32 / CS);
     const int nrows = (leg == LEG_F) ? P.n : P.m;
     dim3 grid((nrows + rb - 1) / rb, width < 1 ? 1 : width);
     update_kernel<T, DP, CS, XF><<<grid, UPD_THREADS, smem, st>>>(P, leg);
 }
 
 #define SKB_V(T, F64, XF, DP, CS) \
-    { F64, XF, DP, Tune<T>::R, CS, (UPD_THREADS / 32) * Tune<T>::R * (32 / CS), \
-      2 * (size_t)(DP + 2) * TileCols<T, CS>::value * sizeof(T), &launch_update<T, DP, CS, XF> }
+    { F64, XF, DP, Tune<T, DP>::R, CS, (UPD_THREADS / 32) * Tune<T, DP>::R * (32 / CS), \
+      2 * (size_t)(DP + 2) * TileCols<T, DP, CS>::value * sizeof(T), &launch_update<T, DP, CS, XF> }
 #define SKB_ROW(DP) \
     SKB_V(float, 0, 0, DP, 1), SKB_V(float, 0, 0, DP, 4), SKB_V(float, 0, 0, DP, 32), \
     SKB_V(double, 1, 0, DP, 1), SKB_V(double, 1, 0, DP, 4), SKB_V(double, 1, 0, DP, 32), \
@@ -41,14 +41,21 @@ const Variant *choose_variant(int W, int n, int m, int d, bool f64, bool fast_ex
 {
     const int DP = padded_dim(d);
     if (DP < 0) return nullptr;
-    // smallest column split that still gives about two waves of CTAs at full width
     const int mn = n < m ? n : m;
-    const int R = 2;
+    int R = 2;
+    for (const Variant &v : g_variants)
+        if (v.f64 == (f64 ? 1 : 0) && v.DP == DP) { R = v.R; break; }
+    // smallest column split that fills its CTAs' rows and gives every SM about four CTAs
     int cs = 32;
+    double best = -1.0;
     for (int c : {1, 4, 32}) {
         const int rb = (UPD_THREADS / 32) * R * (32 / c);
         const long long ctas = (long long)W * ((mn + rb - 1) / rb);
-        if (ctas >= 1184) { cs = c; break; }
+        const double util_n = (double)n / ((double)((n + rb - 1) / rb) * rb);
+        const double util_m = (double)m / ((double)((m + rb - 1) / rb) * rb);
+        const double fill = ctas >= 592 ? 1.0 : (double)ctas / 592.0;
+        const double score = (util_n < util_m ? util_n : util_m) * fill * (c == 32 ? 0.6 : 1.0);
+        if (score > best + 1e-9) { best = score; cs = c; }
     }
     if (force_cs == 1 || force_cs == 4 || force_cs == 32) cs = force_cs;
     for (const Variant &v : g_variants)

@@ -38,12 +38,29 @@ namespace skb {
 
 typedef unsigned long long u64;
 
-template <typename T> struct Tune;
-template <> struct Tune<float> { static constexpr int R = 2, CW = 8; };    // rows per thread, columns per step
-template <> struct Tune<double> { static constexpr int R = 2, CW = 4; };
+// Register tile of one thread: R rows held for the whole kernel x CW adjacent columns per step.
+// More rows per thread means fewer shared-memory bytes per pair; the limit is the register file.
+template <typename T, int DP> struct Tune;
+#ifndef SKB_F32_R16
+#define SKB_F32_R16 4
+#endif
+#ifndef SKB_F32_CW16
+#define SKB_F32_CW16 4
+#endif
+#ifndef SKB_UNROLL_Q
+#define SKB_UNROLL_Q 1
+#endif
+template <int DP> struct Tune<float, DP> {
+    static constexpr int R = DP <= 8 ? 4 : (DP == 16 ? SKB_F32_R16 : 2);
+    static constexpr int CW = DP <= 8 ? 8 : (DP == 16 ? SKB_F32_CW16 : 4);
+};
+template <int DP> struct Tune<double, DP> {
+    static constexpr int R = DP <= 8 ? 4 : 2;
+    static constexpr int CW = 4;
+};
 
-template <typename T, int CS> struct TileCols {
-    static constexpr int value = (Tune<T>::CW * CS * 2 > 128) ? Tune<T>::CW * CS * 2 : 128;   // >= 2 steps per tile
+template <typename T, int DP, int CS> struct TileCols {
+    static constexpr int value = (Tune<T, DP>::CW * CS * 2 > 128) ? Tune<T, DP>::CW * CS * 2 : 128;   // >= 2 steps per tile
 };
 
 __device__ __forceinline__ u64 pack2(float lo, float hi)
@@ -108,12 +125,14 @@ __device__ __forceinline__ void load_tile(T *dst, const T *colc, const T *colt, 
 // columns this thread visited.
 template <int DP, int CS, int FORM>
 __device__ __forceinline__ void stream_f32(float *sm, const float *colc, const float *colt, const float *coll,
-                                           const int cp, const int ncols, const float (&xrow)[2][DP],
-                                           const float (&ph)[2], const int tid, const int cs,
-                                           float (&mx)[2], double (&sd)[2])
+                                           const int cp, const int ncols,
+                                           const float (&xrow)[Tune<float, DP>::R][DP],
+                                           const float (&ph)[Tune<float, DP>::R], const int tid, const int cs,
+                                           float (&mx)[Tune<float, DP>::R], double (&sd)[Tune<float, DP>::R])
 {
-    constexpr int R = 2, CW = 8;
-    constexpr int TJ = TileCols<float, CS>::value;
+    constexpr int R = Tune<float, DP>::R, CW = Tune<float, DP>::CW;
+    constexpr int NP = CW / 2;                       // packed column pairs per step
+    constexpr int TJ = TileCols<float, DP, CS>::value;
     constexpr int STEPS = TJ / (CW * CS);
     constexpr int NR = DP + 1 + (FORM == FORM_DIFF ? 1 : 0);
     constexpr int STAGE = (DP + 2) * TJ;
@@ -143,75 +162,108 @@ __device__ __forceinline__ void stream_f32(float *sm, const float *colc, const f
         }
         __syncthreads();
         const float *st = sm + (t & 1) * STAGE;
-#pragma unroll 1
+        constexpr int UQ = SKB_UNROLL_Q;
+#pragma unroll UQ
         for (int q = 0; q < STEPS; ++q) {
             const int jj = (q * CS + cs) * CW;
-            u64 acc[R][4];
-            const ulonglong2 c0 = *reinterpret_cast<const ulonglong2 *>(st + DP * TJ + jj);
-            const ulonglong2 c1 = *reinterpret_cast<const ulonglong2 *>(st + DP * TJ + jj + 4);
+            u64 acc[R][NP];
+            u64 ct[NP];
+#pragma unroll
+            for (int h = 0; h < NP / 2; ++h) {
+                const ulonglong2 c = *reinterpret_cast<const ulonglong2 *>(st + DP * TJ + jj + 4 * h);
+                ct[2 * h] = c.x; ct[2 * h + 1] = c.y;
+            }
             if (FORM == FORM_DOT) {
 #pragma unroll
-                for (int r = 0; r < R; ++r) { acc[r][0] = c0.x; acc[r][1] = c0.y; acc[r][2] = c1.x; acc[r][3] = c1.y; }
+                for (int r = 0; r < R; ++r)
+#pragma unroll
+                    for (int p = 0; p < NP; ++p) acc[r][p] = ct[p];
 #pragma unroll
                 for (int k = 0; k < DP; ++k) {
-                    const ulonglong2 y0 = *reinterpret_cast<const ulonglong2 *>(st + k * TJ + jj);
-                    const ulonglong2 y1 = *reinterpret_cast<const ulonglong2 *>(st + k * TJ + jj + 4);
+                    u64 y[NP];
 #pragma unroll
-                    for (int r = 0; r < R; ++r) {
-                        acc[r][0] = fma2(xd[r][k], y0.x, acc[r][0]);
-                        acc[r][1] = fma2(xd[r][k], y0.y, acc[r][1]);
-                        acc[r][2] = fma2(xd[r][k], y1.x, acc[r][2]);
-                        acc[r][3] = fma2(xd[r][k], y1.y, acc[r][3]);
+                    for (int h = 0; h < NP / 2; ++h) {
+                        const ulonglong2 v = *reinterpret_cast<const ulonglong2 *>(st + k * TJ + jj + 4 * h);
+                        y[2 * h] = v.x; y[2 * h + 1] = v.y;
                     }
+#pragma unroll
+                    for (int r = 0; r < R; ++r)
+#pragma unroll
+                        for (int p = 0; p < NP; ++p) acc[r][p] = fma2(xd[r][k], y[p], acc[r][p]);
                 }
             } else {
-                u64 sq[R][4];
 #pragma unroll
-                for (int r = 0; r < R; ++r) { sq[r][0] = 0ull; sq[r][1] = 0ull; sq[r][2] = 0ull; sq[r][3] = 0ull; }
+                for (int r = 0; r < R; ++r)
+#pragma unroll
+                    for (int p = 0; p < NP; ++p) acc[r][p] = 0ull;          // |r - c|^2 so far
 #pragma unroll
                 for (int k = 0; k < DP; ++k) {
-                    const ulonglong2 y0 = *reinterpret_cast<const ulonglong2 *>(st + k * TJ + jj);
-                    const ulonglong2 y1 = *reinterpret_cast<const ulonglong2 *>(st + k * TJ + jj + 4);
+                    u64 y[NP];
 #pragma unroll
-                    for (int r = 0; r < R; ++r) {
-                        u64 dk;
-                        dk = sub2(xd[r][k], y0.x); sq[r][0] = fma2(dk, dk, sq[r][0]);
-                        dk = sub2(xd[r][k], y0.y); sq[r][1] = fma2(dk, dk, sq[r][1]);
-                        dk = sub2(xd[r][k], y1.x); sq[r][2] = fma2(dk, dk, sq[r][2]);
-                        dk = sub2(xd[r][k], y1.y); sq[r][3] = fma2(dk, dk, sq[r][3]);
+                    for (int h = 0; h < NP / 2; ++h) {
+                        const ulonglong2 v = *reinterpret_cast<const ulonglong2 *>(st + k * TJ + jj + 4 * h);
+                        y[2 * h] = v.x; y[2 * h + 1] = v.y;
                     }
+#pragma unroll
+                    for (int r = 0; r < R; ++r)
+#pragma unroll
+                        for (int p = 0; p < NP; ++p) {
+                            const u64 dk = sub2(xd[r][k], y[p]);
+                            acc[r][p] = fma2(dk, dk, acc[r][p]);
+                        }
                 }
-                const ulonglong2 l0 = *reinterpret_cast<const ulonglong2 *>(st + (DP + 1) * TJ + jj);
-                const ulonglong2 l1 = *reinterpret_cast<const ulonglong2 *>(st + (DP + 1) * TJ + jj + 4);
+                u64 cl[NP];
+#pragma unroll
+                for (int h = 0; h < NP / 2; ++h) {
+                    const ulonglong2 v = *reinterpret_cast<const ulonglong2 *>(st + (DP + 1) * TJ + jj + 4 * h);
+                    cl[2 * h] = v.x; cl[2 * h + 1] = v.y;
+                }
+#pragma unroll
+                for (int r = 0; r < R; ++r)
+#pragma unroll
+                    for (int p = 0; p < NP; ++p) acc[r][p] = add2(add2(phd[r], ct[p]), sub2(cl[p], acc[r][p]));
+            }
+            // running maxima: one rarely taken branch per step covers all rows
+            float mt[R];
+            bool grow = false;
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                float a[CW];
+#pragma unroll
+                for (int p = 0; p < NP; ++p) unpack2(acc[r][p], a[2 * p], a[2 * p + 1]);
+                mt[r] = fmaxf(a[0], a[1]);
+#pragma unroll
+                for (int e = 2; e < CW; ++e) mt[r] = fmaxf(mt[r], a[e]);
+                grow = grow || (mt[r] > mx[r] + 8.0f);
+            }
+            if (grow) {                                        // lazy rescale: terms stay below 2^9
 #pragma unroll
                 for (int r = 0; r < R; ++r) {
-                    acc[r][0] = add2(add2(phd[r], c0.x), sub2(l0.x, sq[r][0]));
-                    acc[r][1] = add2(add2(phd[r], c0.y), sub2(l0.y, sq[r][1]));
-                    acc[r][2] = add2(add2(phd[r], c1.x), sub2(l1.x, sq[r][2]));
-                    acc[r][3] = add2(add2(phd[r], c1.y), sub2(l1.y, sq[r][3]));
+                    if (mt[r] > mx[r] + 8.0f) {
+                        const float mn = ceilf(mt[r]);
+                        const float fac = pow2i(mx[r] - mn);
+                        float t0, t1;
+                        unpack2(ts[r], t0, t1);
+                        ts[r] = pack2(t0 * fac, t1 * fac);
+                        sd[r] *= (double)fac;
+                        mx[r] = mn;
+                    }
                 }
             }
 #pragma unroll
             for (int r = 0; r < R; ++r) {
-                float a0, a1, a2, a3, a4, a5, a6, a7;
-                unpack2(acc[r][0], a0, a1); unpack2(acc[r][1], a2, a3);
-                unpack2(acc[r][2], a4, a5); unpack2(acc[r][3], a6, a7);
-                const float mt = fmaxf(fmaxf(fmaxf(a0, a1), fmaxf(a2, a3)), fmaxf(fmaxf(a4, a5), fmaxf(a6, a7)));
-                if (mt > mx[r] + 8.0f) {                       // lazy rescale: terms stay below 2^9
-                    const float mn = ceilf(mt);
-                    const float fac = pow2i(mx[r] - mn);
-                    float t0, t1;
-                    unpack2(ts[r], t0, t1);
-                    ts[r] = pack2(t0 * fac, t1 * fac);
-                    sd[r] *= (double)fac;
-                    mx[r] = mn;
-                }
                 const u64 mm = pack2(mx[r], mx[r]);
-                unpack2(sub2(acc[r][0], mm), a0, a1); unpack2(sub2(acc[r][1], mm), a2, a3);
-                unpack2(sub2(acc[r][2], mm), a4, a5); unpack2(sub2(acc[r][3], mm), a6, a7);
-                const u64 e0 = pack2(ex2_fast(a0), ex2_fast(a1)), e1 = pack2(ex2_fast(a2), ex2_fast(a3));
-                const u64 e2 = pack2(ex2_fast(a4), ex2_fast(a5)), e3 = pack2(ex2_fast(a6), ex2_fast(a7));
-                ts[r] = add2(ts[r], add2(add2(e0, e1), add2(e2, e3)));
+                u64 e[NP];
+#pragma unroll
+                for (int p = 0; p < NP; ++p) {
+                    float lo, hi;
+                    unpack2(sub2(acc[r][p], mm), lo, hi);
+                    e[p] = pack2(ex2_fast(lo), ex2_fast(hi));
+                }
+                u64 es = add2(e[0], e[1]);
+#pragma unroll
+                for (int p = 2; p < NP; p += 2) es = add2(es, add2(e[p], e[p + 1]));
+                ts[r] = add2(ts[r], es);
             }
         }
 #pragma unroll
@@ -229,18 +281,21 @@ __device__ __forceinline__ void stream_f32(float *sm, const float *colc, const f
 // XF = 1: exponentials on the fp32 special-function unit; XF = 0: software exp2 in float64.
 template <int DP, int CS, int XF>
 __device__ __forceinline__ void stream_f64(double *sm, const double *colc, const double *colt,
-                                           const int cp, const int ncols, const double (&xr)[2][DP],
-                                           const int tid, const int cs, float (&mx)[2], double (&sd)[2])
+                                           const int cp, const int ncols,
+                                           const double (&xr)[Tune<double, DP>::R][DP],
+                                           const int tid, const int cs,
+                                           float (&mx)[Tune<double, DP>::R], double (&sd)[Tune<double, DP>::R])
 {
-    constexpr int R = 2, CW = 4;
-    constexpr int TJ = TileCols<double, CS>::value;
+    constexpr int R = Tune<double, DP>::R, CW = 4;
+    constexpr int TJ = TileCols<double, DP, CS>::value;
     constexpr int STEPS = TJ / (CW * CS);
     constexpr int NR = DP + 1;
     constexpr int STAGE = (DP + 2) * TJ;
 
     float ts[R];
+    double md[R];
 #pragma unroll
-    for (int r = 0; r < R; ++r) { mx[r] = NEG_BIG; ts[r] = 0.f; sd[r] = 0.0; }
+    for (int r = 0; r < R; ++r) { mx[r] = NEG_BIG; md[r] = (double)NEG_BIG; ts[r] = 0.f; sd[r] = 0.0; }
 
     const int ntiles = (ncols + TJ - 1) / TJ;
     load_tile<double, DP, TJ, NR>(sm, colc, colt, colt, cp, 0, tid);
@@ -277,23 +332,34 @@ __device__ __forceinline__ void stream_f64(double *sm, const double *colc, const
                     acc[r][3] = fma(xr[r][k], y1.y, acc[r][3]);
                 }
             }
+            double mt[R];
+            bool grow = false;
 #pragma unroll
             for (int r = 0; r < R; ++r) {
-                // the maximum only has to be near the true one: track it on fp32 copies
-                const float mt = fmaxf(fmaxf((float)acc[r][0], (float)acc[r][1]), fmaxf((float)acc[r][2], (float)acc[r][3]));
-                if (mt > mx[r] + 8.0f) {
-                    const float mn = ceilf(mt);
-                    const float fac = pow2i(mx[r] - mn);
-                    ts[r] *= fac;
-                    sd[r] *= (double)fac;
-                    mx[r] = mn;
+                mt[r] = fmax(fmax(acc[r][0], acc[r][1]), fmax(acc[r][2], acc[r][3]));
+                grow = grow || (mt[r] > md[r] + 8.0);
+            }
+            if (grow) {
+#pragma unroll
+                for (int r = 0; r < R; ++r) {
+                    if (mt[r] > md[r] + 8.0) {
+                        const float mn = ceilf((float)mt[r]) + 1.0f;       // +1: the fp32 copy may round down
+                        const float fac = pow2i(mx[r] - mn);
+                        ts[r] *= fac;
+                        sd[r] *= (double)fac;
+                        mx[r] = mn;
+                        md[r] = (double)mn;
+                    }
                 }
-                const double md = (double)mx[r];
+            }
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
                 if (XF) {
-                    ts[r] += (ex2_fast((float)(acc[r][0] - md)) + ex2_fast((float)(acc[r][1] - md))) +
-                             (ex2_fast((float)(acc[r][2] - md)) + ex2_fast((float)(acc[r][3] - md)));
+                    ts[r] += (ex2_fast((float)(acc[r][0] - md[r])) + ex2_fast((float)(acc[r][1] - md[r]))) +
+                             (ex2_fast((float)(acc[r][2] - md[r])) + ex2_fast((float)(acc[r][3] - md[r])));
                 } else {
-                    sd[r] += (exp2(acc[r][0] - md) + exp2(acc[r][1] - md)) + (exp2(acc[r][2] - md) + exp2(acc[r][3] - md));
+                    sd[r] += (exp2(acc[r][0] - md[r]) + exp2(acc[r][1] - md[r])) +
+                             (exp2(acc[r][2] - md[r]) + exp2(acc[r][3] - md[r]));
                 }
             }
         }
@@ -308,7 +374,7 @@ __device__ __forceinline__ void stream_f64(double *sm, const double *colc, const
 template <typename T, int DP, int CS, int XF>
 __global__ void __launch_bounds__(UPD_THREADS) update_kernel(const Dev P, const int leg)
 {
-    constexpr int R = Tune<T>::R;
+    constexpr int R = Tune<T, DP>::R;
     constexpr int RG = 32 / CS;                  // row groups per warp
     constexpr int RW = R * RG;                   // rows per warp
     constexpr int NWARP = UPD_THREADS / 32;
@@ -345,7 +411,9 @@ __global__ void __launch_bounds__(UPD_THREADS) update_kernel(const Dev P, const 
     const double *prow = (rows_x ? P.phi[c.parity] : P.gam) + (size_t)slot * rp;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int cs = lane % CS, rg = lane / CS;
+    // lanes that share a row's columns sit RG apart, so that each quarter-warp reads a single
+    // shared-memory address per load when CS <= 4 (a broadcast, the cheapest access pattern)
+    const int cs = lane / RG, rg = lane % RG;
     const int lrow0 = warp * RW + rg;                    // CTA-local row of r = 0; row r: + r*RG
     const int row0 = blockIdx.x * RB + lrow0;
 
@@ -373,8 +441,8 @@ __global__ void __launch_bounds__(UPD_THREADS) update_kernel(const Dev P, const 
     for (int off = 1; off < CS; off <<= 1) {
 #pragma unroll
         for (int r = 0; r < R; ++r) {
-            const float mo = __shfl_xor_sync(0xffffffffu, mx[r], off);
-            const double so = __shfl_xor_sync(0xffffffffu, sd[r], off);
+            const float mo = __shfl_xor_sync(0xffffffffu, mx[r], off * RG);
+            const double so = __shfl_xor_sync(0xffffffffu, sd[r], off * RG);
             const float mn = fmaxf(mx[r], mo);
             sd[r] = sd[r] * (double)pow2i(mx[r] - mn) + so * (double)pow2i(mo - mn);
             mx[r] = mn;
