@@ -179,6 +179,34 @@ skb_status sinkhorn_batch_solve_host(const void *x, const void *y, const float *
 
 void sinkhorn_batch_destroy(skb_batch *h);
 
+/*
+ * Row residual of given potentials without any workspace or allocation.  (The paper has no
+ * counterpart: this is a library convenience for callers that may not allocate device
+ * memory - a host that fixes every component's memory budget at start-up, or a loop that
+ * cannot take the device-wide synchronisation of cudaMalloc.)
+ *
+ * For each lane, r_row = sum_i | sum_j exp((f_i + g_j - |x_i - y_j|^2)/eps) - a_i |, the row
+ * half of Eq. 5, in float64 arithmetic.
+ *   x [W,n,d], y [W,m,d], a [W,n], eps [W]  fp32, device, row-major
+ *   f [W,n], g [W,m]                       float64, device
+ *   r_row [W]                              fp32, device out
+ *   stream                                 cudaStream_t; the call enqueues and returns
+ * The scratch of the reduction is a fixed SKB_STATIC_SCRATCH_BYTES array inside the library
+ * image (held by every GPU that loads the library until exit), so W <= SKB_STATIC_MAX_LANES
+ * and n <= SKB_STATIC_MAX_ROWS; larger shapes return SKB_ERR_SHAPE.  The call performs no
+ * cudaMalloc, cudaFree or other allocating call.  The first call on each device looks the
+ * array's device address up (with that device current); make that first call before any
+ * stream capture begins.  All calls share the one array: calls whose kernels could overlap
+ * on the GPU (different streams, different threads) race and must be ordered by the caller.
+ */
+#define SKB_STATIC_MAX_LANES 256
+#define SKB_STATIC_MAX_ROWS 8192
+#define SKB_STATIC_SCRATCH_BYTES (SKB_STATIC_MAX_LANES * (SKB_STATIC_MAX_ROWS / 128) * 8 + SKB_STATIC_MAX_LANES * 4)
+skb_status sinkhorn_row_residual_static(const float *x, const float *y, const float *a,
+                                        const double *f, const double *g, const float *eps,
+                                        int W, int n, int m, int d, float *r_row, void *stream);
+const char *sinkhorn_row_residual_static_last_error(void);
+
 /* Host string describing the last error on this handle (or of the last failed create
  * when h is null).  Valid until the next call on the same handle. */
 const char *sinkhorn_batch_last_error(const skb_batch *h);

@@ -29,6 +29,8 @@ EXPORTS = (
     "sinkhorn_batch_host_workspace_bytes", "sinkhorn_batch_solve_host",
     "sinkhorn_batch_launch_count", "sinkhorn_batch_profile_update", "sinkhorn_batch_arithmetic",
 )
+# entry points outside the sinkhorn_batch_* family
+EXTRA_EXPORTS = ("sinkhorn_row_residual_static", "sinkhorn_row_residual_static_last_error")
 
 
 class SkbConfig(ctypes.Structure):
@@ -76,6 +78,10 @@ def _load():
     lib.sinkhorn_batch_last_error.restype = ctypes.c_char_p
     lib.sinkhorn_batch_solve_host.argtypes = [vp, vp, vp, vp, vp, ctypes.c_float, cfgp, vp, vp, vp, vp, vp, vp,
                                               ctypes.POINTER(ctypes.c_longlong), ctypes.POINTER(ctypes.c_int)]
+    lib.sinkhorn_row_residual_static.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_int, ctypes.c_int,
+                                                 ctypes.c_int, ctypes.c_int, vp, vp]
+    lib.sinkhorn_row_residual_static.restype = ctypes.c_int
+    lib.sinkhorn_row_residual_static_last_error.restype = ctypes.c_char_p
     for name in EXPORTS:
         if name not in ("sinkhorn_batch_workspace_bytes", "sinkhorn_batch_host_workspace_bytes",
                         "sinkhorn_batch_destroy", "sinkhorn_batch_last_error"):
@@ -138,6 +144,21 @@ def sinkhorn_batch_active(h) -> int:
 
 def sinkhorn_batch_destroy(h):
     lib.sinkhorn_batch_destroy(h)
+
+
+def sinkhorn_row_residual_static(x, y, a, f, g, eps, stream=None):
+    """Row residual of potentials (f, g) per lane, with no workspace and no allocation inside the
+    library (see the header for limits and the sharing rule).  x, y, a, eps: float32 CUDA tensors;
+    f, g: float64.  Returns the library's status code and writes into the tensor it returns."""
+    W, n, d = x.shape
+    m = y.shape[1]
+    out = torch.empty(W, dtype=torch.float32, device=x.device)
+    st = (stream or torch.cuda.current_stream(x.device)).cuda_stream
+    rc = lib.sinkhorn_row_residual_static(_ptr(x), _ptr(y), _ptr(a), _ptr(f), _ptr(g), _ptr(eps), W, n, m, d,
+                                          _ptr(out), st)
+    if rc != SKB_OK:
+        raise SkbError(rc, lib.sinkhorn_row_residual_static_last_error().decode())
+    return out
 
 
 class SinkhornBatch:
