@@ -147,6 +147,8 @@ def main():
     ap.add_argument("--compute", default="auto", choices=["auto", "f32", "mixed", "f64"])
     ap.add_argument("--no-controls", action="store_true", help="skip the static / masked control timings")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--kernel-only", action="store_true",
+                    help="only create the batch and time the update kernel (few launches; for profiler captures)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -174,6 +176,14 @@ def main():
     if w.xy_dtype == "bf16":
         x, y = x.bfloat16(), y.bfloat16()
     a, b, eps = t(w.a), t(w.b), t(w.eps)
+    if args.kernel_only:
+        sb = B.SinkhornBatch(x, y, a, b, eps, w.tol, mode="static", compute=args.compute, max_iter=w.max_iter)
+        sb.step(2)
+        out = {"workload": args.workload, "arithmetic": sb.arithmetic(),
+               "f_leg_ms": sb.profile_update(leg=0, reps=3), "g_leg_ms": sb.profile_update(leg=1, reps=3)}
+        sb.close()
+        print(json.dumps(out), flush=True)
+        return
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)      # > 126 MB L2
 
     def solve(mode, collect=False):
