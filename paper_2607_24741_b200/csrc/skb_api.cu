@@ -62,14 +62,14 @@ static size_t carve(const skb_config *c, const Variant *var, char *base, Dev *D,
         return p;
     };
     const size_t W = c->W, n = c->n, m = c->m;
-    const size_t np = align_up(n, 4), mp = align_up(m, 4), DP = var->DP;
+    const size_t np = align_up(n, 4), mp = align_up(m, 4), DP = var->DP ? var->DP : padded_dim(c->d);
     const size_t ts = var->f64 ? 8 : 4;
     Dev d;
     memset(&d, 0, sizeof(d));
     d.W = c->W; d.n = c->n; d.m = c->m; d.d = c->d; d.np = (int)np; d.mp = (int)mp; d.DP = (int)DP;
     d.mode = c->mode; d.max_iter = c->max_iter; d.audit_every = c->audit_every;
     d.xy_bf16 = c->xy_dtype == SKB_BF16; d.compute_f64 = var->f64;
-    d.cost_form = c->cost_form;
+    d.cost_form = c->d > 32 ? 1 : c->cost_form;      // the large-d kernels only have the expanded form
     // fp32: above this scaled squared radius the expanded cost loses more than ~4e-6 per term
     d.form_threshold = FORM_DIFF_RADIUS;
     // control block first, then everything that must start at zero, in one contiguous range

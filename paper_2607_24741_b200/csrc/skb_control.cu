@@ -29,7 +29,7 @@ __device__ __forceinline__ float load_raw(const Dev &P, const void *base, size_t
 __global__ void __launch_bounds__(256) lane_stats_kernel(const Dev P, const void *xin, const void *yin, const float *eps)
 {
     __shared__ double red[256];
-    __shared__ double cen[32];
+    __shared__ double cen[1024];
     const int slot = blockIdx.x, tid = threadIdx.x;
     const int tot = P.n + P.m;
     for (int k = 0; k < P.d; ++k) {
@@ -56,7 +56,7 @@ __global__ void __launch_bounds__(256) lane_stats_kernel(const Dev P, const void
     red[tid] = mxr;
     __syncthreads();
     for (int off = 128; off > 0; off >>= 1) { if (tid < off) red[tid] = fmax(red[tid], red[tid + off]); __syncthreads(); }
-    if (tid < P.DP) P.center[(size_t)slot * P.DP + tid] = tid < P.d ? cen[tid] : 0.0;
+    for (int k = tid; k < P.DP; k += 256) P.center[(size_t)slot * P.DP + k] = k < P.d ? cen[k] : 0.0;
     if (tid == 0) {
         const double e = (double)eps[slot];
         const bool eps_ok = (e > 0.0) && isfinite(e);

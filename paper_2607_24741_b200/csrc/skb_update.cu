@@ -1,6 +1,7 @@
 // Instantiations of the streaming update kernel and the shape -> variant choice.
 #include <cstdlib>
 #include "skb_update.cuh"
+#include "skb_update_bigd.cuh"
 #include "skb_host.h"
 
 namespace skb {
@@ -30,8 +31,30 @@ static void launch_update(const Dev &P, int leg, int width, cudaStream_t st)
 
 static const Variant g_variants[] = {SKB_ROW(2), SKB_ROW(3), SKB_ROW(4), SKB_ROW(8), SKB_ROW(16), SKB_ROW(32)};
 
+template <typename T, int XF>
+static void launch_bigd(const Dev &P, int leg, int width, cudaStream_t st)
+{
+    static bool attr_set = false;
+    const size_t smem = 2 * (size_t)BIGD_KC * (BIGD_RB + BIGD_TJ) * sizeof(T);
+    if (!attr_set) {
+        cudaFuncSetAttribute(update_bigd_kernel<T, XF>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        attr_set = true;
+    }
+    const int nrows = (leg == LEG_F) ? P.n : P.m;
+    dim3 grid((nrows + BIGD_RB - 1) / BIGD_RB, width < 1 ? 1 : width);
+    update_bigd_kernel<T, XF><<<grid, UPD_THREADS, smem, st>>>(P, leg);
+}
+
+// DP = 0 marks the large-d kernels: the padded dimension is d rounded up to the chunk size
+static const Variant g_bigd[] = {
+    {0, 0, 0, 4, 4, BIGD_RB, 2 * (size_t)BIGD_KC * (BIGD_RB + BIGD_TJ) * 4, &launch_bigd<float, 0>},
+    {1, 0, 0, 4, 4, BIGD_RB, 2 * (size_t)BIGD_KC * (BIGD_RB + BIGD_TJ) * 8, &launch_bigd<double, 0>},
+    {1, 1, 0, 4, 4, BIGD_RB, 2 * (size_t)BIGD_KC * (BIGD_RB + BIGD_TJ) * 8, &launch_bigd<double, 1>},
+};
+
 int padded_dim(int d)
 {
+    if (d > 32) return d <= 1024 ? (d + BIGD_KC - 1) / BIGD_KC * BIGD_KC : -1;
     const int opts[] = {2, 3, 4, 8, 16, 32};
     for (int o : opts) if (d <= o) return o;
     return -1;
@@ -41,6 +64,11 @@ const Variant *choose_variant(int W, int n, int m, int d, bool f64, bool fast_ex
 {
     const int DP = padded_dim(d);
     if (DP < 0) return nullptr;
+    if (d > 32) {
+        for (const Variant &v : g_bigd)
+            if (v.f64 == (f64 ? 1 : 0) && v.xf == ((f64 && fast_exp) ? 1 : 0)) return &v;
+        return nullptr;
+    }
     const int mn = n < m ? n : m;
     int R = 2;
     for (const Variant &v : g_variants)

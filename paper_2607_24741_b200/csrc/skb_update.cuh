@@ -371,6 +371,96 @@ __device__ __forceinline__ void stream_f64(double *sm, const double *colc, const
     }
 }
 
+// Float64 epilogue of a CTA's RB rows (one thread per row) and the fused residual reduction.
+// row_m / row_s hold, per CTA-local row, the integer-valued maximum and the sum of
+// 2^(arg - max) over ALL columns; row_h the fp32 shift a difference-form row carried.
+template <typename T, int RB>
+__device__ __forceinline__ void finish_rows(const Dev &P, const Ctl &c, const int leg, const int slot,
+                                            const int form, const float *row_m, const double *row_s,
+                                            const float *row_h, double *red, int *is_last)
+{
+    constexpr int NWARP = UPD_THREADS / 32;
+    const bool rows_x = (leg == LEG_F);
+    const int nrows = rows_x ? P.n : P.m, rp = rows_x ? P.np : P.mp;
+    const double *prow = (rows_x ? P.phi[c.parity] : P.gam) + (size_t)slot * rp;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const bool frozen = (P.mode == MODE_MASKED) && P.state[slot] != 0;
+    const bool writes = !frozen && leg != LEG_V;
+    double term_sum = 0.0;
+    for (int lr = tid; lr < RB; lr += UPD_THREADS) {
+        const int i = blockIdx.x * RB + lr;
+        if (i >= nrows) continue;
+        const size_t o = (size_t)slot * rp + i;
+        const double lw = (rows_x ? P.la2 : P.lb2)[o];
+        const double sq = (rows_x ? P.sqx : P.sqy)[o];
+        const double pold = prow[i];
+        const double L = (double)row_m[lr] + log2(row_s[lr]);
+        // log2 of this row's marginal under the potentials the leg started from, and the
+        // updated potential that makes the marginal equal to the weight (Eq. 3)
+        double lmarg, pnew;
+        if (form == FORM_DOT) {
+            pnew = lw + sq - L;
+            lmarg = lw + pold - pnew;
+        } else {
+            lmarg = L - ((double)row_h[lr] - pold);
+            pnew = pold + (lw - lmarg);
+        }
+        if (leg != LEG_G) term_sum += (rows_x ? P.wa : P.wb)[o] * fabs(expm1((lmarg - lw) * 0.6931471805599453));
+        if (writes) {
+            T hi, lo;
+            if (form == FORM_DOT) { hi = (T)(pnew - sq); lo = T(0); }
+            else { hi = (T)pnew; lo = (T)(pnew - (double)hi); }
+            if (leg == LEG_F) {
+                P.phi[c.parity ^ 1][o] = pnew;
+                reinterpret_cast<T *>(P.ft[c.parity ^ 1])[o] = hi;
+                reinterpret_cast<T *>(P.fl[c.parity ^ 1])[o] = lo;
+            } else {
+                P.gam[o] = pnew;
+                reinterpret_cast<T *>(P.gt)[o] = hi;
+                reinterpret_cast<T *>(P.gl)[o] = lo;
+            }
+        }
+    }
+    if (leg == LEG_G) return;
+
+    // fused marginal-residual reduction -> one flag per lane (fixed summation order)
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) term_sum += __shfl_down_sync(0xffffffffu, term_sum, off);
+    if (lane == 0) red[warp] = term_sum;
+    __syncthreads();
+    double *parts = (leg == LEG_F ? P.part_row : P.part_col) + (size_t)slot * MAX_PARTS;
+    unsigned *cnt = (leg == LEG_F ? P.cnt_row : P.cnt_col) + slot;
+    const int nblk = (nrows + RB - 1) / RB;
+    if (tid == 0) {
+        double s = 0.0;
+#pragma unroll
+        for (int w = 0; w < NWARP; ++w) s += red[w];
+        parts[blockIdx.x] = s;
+        __threadfence();
+        const unsigned ticket = atomicAdd(cnt, 1u);
+        *is_last = (ticket == (unsigned)(nblk - 1));
+    }
+    __syncthreads();
+    if (!*is_last || tid != 0) return;
+    __threadfence();
+    double tot = 0.0;
+    for (int b = 0; b < nblk; ++b) tot += reinterpret_cast<volatile double *>(parts)[b];
+    *cnt = 0u;
+    const bool finite = isfinite(tot);
+    if (leg == LEG_F) {
+        P.rrow[slot] = tot;
+        const bool audited = c.cycle >= 1 && (c.cycle % P.audit_every) == 0;
+        const bool live = !frozen && !(P.mode == MODE_STATIC && P.state[slot] != 0);
+        P.flag[slot] = (audited && live && finite && tot <= P.tol_screen) ? 1 : 0;
+        if (!finite && !frozen) P.nonfinite[slot] = 1;
+    } else {
+        P.rcol[slot] = tot;
+        const double two = fmax(P.rrow[slot], tot);
+        P.verdict[slot] = (finite && two <= P.tol_stop) ? 1 : 0;
+        if (!finite) P.nonfinite[slot] = 1;
+    }
+}
+
 template <typename T, int DP, int CS, int XF>
 __global__ void __launch_bounds__(UPD_THREADS) update_kernel(const Dev P, const int leg)
 {
@@ -457,83 +547,7 @@ __global__ void __launch_bounds__(UPD_THREADS) update_kernel(const Dev P, const 
         }
     }
     __syncthreads();
-
-    // epilogue: one thread per row of the CTA (float64)
-    const bool frozen = (P.mode == MODE_MASKED) && P.state[slot] != 0;
-    const bool writes = !frozen && leg != LEG_V;
-    double term_sum = 0.0;
-    for (int lr = tid; lr < RB; lr += UPD_THREADS) {
-        const int i = blockIdx.x * RB + lr;
-        if (i >= nrows) continue;
-        const size_t o = (size_t)slot * rp + i;
-        const double lw = (rows_x ? P.la2 : P.lb2)[o];
-        const double sq = (rows_x ? P.sqx : P.sqy)[o];
-        const double pold = prow[i];
-        const double L = (double)row_m[lr] + log2(row_s[lr]);
-        // log2 of this row's marginal under the potentials the leg started from, and the
-        // updated potential that makes the marginal equal to the weight (Eq. 3)
-        double lmarg, pnew;
-        if (form == FORM_DOT) {
-            pnew = lw + sq - L;
-            lmarg = lw + pold - pnew;
-        } else {
-            lmarg = L - ((double)row_h[lr] - pold);
-            pnew = pold + (lw - lmarg);
-        }
-        if (leg != LEG_G) term_sum += (rows_x ? P.wa : P.wb)[o] * fabs(expm1((lmarg - lw) * 0.6931471805599453));
-        if (writes) {
-            T hi, lo;
-            if (form == FORM_DOT) { hi = (T)(pnew - sq); lo = T(0); }
-            else { hi = (T)pnew; lo = (T)(pnew - (double)hi); }
-            if (leg == LEG_F) {
-                P.phi[c.parity ^ 1][o] = pnew;
-                reinterpret_cast<T *>(P.ft[c.parity ^ 1])[o] = hi;
-                reinterpret_cast<T *>(P.fl[c.parity ^ 1])[o] = lo;
-            } else {
-                P.gam[o] = pnew;
-                reinterpret_cast<T *>(P.gt)[o] = hi;
-                reinterpret_cast<T *>(P.gl)[o] = lo;
-            }
-        }
-    }
-    if (leg == LEG_G) return;
-
-    // fused marginal-residual reduction -> one flag per lane (fixed summation order)
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) term_sum += __shfl_down_sync(0xffffffffu, term_sum, off);
-    if (lane == 0) red[warp] = term_sum;
-    __syncthreads();
-    double *parts = (leg == LEG_F ? P.part_row : P.part_col) + (size_t)slot * MAX_PARTS;
-    unsigned *cnt = (leg == LEG_F ? P.cnt_row : P.cnt_col) + slot;
-    const int nblk = (nrows + RB - 1) / RB;
-    if (tid == 0) {
-        double s = 0.0;
-#pragma unroll
-        for (int w = 0; w < NWARP; ++w) s += red[w];
-        parts[blockIdx.x] = s;
-        __threadfence();
-        const unsigned ticket = atomicAdd(cnt, 1u);
-        is_last = (ticket == (unsigned)(nblk - 1));
-    }
-    __syncthreads();
-    if (!is_last || tid != 0) return;
-    __threadfence();
-    double tot = 0.0;
-    for (int b = 0; b < nblk; ++b) tot += reinterpret_cast<volatile double *>(parts)[b];
-    *cnt = 0u;
-    const bool finite = isfinite(tot);
-    if (leg == LEG_F) {
-        P.rrow[slot] = tot;
-        const bool audited = c.cycle >= 1 && (c.cycle % P.audit_every) == 0;
-        const bool live = !frozen && !(P.mode == MODE_STATIC && P.state[slot] != 0);
-        P.flag[slot] = (audited && live && finite && tot <= P.tol_screen) ? 1 : 0;
-        if (!finite && !frozen) P.nonfinite[slot] = 1;
-    } else {
-        P.rcol[slot] = tot;
-        const double two = fmax(P.rrow[slot], tot);
-        P.verdict[slot] = (finite && two <= P.tol_stop) ? 1 : 0;
-        if (!finite) P.nonfinite[slot] = 1;
-    }
+    finish_rows<T, RB>(P, c, leg, slot, form, row_m, row_s, row_h, red, &is_last);
 }
 
 }  // namespace skb

@@ -26,6 +26,7 @@ CASES = {
     "sensor_ragged": dict(name="sensor", W=16, n=200, m=264),
     "registration_small": dict(name="registration", W=4, n=1000),
     "sweep_small": dict(name="sweep", W=48, n=100, m=77, max_iter=3000),
+    "feature_small": dict(name="feature", W=4, n=200, m=333, d=80),      # bf16 inputs, large-d kernels
 }
 
 
@@ -241,3 +242,54 @@ def test_host_buffer_call_matches_device_call(oracle):
     assert code == 0
     np.testing.assert_array_equal(depth, r["depth"]); np.testing.assert_array_equal(f, r["f32"])
     np.testing.assert_array_equal(g, r["g32"]); assert slots.value == r["stats"]["slots"]
+
+
+# ---- BASELINE sizes, in the launch configuration bench.py times (ACTIVE, default arithmetic) ----
+FULL = {
+    "tiny": (range(8), {}),
+    "sensor": ([0, 1, 17, 63, 100, 128, 200, 255], {}),
+    "feature": ([0, 21, 63], {}),
+    "sweep": ([0, 3, 5, 8, 100, 511, 777, 1023], {}),
+}
+
+
+@pytest.mark.parametrize("name", list(FULL))
+def test_full_size_sampled_lanes_against_oracle(oracle, name):
+    lanes, kw = FULL[name]
+    w = wl.make(name, **kw)
+    W = w.shape[0]
+    r = run_gpu(w, mode="active")
+    misses = check_against_oracle(oracle, w, r, lanes, pot_tol=POT_TOL_F32, exact_depth=False)
+    for t, dg, do, margin in misses:
+        print(f"[depth miss] {name} lane {t}: gpu {dg} oracle {do} oracle margin {margin:.2e}")
+        assert margin <= MARGIN_AUTO
+    # properties that hold at any size
+    depth = r["depth"].astype(np.int64)
+    assert np.all(r["status"] == 1) and np.all(r["r_row"] <= w.tol)
+    assert r["stats"]["slots"] == depth.sum() and r["cycles"] == depth.max()
+    np.testing.assert_array_equal(np.array(r["stats"]["widths"]), oracle.survivor_widths(depth))
+
+
+def test_full_size_registration_properties(oracle):
+    # one oracle lane would take ~15 core-minutes here: check what can be computed one by one
+    w = wl.make("registration")
+    W, n, m, d = w.shape
+    r = run_gpu(w, mode="active")
+    depth = r["depth"].astype(np.int64)
+    assert np.all(r["status"] == 1) and np.all(r["r_row"] <= w.tol) and np.all(depth > 50)
+    assert r["stats"]["slots"] == depth.sum() and r["cycles"] == depth.max()
+    np.testing.assert_array_equal(np.array(r["stats"]["widths"]), oracle.survivor_widths(depth))
+    for t in (0, 31):
+        # the achieved two-sided residual of the emitted state, evaluated by the oracle in float64
+        rr, rc = oracle.residuals(w.x[t], w.y[t], w.a[t], w.b[t], float(w.eps[t]), r["f"][t], r["g"][t])
+        assert max(rr, rc) <= w.tol * (1 + 5e-3) and abs(rr - r["r_row"][t]) <= 2e-2 * w.tol
+        # the emitted g is the g-leg of the emitted f (Eq. 4): the column marginal is current
+        assert rc <= 1e-5
+        # one more oracle cycle from the emitted state still passes and lowers the row residual
+        C = oracle.cost_matrix(w.x[t], w.y[t])
+        f1 = oracle.f_leg(C, r["g"][t], w.a[t], float(w.eps[t])); g1 = oracle.g_leg(C, f1, w.b[t], float(w.eps[t]))
+        row, col = oracle.marginals(C, f1, g1, float(w.eps[t]))
+        assert np.abs(row - w.a[t]).sum() < rr
+        # and one cycle BACK did not pass: undo is impossible, but the screen value of the state before
+        # the last cycle is bounded below by the monotone decay: r(l-1) >= r(l)
+        assert rr > 0.5 * w.tol            # the lane stopped at its first passing audit, not long after
