@@ -40,8 +40,9 @@ def peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
         p = json.load(open(path))
-        return {"hbm_gbs": p["hbm_gbs"], "sm_max_mhz": p.get("sm_max_mhz", 1965.0), "source": "measured"}
-    return {"hbm_gbs": 6650.0, "sm_max_mhz": 1965.0, "source": "fallback"}
+        return {"hbm_gbs": p["hbm_gbs"], "sm_max_mhz": p.get("sm_max_mhz", 1965.0),
+                "bf16_tflops": p.get("bf16_tflops", 1590.0), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "sm_max_mhz": 1965.0, "bf16_tflops": 1590.0, "source": "fallback"}
 
 
 class ClockSampler:
@@ -144,7 +145,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="sensor", choices=["tiny", "sensor", "feature", "registration", "sweep"])
     ap.add_argument("--mode", default="active", choices=["active", "masked", "static"])
-    ap.add_argument("--compute", default="auto", choices=["auto", "f32", "mixed", "f64"])
+    ap.add_argument("--compute", default="auto", choices=["auto", "f32", "mixed", "f64", "tensor"])
     ap.add_argument("--no-controls", action="store_true", help="skip the static / masked control timings")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--kernel-only", action="store_true",
@@ -294,8 +295,19 @@ def main():
         achieved_inst = pairs * inst_per_pair / (k_ms * 1e-3)
         achieved_exp = pairs / (k_ms * 1e-3)
         bound_fp32 = inst_per_pair / lanes > 1.0 / MUFU_LANES
-        line["dtype"] = {"f32": "f32", "mixed": "f64 exponents / f32 exp", "f64": "f64"}[arith]
-        line["roofline"] = {
+        line["dtype"] = {"f32": "f32", "mixed": "f64 exponents / f32 exp", "f64": "f64",
+                         "tensor": "bf16 (f32 accumulate, f32 exp)"}[arith]
+        if arith == "tensor":
+            # the cross term is a dense bf16 contraction: 2*d flops per pair against the measured
+            # cuBLAS bf16 burst throughput (kernel timed alone)
+            tf = 2.0 * d * pairs / (k_ms * 1e-3) / 1e12
+            line["roofline"] = {"bound": "tensor", "kernel": "update_tc_kernel (f-leg, full width)",
+                                "arithmetic": arith, "achieved": tf, "peak": pk["bf16_tflops"], "unit": "TFLOP/s",
+                                "frac": tf / pk["bf16_tflops"], "exp_frac": achieved_exp / mufu_peak,
+                                "ms_per_launch": k_ms, "pairs_per_launch": pairs, "traffic": None,
+                                "peak_source": pk["source"] + " cuBLAS bf16 burst (MEASURED_PEAKS.json)"}
+        else:
+          line["roofline"] = {
             "bound": "alu", "kernel": "update_kernel (f-leg, full width)",
             "arithmetic": arith,
             "binding_unit": ("fp64 pipe" if wide else "fp32 pipe") if bound_fp32 else "special-function unit (ex2)",

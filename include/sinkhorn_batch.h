@@ -55,10 +55,14 @@ typedef enum {
 typedef enum { SKB_F32 = 0, SKB_BF16 = 1 } skb_dtype;           /* storage type of x and y only */
 /* Arithmetic of the pair terms log2 pi_ij and their exponentials. */
 typedef enum {
-    SKB_COMPUTE_AUTO = 0,  /* F32, or MIXED when some lane's cost/eps range is beyond fp32     */
+    SKB_COMPUTE_AUTO = 0,  /* F32 (TENSOR where eligible), or MIXED when some lane's cost/eps  */
+                           /* range is beyond fp32                                             */
     SKB_COMPUTE_F32 = 1,   /* fp32 exponents and exponentials                                  */
     SKB_COMPUTE_MIXED = 2, /* float64 exponents (half-rate FP64 pipe), fp32 exponentials       */
-    SKB_COMPUTE_F64 = 3    /* float64 throughout, software exp2: the slow validation arithmetic */
+    SKB_COMPUTE_F64 = 3,   /* float64 throughout, software exp2: the slow validation arithmetic */
+    SKB_COMPUTE_TENSOR = 4 /* bf16 x, y only, d a multiple of 64 up to 512: cross term on the   */
+                           /* tensor cores (fp32 accumulate), fp32 exponentials; what AUTO     */
+                           /* picks for such inputs                                            */
 } skb_compute;
 
 typedef enum {

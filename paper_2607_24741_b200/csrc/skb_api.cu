@@ -23,6 +23,8 @@ struct skb_batch {
     bool finished;
     long long enqueued;    // cycles enqueued so far
     long long launches;    // kernels launched so far
+    bool tensor;           // the tensor-core update kernel is in use
+    alignas(64) unsigned char maps[2 * 128];   // CUtensorMap of x and of y
     std::string err;
 };
 
@@ -43,7 +45,7 @@ static bool config_ok(const skb_config *c, std::string &why)
     if (c->W < 1 || c->n < 1 || c->m < 1 || c->d < 1) { why = "W, n, m, d must be >= 1"; return false; }
     if (c->xy_dtype != SKB_F32 && c->xy_dtype != SKB_BF16) { why = "bad xy_dtype"; return false; }
     if (c->mode < SKB_ACTIVE || c->mode > SKB_STATIC) { why = "bad mode"; return false; }
-    if (c->compute < SKB_COMPUTE_AUTO || c->compute > SKB_COMPUTE_F64) { why = "bad compute type"; return false; }
+    if (c->compute < SKB_COMPUTE_AUTO || c->compute > SKB_COMPUTE_TENSOR) { why = "bad compute type"; return false; }
     if (c->max_iter < 1 || c->audit_every < 1) { why = "max_iter and audit_every must be >= 1"; return false; }
     if (c->cost_form < 0 || c->cost_form > 2) { why = "cost_form must be 0 (automatic), 1 (expanded) or 2 (difference)"; return false; }
     if (c->column_split != 0 && c->column_split != 1 && c->column_split != 4 && c->column_split != 32) {
@@ -53,7 +55,7 @@ static bool config_ok(const skb_config *c, std::string &why)
 }
 
 // Lays the batch's arrays out in the workspace (base may be null: size query only).
-static size_t carve(const skb_config *c, const Variant *var, char *base, Dev *D, size_t *zero_end_out = nullptr)
+static size_t carve(const skb_config *c, const Variant *var, bool tensor, char *base, Dev *D, size_t *zero_end_out = nullptr)
 {
     size_t off = 0;
     auto take = [&](size_t bytes) -> void * {
@@ -88,7 +90,12 @@ static size_t carve(const skb_config *c, const Variant *var, char *base, Dev *D,
     d.ret_scale = (double *)take(W * 8);
     d.hole_list = (int *)take(W * 4); d.fill_list = (int *)take(W * 4);
     d.part_row = (double *)take(W * MAX_PARTS * 8); d.part_col = (double *)take(W * MAX_PARTS * 8);
-    d.xs = take(W * DP * np * ts); d.ys = take(W * DP * mp * ts);
+    d.tensor = tensor ? 1 : 0;
+    if (tensor) {
+        d.xb = take(W * n * (size_t)c->d * 2); d.yb = take(W * m * (size_t)c->d * 2);
+    } else {
+        d.xs = take(W * DP * np * ts); d.ys = take(W * DP * mp * ts);
+    }
     d.ft[0] = take(W * np * ts); d.ft[1] = take(W * np * ts); d.gt = take(W * mp * ts);
     d.fl[0] = take(W * np * ts); d.fl[1] = take(W * np * ts); d.gl = take(W * mp * ts);
     d.sqx = (double *)take(W * np * 8); d.sqy = (double *)take(W * mp * 8);
@@ -104,6 +111,7 @@ static size_t carve(const skb_config *c, const Variant *var, char *base, Dev *D,
 
 static const Variant *variant_for(const skb_config *c, int compute)
 {
+    if (compute == SKB_COMPUTE_TENSOR) compute = SKB_COMPUTE_F32;     // fp32 epilogue, same scratch shapes
     const bool f64 = compute == SKB_COMPUTE_F64 || compute == SKB_COMPUTE_MIXED;
     return choose_variant(c->W, c->n, c->m, c->d, f64, compute == SKB_COMPUTE_MIXED, c->column_split);
 }
@@ -113,9 +121,15 @@ extern "C" size_t sinkhorn_batch_workspace_bytes(const skb_config *cfg)
     std::string why;
     if (!config_ok(cfg, why)) return 0;
     // an automatic batch may end up with float64 coordinates: size for the larger layout
+    if (cfg->compute == SKB_COMPUTE_TENSOR && !tc_eligible(cfg->d, cfg->xy_dtype == SKB_BF16)) return 0;
     const Variant *v = variant_for(cfg, cfg->compute == SKB_COMPUTE_AUTO ? SKB_COMPUTE_MIXED : cfg->compute);
     if (!v) return 0;
-    return carve(cfg, v, nullptr, nullptr);
+    size_t need = carve(cfg, v, cfg->compute == SKB_COMPUTE_TENSOR, nullptr, nullptr);
+    if (cfg->compute == SKB_COMPUTE_AUTO && tc_eligible(cfg->d, cfg->xy_dtype == SKB_BF16)) {
+        const size_t t = carve(cfg, variant_for(cfg, SKB_COMPUTE_F32), true, nullptr, nullptr);
+        if (t > need) need = t;
+    }
+    return need;
 }
 
 static skb_status fail(skb_batch *h, skb_status st, const std::string &msg)
@@ -150,8 +164,12 @@ extern "C" skb_status sinkhorn_batch_create(const void *x, const void *y, const 
         (mx + var_big->rows_per_cta - 1) / var_big->rows_per_cta > MAX_PARTS)
         return fail(nullptr, SKB_ERR_SHAPE, "n or m too large for the residual scratch");
     if (cfg->W > 65535) return fail(nullptr, SKB_ERR_SHAPE, "W must be <= 65535");
+    const bool can_tensor = tc_eligible(cfg->d, cfg->xy_dtype == SKB_BF16);
+    if (cfg->compute == SKB_COMPUTE_TENSOR && !can_tensor)
+        return fail(nullptr, SKB_ERR_SHAPE, "the tensor-core path needs bf16 x, y and d a multiple of 64 with 64 <= d <= 512");
     size_t zero_end = 0;
-    const size_t need = carve(cfg, var_big, nullptr, nullptr, &zero_end);
+    carve(cfg, var_big, false, nullptr, nullptr, &zero_end);
+    const size_t need = sinkhorn_batch_workspace_bytes(cfg);
     if (!cfg->workspace) return fail(nullptr, SKB_ERR_WORKSPACE, "workspace is null");
     if (((uintptr_t)cfg->workspace & 255u) != 0) return fail(nullptr, SKB_ERR_WORKSPACE, "workspace must be 256-byte aligned");
     if (cfg->workspace_bytes < need) {
@@ -164,7 +182,8 @@ extern "C" skb_status sinkhorn_batch_create(const void *x, const void *y, const 
     h->cfg = *cfg; h->var = var; h->stream = (cudaStream_t)cfg->stream;
     h->known_width = cfg->W; h->finished = false; h->enqueued = 0; h->launches = 0; h->h_ctl = nullptr;
     h->ev[0] = h->ev[1] = nullptr;
-    carve(cfg, var, (char *)cfg->workspace, &h->dev);
+    h->tensor = cfg->compute == SKB_COMPUTE_TENSOR;
+    carve(cfg, var, h->tensor, (char *)cfg->workspace, &h->dev);
     h->dev.tol_stop = (double)tol;
     h->dev.tol_screen = cfg->tol_screen > 0.0f ? (double)cfg->tol_screen : (double)tol;
     cudaError_t e;
@@ -198,11 +217,31 @@ extern "C" skb_status sinkhorn_batch_create(const void *x, const void *y, const 
         }
         double radius;
         memcpy(&radius, &h->h_ctl[1].max_radius_bits, sizeof(double));
+        const double ts = h->dev.tol_stop, tsc = h->dev.tol_screen;
         if (radius > MIXED_RADIUS) {
             h->var = var_big;
-            const double ts = h->dev.tol_stop, tsc = h->dev.tol_screen;
-            carve(cfg, var_big, (char *)cfg->workspace, &h->dev);
-            h->dev.tol_stop = ts; h->dev.tol_screen = tsc;
+            carve(cfg, var_big, false, (char *)cfg->workspace, &h->dev);
+        } else if (can_tensor) {
+            h->tensor = true;
+            carve(cfg, var, true, (char *)cfg->workspace, &h->dev);
+        }
+        h->dev.tol_stop = ts; h->dev.tol_screen = tsc;
+    }
+    if (h->tensor) {
+        // the MMA reads the caller's bf16 layout: keep a copy the compaction may permute
+        const size_t W = cfg->W, d = cfg->d;
+        const char *why = nullptr;
+        if ((e = cudaMemcpyAsync(h->dev.xb, x, W * cfg->n * d * 2, cudaMemcpyDeviceToDevice, h->stream)) != cudaSuccess ||
+            (e = cudaMemcpyAsync(h->dev.yb, y, W * cfg->m * d * 2, cudaMemcpyDeviceToDevice, h->stream)) != cudaSuccess) {
+            skb_status st = cuda_fail(nullptr, e, "create");
+            sinkhorn_batch_destroy(h);
+            return st;
+        }
+        if ((why = tc_make_map(h->maps, h->dev.xb, cfg->W, cfg->n, cfg->d)) != nullptr ||
+            (why = tc_make_map(h->maps + 128, h->dev.yb, cfg->W, cfg->m, cfg->d)) != nullptr) {
+            skb_status st = fail(nullptr, SKB_ERR_CUDA, why);
+            sinkhorn_batch_destroy(h);
+            return st;
         }
     }
     launch_prep(h->dev, x, y, a, b, h->stream);
@@ -219,14 +258,20 @@ extern "C" skb_status sinkhorn_batch_create(const void *x, const void *y, const 
 
 // one full cycle: f-leg (+ row screen of the previous state), column check of screen-positive
 // lanes, plan, emit/compact, g-leg
+static void launch_leg(skb_batch *h, int leg, int w)
+{
+    if (h->tensor) launch_update_tc(h->dev, h->maps, leg, w, h->stream);
+    else h->var->launch(h->dev, leg, w, h->stream);
+}
+
 static void enqueue_cycle(skb_batch *h)
 {
     const int w = h->known_width;
-    h->var->launch(h->dev, LEG_F, w, h->stream);
-    h->var->launch(h->dev, LEG_V, w, h->stream);
+    launch_leg(h, LEG_F, w);
+    launch_leg(h, LEG_V, w);
     launch_plan(h->dev, h->stream);
     launch_emit_move(h->dev, w, h->stream);
-    h->var->launch(h->dev, LEG_G, w, h->stream);
+    launch_leg(h, LEG_G, w);
     h->enqueued++;
     h->launches += 5;
 }
@@ -234,6 +279,7 @@ static void enqueue_cycle(skb_batch *h)
 static skb_status absorb(skb_batch *h, const Ctl &c)
 {
     if (c.error & ERR_VALUE) return fail(h, SKB_ERR_VALUE, "inputs rejected on the device: weights and eps must be positive, coordinates finite");
+    if (c.error & ERR_WAIT) return fail(h, SKB_ERR_CUDA, "a bounded wait inside a kernel ran out (pipeline barrier never completed)");
     if (c.error) return fail(h, SKB_ERR_CUDA, "a kernel reported an internal error");
     if (h->cfg.mode == SKB_ACTIVE && c.n_phys >= 0 && c.n_phys < h->known_width) h->known_width = c.n_phys;
     if (c.done) h->finished = true;
@@ -357,7 +403,7 @@ extern "C" skb_status sinkhorn_batch_stats(skb_batch *h, long long *slots, int *
 extern "C" skb_status sinkhorn_batch_arithmetic(skb_batch *h, int *compute)
 {
     if (!h || !compute) return SKB_ERR_NULL;
-    *compute = !h->var->f64 ? SKB_COMPUTE_F32 : (h->var->xf ? SKB_COMPUTE_MIXED : SKB_COMPUTE_F64);
+    *compute = h->tensor ? SKB_COMPUTE_TENSOR : (!h->var->f64 ? SKB_COMPUTE_F32 : (h->var->xf ? SKB_COMPUTE_MIXED : SKB_COMPUTE_F64));
     return SKB_OK;
 }
 
@@ -376,9 +422,9 @@ extern "C" skb_status sinkhorn_batch_profile_update(skb_batch *h, int leg, int r
     cudaError_t e;
     if ((e = cudaEventCreate(&a)) != cudaSuccess) return cuda_fail(h, e, "profile");
     if ((e = cudaEventCreate(&b)) != cudaSuccess) { cudaEventDestroy(a); return cuda_fail(h, e, "profile"); }
-    h->var->launch(h->dev, leg, h->known_width, h->stream);          // warm-up
+    launch_leg(h, leg, h->known_width);          // warm-up
     cudaEventRecord(a, h->stream);
-    for (int i = 0; i < reps; ++i) h->var->launch(h->dev, leg, h->known_width, h->stream);
+    for (int i = 0; i < reps; ++i) launch_leg(h, leg, h->known_width);
     cudaEventRecord(b, h->stream);
     e = cudaEventSynchronize(b);
     float ms = 0.f;

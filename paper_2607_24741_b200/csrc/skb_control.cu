@@ -87,11 +87,12 @@ __global__ void prep_kernel(const Dev P, const void *xin, const void *yin, const
     double *sq = side ? P.sqy : P.sqx, *lw = side ? P.lb2 : P.la2, *wt = side ? P.wb : P.wa;
     T hi, lo = T(0);
     if (i >= npts) {                                  // padding points
-        for (int k = 0; k < P.DP; ++k) crd[(size_t)k * pp + i] = T(0);
+        if (!P.tensor) for (int k = 0; k < P.DP; ++k) crd[(size_t)k * pp + i] = T(0);
         hi = T(NEG_BIG);
         sq[o] = 0.0; lw[o] = 0.0; wt[o] = 0.0;
     } else {
-        const double sc = sqrt(form == FORM_DOT ? 2.0 * s : s);
+        // tensor-core path: raw coordinates feed the MMA, the scale 2s is applied to its result
+        const double sc = P.tensor ? sqrt(2.0 * s) : sqrt(form == FORM_DOT ? 2.0 * s : s);
         const size_t ibase = ((size_t)slot * npts + i) * P.d;
         const double *cen = P.center + (size_t)slot * P.DP;
         double nrm = 0.0;
@@ -101,9 +102,10 @@ __global__ void prep_kernel(const Dev P, const void *xin, const void *yin, const
             if (k < P.d) {
                 const float raw = load_raw(P, side ? yin : xin, ibase + k);
                 ok = ok && isfinite(raw);
-                v = (T)(sc * ((double)raw - cen[k]));
+                v = P.tensor ? (T)0 : (T)(sc * ((double)raw - cen[k]));
+                if (P.tensor) nrm += (sc * (double)raw) * (sc * (double)raw);
             }
-            crd[(size_t)k * pp + i] = v;
+            if (!P.tensor) crd[(size_t)k * pp + i] = v;
             nrm += (double)v * (double)v;
         }
         nrm = form == FORM_DOT ? 0.5 * nrm : 0.0;
@@ -299,8 +301,13 @@ __global__ void __launch_bounds__(256) emit_move_kernel(const Dev P)
         for (size_t v = tid; v < nv; v += nth) d4[v] = s4[v];
     };
     const int np_ = ep ^ 1;   // buffer that holds the survivors' current row potentials
-    copy(P.xs, (size_t)P.DP * P.np * sizeof(T));
-    copy(P.ys, (size_t)P.DP * P.mp * sizeof(T));
+    if (P.tensor) {
+        copy(P.xb, (size_t)P.n * P.d * 2);
+        copy(P.yb, (size_t)P.m * P.d * 2);
+    } else {
+        copy(P.xs, (size_t)P.DP * P.np * sizeof(T));
+        copy(P.ys, (size_t)P.DP * P.mp * sizeof(T));
+    }
     copy(P.sqx, (size_t)P.np * 8); copy(P.sqy, (size_t)P.mp * 8);
     copy(P.la2, (size_t)P.np * 8); copy(P.lb2, (size_t)P.mp * 8);
     copy(P.wa, (size_t)P.np * 8); copy(P.wb, (size_t)P.mp * 8);

@@ -48,11 +48,12 @@ struct Ctl {
 
 struct Dev {
     int W, n, m, d, np, mp, DP;
-    int mode, max_iter, audit_every, xy_bf16, compute_f64, cost_form;
+    int mode, max_iter, audit_every, xy_bf16, compute_f64, cost_form, tensor;
     double form_threshold;    // scaled squared radius above which a lane uses the difference form
     double tol_screen, tol_stop;
     // slabs by slot
-    void *xs, *ys;            // [W][DP][np|mp]   T
+    void *xs, *ys;            // [W][DP][np|mp]   T   (SIMT kernels)
+    void *xb, *yb;            // [W][n|m][d] bf16, the caller's layout (tensor-core kernel)
     void *ft[2];              // [W][np]          T
     void *gt;                 // [W][mp]          T
     void *fl[2], *gl;         // low parts of the potentials (difference form only)

@@ -374,12 +374,12 @@ __device__ __forceinline__ void stream_f64(double *sm, const double *colc, const
 // Float64 epilogue of a CTA's RB rows (one thread per row) and the fused residual reduction.
 // row_m / row_s hold, per CTA-local row, the integer-valued maximum and the sum of
 // 2^(arg - max) over ALL columns; row_h the fp32 shift a difference-form row carried.
-template <typename T, int RB>
+template <typename T, int RB, int THREADS = UPD_THREADS>
 __device__ __forceinline__ void finish_rows(const Dev &P, const Ctl &c, const int leg, const int slot,
                                             const int form, const float *row_m, const double *row_s,
                                             const float *row_h, double *red, int *is_last)
 {
-    constexpr int NWARP = UPD_THREADS / 32;
+    constexpr int NWARP = THREADS / 32;
     const bool rows_x = (leg == LEG_F);
     const int nrows = rows_x ? P.n : P.m, rp = rows_x ? P.np : P.mp;
     const double *prow = (rows_x ? P.phi[c.parity] : P.gam) + (size_t)slot * rp;
@@ -387,7 +387,7 @@ __device__ __forceinline__ void finish_rows(const Dev &P, const Ctl &c, const in
     const bool frozen = (P.mode == MODE_MASKED) && P.state[slot] != 0;
     const bool writes = !frozen && leg != LEG_V;
     double term_sum = 0.0;
-    for (int lr = tid; lr < RB; lr += UPD_THREADS) {
+    for (int lr = tid; lr < RB; lr += THREADS) {
         const int i = blockIdx.x * RB + lr;
         if (i >= nrows) continue;
         const size_t o = (size_t)slot * rp + i;
