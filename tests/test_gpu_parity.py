@@ -293,3 +293,46 @@ def test_full_size_registration_properties(oracle):
         # and one cycle BACK did not pass: undo is impossible, but the screen value of the state before
         # the last cycle is bounded below by the monotone decay: r(l-1) >= r(l)
         assert rr > 0.5 * w.tol            # the lane stopped at its first passing audit, not long after
+
+
+# ---- tensor-core cross term (bf16 inputs, d a multiple of 64) ------------------------------------
+POT_TOL_BF16 = 5e-3     # acceptance bar for bf16 inputs; measured errors are ~1e-6
+
+
+@pytest.mark.parametrize("kw", [dict(W=3, n=200, m=333, d=64), dict(W=2, n=256, d=128), dict(W=2, n=129, m=640, d=512)])
+def test_tensor_core_path_against_oracle(oracle, kw):
+    w = wl.make("feature", **kw)
+    W = w.shape[0]
+    r = run_gpu(w, mode="active", compute="tensor")
+    misses = check_against_oracle(oracle, w, r, range(W), pot_tol=POT_TOL_F32, exact_depth=False)
+    for t, dg, do, margin in misses:
+        print(f"[depth miss] tensor {kw} lane {t}: gpu {dg} oracle {do} oracle margin {margin:.2e}")
+        assert margin <= MARGIN_F32
+    check_accounting(oracle, r, W, "active")
+    # what AUTO picks for such inputs is this very path: bit-identical results
+    ra = run_gpu(w, mode="active")
+    np.testing.assert_array_equal(ra["f"], r["f"]); np.testing.assert_array_equal(ra["depth"], r["depth"])
+
+
+def test_tensor_core_modes_and_compaction(oracle):
+    w = wl.make("feature", W=6, n=256, d=128)
+    ra = run_gpu(w, mode="active", compute="tensor")
+    rm = run_gpu(w, mode="masked", compute="tensor")
+    rs = run_gpu(w, mode="static", compute="tensor")
+    np.testing.assert_array_equal(ra["depth"], rm["depth"]); np.testing.assert_array_equal(ra["depth"], rs["depth"])
+    np.testing.assert_array_equal(ra["f"], rm["f"]); np.testing.assert_array_equal(ra["g"], rm["g"])
+    assert len(set(ra["depth"].tolist())) > 1                    # lanes really leave at different depths
+    check_accounting(oracle, ra, 6, "active"); check_accounting(oracle, rs, 6, "static")
+    ref = oracle.solve_batch(w.x, w.y, w.a, w.b, w.eps, w.tol, max_iter=w.max_iter)
+    np.testing.assert_array_equal(ra["depth"], ref.depth)
+    assert pot_err(ra["f"], ra["g"], ref.f, ref.g, w.eps.astype(np.float64)).max() <= POT_TOL_F32
+
+
+def test_tensor_core_request_on_ineligible_input_is_refused():
+    import torch
+    from paper_2607_24741_b200 import binding as B
+    w = wl.make("tiny")
+    t = lambda v: torch.from_numpy(v).to("cuda:0")
+    with pytest.raises(B.SkbError) as e:
+        B.SinkhornBatch(t(w.x), t(w.y), t(w.a), t(w.b), t(w.eps), w.tol, compute="tensor")
+    assert e.value.code == 2
