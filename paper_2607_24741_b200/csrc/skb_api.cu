@@ -269,7 +269,7 @@ static void enqueue_cycle(skb_batch *h)
     const int w = h->known_width;
     launch_leg(h, LEG_F, w);
     launch_leg(h, LEG_V, w);
-    launch_plan(h->dev, h->stream);
+    launch_plan(h->dev, w, h->stream);
     launch_emit_move(h->dev, w, h->stream);
     launch_leg(h, LEG_G, w);
     h->enqueued++;

@@ -127,7 +127,7 @@ __global__ void prep_kernel(const Dev P, const void *xin, const void *yin, const
 }
 
 // ---------------------------------------------------------------- plan
-constexpr int PLAN_THREADS = 1024;
+constexpr int PLAN_THREADS = 1024;   // upper bound; the launch sizes the block to the width
 
 // exclusive prefix sums of up to three 0/1 flags over the block, by warp ballot + popc
 __device__ __forceinline__ void block_scan3(int f0, int f1, int f2, int (&ex)[3], int (&tot)[3], int (*wsum)[3])
@@ -141,7 +141,8 @@ __device__ __forceinline__ void block_scan3(int f0, int f1, int f2, int (&ex)[3]
     if (lane == 0) { wsum[warp][0] = __popc(b0); wsum[warp][1] = __popc(b1); wsum[warp][2] = __popc(b2); }
     __syncthreads();
     int run[3] = {0, 0, 0};
-    for (int w = 0; w < PLAN_THREADS / 32; ++w) {
+    const int nwarp = blockDim.x >> 5;
+    for (int w = 0; w < nwarp; ++w) {
         if (w == warp) { ex[0] += run[0]; ex[1] += run[1]; ex[2] += run[2]; }
         run[0] += wsum[w][0]; run[1] += wsum[w][1]; run[2] += wsum[w][2];
     }
@@ -152,14 +153,14 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_kernel(const Dev P)
 {
     __shared__ int wsum[PLAN_THREADS / 32][3];
     Ctl c = *P.ctl;
-    const int tid = threadIdx.x;
+    const int tid = threadIdx.x, NT = blockDim.x;
     if (c.done) { if (tid == 0) P.ctl->n_retire = 0; return; }
     const int k = c.cycle;                           // cycles completed by the audited state
     const int A = c.n_phys;
     const bool limit = k >= P.max_iter;
 
     if (P.mode == MODE_STATIC && c.static_final) {   // emit every lane at the common boundary
-        for (int s = tid; s < P.W; s += PLAN_THREADS) {
+        for (int s = tid; s < P.W; s += NT) {
             P.ret_slot[s] = s; P.ret_lane[s] = s; P.ret_src[s] = -1; P.ret_scale[s] = P.scale[s];
             P.res_row[s] = P.rrow[s]; P.res_col[s] = P.rcol[s];
             if (P.nonfinite[s]) P.status[s] = LANE_NONFINITE;
@@ -185,7 +186,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_kernel(const Dev P)
 
     // pass 1: count retirees and screen-positive lanes
     int cnt = 0, nflag = 0;
-    for (int s = tid; s < A; s += PLAN_THREADS) {
+    for (int s = tid; s < A; s += NT) {
         int r, st; decide(s, r, st); cnt += r;
         nflag += (P.flag[s] != 0);
     }
@@ -196,13 +197,14 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_kernel(const Dev P)
     if ((tid & 31) == 0) { wsum[tid >> 5][0] = cnt; wsum[tid >> 5][1] = nflag; }
     __syncthreads();
     int nret = 0, nflagged = 0;
-    for (int w = 0; w < PLAN_THREADS / 32; ++w) { nret += wsum[w][0]; nflagged += wsum[w][1]; }
+    for (int w = 0; w < (NT >> 5); ++w) { nret += wsum[w][0]; nflagged += wsum[w][1]; }
     __syncthreads();
     const int Anew = (P.mode == MODE_ACTIVE) ? A - nret : A;
 
-    // pass 2: ordered lists (retirees, holes below Anew, survivors at or above Anew)
+    // pass 2: ordered lists (retirees, holes below Anew, survivors at or above Anew);
+    // most audits retire nobody and skip it
     int base[3] = {0, 0, 0};
-    for (int s0 = 0; s0 < A; s0 += PLAN_THREADS) {
+    for (int s0 = 0; s0 < (nret > 0 ? A : 0); s0 += NT) {
         const int s = s0 + tid;
         int r, st; decide(s, r, st);
         const int hole = (P.mode == MODE_ACTIVE) && r && s < Anew;
@@ -231,12 +233,12 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_kernel(const Dev P)
     __syncthreads();
     const int nholes = base[1];
     // resolve each hole's source, then move the per-slot scalars
-    for (int r = tid; r < nret; r += PLAN_THREADS) {
+    for (int r = tid; r < nret; r += NT) {
         const int code = P.ret_src[r];
         if (code <= -2) P.ret_src[r] = P.fill_list[-(code + 2)];
     }
     __syncthreads();
-    for (int h = tid; h < nholes; h += PLAN_THREADS) {
+    for (int h = tid; h < nholes; h += NT) {
         const int dst = P.hole_list[h], src = P.fill_list[h];
         P.lane_id[dst] = P.lane_id[src];
         P.scale[dst] = P.scale[src];
@@ -274,11 +276,18 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_kernel(const Dev P)
 
 // ---------------------------------------------------------------- emit + move
 template <typename T>
+__device__ __forceinline__ void emit_move_one(const Dev &P, const Ctl &c, const int r);
+
+template <typename T>
 __global__ void __launch_bounds__(256) emit_move_kernel(const Dev P)
 {
     const Ctl c = *P.ctl;
-    const int r = blockIdx.y;
-    if (r >= c.n_retire) return;
+    for (int r = blockIdx.y; r < c.n_retire; r += gridDim.y) emit_move_one<T>(P, c, r);
+}
+
+template <typename T>
+__device__ __forceinline__ void emit_move_one(const Dev &P, const Ctl &c, const int r)
+{
     const int slot = P.ret_slot[r], lane = P.ret_lane[r], src = P.ret_src[r];
     const double inv_s = 1.0 / P.ret_scale[r];
     const int tid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
@@ -366,14 +375,20 @@ void launch_prep(const Dev &P, const void *x, const void *y, const float *a, con
     if (P.compute_f64) prep_kernel<double><<<grid, 128, 0, st>>>(P, x, y, a, b);
     else prep_kernel<float><<<grid, 128, 0, st>>>(P, x, y, a, b);
 }
-void launch_plan(const Dev &P, cudaStream_t st) { plan_kernel<<<1, PLAN_THREADS, 0, st>>>(P); }
+void launch_plan(const Dev &P, int width, cudaStream_t st)
+{
+    int nt = (width + 31) / 32 * 32;
+    if (P.mode == MODE_STATIC) nt = (P.W + 31) / 32 * 32;
+    nt = nt < 128 ? 128 : (nt > PLAN_THREADS ? PLAN_THREADS : nt);
+    plan_kernel<<<1, nt, 0, st>>>(P);
+}
 void launch_emit_move(const Dev &P, int width, cudaStream_t st)
 {
     if (width < 1) width = 1;
     const size_t bytes = (size_t)P.DP * (P.np + P.mp) * (P.compute_f64 ? 8 : 4);
     int gx = (int)(bytes / (256 * 16 * 4)) + 1;
     if (gx > 64) gx = 64;
-    dim3 grid(gx, width);
+    dim3 grid(gx, width > 128 ? 128 : width);
     if (P.compute_f64) emit_move_kernel<double><<<grid, 256, 0, st>>>(P);
     else emit_move_kernel<float><<<grid, 256, 0, st>>>(P);
 }

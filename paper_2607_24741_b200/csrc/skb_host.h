@@ -19,7 +19,7 @@ int padded_dim(int d);
 
 void launch_lane_stats(const Dev &P, const void *x, const void *y, const float *eps, double *max_radius, cudaStream_t st);
 void launch_prep(const Dev &P, const void *x, const void *y, const float *a, const float *b, cudaStream_t st);
-void launch_plan(const Dev &P, cudaStream_t st);
+void launch_plan(const Dev &P, int width, cudaStream_t st);
 // tensor-core update kernel (bf16 inputs, d a multiple of 64 up to 512)
 bool tc_eligible(int d, bool bf16);
 const char *tc_make_map(void *out_map, void *base, int W, int npts, int d);
