@@ -12,7 +12,8 @@
 //              fma with the column term, online logsumexp entirely in registers (no shuffles)
 //   warp 4     producer: one lane issues TMA loads (3-D tensor maps over [lane, point, d],
 //              128-byte swizzle, out-of-range points read as zero): the row block once
-//              (d/64 chunks of 16 KB), then column chunks through a 4-stage ring
+//              (d/64 chunks of 16 KB, riding on the first tile's barriers), and column
+//              chunks through a ring of 2 (d <= 256: two CTAs per SM) or 4 stages
 //   warp 5     allocates 256 TMEM columns (two 128-column accumulators); one lane issues the
 //              MMAs (4 x K=16 per 64-wide chunk) and commits to the ring's empty barriers and
 //              to the accumulator-full barrier, so the next tile's MMAs overlap this tile's
@@ -29,7 +30,7 @@
 namespace skb {
 
 constexpr int TC_THREADS = 192;
-constexpr int TC_STAGES = 4;
+constexpr int TC_MAX_STAGES = 4;
 constexpr int TC_BM = 128, TC_BN = 128, TC_BK = 64;
 constexpr uint32_t TC_CHUNK = TC_BM * TC_BK * 2;          // 16 KB: 128 points x 64 bf16
 constexpr long long TC_WAIT_CLOCKS = 2000000000LL;        // ~1 s
@@ -105,11 +106,12 @@ __device__ __forceinline__ uint64_t tc_desc(uint32_t saddr)
 // instruction descriptor: D fp32, A and B bf16, both K-major, M = 128, N = 128
 constexpr uint32_t TC_IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(TC_BN >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
 
+template <int TC_STAGES>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 update_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUtensorMap tmy, const Dev P, const int leg)
 {
     extern __shared__ __align__(1024) unsigned char smem_tc[];
-    __shared__ __align__(8) unsigned long long bars[2 * TC_STAGES + 5];
+    __shared__ __align__(8) unsigned long long bars[2 * TC_MAX_STAGES + 5];
     __shared__ uint32_t tmem_holder;
     __shared__ int abort_flag;
     __shared__ float gts[2][TC_BN];
@@ -168,14 +170,15 @@ update_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant_
     if (warp == 4) {
         // ---------------- producer
         if (lane == 0) {
-            mbar_expect_tx(b_a, (uint32_t)nkc * TC_CHUNK);
-            for (int kc = 0; kc < nkc; ++kc) tma_load_3d(sA + kc * TC_CHUNK, tm_row, kc * TC_BK, i0, slot, b_a);
+            // the row block rides on the first tile's ring barriers, chunk by chunk, so the first
+            // MMAs start as soon as one chunk of each operand has landed
             int it = 0;
             for (int t = 0; t < ntiles && !*ab; ++t) {
                 for (int kc = 0; kc < nkc; ++kc, ++it) {
                     const int s = it % TC_STAGES;
                     if (it >= TC_STAGES && !mbar_wait(b_empty + 8 * s, ((it / TC_STAGES) - 1) & 1, ab)) break;
-                    mbar_expect_tx(b_full + 8 * s, TC_CHUNK);
+                    mbar_expect_tx(b_full + 8 * s, t == 0 ? 2 * TC_CHUNK : TC_CHUNK);
+                    if (t == 0) tma_load_3d(sA + kc * TC_CHUNK, tm_row, kc * TC_BK, i0, slot, b_full + 8 * s);
                     tma_load_3d(sB + s * TC_CHUNK, tm_col, kc * TC_BK, t * TC_BN, slot, b_full + 8 * s);
                 }
             }
@@ -183,7 +186,7 @@ update_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant_
     } else if (warp == 5) {
         // ---------------- MMA issuer
         if (lane == 0) {
-            bool ok = mbar_wait(b_a, 0, ab);
+            bool ok = true;
             int it = 0;
             for (int t = 0; t < ntiles && ok; ++t) {
                 const int buf = t & 1;
@@ -274,7 +277,10 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
 
 bool tc_eligible(int d, bool bf16) { return bf16 && d >= 64 && d <= 512 && d % 64 == 0; }
 
-size_t tc_smem_bytes(int d) { return (size_t)(d / TC_BK + TC_STAGES) * TC_CHUNK + 1024; }
+// two ring stages when that lets two CTAs share an SM (d <= 256: the second CTA's MMAs cover
+// this CTA's prologue and epilogue), four otherwise
+static int tc_stages(int d) { return d <= 256 ? 2 : 4; }
+size_t tc_smem_bytes(int d) { return (size_t)(d / TC_BK + tc_stages(d)) * TC_CHUNK + 1024; }
 
 // Builds the [lane, point, d] bf16 tensor map of one operand array.  Returns a CUDA error string or null.
 const char *tc_make_map(void *out_map, void *base, int W, int npts, int d)
@@ -302,13 +308,15 @@ void launch_update_tc(const Dev &P, const void *maps, int leg, int width, cudaSt
     static bool attr_set = false;
     const size_t smem = tc_smem_bytes(P.d);
     if (!attr_set) {
-        cudaFuncSetAttribute(update_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc_smem_bytes(512));
+        cudaFuncSetAttribute(update_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc_smem_bytes(256));
+        cudaFuncSetAttribute(update_tc_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc_smem_bytes(512));
         attr_set = true;
     }
     const CUtensorMap *tm = reinterpret_cast<const CUtensorMap *>(maps);
     const int nrows = (leg == LEG_F) ? P.n : P.m;
     dim3 grid((nrows + TC_BM - 1) / TC_BM, width < 1 ? 1 : width);
-    update_tc_kernel<<<grid, TC_THREADS, smem, st>>>(tm[0], tm[1], P, leg);
+    if (tc_stages(P.d) == 2) update_tc_kernel<2><<<grid, TC_THREADS, smem, st>>>(tm[0], tm[1], P, leg);
+    else update_tc_kernel<4><<<grid, TC_THREADS, smem, st>>>(tm[0], tm[1], P, leg);
 }
 
 }  // namespace skb
