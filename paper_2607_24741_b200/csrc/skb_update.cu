@@ -82,7 +82,9 @@ const Variant *choose_variant(int W, int n, int m, int d, bool f64, bool fast_ex
         const double util_n = (double)n / ((double)((n + rb - 1) / rb) * rb);
         const double util_m = (double)m / ((double)((m + rb - 1) / rb) * rb);
         const double fill = ctas >= 592 ? 1.0 : (double)ctas / 592.0;
-        const double score = (util_n < util_m ? util_n : util_m) * fill * (c == 32 ? 0.6 : 1.0);
+        // a whole lane per CTA (c == 1) is marginally faster at full width but leaves the narrow tail of
+        // an active batch to one CTA per lane, so it only wins when the 4-way split would idle rows
+        const double score = (util_n < util_m ? util_n : util_m) * fill * (c == 32 ? 0.6 : (c == 1 ? 0.85 : 1.0));
         if (score > best + 1e-9) { best = score; cs = c; }
     }
     if (force_cs == 1 || force_cs == 4 || force_cs == 32) cs = force_cs;

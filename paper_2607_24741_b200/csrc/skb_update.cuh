@@ -54,8 +54,11 @@ template <int DP> struct Tune<float, DP> {
     static constexpr int R = DP <= 8 ? 4 : (DP == 16 ? SKB_F32_R16 : 2);
     static constexpr int CW = DP <= 8 ? 8 : (DP == 16 ? SKB_F32_CW16 : 4);
 };
+#ifndef SKB_F64_R
+#define SKB_F64_R 2
+#endif
 template <int DP> struct Tune<double, DP> {
-    static constexpr int R = DP <= 8 ? 4 : 2;
+    static constexpr int R = DP <= 8 ? SKB_F64_R : 2;
     static constexpr int CW = 4;
 };
 
@@ -90,6 +93,12 @@ __device__ __forceinline__ u64 sub2(u64 a, u64 b)
     u64 d;
     asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
     return d;
+}
+// order-preserving 32-bit key of a float64 (its high word, sign-magnitude -> two's complement)
+__device__ __forceinline__ int dkey(double v)
+{
+    const int hi = __double2hiint(v);
+    return hi ^ ((hi >> 31) & 0x7fffffff);
 }
 // 2^k for an integer-valued k <= 0 (exact; flushes to 0 below the normal range)
 __device__ __forceinline__ float pow2i(float k)
@@ -294,8 +303,9 @@ __device__ __forceinline__ void stream_f64(double *sm, const double *colc, const
 
     float ts[R];
     double md[R];
+    int kmax[R];
 #pragma unroll
-    for (int r = 0; r < R; ++r) { mx[r] = NEG_BIG; md[r] = (double)NEG_BIG; ts[r] = 0.f; sd[r] = 0.0; }
+    for (int r = 0; r < R; ++r) { mx[r] = NEG_BIG; md[r] = (double)NEG_BIG; kmax[r] = dkey(md[r]); ts[r] = 0.f; sd[r] = 0.0; }
 
     const int ntiles = (ncols + TJ - 1) / TJ;
     load_tile<double, DP, TJ, NR>(sm, colc, colt, colt, cp, 0, tid);
@@ -332,23 +342,27 @@ __device__ __forceinline__ void stream_f64(double *sm, const double *colc, const
                     acc[r][3] = fma(xr[r][k], y1.y, acc[r][3]);
                 }
             }
-            double mt[R];
+            // the maximum only steers the rescale, so compare monotone integer keys of the high
+            // words (ALU pipe) instead of float64 values (FP64 pipe)
+            int kt[R];
             bool grow = false;
 #pragma unroll
             for (int r = 0; r < R; ++r) {
-                mt[r] = fmax(fmax(acc[r][0], acc[r][1]), fmax(acc[r][2], acc[r][3]));
-                grow = grow || (mt[r] > md[r] + 8.0);
+                kt[r] = max(max(dkey(acc[r][0]), dkey(acc[r][1])), max(dkey(acc[r][2]), dkey(acc[r][3])));
+                grow = grow || (kt[r] > kmax[r]);
             }
             if (grow) {
 #pragma unroll
                 for (int r = 0; r < R; ++r) {
-                    if (mt[r] > md[r] + 8.0) {
-                        const float mn = ceilf((float)mt[r]) + 1.0f;       // +1: the fp32 copy may round down
+                    if (kt[r] > kmax[r]) {
+                        const double mt = fmax(fmax(acc[r][0], acc[r][1]), fmax(acc[r][2], acc[r][3]));
+                        const float mn = ceilf((float)mt) + 1.0f;          // +1: the fp32 copy may round down
                         const float fac = pow2i(mx[r] - mn);
                         ts[r] *= fac;
                         sd[r] *= (double)fac;
                         mx[r] = mn;
                         md[r] = (double)mn;
+                        kmax[r] = dkey(md[r] + 7.0);                       // rescale once a term would exceed 2^7
                     }
                 }
             }
