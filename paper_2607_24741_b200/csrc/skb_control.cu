@@ -152,6 +152,7 @@ __device__ __forceinline__ void block_scan3(int f0, int f1, int f2, int (&ex)[3]
 __global__ void __launch_bounds__(PLAN_THREADS) plan_kernel(const Dev P)
 {
     __shared__ int wsum[PLAN_THREADS / 32][3];
+    pdl_enter();
     Ctl c = *P.ctl;
     const int tid = threadIdx.x, NT = blockDim.x;
     if (c.done) { if (tid == 0) P.ctl->n_retire = 0; return; }
@@ -281,6 +282,7 @@ __device__ __forceinline__ void emit_move_one(const Dev &P, const Ctl &c, const 
 template <typename T>
 __global__ void __launch_bounds__(256) emit_move_kernel(const Dev P)
 {
+    pdl_enter();
     const Ctl c = *P.ctl;
     for (int r = blockIdx.y; r < c.n_retire; r += gridDim.y) emit_move_one<T>(P, c, r);
 }
@@ -380,7 +382,7 @@ void launch_plan(const Dev &P, int width, cudaStream_t st)
     int nt = (width + 31) / 32 * 32;
     if (P.mode == MODE_STATIC) nt = (P.W + 31) / 32 * 32;
     nt = nt < 128 ? 128 : (nt > PLAN_THREADS ? PLAN_THREADS : nt);
-    plan_kernel<<<1, nt, 0, st>>>(P);
+    launch_pdl(plan_kernel, dim3(1), dim3(nt), 0, st, P);
 }
 void launch_emit_move(const Dev &P, int width, cudaStream_t st)
 {
@@ -389,8 +391,8 @@ void launch_emit_move(const Dev &P, int width, cudaStream_t st)
     int gx = (int)(bytes / (256 * 16 * 4)) + 1;
     if (gx > 64) gx = 64;
     dim3 grid(gx, width > 128 ? 128 : width);
-    if (P.compute_f64) emit_move_kernel<double><<<grid, 256, 0, st>>>(P);
-    else emit_move_kernel<float><<<grid, 256, 0, st>>>(P);
+    if (P.compute_f64) launch_pdl(emit_move_kernel<double>, grid, dim3(256), 0, st, P);
+    else launch_pdl(emit_move_kernel<float>, grid, dim3(256), 0, st, P);
 }
 void launch_gather(const Dev &P, void *f, void *g, bool f64, cudaStream_t st)
 {

@@ -95,6 +95,15 @@ __device__ __forceinline__ float ex2_fast(float x)
 __device__ __forceinline__ float ex2_t(float x) { return ex2_fast(x); }
 __device__ __forceinline__ double ex2_t(double x) { return exp2(x); }
 
+// Programmatic dependent launch: wait until the kernels this launch depends on have completed
+// and their writes are visible, then let the NEXT kernel in the stream start launching (it
+// blocks at its own wait), so launch latency overlaps execution.  A no-op for plain launches.
+__device__ __forceinline__ void pdl_enter()
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 __device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src)
 {
     unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);

@@ -5,6 +5,19 @@
 
 namespace skb {
 
+// Launch with programmatic stream serialization allowed (the kernel must call pdl_enter()).
+template <typename... KArgs, typename... Args>
+inline void launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+
 // Update-kernel variant: compute type, padded dimension, rows per thread, column split.
 struct Variant {
     int f64, xf, DP, R, CS;   // xf: float64 arguments with fp32 special-function exponentials

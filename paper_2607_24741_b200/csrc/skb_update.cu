@@ -18,7 +18,7 @@ static void launch_update(const Dev &P, int leg, int width, cudaStream_t st)
     const int rb = (UPD_THREADS / 32) * Tune<T, DP>::R * (32 / CS);
     const int nrows = (leg == LEG_F) ? P.n : P.m;
     dim3 grid((nrows + rb - 1) / rb, width < 1 ? 1 : width);
-    update_kernel<T, DP, CS, XF><<<grid, UPD_THREADS, smem, st>>>(P, leg);
+    launch_pdl(update_kernel<T, DP, CS, XF>, grid, dim3(UPD_THREADS), smem, st, P, leg);
 }
 
 #define SKB_V(T, F64, XF, DP, CS) \
@@ -42,7 +42,7 @@ static void launch_bigd(const Dev &P, int leg, int width, cudaStream_t st)
     }
     const int nrows = (leg == LEG_F) ? P.n : P.m;
     dim3 grid((nrows + BIGD_RB - 1) / BIGD_RB, width < 1 ? 1 : width);
-    update_bigd_kernel<T, XF><<<grid, UPD_THREADS, smem, st>>>(P, leg);
+    launch_pdl(update_bigd_kernel<T, XF>, grid, dim3(UPD_THREADS), smem, st, P, leg);
 }
 
 // DP = 0 marks the large-d kernels: the padded dimension is d rounded up to the chunk size

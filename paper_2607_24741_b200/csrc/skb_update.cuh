@@ -492,6 +492,7 @@ __global__ void __launch_bounds__(UPD_THREADS) update_kernel(const Dev P, const 
     __shared__ double red[NWARP];
     __shared__ int is_last;
 
+    pdl_enter();
     const Ctl c = *P.ctl;
     if (c.done) return;
     const int slot = blockIdx.y;

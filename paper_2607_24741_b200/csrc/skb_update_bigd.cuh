@@ -41,6 +41,7 @@ __global__ void __launch_bounds__(UPD_THREADS) update_bigd_kernel(const Dev P, c
     __shared__ double red[UPD_THREADS / 32];
     __shared__ int is_last;
 
+    pdl_enter();
     const Ctl c = *P.ctl;
     if (c.done) return;
     const int slot = blockIdx.y;

@@ -121,6 +121,7 @@ update_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant_
     __shared__ double red[TC_THREADS / 32];
     __shared__ int is_last;
 
+    pdl_enter();
     const Ctl c = *P.ctl;
     if (c.done) return;
     const int slot = blockIdx.y;
@@ -315,8 +316,8 @@ void launch_update_tc(const Dev &P, const void *maps, int leg, int width, cudaSt
     const CUtensorMap *tm = reinterpret_cast<const CUtensorMap *>(maps);
     const int nrows = (leg == LEG_F) ? P.n : P.m;
     dim3 grid((nrows + TC_BM - 1) / TC_BM, width < 1 ? 1 : width);
-    if (tc_stages(P.d) == 2) update_tc_kernel<2><<<grid, TC_THREADS, smem, st>>>(tm[0], tm[1], P, leg);
-    else update_tc_kernel<4><<<grid, TC_THREADS, smem, st>>>(tm[0], tm[1], P, leg);
+    if (tc_stages(P.d) == 2) launch_pdl(update_tc_kernel<2>, grid, dim3(TC_THREADS), smem, st, tm[0], tm[1], P, leg);
+    else launch_pdl(update_tc_kernel<4>, grid, dim3(TC_THREADS), smem, st, tm[0], tm[1], P, leg);
 }
 
 }  // namespace skb
