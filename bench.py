@@ -148,6 +148,10 @@ def main():
     ap.add_argument("--compute", default="auto", choices=["auto", "f32", "mixed", "f64", "tensor"])
     ap.add_argument("--no-controls", action="store_true", help="skip the static / masked control timings")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--tol", type=float, default=None, help="override the workload's stopping tolerance")
+    ap.add_argument("--tol-sweep", action="store_true",
+                    help="completion-depth disagreement report: every tolerance of the sweep grid in static, "
+                         "masked and active mode, slots spent against W*l_max and sum l_t (one JSON line)")
     ap.add_argument("--kernel-only", action="store_true",
                     help="only create the batch and time the update kernel (few launches; for profiler captures)")
     args = ap.parse_args()
@@ -171,12 +175,44 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
 
     w = make_workload(args.workload)
+    if args.tol is not None:
+        w.tol = args.tol
     W, n, m, d = w.shape
     t = lambda v: torch.from_numpy(v).to(dev)
     x, y = t(w.x), t(w.y)
     if w.xy_dtype == "bf16":
         x, y = x.bfloat16(), y.bfloat16()
     a, b, eps = t(w.a), t(w.b), t(w.eps)
+    if args.tol_sweep:
+        from paper_2607_24741_b200 import workloads as wlmod
+        rows = []
+        for tol in wlmod.SWEEP_TOLS:
+            row = {"tol": tol}
+            for mode in ("static", "masked", "active"):
+                best, info = None, None
+                for rep in range(3):
+                    torch.cuda.synchronize()
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                    sb = B.SinkhornBatch(x, y, a, b, eps, tol, mode=mode, compute=args.compute, max_iter=w.max_iter)
+                    sb.drain()
+                    e1.record(); torch.cuda.synchronize()
+                    ms_ = e0.elapsed_time(e1)
+                    if best is None or ms_ < best:
+                        best = ms_
+                    depth, status = sb.depths(); st = sb.stats()
+                    info = {"slots": st["slots"], "l_max": st["cycles"], "sum_depth": int(depth.sum().item()),
+                            "done": int((status == 1).sum().item())}
+                    sb.close()
+                row[mode] = {"ms": best, **info}
+            row["W_lmax"] = W * row["active"]["l_max"]
+            row["removed_slots"] = row["static"]["slots"] - row["active"]["slots"]
+            row["static_over_active"] = row["static"]["ms"] / row["active"]["ms"]
+            row["masked_over_active"] = row["masked"]["ms"] / row["active"]["ms"]
+            rows.append(row)
+        print(json.dumps({"report": "tol-sweep", "workload": args.workload, "W": W, "n": n, "m": m, "d": d,
+                          "rows": rows}), flush=True)
+        return
     if args.kernel_only:
         sb = B.SinkhornBatch(x, y, a, b, eps, w.tol, mode="static", compute=args.compute, max_iter=w.max_iter)
         sb.step(2)

@@ -75,7 +75,11 @@ def check_against_oracle(oracle, w, r, lanes, *, pot_tol, exact_depth, tol=None,
             if audit_every == 1:
                 hist = np.maximum(o.hist_row, o.hist_col)
                 k = min(dg, do)                       # the audit the two sides disagree on
-                misses.append((t, dg, do, abs(hist[k - 1] - tol) / tol))
+                margin = abs(hist[k - 1] - tol) / tol
+                # relative decay of the oracle residual per cycle around that audit: an error injected
+                # every cycle is remembered for about 1/decay cycles
+                decay = abs(hist[max(k - 2, 0)] - hist[k - 1]) / tol if k >= 2 else 1.0
+                misses.append((t, dg, do, margin, decay))
         if dg == do or audit_every == 1:
             e = pot_err(r["f"][t][None], r["g"][t][None], fo[None], go[None], float(w.eps[t]))[0]
             assert e <= pot_tol, f"lane {t}: potential error {e:.3e} > {pot_tol}"
@@ -86,6 +90,13 @@ def check_against_oracle(oracle, w, r, lanes, *, pot_tol, exact_depth, tol=None,
             assert r["r_row"][t] <= tol
             assert abs(r["r_row"][t] - rr) <= 2e-2 * tol
     return misses
+
+
+def miss_allowed(margin, decay, floor):
+    """A lane may sit one audit away if the oracle's margin at the disputed audit is below the
+    arithmetic's residual error: a floor, or for slowly converging lanes the fp32 exponential
+    error 2^-22 accumulated over the ~1/decay cycles the iteration remembers (factor 4 slack)."""
+    return margin <= max(floor, 4.0 * 2.0 ** -22 / max(decay, 1e-12))
 
 
 def check_accounting(oracle, r, W, mode):
