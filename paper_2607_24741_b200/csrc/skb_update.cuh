@@ -57,9 +57,12 @@ template <int DP> struct Tune<float, DP> {
 #ifndef SKB_F64_R
 #define SKB_F64_R 2
 #endif
+#ifndef SKB_F64_CW
+#define SKB_F64_CW 4
+#endif
 template <int DP> struct Tune<double, DP> {
     static constexpr int R = DP <= 8 ? SKB_F64_R : 2;
-    static constexpr int CW = 4;
+    static constexpr int CW = DP <= 8 ? SKB_F64_CW : 4;
 };
 
 template <typename T, int DP, int CS> struct TileCols {
@@ -93,12 +96,6 @@ __device__ __forceinline__ u64 sub2(u64 a, u64 b)
     u64 d;
     asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
     return d;
-}
-// order-preserving 32-bit key of a float64 (its high word, sign-magnitude -> two's complement)
-__device__ __forceinline__ int dkey(double v)
-{
-    const int hi = __double2hiint(v);
-    return hi ^ ((hi >> 31) & 0x7fffffff);
 }
 // 2^k for an integer-valued k <= 0 (exact; flushes to 0 below the normal range)
 __device__ __forceinline__ float pow2i(float k)
@@ -295,7 +292,7 @@ __device__ __forceinline__ void stream_f64(double *sm, const double *colc, const
                                            const int tid, const int cs,
                                            float (&mx)[Tune<double, DP>::R], double (&sd)[Tune<double, DP>::R])
 {
-    constexpr int R = Tune<double, DP>::R, CW = 4;
+    constexpr int R = Tune<double, DP>::R, CW = Tune<double, DP>::CW;
     constexpr int TJ = TileCols<double, DP, CS>::value;
     constexpr int STEPS = TJ / (CW * CS);
     constexpr int NR = DP + 1;
@@ -303,9 +300,8 @@ __device__ __forceinline__ void stream_f64(double *sm, const double *colc, const
 
     float ts[R];
     double md[R];
-    int kmax[R];
 #pragma unroll
-    for (int r = 0; r < R; ++r) { mx[r] = NEG_BIG; md[r] = (double)NEG_BIG; kmax[r] = dkey(md[r]); ts[r] = 0.f; sd[r] = 0.0; }
+    for (int r = 0; r < R; ++r) { mx[r] = NEG_BIG; md[r] = (double)NEG_BIG; ts[r] = 0.f; sd[r] = 0.0; }
 
     const int ntiles = (ncols + TJ - 1) / TJ;
     load_tile<double, DP, TJ, NR>(sm, colc, colt, colt, cp, 0, tid);
@@ -323,57 +319,77 @@ __device__ __forceinline__ void stream_f64(double *sm, const double *colc, const
 #pragma unroll 1
         for (int q = 0; q < STEPS; ++q) {
             const int jj = (q * CS + cs) * CW;
-            double acc[R][4];
-            {
-                const double2 c0 = *reinterpret_cast<const double2 *>(st + DP * TJ + jj);
-                const double2 c1 = *reinterpret_cast<const double2 *>(st + DP * TJ + jj + 2);
+            double acc[R][CW];
 #pragma unroll
-                for (int r = 0; r < R; ++r) { acc[r][0] = c0.x; acc[r][1] = c0.y; acc[r][2] = c1.x; acc[r][3] = c1.y; }
+            for (int h = 0; h < CW / 2; ++h) {
+                const double2 c0 = *reinterpret_cast<const double2 *>(st + DP * TJ + jj + 2 * h);
+#pragma unroll
+                for (int r = 0; r < R; ++r) { acc[r][2 * h] = c0.x; acc[r][2 * h + 1] = c0.y; }
             }
 #pragma unroll
             for (int k = 0; k < DP; ++k) {
-                const double2 y0 = *reinterpret_cast<const double2 *>(st + k * TJ + jj);
-                const double2 y1 = *reinterpret_cast<const double2 *>(st + k * TJ + jj + 2);
 #pragma unroll
-                for (int r = 0; r < R; ++r) {
-                    acc[r][0] = fma(xr[r][k], y0.x, acc[r][0]);
-                    acc[r][1] = fma(xr[r][k], y0.y, acc[r][1]);
-                    acc[r][2] = fma(xr[r][k], y1.x, acc[r][2]);
-                    acc[r][3] = fma(xr[r][k], y1.y, acc[r][3]);
-                }
-            }
-            // the maximum only steers the rescale, so compare monotone integer keys of the high
-            // words (ALU pipe) instead of float64 values (FP64 pipe)
-            int kt[R];
-            bool grow = false;
+                for (int h = 0; h < CW / 2; ++h) {
+                    const double2 y0 = *reinterpret_cast<const double2 *>(st + k * TJ + jj + 2 * h);
 #pragma unroll
-            for (int r = 0; r < R; ++r) {
-                kt[r] = max(max(dkey(acc[r][0]), dkey(acc[r][1])), max(dkey(acc[r][2]), dkey(acc[r][3])));
-                grow = grow || (kt[r] > kmax[r]);
-            }
-            if (grow) {
-#pragma unroll
-                for (int r = 0; r < R; ++r) {
-                    if (kt[r] > kmax[r]) {
-                        const double mt = fmax(fmax(acc[r][0], acc[r][1]), fmax(acc[r][2], acc[r][3]));
-                        const float mn = ceilf((float)mt) + 1.0f;          // +1: the fp32 copy may round down
-                        const float fac = pow2i(mx[r] - mn);
-                        ts[r] *= fac;
-                        sd[r] *= (double)fac;
-                        mx[r] = mn;
-                        md[r] = (double)mn;
-                        kmax[r] = dkey(md[r] + 7.0);                       // rescale once a term would exceed 2^7
+                    for (int r = 0; r < R; ++r) {
+                        acc[r][2 * h] = fma(xr[r][k], y0.x, acc[r][2 * h]);
+                        acc[r][2 * h + 1] = fma(xr[r][k], y0.y, acc[r][2 * h + 1]);
                     }
                 }
             }
+            if (XF) {
+                // shifted arguments in fp32 (needed for ex2 anyway); their maximum steers the rescale
+                float v[R][CW];
+                bool grow = false;
 #pragma unroll
-            for (int r = 0; r < R; ++r) {
-                if (XF) {
-                    ts[r] += (ex2_fast((float)(acc[r][0] - md[r])) + ex2_fast((float)(acc[r][1] - md[r]))) +
-                             (ex2_fast((float)(acc[r][2] - md[r])) + ex2_fast((float)(acc[r][3] - md[r])));
-                } else {
-                    sd[r] += (exp2(acc[r][0] - md[r]) + exp2(acc[r][1] - md[r])) +
-                             (exp2(acc[r][2] - md[r]) + exp2(acc[r][3] - md[r]));
+                for (int r = 0; r < R; ++r) {
+#pragma unroll
+                    for (int e = 0; e < CW; ++e) v[r][e] = (float)(acc[r][e] - md[r]);
+                    float vm = v[r][0];
+#pragma unroll
+                    for (int e = 1; e < CW; ++e) vm = fmaxf(vm, v[r][e]);
+                    grow = grow || (vm > 8.0f);
+                }
+                if (grow) {                                   // rare: move the reference point up
+#pragma unroll
+                    for (int r = 0; r < R; ++r) {
+                        double mt = acc[r][0];
+#pragma unroll
+                        for (int e = 1; e < CW; ++e) mt = fmax(mt, acc[r][e]);
+                        if (mt > md[r] + 8.0) {
+                            const float mn = ceilf((float)mt) + 1.0f;      // +1: the fp32 copy may round down
+                            const float fac = pow2i(mx[r] - mn);
+                            ts[r] *= fac;
+                            sd[r] *= (double)fac;
+                            mx[r] = mn;
+                            md[r] = (double)mn;
+#pragma unroll
+                            for (int e = 0; e < CW; ++e) v[r][e] = (float)(acc[r][e] - md[r]);
+                        }
+                    }
+                }
+#pragma unroll
+                for (int r = 0; r < R; ++r) {
+                    float e2 = 0.f;
+#pragma unroll
+                    for (int e = 0; e < CW; ++e) e2 += ex2_fast(v[r][e]);
+                    ts[r] += e2;
+                }
+            } else {
+#pragma unroll
+                for (int r = 0; r < R; ++r) {
+                    double mt = acc[r][0];
+#pragma unroll
+                    for (int e = 1; e < CW; ++e) mt = fmax(mt, acc[r][e]);
+                    if (mt > md[r] + 8.0) {
+                        const float mn = ceilf((float)mt) + 1.0f;
+                        sd[r] *= (double)pow2i(mx[r] - mn);
+                        mx[r] = mn;
+                        md[r] = (double)mn;
+                    }
+#pragma unroll
+                    for (int e = 0; e < CW; ++e) sd[r] += exp2(acc[r][e] - md[r]);
                 }
             }
         }
