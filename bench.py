@@ -152,6 +152,9 @@ def main():
     ap.add_argument("--tol-sweep", action="store_true",
                     help="completion-depth disagreement report: every tolerance of the sweep grid in static, "
                          "masked and active mode, slots spent against W*l_max and sum l_t (one JSON line)")
+    ap.add_argument("--width-sweep", action="store_true",
+                    help="width report: W in {1,2,4,8,16} lanes of the registration law at n = 4096, solved "
+                         "one lane at a time (width-one), static-packed and active-packed (one JSON line)")
     ap.add_argument("--kernel-only", action="store_true",
                     help="only create the batch and time the update kernel (few launches; for profiler captures)")
     args = ap.parse_args()
@@ -174,6 +177,38 @@ def main():
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         dist.init_process_group("nccl", device_id=dev)
 
+    if args.width_sweep:
+        from paper_2607_24741_b200 import workloads as wlmod
+        big = wlmod.make("registration", W=16, n=4096)
+        tt = lambda v: torch.from_numpy(v).to(dev)
+        X, Y, A_, B_, E_ = tt(big.x), tt(big.y), tt(big.a), tt(big.b), tt(big.eps)
+
+        def run(sl, mode):
+            best = None
+            for rep in range(2):
+                torch.cuda.synchronize()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                sb = B.SinkhornBatch(X[sl], Y[sl], A_[sl], B_[sl], E_[sl], big.tol, mode=mode, compute=args.compute,
+                                     max_iter=big.max_iter)
+                sb.drain()
+                e1.record(); torch.cuda.synchronize()
+                ms_ = e0.elapsed_time(e1)
+                st = sb.stats(); sb.close()
+                best = ms_ if best is None or ms_ < best else best
+            return best, st["slots"], st["cycles"]
+
+        rows = []
+        for Wd in (1, 2, 4, 8, 16):
+            one = sum(run(slice(t0, t0 + 1), "active")[0] for t0 in range(Wd))
+            st_ms, st_slots, lmax = run(slice(0, Wd), "static")
+            ac_ms, ac_slots, _ = run(slice(0, Wd), "active")
+            rows.append({"W": Wd, "width_one_ms": one, "static_ms": st_ms, "active_ms": ac_ms, "l_max": lmax,
+                         "static_slots": st_slots, "active_slots": ac_slots,
+                         "width_one_over_static": one / st_ms, "static_over_active": st_ms / ac_ms,
+                         "width_one_over_active": one / ac_ms})
+        print(json.dumps({"report": "width-sweep", "law": "registration", "n": 4096, "d": 3, "rows": rows}), flush=True)
+        return
     w = make_workload(args.workload)
     if args.tol is not None:
         w.tol = args.tol
