@@ -104,6 +104,31 @@ __device__ __forceinline__ float pow2i(float k)
     return __int_as_float(e << 23);
 }
 
+// R consecutive values as one (or two) aligned vector loads; zeros when `ok` is false.
+template <typename T, int R>
+__device__ __forceinline__ void load_rows(const T *p, const bool ok, T (&v)[R])
+{
+    constexpr int BYTES = R * (int)sizeof(T);
+    if (!ok) {
+#pragma unroll
+        for (int r = 0; r < R; ++r) v[r] = T(0);
+        return;
+    }
+    if constexpr (BYTES == 8) {
+        const uint2 t = *reinterpret_cast<const uint2 *>(p);
+        memcpy(v, &t, 8);
+    } else if constexpr (BYTES == 16) {
+        const uint4 t = *reinterpret_cast<const uint4 *>(p);
+        memcpy(v, &t, 16);
+    } else {
+        static_assert(BYTES == 32, "unsupported row vector");
+        const uint4 t0 = *reinterpret_cast<const uint4 *>(p);
+        const uint4 t1 = *reinterpret_cast<const uint4 *>(reinterpret_cast<const char *>(p) + 16);
+        memcpy(v, &t0, 16);
+        memcpy(reinterpret_cast<char *>(v) + 16, &t1, 16);
+    }
+}
+
 // Column-tile loader shared by all arithmetic flavours: NR rows of TJ elements per stage.
 template <typename T, int DP, int TJ, int NR>
 __device__ __forceinline__ void load_tile(T *dst, const T *colc, const T *colt, const T *coll,
@@ -535,18 +560,21 @@ __global__ void __launch_bounds__(UPD_THREADS) update_kernel(const Dev P, const 
     // lanes that share a row's columns sit RG apart, so that each quarter-warp reads a single
     // shared-memory address per load when CS <= 4 (a broadcast, the cheapest access pattern)
     const int cs = lane / RG, rg = lane % RG;
-    const int lrow0 = warp * RW + rg;                    // CTA-local row of r = 0; row r: + r*RG
+    const int lrow0 = warp * RW + rg * R;                // this thread's R consecutive CTA-local rows
     const int row0 = blockIdx.x * RB + lrow0;
 
+    // R consecutive rows of one dimension are one aligned vector load (padding rows hold zeros)
     T xr[R][DP];
     T ph[R];
 #pragma unroll
-    for (int r = 0; r < R; ++r) {
-        const int i = row0 + r * RG;
+    for (int k = 0; k < DP; ++k) {
+        T v[R];
+        load_rows<T, R>(rowc + (size_t)k * rp + row0, row0 < rp, v);
 #pragma unroll
-        for (int k = 0; k < DP; ++k) xr[r][k] = (i < nrows) ? rowc[(size_t)k * rp + i] : T(0);
-        ph[r] = (i < nrows && form == FORM_DIFF) ? (T)prow[i] : T(0);
+        for (int r = 0; r < R; ++r) xr[r][k] = v[r];
     }
+#pragma unroll
+    for (int r = 0; r < R; ++r) ph[r] = (row0 + r < nrows && form == FORM_DIFF) ? (T)prow[row0 + r] : T(0);
 
     float mx[R];
     double sd[R];
@@ -572,9 +600,9 @@ __global__ void __launch_bounds__(UPD_THREADS) update_kernel(const Dev P, const 
     if (cs == 0) {
 #pragma unroll
         for (int r = 0; r < R; ++r) {
-            row_m[lrow0 + r * RG] = mx[r];
-            row_s[lrow0 + r * RG] = sd[r];
-            row_h[lrow0 + r * RG] = (float)ph[r];
+            row_m[lrow0 + r] = mx[r];
+            row_s[lrow0 + r] = sd[r];
+            row_h[lrow0 + r] = (float)ph[r];
         }
     }
     __syncthreads();
