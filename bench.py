@@ -31,6 +31,11 @@ sys.path.insert(0, ROOT)
 METRIC = "active lane*n*m updates/s (batch time-to-tol 1e-3)"
 UNIT = "lane*n*m updates/s"
 
+# DRAM bytes (read + write) of ONE full-width f-leg launch of the dominant kernel, from the ncu
+# captures summarised in profiles/update_kernel_sensor_registration_sweep.md and
+# profiles/update_tc_kernel_feature.md (one launch each; equal to the lanes' operands read once)
+NCU_TRAFFIC_BYTES = {"sensor": 20.5e6, "registration": 13.7e6, "sweep": 42.0e6, "feature": 141.0e6}
+
 # nominal unit counts (148 SMs, 128 FP32 lanes and 16 special-function lanes per SM per clock,
 # 64 FP64 lanes) at the maximum SM clock; the fraction reported is against these
 SM_COUNT, FP32_LANES, MUFU_LANES, FP64_LANES = 148, 128, 16, 64
@@ -375,7 +380,8 @@ def main():
             line["roofline"] = {"bound": "tensor", "kernel": "update_tc_kernel (f-leg, full width)",
                                 "arithmetic": arith, "achieved": tf, "peak": pk["bf16_tflops"], "unit": "TFLOP/s",
                                 "frac": tf / pk["bf16_tflops"], "exp_frac": achieved_exp / mufu_peak,
-                                "ms_per_launch": k_ms, "pairs_per_launch": pairs, "traffic": None,
+                                "ms_per_launch": k_ms, "pairs_per_launch": pairs,
+                                "traffic": NCU_TRAFFIC_BYTES.get(args.workload),
                                 "peak_source": pk["source"] + " cuBLAS bf16 burst (MEASURED_PEAKS.json)"}
         else:
           line["roofline"] = {
@@ -388,7 +394,8 @@ def main():
             "frac": (achieved_inst / fp32_peak) if bound_fp32 else (achieved_exp / mufu_peak),
             "exp_frac": achieved_exp / mufu_peak, "pipe_frac": achieved_inst / fp32_peak,
             "ms_per_launch": k_ms, "pairs_per_launch": pairs, "peak_clock_mhz": pk["sm_max_mhz"],
-            "traffic": None, "peak_source": "unit counts x max SM clock"}
+            "traffic": NCU_TRAFFIC_BYTES.get(args.workload), "traffic_unit": "bytes per launch (ncu)",
+            "peak_source": "unit counts x max SM clock"}
 
         # ---- static / masked controls on the same kernels
         if not args.no_controls:
@@ -398,19 +405,23 @@ def main():
                 ctl[mode] = {"ms": cms, "slots": cinfo["slots"]}
             line["controls"] = ctl
 
-        # ---- the oracle on the host cores, bounded sample
+        # ---- the oracle on the host cores, bounded sample (about 10 s of wall time at most)
         if not args.no_cpu_baseline:
             import oracle
             cores = os.cpu_count() or 1
-            lanes = min(W, max(cores, 64)) if n * m <= 512 * 512 else min(W, cores)
+            cap = min(w.max_iter, 40) if n * m > 2048 * 2048 else w.max_iter
+            done_lanes, units, threads = 0, 0.0, 1
             t0 = time.perf_counter()
-            r = oracle.solve_batch(w.x[:lanes], w.y[:lanes], w.a[:lanes], w.b[:lanes], w.eps[:lanes], w.tol,
-                                   max_iter=min(w.max_iter, 40) if n * m > 2048 * 2048 else w.max_iter)
+            while done_lanes < W and time.perf_counter() - t0 < 8.0:
+                sl = slice(done_lanes, min(W, done_lanes + cores))
+                r = oracle.solve_batch(w.x[sl], w.y[sl], w.a[sl], w.b[sl], w.eps[sl], w.tol, max_iter=cap)
+                units += float(r.depth.sum()) * n * m
+                threads = max(threads, r.threads)
+                done_lanes = sl.stop
             dt = time.perf_counter() - t0
-            line["cpu_baseline"] = {"value": float(r.depth.sum()) * n * m / dt, "unit": UNIT, "cores": r.threads,
-                                    "kind": "oracle", "seconds": dt,
-                                    "sample": f"lanes 0..{lanes - 1} of {W}, each to its own depth"
-                                              + (" (capped at 40 cycles)" if n * m > 2048 * 2048 else "")}
+            line["cpu_baseline"] = {"value": units / dt, "unit": UNIT, "cores": threads, "kind": "oracle", "seconds": dt,
+                                    "sample": f"lanes 0..{done_lanes - 1} of {W}, each to its own depth"
+                                              + (f" (capped at {cap} cycles)" if cap < w.max_iter else "")}
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.barrier()
