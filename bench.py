@@ -31,9 +31,9 @@ sys.path.insert(0, ROOT)
 METRIC = "active lane*n*m updates/s (batch time-to-tol 1e-3)"
 UNIT = "lane*n*m updates/s"
 
-# DRAM bytes (read + write) of ONE full-width f-leg launch of the dominant kernel, from the ncu
-# captures summarised in profiles/update_kernel_sensor_registration_sweep.md and
-# profiles/update_tc_kernel_feature.md (one launch each; equal to the lanes' operands read once)
+# DRAM bytes (read + write) of ONE full-width f-leg launch of the dominant kernel, taken from ncu
+# captures of `bench.py --workload <name> --kernel-only` (one launch each; they equal the lanes'
+# operands read once)
 NCU_TRAFFIC_BYTES = {"sensor": 20.5e6, "registration": 13.7e6, "sweep": 42.0e6, "feature": 141.0e6}
 
 # nominal unit counts (148 SMs, 128 FP32 lanes and 16 special-function lanes per SM per clock,

@@ -155,6 +155,16 @@ skb_status sinkhorn_batch_stats(skb_batch *h, long long *slots, int *cycles, int
  * batch resolved to from its data.  Host out. */
 skb_status sinkhorn_batch_arithmetic(skb_batch *h, int *compute);
 
+/*
+ * Self-test of the kernels' failure detection.  The tensor-core kernel synchronises its
+ * warps through mbarriers; every such wait has a clock budget, after which the kernel
+ * records an error instead of hanging (the host then reports SKB_ERR_CUDA).  This call runs
+ * one such wait on a barrier that nothing completes, with the given budget in milliseconds
+ * (at ~2 GHz), and writes three ints to out3 (device): 1 if the wait gave up, the abort flag
+ * it raised, and the kilo-clocks it spent.  Enqueues only.
+ */
+skb_status sinkhorn_batch_selftest_bounded_wait(int *out3, float budget_ms, void *stream);
+
 /* Number of kernels this handle has launched so far (host out). */
 skb_status sinkhorn_batch_launch_count(skb_batch *h, long long *launches);
 

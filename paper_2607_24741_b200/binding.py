@@ -28,6 +28,7 @@ EXPORTS = (
     "sinkhorn_batch_stats", "sinkhorn_batch_destroy", "sinkhorn_batch_last_error",
     "sinkhorn_batch_host_workspace_bytes", "sinkhorn_batch_solve_host",
     "sinkhorn_batch_launch_count", "sinkhorn_batch_profile_update", "sinkhorn_batch_arithmetic",
+    "sinkhorn_batch_selftest_bounded_wait",
 )
 # entry points outside the sinkhorn_batch_* family
 EXTRA_EXPORTS = ("sinkhorn_row_residual_static", "sinkhorn_row_residual_static_last_error")
@@ -69,6 +70,7 @@ def _load():
     lib.sinkhorn_batch_residuals.argtypes = [vp, vp, vp]
     lib.sinkhorn_batch_stats.argtypes = [vp, ctypes.POINTER(ctypes.c_longlong), ctypes.POINTER(ctypes.c_int),
                                          vp, ctypes.c_int, ctypes.POINTER(ctypes.c_longlong)]
+    lib.sinkhorn_batch_selftest_bounded_wait.argtypes = [vp, ctypes.c_float, vp]
     lib.sinkhorn_batch_arithmetic.argtypes = [vp, ctypes.POINTER(ctypes.c_int)]
     lib.sinkhorn_batch_launch_count.argtypes = [vp, ctypes.POINTER(ctypes.c_longlong)]
     lib.sinkhorn_batch_profile_update.argtypes = [vp, ctypes.c_int, ctypes.c_int, ctypes.POINTER(ctypes.c_float)]

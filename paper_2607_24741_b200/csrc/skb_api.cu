@@ -407,6 +407,15 @@ extern "C" skb_status sinkhorn_batch_arithmetic(skb_batch *h, int *compute)
     return SKB_OK;
 }
 
+extern "C" skb_status sinkhorn_batch_selftest_bounded_wait(int *out3, float budget_ms, void *stream)
+{
+    if (!out3) return SKB_ERR_NULL;
+    if (!(budget_ms > 0.0f) || budget_ms > 2000.0f) return fail(nullptr, SKB_ERR_VALUE, "budget must be in (0, 2000] ms");
+    launch_wait_probe(out3, (long long)(budget_ms * 2.0e6f), (cudaStream_t)stream);
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? SKB_OK : cuda_fail(nullptr, e, "selftest");
+}
+
 extern "C" skb_status sinkhorn_batch_launch_count(skb_batch *h, long long *launches)
 {
     if (!h || !launches) return SKB_ERR_NULL;

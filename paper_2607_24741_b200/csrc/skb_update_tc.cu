@@ -34,6 +34,7 @@ constexpr int TC_MAX_STAGES = 4;
 constexpr int TC_BM = 128, TC_BN = 128, TC_BK = 64;
 constexpr uint32_t TC_CHUNK = TC_BM * TC_BK * 2;          // 16 KB: 128 points x 64 bf16
 constexpr long long TC_WAIT_CLOCKS = 2000000000LL;        // ~1 s
+__device__ long long g_wait_clocks = TC_WAIT_CLOCKS;      // budget of every bounded wait (a self-test shortens it)
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint32_t a, uint32_t count)
@@ -61,7 +62,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t a, uint32_t parity, volatile 
     const long long t0 = clock64();
     while (!mbar_try_wait(a, parity)) {
         if (*abort_flag) return false;
-        if (clock64() - t0 > TC_WAIT_CLOCKS) { *abort_flag = 1; return false; }
+        if (clock64() - t0 > g_wait_clocks) { *abort_flag = 1; return false; }
     }
     return true;
 }
@@ -269,6 +270,32 @@ update_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant_
         if (tid == 0) atomicOr(&P.ctl->error, ERR_WAIT);
     }
     finish_rows<float, TC_BM, TC_THREADS>(P, c, leg, slot, (int)FORM_DOT, row_m, row_s, row_h, red, &is_last);
+}
+
+// Self-test of the bounded wait: one thread waits on a barrier that nothing will ever complete
+// and must come back with `false` once its clock budget is spent.
+__global__ void wait_probe_kernel(int *out, long long budget)
+{
+    __shared__ __align__(8) unsigned long long bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        const long long saved = g_wait_clocks;
+        g_wait_clocks = budget;
+        const long long t0 = clock64();
+        const bool ok = mbar_wait(smem_u32(&bar), 0, &abort_flag);
+        out[0] = ok ? 0 : 1;                       // 1: the wait gave up
+        out[1] = abort_flag;
+        out[2] = (int)((clock64() - t0) >> 10);    // kilo-clocks spent
+        g_wait_clocks = saved;
+    }
+}
+
+void launch_wait_probe(int *out, long long budget_clocks, cudaStream_t st)
+{
+    wait_probe_kernel<<<1, 32, 0, st>>>(out, budget_clocks);
 }
 
 // ---------------------------------------------------------------- host side

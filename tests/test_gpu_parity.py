@@ -352,3 +352,18 @@ def test_other_tolerances_of_the_sweep_grid(oracle, tol):
     np.testing.assert_array_equal(rs["depth"], r["depth"])
     lmax = int(r["depth"].max())
     assert rs["stats"]["slots"] == 24 * lmax and r["stats"]["slots"] == int(r["depth"].sum())
+
+
+def test_bounded_wait_gives_up_instead_of_hanging():
+    # failure detection without a fault: a barrier nothing completes, a 5 ms budget
+    import torch
+    from paper_2607_24741_b200 import binding as B
+    out = torch.zeros(3, dtype=torch.int32, device="cuda:0")
+    rc = B.lib.sinkhorn_batch_selftest_bounded_wait(out.data_ptr(), 5.0, None)
+    assert rc == 0
+    torch.cuda.synchronize()
+    gave_up, abort_flag, kclk = out.cpu().tolist()
+    assert gave_up == 1 and abort_flag == 1
+    assert 5e3 <= kclk <= 5e5           # ~10 M clocks budget: it neither returned at once nor spun for long
+    # the context is still usable
+    assert int(torch.arange(10, device="cuda:0").sum().item()) == 45
