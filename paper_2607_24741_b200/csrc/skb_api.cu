@@ -92,7 +92,7 @@ static size_t carve(const skb_config *c, const Variant *var, bool tensor, char *
     d.part_row = (double *)take(W * MAX_PARTS * 8); d.part_col = (double *)take(W * MAX_PARTS * 8);
     d.tensor = tensor ? 1 : 0;
     if (tensor) {
-        d.xb = take(W * n * (size_t)c->d * 2); d.yb = take(W * m * (size_t)c->d * 2);
+        d.xb = take(tc_tiled_bytes(c->W, c->n, c->d)); d.yb = take(tc_tiled_bytes(c->W, c->m, c->d));
     } else {
         d.xs = take(W * DP * np * ts); d.ys = take(W * DP * mp * ts);
     }
@@ -228,15 +228,11 @@ extern "C" skb_status sinkhorn_batch_create(const void *x, const void *y, const 
         h->dev.tol_stop = ts; h->dev.tol_screen = tsc;
     }
     if (h->tensor) {
-        // the MMA reads the caller's bf16 layout: keep a copy the compaction may permute
-        const size_t W = cfg->W, d = cfg->d;
+        // the MMA operands: tiled copies of x and y that the compaction may permute
         const char *why = nullptr;
-        if ((e = cudaMemcpyAsync(h->dev.xb, x, W * cfg->n * d * 2, cudaMemcpyDeviceToDevice, h->stream)) != cudaSuccess ||
-            (e = cudaMemcpyAsync(h->dev.yb, y, W * cfg->m * d * 2, cudaMemcpyDeviceToDevice, h->stream)) != cudaSuccess) {
-            skb_status st = cuda_fail(nullptr, e, "create");
-            sinkhorn_batch_destroy(h);
-            return st;
-        }
+        launch_retile(x, h->dev.xb, cfg->W, cfg->n, cfg->d, h->stream);
+        launch_retile(y, h->dev.yb, cfg->W, cfg->m, cfg->d, h->stream);
+        h->launches += 2;
         if ((why = tc_make_map(h->maps, h->dev.xb, cfg->W, cfg->n, cfg->d)) != nullptr ||
             (why = tc_make_map(h->maps + 128, h->dev.yb, cfg->W, cfg->m, cfg->d)) != nullptr) {
             skb_status st = fail(nullptr, SKB_ERR_CUDA, why);

@@ -313,8 +313,8 @@ __device__ __forceinline__ void emit_move_one(const Dev &P, const Ctl &c, const 
     };
     const int np_ = ep ^ 1;   // buffer that holds the survivors' current row potentials
     if (P.tensor) {
-        copy(P.xb, (size_t)P.n * P.d * 2);
-        copy(P.yb, (size_t)P.m * P.d * 2);
+        copy(P.xb, (size_t)((P.n + 127) / 128) * P.d * 256);      // tiled copies: 128-point tiles x d bf16
+        copy(P.yb, (size_t)((P.m + 127) / 128) * P.d * 256);
     } else {
         copy(P.xs, (size_t)P.DP * P.np * sizeof(T));
         copy(P.ys, (size_t)P.DP * P.mp * sizeof(T));

@@ -53,7 +53,7 @@ struct Dev {
     double tol_screen, tol_stop;
     // slabs by slot
     void *xs, *ys;            // [W][DP][np|mp]   T   (SIMT kernels)
-    void *xb, *yb;            // [W][n|m][d] bf16, the caller's layout (tensor-core kernel)
+    void *xb, *yb;            // bf16 copies tiled [W][128-point tile][64-dim chunk][128][64] (tensor-core kernel)
     void *ft[2];              // [W][np]          T
     void *gt;                 // [W][mp]          T
     void *fl[2], *gl;         // low parts of the potentials (difference form only)

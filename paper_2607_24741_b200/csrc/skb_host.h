@@ -36,6 +36,8 @@ void launch_plan(const Dev &P, int width, cudaStream_t st);
 // tensor-core update kernel (bf16 inputs, d a multiple of 64 up to 512)
 bool tc_eligible(int d, bool bf16);
 const char *tc_make_map(void *out_map, void *base, int W, int npts, int d);
+size_t tc_tiled_bytes(int W, int npts, int d);
+void launch_retile(const void *src, void *dst, int W, int npts, int d, cudaStream_t st);
 void launch_wait_probe(int *out, long long budget_clocks, cudaStream_t st);
 void launch_update_tc(const Dev &P, const void *maps, int leg, int width, cudaStream_t st);
 void launch_emit_move(const Dev &P, int width, cudaStream_t st);

@@ -10,8 +10,10 @@
 // Warp roles (192 threads):
 //   warps 0-3  epilogue: thread e owns row e = TMEM lane e; tcgen05.ld 32 columns at a time,
 //              fma with the column term, online logsumexp entirely in registers (no shuffles)
-//   warp 4     producer: one lane issues TMA loads (3-D tensor maps over [lane, point, d],
-//              128-byte swizzle, out-of-range points read as zero): the row block once
+//   warp 4     producer: one lane issues TMA loads of pre-tiled operand copies (every
+//              128-point x 64-dimension chunk is one contiguous 16 KB block in the workspace,
+//              which TMA streams at about twice the rate of 1 KB-strided rows; 128-byte
+//              swizzle; points past the end are stored as zeros): the row block once
 //              (d/64 chunks of 16 KB, riding on the first tile's barriers), and column
 //              chunks through a ring of 2 (d <= 256: two CTAs per SM) or 4 stages
 //   warp 5     allocates 256 TMEM columns (two 128-column accumulators); one lane issues the
@@ -66,10 +68,11 @@ __device__ __forceinline__ bool mbar_wait(uint32_t a, uint32_t parity, volatile 
     }
     return true;
 }
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *tm, int c0, int c1, int c2, uint32_t mbar)
+// one pre-tiled chunk (128 points x 64 bf16, contiguous 16 KB in global memory) -> shared memory
+__device__ __forceinline__ void tma_load_chunk(uint32_t dst, const CUtensorMap *tm, int row, uint32_t mbar)
 {
-    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
-                 ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(c0), "r"(c1), "r"(c2), "r"(mbar) : "memory");
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(0), "r"(row), "r"(mbar) : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -139,6 +142,10 @@ update_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant_
                                : reinterpret_cast<const float *>(P.ft[c.parity]) + (size_t)slot * cp;
     const int nkc = P.d / TC_BK;
     const int ntiles = (ncols + TC_BN - 1) / TC_BN;
+    // chunk index of this CTA's row block and of the lane's first column tile in the tiled copies
+    const int nrt = (nrows + TC_BM - 1) / TC_BM;
+    const int row_tile0 = (slot * nrt + (int)blockIdx.x) * nkc;
+    const int col_tile0 = slot * ntiles * nkc;
     const float two_s = (float)(2.0 * P.scale[slot]);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -180,8 +187,8 @@ update_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant_
                     const int s = it % TC_STAGES;
                     if (it >= TC_STAGES && !mbar_wait(b_empty + 8 * s, ((it / TC_STAGES) - 1) & 1, ab)) break;
                     mbar_expect_tx(b_full + 8 * s, t == 0 ? 2 * TC_CHUNK : TC_CHUNK);
-                    if (t == 0) tma_load_3d(sA + kc * TC_CHUNK, tm_row, kc * TC_BK, i0, slot, b_full + 8 * s);
-                    tma_load_3d(sB + s * TC_CHUNK, tm_col, kc * TC_BK, t * TC_BN, slot, b_full + 8 * s);
+                    if (t == 0) tma_load_chunk(sA + kc * TC_CHUNK, tm_row, (row_tile0 + kc) * TC_BM, b_full + 8 * s);
+                    tma_load_chunk(sB + s * TC_CHUNK, tm_col, (col_tile0 + t * nkc + kc) * TC_BN, b_full + 8 * s);
                 }
             }
         }
@@ -310,7 +317,7 @@ bool tc_eligible(int d, bool bf16) { return bf16 && d >= 64 && d <= 512 && d % 6
 static int tc_stages(int d) { return d <= 256 ? 2 : 4; }
 size_t tc_smem_bytes(int d) { return (size_t)(d / TC_BK + tc_stages(d)) * TC_CHUNK + 1024; }
 
-// Builds the [lane, point, d] bf16 tensor map of one operand array.  Returns a CUDA error string or null.
+// Tensor map of one tiled operand copy: rows of 64 bf16 (128 B, contiguous), 128-row boxes.
 const char *tc_make_map(void *out_map, void *base, int W, int npts, int d)
 {
     static EncodeTiledFn fn = nullptr;
@@ -321,14 +328,37 @@ const char *tc_make_map(void *out_map, void *base, int W, int npts, int d)
             return "cuTensorMapEncodeTiled is not available";
         fn = (EncodeTiledFn)p;
     }
-    const cuuint64_t gdim[3] = {(cuuint64_t)d, (cuuint64_t)npts, (cuuint64_t)W};
-    const cuuint64_t gstr[2] = {(cuuint64_t)d * 2, (cuuint64_t)npts * d * 2};
-    const cuuint32_t box[3] = {TC_BK, TC_BM, 1};
-    const cuuint32_t estr[3] = {1, 1, 1};
-    const CUresult r = fn((CUtensorMap *)out_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, gdim, gstr, box, estr,
+    const cuuint64_t rows = (cuuint64_t)W * ((npts + TC_BM - 1) / TC_BM) * (d / TC_BK) * TC_BM;
+    const cuuint64_t gdim[2] = {(cuuint64_t)TC_BK, rows};
+    const cuuint64_t gstr[1] = {(cuuint64_t)TC_BK * 2};
+    const cuuint32_t box[2] = {TC_BK, TC_BM};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = fn((CUtensorMap *)out_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, gdim, gstr, box, estr,
                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? nullptr : "cuTensorMapEncodeTiled failed";
+}
+
+size_t tc_tiled_bytes(int W, int npts, int d) { return (size_t)W * ((npts + TC_BM - 1) / TC_BM) * (d / TC_BK) * TC_CHUNK; }
+
+// Copies [W][npts][d] bf16 into the tiled layout [W][tile][chunk][128][64]; points past npts become zeros.
+__global__ void __launch_bounds__(256) retile_kernel(const uint4 *__restrict__ src, uint4 *__restrict__ dst, int npts, int d)
+{
+    const int nkc = d / TC_BK, ntile = (npts + TC_BM - 1) / TC_BM;
+    const int blk = blockIdx.x, tile = blk / nkc, kc = blk % nkc, slot = blockIdx.y;
+    uint4 *out = dst + ((size_t)(slot * ntile + tile) * nkc + kc) * (TC_CHUNK / 16);
+    for (int q = threadIdx.x; q < TC_BM * 8; q += 256) {
+        const int r = q >> 3, c = q & 7, pt = tile * TC_BM + r;
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (pt < npts) v = src[((size_t)(slot * (size_t)npts + pt) * d + kc * TC_BK) / 8 + c];
+        out[q] = v;
+    }
+}
+
+void launch_retile(const void *src, void *dst, int W, int npts, int d, cudaStream_t st)
+{
+    dim3 grid(((npts + TC_BM - 1) / TC_BM) * (d / TC_BK), W);
+    retile_kernel<<<grid, 256, 0, st>>>((const uint4 *)src, (uint4 *)dst, npts, d);
 }
 
 void launch_update_tc(const Dev &P, const void *maps, int leg, int width, cudaStream_t st)
