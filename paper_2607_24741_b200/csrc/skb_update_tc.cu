@@ -15,9 +15,10 @@
 //              which TMA streams at about twice the rate of 1 KB-strided rows; 128-byte
 //              swizzle; points past the end are stored as zeros): the row block once
 //              (d/64 chunks of 16 KB, riding on the first tile's barriers), and column
-//              chunks through a ring of 2 (d <= 256: two CTAs per SM) or 4 stages
-//   warp 5     allocates 256 TMEM columns (two 128-column accumulators); one lane issues the
-//              MMAs (4 x K=16 per 64-wide chunk) and commits to the ring's empty barriers and
+//              chunks through a ring of 2 (d <= 256, 128-column tiles, two CTAs per SM) or
+//              3 stages (d > 256, 256-column tiles of two chunks each)
+//   warp 5     allocates the TMEM columns of two accumulators (2 x 128 or 2 x 256); one lane issues
+//              the MMAs (4 x K=16 per 64-wide chunk) and commits to the ring's empty barriers and
 //              to the accumulator-full barrier, so the next tile's MMAs overlap this tile's
 //              exponentials.
 // Every mbarrier wait is bounded by a clock budget; on expiry the kernel raises ERR_WAIT in
@@ -25,6 +26,7 @@
 // returns (the host reports SKB_ERR_CUDA).
 #include <cuda.h>
 #include <cuda_runtime.h>
+#include <cstdio>
 
 #include "skb_update.cuh"
 #include "skb_host.h"
@@ -33,7 +35,7 @@ namespace skb {
 
 constexpr int TC_THREADS = 192;
 constexpr int TC_MAX_STAGES = 4;
-constexpr int TC_BM = 128, TC_BN = 128, TC_BK = 64;
+constexpr int TC_BM = 128, TC_BK = 64;
 constexpr uint32_t TC_CHUNK = TC_BM * TC_BK * 2;          // 16 KB: 128 points x 64 bf16
 constexpr long long TC_WAIT_CLOCKS = 2000000000LL;        // ~1 s
 __device__ long long g_wait_clocks = TC_WAIT_CLOCKS;      // budget of every bounded wait (a self-test shortens it)
@@ -69,6 +71,11 @@ __device__ __forceinline__ bool mbar_wait(uint32_t a, uint32_t parity, volatile 
     return true;
 }
 // one pre-tiled chunk (128 points x 64 bf16, contiguous 16 KB in global memory) -> shared memory
+#ifdef SKB_TC_DEBUG
+#define TC_TIMED_WAIT(acc, call) ({ const long long _t = clock64(); const bool _r = (call); (acc) += clock64() - _t; _r; })
+#else
+#define TC_TIMED_WAIT(acc, call) (call)
+#endif
 __device__ __forceinline__ void tma_load_chunk(uint32_t dst, const CUtensorMap *tm, int row, uint32_t mbar)
 {
     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
@@ -108,9 +115,9 @@ __device__ __forceinline__ uint64_t tc_desc(uint32_t saddr)
     return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(1024u >> 4) << 32) | (1ull << 46) | (2ull << 61);
 }
 // instruction descriptor: D fp32, A and B bf16, both K-major, M = 128, N = 128
-constexpr uint32_t TC_IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(TC_BN >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
+__host__ __device__ constexpr uint32_t tc_idesc(int bn) { return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24); }
 
-template <int TC_STAGES>
+template <int TC_STAGES, int TC_BN>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 update_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUtensorMap tmy, const Dev P, const int leg)
 {
@@ -118,10 +125,13 @@ update_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant_
     __shared__ __align__(8) unsigned long long bars[2 * TC_MAX_STAGES + 5];
     __shared__ uint32_t tmem_holder;
     __shared__ int abort_flag;
-    __shared__ float gts[2][TC_BN];
-    __shared__ double row_s[TC_BM];
-    __shared__ float row_m[TC_BM];
-    __shared__ float row_h[TC_BM];
+    // column terms of two tiles while streaming; the per-row results afterwards (same bytes)
+    __shared__ __align__(16) unsigned char small_buf[2 * TC_BN * 4 > 2048 ? 2 * TC_BN * 4 : 2048];
+    float (*gts)[TC_BN] = reinterpret_cast<float (*)[TC_BN]>(small_buf);
+    double *row_s = reinterpret_cast<double *>(small_buf);
+    float *row_m = reinterpret_cast<float *>(small_buf + 1024);
+    float *row_h = reinterpret_cast<float *>(small_buf + 1536);
+    constexpr uint32_t STAGE_BYTES = (TC_BN / 128) * TC_CHUNK;     // one or two 128-point chunks per stage
     __shared__ double red[TC_THREADS / 32];
     __shared__ int is_last;
 
@@ -145,7 +155,8 @@ update_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant_
     // chunk index of this CTA's row block and of the lane's first column tile in the tiled copies
     const int nrt = (nrows + TC_BM - 1) / TC_BM;
     const int row_tile0 = (slot * nrt + (int)blockIdx.x) * nkc;
-    const int col_tile0 = slot * ntiles * nkc;
+    const int nct128 = (ncols + 127) / 128;                     // 128-point tiles of the column operand
+    const int col_tile0 = slot * nct128 * nkc;
     const float two_s = (float)(2.0 * P.scale[slot]);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -164,7 +175,8 @@ update_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant_
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 5) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 256;" ::"r"(smem_u32(&tmem_holder)) : "memory");
+        if (TC_BN == 256) asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(&tmem_holder)) : "memory");
+        else asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 256;" ::"r"(smem_u32(&tmem_holder)) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
@@ -175,6 +187,9 @@ update_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant_
 
     float mx = NEG_BIG;
     double sd = 0.0;
+    long long dbg_w0 = 0, dbg_w1 = 0;   // clocks spent in waits (debug builds)
+    const long long dbg_t0 = clock64();
+    (void)dbg_w0; (void)dbg_w1; (void)dbg_t0;
 
     if (warp == 4) {
         // ---------------- producer
@@ -185,10 +200,18 @@ update_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant_
             for (int t = 0; t < ntiles && !*ab; ++t) {
                 for (int kc = 0; kc < nkc; ++kc, ++it) {
                     const int s = it % TC_STAGES;
-                    if (it >= TC_STAGES && !mbar_wait(b_empty + 8 * s, ((it / TC_STAGES) - 1) & 1, ab)) break;
-                    mbar_expect_tx(b_full + 8 * s, t == 0 ? 2 * TC_CHUNK : TC_CHUNK);
+                    if (it >= TC_STAGES && !TC_TIMED_WAIT(dbg_w0, mbar_wait(b_empty + 8 * s, ((it / TC_STAGES) - 1) & 1, ab))) break;
+                    mbar_expect_tx(b_full + 8 * s, t == 0 ? STAGE_BYTES + TC_CHUNK : STAGE_BYTES);
                     if (t == 0) tma_load_chunk(sA + kc * TC_CHUNK, tm_row, (row_tile0 + kc) * TC_BM, b_full + 8 * s);
-                    tma_load_chunk(sB + s * TC_CHUNK, tm_col, (col_tile0 + t * nkc + kc) * TC_BN, b_full + 8 * s);
+#pragma unroll
+                    for (int h = 0; h < TC_BN / 128; ++h) {
+                        // 128-point tile index of this half of the column tile; tiles past the end read as zeros
+                        const int pt = t * (TC_BN / 128) + h;
+                        if (pt < nct128)
+                            tma_load_chunk(sB + s * STAGE_BYTES + h * TC_CHUNK, tm_col, (col_tile0 + pt * nkc + kc) * 128, b_full + 8 * s);
+                        else
+                            tma_load_chunk(sB + s * STAGE_BYTES + h * TC_CHUNK, tm_col, 0x7fffff80, b_full + 8 * s);
+                    }
                 }
             }
         }
@@ -199,20 +222,20 @@ update_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant_
             int it = 0;
             for (int t = 0; t < ntiles && ok; ++t) {
                 const int buf = t & 1;
-                if (t >= 2) ok = mbar_wait(b_tempty + 8 * buf, ((t >> 1) - 1) & 1, ab);
+                if (t >= 2) ok = TC_TIMED_WAIT(dbg_w1, mbar_wait(b_tempty + 8 * buf, ((t >> 1) - 1) & 1, ab));
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem + (uint32_t)buf * TC_BN;
                 for (int kc = 0; kc < nkc && ok; ++kc, ++it) {
                     const int s = it % TC_STAGES;
-                    ok = mbar_wait(b_full + 8 * s, (it / TC_STAGES) & 1, ab);
+                    ok = TC_TIMED_WAIT(dbg_w0, mbar_wait(b_full + 8 * s, (it / TC_STAGES) & 1, ab));
                     if (!ok) break;
                     tc_fence_after();
 #pragma unroll
                     for (int k = 0; k < TC_BK / 16; ++k) {
+                        const uint64_t bd = tc_desc(sB + s * STAGE_BYTES + k * 32);
                         const uint64_t ad = tc_desc(sA + kc * TC_CHUNK + k * 32);
-                        const uint64_t bd = tc_desc(sB + s * TC_CHUNK + k * 32);
-                        tc_mma(d_tmem, ad, bd, TC_IDESC, (kc | k) ? 1u : 0u);
+                        tc_mma(d_tmem, ad, bd, tc_idesc(TC_BN), (kc | k) ? 1u : 0u);
                     }
                     tc_commit(b_empty + 8 * s);             // frees the ring stage when these MMAs retire
                 }
@@ -226,12 +249,13 @@ update_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant_
         bool ok = true;
         for (int t = 0; t < ntiles && ok; ++t) {
             const int buf = t & 1;
-            {
-                const int j = t * TC_BN + e;
-                gts[buf][e] = (j < cp) ? colt[j] : NEG_BIG;
+#pragma unroll
+            for (int h = 0; h < TC_BN / 128; ++h) {
+                const int j = t * TC_BN + h * 128 + e;
+                gts[buf][h * 128 + e] = (j < cp) ? colt[j] : NEG_BIG;
             }
             asm volatile("bar.sync 1, 128;" ::: "memory");
-            ok = mbar_wait(b_tfull + 8 * buf, (t >> 1) & 1, ab);
+            ok = TC_TIMED_WAIT(dbg_w0, mbar_wait(b_tfull + 8 * buf, (t >> 1) & 1, ab));
             if (!ok) break;
             tc_fence_after();
             float ts = 0.f;
@@ -259,6 +283,7 @@ update_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant_
             tc_fence_before();
             mbar_arrive(b_tempty + 8 * buf);                // all 128 rows have read this accumulator
         }
+        asm volatile("bar.sync 1, 128;" ::: "memory");     // every row is done with the column terms
         row_m[e] = mx;
         row_s[e] = ok ? sd : __longlong_as_double(0x7ff8000000000000LL);
         row_h[e] = 0.f;
@@ -269,10 +294,18 @@ update_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant_
         const long long t0 = clock64();
         while (clock64() - t0 < 200000LL) { }
     }
+#ifdef SKB_TC_DEBUG
+    if (blockIdx.x == 1 && blockIdx.y == 3 && leg == LEG_F && (lane == 0) && (warp == 0 || warp >= 4))
+        printf("[tc dbg] warp %d: total %lld clk, wait0 %lld, wait1 %lld (producer: empty; mma: full, tmem-empty; epilogue: tmem-full) tiles %d chunks/tile %d\n",
+               warp, clock64() - dbg_t0, dbg_w0, dbg_w1, ntiles, nkc);
+#endif
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    if (warp == 5) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 256;" ::"r"(tmem) : "memory");
+    if (warp == 5) {
+        if (TC_BN == 256) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
+        else asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 256;" ::"r"(tmem) : "memory");
+    }
     if (abort_flag) {
         if (tid == 0) atomicOr(&P.ctl->error, ERR_WAIT);
     }
@@ -314,8 +347,12 @@ bool tc_eligible(int d, bool bf16) { return bf16 && d >= 64 && d <= 512 && d % 6
 
 // two ring stages when that lets two CTAs share an SM (d <= 256: the second CTA's MMAs cover
 // this CTA's prologue and epilogue), four otherwise
-static int tc_stages(int d) { return d <= 256 ? 2 : 4; }
-size_t tc_smem_bytes(int d) { return (size_t)(d / TC_BK + tc_stages(d)) * TC_CHUNK + 1024; }
+// beyond d = 256 the row block lives in tensor memory, which leaves shared memory to a 12-stage ring
+// d <= 256: 128-column tiles, two ring stages, small enough for two CTAs per SM (the second CTA's MMAs
+// cover this CTA's prologue and epilogue).  d > 256: 256-column tiles (the tensor pipe runs 128x256 MMAs
+// about twice as efficiently as 128x128 ones), three 32 KB stages beside the 128 KB row block.
+static bool tc_wide(int d) { return d > 256; }
+size_t tc_smem_bytes(int d) { return (size_t)(d / TC_BK + (tc_wide(d) ? 6 : 2)) * TC_CHUNK; }
 
 // Tensor map of one tiled operand copy: rows of 64 bf16 (128 B, contiguous), 128-row boxes.
 const char *tc_make_map(void *out_map, void *base, int W, int npts, int d)
@@ -363,18 +400,24 @@ void launch_retile(const void *src, void *dst, int W, int npts, int d, cudaStrea
 
 void launch_update_tc(const Dev &P, const void *maps, int leg, int width, cudaStream_t st)
 {
+    // dynamic shared memory: the tiles, plus what it takes to start them on a 1024-byte boundary
+    static size_t pad[2] = {0, 0};
     static bool attr_set = false;
-    const size_t smem = tc_smem_bytes(P.d);
     if (!attr_set) {
-        cudaFuncSetAttribute(update_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc_smem_bytes(256));
-        cudaFuncSetAttribute(update_tc_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc_smem_bytes(512));
+        cudaFuncAttributes fa;
+        cudaFuncGetAttributes(&fa, update_tc_kernel<2, 128>);
+        pad[0] = (1024 - fa.sharedSizeBytes % 1024) % 1024;
+        cudaFuncGetAttributes(&fa, update_tc_kernel<3, 256>);
+        pad[1] = (1024 - fa.sharedSizeBytes % 1024) % 1024;
+        cudaFuncSetAttribute(update_tc_kernel<2, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(tc_smem_bytes(256) + pad[0]));
+        cudaFuncSetAttribute(update_tc_kernel<3, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(tc_smem_bytes(512) + pad[1]));
         attr_set = true;
     }
     const CUtensorMap *tm = reinterpret_cast<const CUtensorMap *>(maps);
     const int nrows = (leg == LEG_F) ? P.n : P.m;
     dim3 grid((nrows + TC_BM - 1) / TC_BM, width < 1 ? 1 : width);
-    if (tc_stages(P.d) == 2) launch_pdl(update_tc_kernel<2>, grid, dim3(TC_THREADS), smem, st, tm[0], tm[1], P, leg);
-    else launch_pdl(update_tc_kernel<4>, grid, dim3(TC_THREADS), smem, st, tm[0], tm[1], P, leg);
+    if (!tc_wide(P.d)) launch_pdl(update_tc_kernel<2, 128>, grid, dim3(TC_THREADS), tc_smem_bytes(P.d) + pad[0], st, tm[0], tm[1], P, leg);
+    else launch_pdl(update_tc_kernel<3, 256>, grid, dim3(TC_THREADS), tc_smem_bytes(P.d) + pad[1], st, tm[0], tm[1], P, leg);
 }
 
 }  // namespace skb
