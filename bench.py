@@ -34,7 +34,7 @@ UNIT = "lane*n*m updates/s"
 # DRAM bytes (read + write) of ONE full-width f-leg launch of the dominant kernel, taken from ncu
 # captures of `bench.py --workload <name> --kernel-only` (one launch each; they equal the lanes'
 # operands read once)
-NCU_TRAFFIC_BYTES = {"sensor": 20.5e6, "registration": 13.7e6, "sweep": 42.0e6, "feature": 141.0e6}
+NCU_TRAFFIC_BYTES = {"sensor": 20.5e6, "registration": 13.7e6, "sweep": 42.0e6, "feature": 140.8e6}
 
 # nominal unit counts (148 SMs, 128 FP32 lanes and 16 special-function lanes per SM per clock,
 # 64 FP64 lanes) at the maximum SM clock; the fraction reported is against these
