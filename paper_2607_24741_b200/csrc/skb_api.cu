@@ -296,7 +296,7 @@ extern "C" skb_status sinkhorn_batch_drain(skb_batch *h, int *cycles_run)
 {
     if (!h) return SKB_ERR_NULL;
     cudaError_t e;
-    int chunk = 2, snap = 0;
+    int chunk = 2, snap = 0, rounds = 0;
     bool have_prev = false;
     // every lane is retired by the audit that follows cycle max_iter; STATIC needs one more pass
     const long long hard_cap = (long long)h->cfg.max_iter + 4;
@@ -312,7 +312,9 @@ extern "C" skb_status sinkhorn_batch_drain(skb_batch *h, int *cycles_run)
         }
         have_prev = true;
         snap ^= 1;
-        if (chunk < 16) chunk *= 2;
+        // grow the chunk every other round: cycles enqueued past completion are empty launches that
+        // still have to drain, which matters for batches that finish within a dozen cycles
+        if (chunk < 16 && (++rounds & 1) == 0) chunk *= 2;
         if (h->enqueued > hard_cap + 64) break;
     }
     if ((e = cudaStreamSynchronize(h->stream)) != cudaSuccess) return cuda_fail(h, e, "drain");
