@@ -18,7 +18,9 @@
  * Conventions
  *   - Every data pointer is DEVICE memory owned by the caller unless it says
  *     "host".  Inputs are const and never modified.  The library allocates no
- *     device memory: all of its state lives in the caller's workspace.
+ *     device memory: all of its state lives in the caller's workspace.  (Host side, a
+ *     handle borrows a 128-byte pinned block and two events from a small per-device pool
+ *     that the library keeps for the life of the process.)
  *   - All work is enqueued on the stream given at creation.
  *   - Every call returns an skb_status; nothing throws or aborts.  The text of
  *     the last error is available from sinkhorn_batch_last_error().

@@ -5,7 +5,9 @@
 #include <cstdio>
 #include <cstring>
 #include <new>
+#include <mutex>
 #include <string>
+#include <vector>
 
 #include "../../include/sinkhorn_batch.h"
 #include "skb_host.h"
@@ -23,12 +25,45 @@ struct skb_batch {
     bool finished;
     long long enqueued;    // cycles enqueued so far
     long long launches;    // kernels launched so far
+    int res_device;        // device the pooled host resources belong to
     bool tensor;           // the tensor-core update kernel is in use
     alignas(64) unsigned char maps[2 * 128];   // CUtensorMap of x and of y
     std::string err;
 };
 
 static std::string g_create_err;
+
+// Host-side resources of a handle (a pinned control-block pair and two events) are recycled
+// through a small per-device pool: allocating and freeing pinned memory costs hundreds of
+// microseconds, which would dominate short solves created in a loop.
+struct HostRes { Ctl *pinned; cudaEvent_t ev[2]; int device; };
+static std::mutex g_pool_mu;
+static std::vector<HostRes> g_pool;
+
+static cudaError_t host_res_get(HostRes *r)
+{
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    {
+        std::lock_guard<std::mutex> lk(g_pool_mu);
+        for (size_t i = 0; i < g_pool.size(); ++i)
+            if (g_pool[i].device == dev) { *r = g_pool[i]; g_pool.erase(g_pool.begin() + i); return cudaSuccess; }
+    }
+    r->device = dev; r->pinned = nullptr; r->ev[0] = r->ev[1] = nullptr;
+    if ((e = cudaHostAlloc((void **)&r->pinned, 2 * sizeof(Ctl), cudaHostAllocDefault)) != cudaSuccess) return e;
+    if ((e = cudaEventCreateWithFlags(&r->ev[0], cudaEventDisableTiming)) != cudaSuccess) return e;
+    return cudaEventCreateWithFlags(&r->ev[1], cudaEventDisableTiming);
+}
+
+static void host_res_put(const HostRes &r)
+{
+    std::lock_guard<std::mutex> lk(g_pool_mu);
+    if (g_pool.size() < 64) { g_pool.push_back(r); return; }
+    if (r.ev[0]) cudaEventDestroy(r.ev[0]);
+    if (r.ev[1]) cudaEventDestroy(r.ev[1]);
+    if (r.pinned) cudaFreeHost(r.pinned);
+}
 
 // fp32 arithmetic: the expanded cost |x|^2+|y|^2-2x.y carries an error of about one ulp of the
 // scaled squared radius M = s*max|x-c|^2 into every exponent.  Above FORM_DIFF_RADIUS a lane
@@ -187,9 +222,10 @@ extern "C" skb_status sinkhorn_batch_create(const void *x, const void *y, const 
     h->dev.tol_stop = (double)tol;
     h->dev.tol_screen = cfg->tol_screen > 0.0f ? (double)cfg->tol_screen : (double)tol;
     cudaError_t e;
-    if ((e = cudaHostAlloc((void **)&h->h_ctl, 2 * sizeof(Ctl), cudaHostAllocDefault)) != cudaSuccess ||
-        (e = cudaEventCreateWithFlags(&h->ev[0], cudaEventDisableTiming)) != cudaSuccess ||
-        (e = cudaEventCreateWithFlags(&h->ev[1], cudaEventDisableTiming)) != cudaSuccess) {
+    HostRes res;
+    e = host_res_get(&res);
+    h->h_ctl = res.pinned; h->ev[0] = res.ev[0]; h->ev[1] = res.ev[1]; h->res_device = res.device;
+    if (e != cudaSuccess) {
         skb_status st = cuda_fail(nullptr, e, "create");
         sinkhorn_batch_destroy(h);
         return st;
@@ -518,9 +554,14 @@ extern "C" void sinkhorn_batch_destroy(skb_batch *h)
 {
     if (!h) return;
     if (h->stream || h->h_ctl) cudaStreamSynchronize(h->stream);
-    if (h->ev[0]) cudaEventDestroy(h->ev[0]);
-    if (h->ev[1]) cudaEventDestroy(h->ev[1]);
-    if (h->h_ctl) cudaFreeHost(h->h_ctl);
+    if (h->h_ctl && h->ev[0] && h->ev[1]) {
+        HostRes r; r.pinned = h->h_ctl; r.ev[0] = h->ev[0]; r.ev[1] = h->ev[1]; r.device = h->res_device;
+        host_res_put(r);
+    } else {
+        if (h->ev[0]) cudaEventDestroy(h->ev[0]);
+        if (h->ev[1]) cudaEventDestroy(h->ev[1]);
+        if (h->h_ctl) cudaFreeHost(h->h_ctl);
+    }
     delete h;
 }
 
