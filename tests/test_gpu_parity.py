@@ -367,3 +367,23 @@ def test_bounded_wait_gives_up_instead_of_hanging():
     assert 5e3 <= kclk <= 5e5           # ~10 M clocks budget: it neither returned at once nor spun for long
     # the context is still usable
     assert int(torch.arange(10, device="cuda:0").sum().item()) == 45
+
+
+def test_very_wide_batch_and_rectangular_lanes(oracle):
+    # more lanes than the planner has threads: its scans run in several chunks, holes and fillers
+    # pair up across chunks
+    w = wl.make("sweep", W=2500, n=8, m=9, max_iter=600)
+    r = run_gpu(w, mode="active", compute="f64")
+    lanes = [0, 1, 1023, 1024, 1025, 2047, 2048, 2499] + list(range(300, 2500, 211))
+    assert check_against_oracle(oracle, w, r, lanes, pot_tol=POT_TOL_F64, exact_depth=True, max_iter=600) == []
+    check_accounting(oracle, r, 2500, "active")
+    rm = run_gpu(w, mode="masked", compute="f64")
+    np.testing.assert_array_equal(rm["depth"], r["depth"]); np.testing.assert_array_equal(rm["f"], r["f"])
+    # few sources, many targets (and the reverse): row blocks and column tiles of very different counts
+    for n, m in ((5, 700), (700, 5)):
+        w = wl.make("sensor", W=3, n=n, m=m)
+        for compute in ("f64", "auto"):
+            r = run_gpu(w, compute=compute)
+            misses = check_against_oracle(oracle, w, r, range(3), pot_tol=POT_TOL_F64 if compute == "f64" else POT_TOL_F32,
+                                          exact_depth=compute == "f64")
+            assert misses == []
