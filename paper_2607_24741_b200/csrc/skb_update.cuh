@@ -315,6 +315,7 @@ __device__ __forceinline__ void stream_f64(double *sm, const double *colc, const
                                            const int cp, const int ncols,
                                            const double (&xr)[Tune<double, DP>::R][DP],
                                            const int tid, const int cs,
+                                           const float (&m0)[Tune<double, DP>::R],
                                            float (&mx)[Tune<double, DP>::R], double (&sd)[Tune<double, DP>::R])
 {
     constexpr int R = Tune<double, DP>::R, CW = Tune<double, DP>::CW;
@@ -326,7 +327,7 @@ __device__ __forceinline__ void stream_f64(double *sm, const double *colc, const
     float ts[R];
     double md[R];
 #pragma unroll
-    for (int r = 0; r < R; ++r) { mx[r] = NEG_BIG; md[r] = (double)NEG_BIG; ts[r] = 0.f; sd[r] = 0.0; }
+    for (int r = 0; r < R; ++r) { mx[r] = m0[r]; md[r] = (double)m0[r]; ts[r] = 0.f; sd[r] = 0.0; }
 
     const int ntiles = (ncols + TJ - 1) / TJ;
     load_tile<double, DP, TJ, NR>(sm, colc, colt, colt, cp, 0, tid);
@@ -578,24 +579,59 @@ __global__ void __launch_bounds__(UPD_THREADS) update_kernel(const Dev P, const 
 
     float mx[R];
     double sd[R];
-    if constexpr (sizeof(T) == 4) {
-        if (form == FORM_DOT) stream_f32<DP, CS, FORM_DOT>(sm, colc, colt, coll, cp, ncols, xr, ph, tid, cs, mx, sd);
-        else stream_f32<DP, CS, FORM_DIFF>(sm, colc, colt, coll, cp, ncols, xr, ph, tid, cs, mx, sd);
-    } else {
-        stream_f64<DP, CS, XF>(sm, colc, colt, cp, ncols, xr, tid, cs, mx, sd);
-    }
-
-    // merge the CS column splits of each row: maxima are integers, so the scalings are exact
+    // Where the exponential runs in fp32 on float64 arguments, the reference point of each row
+    // starts at the value its log-sum-exp takes if the potential does not move in this leg
+    // (Eq. 3 solved for the sum: L = log2 w + s|x|^2 - phi_old).  Near convergence that is within
+    // a fraction of a unit of the truth, so the rescale branch of the streaming loop stays cold.
+    // A reference far too HIGH would push every term towards the flush-to-zero range: such a CTA
+    // repeats the pass from "minus infinity", as the other arithmetic modes always do.
+    float m0[R];
 #pragma unroll
-    for (int off = 1; off < CS; off <<= 1) {
+    for (int r = 0; r < R; ++r) m0[r] = NEG_BIG;
+    if constexpr (sizeof(T) == 8 && XF != 0) {
 #pragma unroll
         for (int r = 0; r < R; ++r) {
-            const float mo = __shfl_xor_sync(0xffffffffu, mx[r], off * RG);
-            const double so = __shfl_xor_sync(0xffffffffu, sd[r], off * RG);
-            const float mn = fmaxf(mx[r], mo);
-            sd[r] = sd[r] * (double)pow2i(mx[r] - mn) + so * (double)pow2i(mo - mn);
-            mx[r] = mn;
+            if (row0 + r < nrows) {
+                const size_t o = (size_t)slot * rp + row0 + r;
+                const double est = (rows_x ? P.la2 : P.lb2)[o] + (rows_x ? P.sqx : P.sqy)[o] - prow[row0 + r];
+                if (fabs(est) < 1.0e7) m0[r] = ceilf((float)est);
+            }
         }
+    }
+#pragma unroll 1
+    for (int pass = 0; pass < 2; ++pass) {
+        if constexpr (sizeof(T) == 4) {
+            if (form == FORM_DOT) stream_f32<DP, CS, FORM_DOT>(sm, colc, colt, coll, cp, ncols, xr, ph, tid, cs, mx, sd);
+            else stream_f32<DP, CS, FORM_DIFF>(sm, colc, colt, coll, cp, ncols, xr, ph, tid, cs, mx, sd);
+        } else {
+            stream_f64<DP, CS, XF>(sm, colc, colt, cp, ncols, xr, tid, cs, m0, mx, sd);
+        }
+
+        // merge the CS column splits of each row: maxima are integers, so the scalings are exact
+#pragma unroll
+        for (int off = 1; off < CS; off <<= 1) {
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                const float mo = __shfl_xor_sync(0xffffffffu, mx[r], off * RG);
+                const double so = __shfl_xor_sync(0xffffffffu, sd[r], off * RG);
+                const float mn = fmaxf(mx[r], mo);
+                sd[r] = sd[r] * (double)pow2i(mx[r] - mn) + so * (double)pow2i(mo - mn);
+                mx[r] = mn;
+            }
+        }
+        if constexpr (sizeof(T) == 8 && XF != 0) {
+            if (pass == 0) {
+                bool low = false;
+#pragma unroll
+                for (int r = 0; r < R; ++r)
+                    low = low || (row0 + r < nrows && m0[r] != NEG_BIG && !(sd[r] >= 0x1p-20));
+                if (!__syncthreads_or(low ? 1 : 0)) break;
+#pragma unroll
+                for (int r = 0; r < R; ++r) m0[r] = NEG_BIG;
+                continue;
+            }
+        }
+        break;
     }
     if (cs == 0) {
 #pragma unroll

@@ -387,3 +387,24 @@ def test_very_wide_batch_and_rectangular_lanes(oracle):
             misses = check_against_oracle(oracle, w, r, range(3), pot_tol=POT_TOL_F64 if compute == "f64" else POT_TOL_F32,
                                           exact_depth=compute == "f64")
             assert misses == []
+
+
+def test_mixed_arithmetic_with_a_useless_reference_estimate(oracle):
+    # Clouds ten units apart at a small eps: starting from zero potentials, the first legs move
+    # every potential by thousands of log2 units, so a reference point estimated from the old
+    # potential is off by far more than the fp32 exponent range.  The kernel must notice and
+    # repeat such a pass from scratch; otherwise every term flushes to zero and the lanes blow up.
+    rng = np.random.default_rng(7)
+    W, n, m, d = 6, 70, 90, 3
+    x = rng.random((W, n, d), dtype=np.float32)
+    y = rng.random((W, m, d), dtype=np.float32) + np.float32(10.0)
+    a = rng.random((W, n), dtype=np.float32) + 0.5; a /= a.sum(1, keepdims=True)
+    b = rng.random((W, m), dtype=np.float32) + 0.5; b /= b.sum(1, keepdims=True)
+    eps = np.linspace(0.03, 0.2, W).astype(np.float32)
+    w = wl.Workload("far_apart", x, y, a.astype(np.float32), b.astype(np.float32), eps, 1e-5, 5000)
+    for mode in ("active", "static"):
+        r = run_gpu(w, mode=mode, compute="mixed")
+        assert (r["status"] == oracle.DONE).all()
+        misses = check_against_oracle(oracle, w, r, range(W), pot_tol=POT_TOL_F32, exact_depth=False)
+        for t, dg, do, margin, decay in misses:
+            assert miss_allowed(margin, decay, MARGIN_AUTO)
