@@ -427,77 +427,63 @@ __device__ __forceinline__ void stream_f64(double *sm, const double *colc, const
     }
 }
 
-// Float64 epilogue of a CTA's RB rows (one thread per row) and the fused residual reduction.
-// row_m / row_s hold, per CTA-local row, the integer-valued maximum and the sum of
-// 2^(arg - max) over ALL columns; row_h the fp32 shift a difference-form row carried.
-template <typename T, int RB, int THREADS = UPD_THREADS>
-__device__ __forceinline__ void finish_rows(const Dev &P, const Ctl &c, const int leg, const int slot,
-                                            const int form, const float *row_m, const double *row_s,
-                                            const float *row_h, double *red, int *is_last)
+// Float64 epilogue of ONE row of a leg: `m` is the integer-valued maximum and `s` the sum of
+// 2^(arg - m) over ALL columns, `h` the fp32 shift a difference-form row carried.  Writes the
+// updated potential (unless the leg only checks, or the lane is frozen) and returns the row's
+// term of the marginal residual (zero for the g-leg, which measures nothing).
+template <typename T>
+__device__ __forceinline__ double finish_one_row(const Dev &P, const Ctl &c, const int leg, const int slot, const int form,
+                                                 const int i, const float m, const double s, const float h, const bool writes)
 {
-    constexpr int NWARP = THREADS / 32;
     const bool rows_x = (leg == LEG_F);
-    const int nrows = rows_x ? P.n : P.m, rp = rows_x ? P.np : P.mp;
+    const int rp = rows_x ? P.np : P.mp;
     const double *prow = (rows_x ? P.phi[c.parity] : P.gam) + (size_t)slot * rp;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const bool frozen = (P.mode == MODE_MASKED) && P.state[slot] != 0;
-    const bool writes = !frozen && leg != LEG_V;
-    double term_sum = 0.0;
-    for (int lr = tid; lr < RB; lr += THREADS) {
-        const int i = blockIdx.x * RB + lr;
-        if (i >= nrows) continue;
-        const size_t o = (size_t)slot * rp + i;
-        const double lw = (rows_x ? P.la2 : P.lb2)[o];
-        const double sq = (rows_x ? P.sqx : P.sqy)[o];
-        const double pold = prow[i];
-        const double L = (double)row_m[lr] + log2(row_s[lr]);
-        // log2 of this row's marginal under the potentials the leg started from, and the
-        // updated potential that makes the marginal equal to the weight (Eq. 3)
-        double lmarg, pnew;
-        if (form == FORM_DOT) {
-            pnew = lw + sq - L;
-            lmarg = lw + pold - pnew;
+    const size_t o = (size_t)slot * rp + i;
+    const double lw = (rows_x ? P.la2 : P.lb2)[o];
+    const double sq = (rows_x ? P.sqx : P.sqy)[o];
+    const double pold = prow[i];
+    const double L = (double)m + log2(s);
+    // log2 of this row's marginal under the potentials the leg started from, and the
+    // updated potential that makes the marginal equal to the weight (Eq. 3)
+    double lmarg, pnew;
+    if (form == FORM_DOT) {
+        pnew = lw + sq - L;
+        lmarg = lw + pold - pnew;
+    } else {
+        lmarg = L - ((double)h - pold);
+        pnew = pold + (lw - lmarg);
+    }
+    double term = 0.0;
+    if (leg != LEG_G) term = (rows_x ? P.wa : P.wb)[o] * fabs(expm1((lmarg - lw) * 0.6931471805599453));
+    if (writes) {
+        T hi, lo;
+        if (form == FORM_DOT) { hi = (T)(pnew - sq); lo = T(0); }
+        else { hi = (T)pnew; lo = (T)(pnew - (double)hi); }
+        if (leg == LEG_F) {
+            P.phi[c.parity ^ 1][o] = pnew;
+            reinterpret_cast<T *>(P.ft[c.parity ^ 1])[o] = hi;
+            reinterpret_cast<T *>(P.fl[c.parity ^ 1])[o] = lo;
         } else {
-            lmarg = L - ((double)row_h[lr] - pold);
-            pnew = pold + (lw - lmarg);
-        }
-        if (leg != LEG_G) term_sum += (rows_x ? P.wa : P.wb)[o] * fabs(expm1((lmarg - lw) * 0.6931471805599453));
-        if (writes) {
-            T hi, lo;
-            if (form == FORM_DOT) { hi = (T)(pnew - sq); lo = T(0); }
-            else { hi = (T)pnew; lo = (T)(pnew - (double)hi); }
-            if (leg == LEG_F) {
-                P.phi[c.parity ^ 1][o] = pnew;
-                reinterpret_cast<T *>(P.ft[c.parity ^ 1])[o] = hi;
-                reinterpret_cast<T *>(P.fl[c.parity ^ 1])[o] = lo;
-            } else {
-                P.gam[o] = pnew;
-                reinterpret_cast<T *>(P.gt)[o] = hi;
-                reinterpret_cast<T *>(P.gl)[o] = lo;
-            }
+            P.gam[o] = pnew;
+            reinterpret_cast<T *>(P.gt)[o] = hi;
+            reinterpret_cast<T *>(P.gl)[o] = lo;
         }
     }
-    if (leg == LEG_G) return;
+    return term;
+}
 
-    // fused marginal-residual reduction -> one flag per lane (fixed summation order)
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) term_sum += __shfl_down_sync(0xffffffffu, term_sum, off);
-    if (lane == 0) red[warp] = term_sum;
-    __syncthreads();
+// One thread per row block hands in its block's residual sum; the last block of the lane to
+// arrive adds all of them in block order (fixed summation order) and sets the lane's flags.
+// Returns true for that last block.
+__device__ __forceinline__ bool finish_lane_residual(const Dev &P, const Ctl &c, const int leg, const int slot,
+                                                     const int nblk, const int blk, const double block_sum, const bool frozen)
+{
     double *parts = (leg == LEG_F ? P.part_row : P.part_col) + (size_t)slot * MAX_PARTS;
     unsigned *cnt = (leg == LEG_F ? P.cnt_row : P.cnt_col) + slot;
-    const int nblk = (nrows + RB - 1) / RB;
-    if (tid == 0) {
-        double s = 0.0;
-#pragma unroll
-        for (int w = 0; w < NWARP; ++w) s += red[w];
-        parts[blockIdx.x] = s;
-        __threadfence();
-        const unsigned ticket = atomicAdd(cnt, 1u);
-        *is_last = (ticket == (unsigned)(nblk - 1));
-    }
-    __syncthreads();
-    if (!*is_last || tid != 0) return;
+    parts[blk] = block_sum;
+    __threadfence();
+    const unsigned ticket = atomicAdd(cnt, 1u);
+    if (ticket != (unsigned)(nblk - 1)) return false;
     __threadfence();
     double tot = 0.0;
     for (int b = 0; b < nblk; ++b) tot += reinterpret_cast<volatile double *>(parts)[b];
@@ -515,6 +501,42 @@ __device__ __forceinline__ void finish_rows(const Dev &P, const Ctl &c, const in
         P.verdict[slot] = (finite && two <= P.tol_stop) ? 1 : 0;
         if (!finite) P.nonfinite[slot] = 1;
     }
+    return true;
+}
+
+// Float64 epilogue of a CTA's RB rows (one thread per row) and the fused residual reduction.
+// row_m / row_s hold, per CTA-local row, the integer-valued maximum and the sum of
+// 2^(arg - max) over ALL columns; row_h the fp32 shift a difference-form row carried.
+template <typename T, int RB, int THREADS = UPD_THREADS>
+__device__ __forceinline__ void finish_rows(const Dev &P, const Ctl &c, const int leg, const int slot,
+                                            const int form, const float *row_m, const double *row_s,
+                                            const float *row_h, double *red, int *is_last)
+{
+    constexpr int NWARP = THREADS / 32;
+    const int nrows = (leg == LEG_F) ? P.n : P.m;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const bool frozen = (P.mode == MODE_MASKED) && P.state[slot] != 0;
+    const bool writes = !frozen && leg != LEG_V;
+    double term_sum = 0.0;
+    for (int lr = tid; lr < RB; lr += THREADS) {
+        const int i = blockIdx.x * RB + lr;
+        if (i >= nrows) continue;
+        term_sum += finish_one_row<T>(P, c, leg, slot, form, i, row_m[lr], row_s[lr], row_h[lr], writes);
+    }
+    if (leg == LEG_G) return;
+
+    // fused marginal-residual reduction -> one flag per lane
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) term_sum += __shfl_down_sync(0xffffffffu, term_sum, off);
+    if (lane == 0) red[warp] = term_sum;
+    __syncthreads();
+    if (tid == 0) {
+        double s = 0.0;
+#pragma unroll
+        for (int w = 0; w < NWARP; ++w) s += red[w];
+        finish_lane_residual(P, c, leg, slot, (nrows + RB - 1) / RB, blockIdx.x, s, frozen);
+    }
+    (void)is_last;
 }
 
 template <typename T, int DP, int CS, int XF>

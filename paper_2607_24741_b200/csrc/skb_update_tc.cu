@@ -27,13 +27,16 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <cstdio>
+#include <cstdlib>
 
 #include "skb_update.cuh"
 #include "skb_host.h"
 
 namespace skb {
 
-constexpr int TC_THREADS = 192;
+constexpr int TC_EPI_WARPS = 8;                            // two per scheduler: lanes (w & 3), column half (w >> 2)
+constexpr int TC_EPI_THREADS = TC_EPI_WARPS * 32;
+constexpr int TC_THREADS = TC_EPI_THREADS + 64;            // + producer warp + MMA warp
 constexpr int TC_MAX_STAGES = 4;
 constexpr int TC_BM = 128, TC_BK = 64;
 constexpr uint32_t TC_CHUNK = TC_BM * TC_BK * 2;          // 16 KB: 128 points x 64 bf16
@@ -63,6 +66,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t a, uint32_t parity)
 // Bounded wait: false if the budget ran out or another role already gave up.
 __device__ __forceinline__ bool mbar_wait(uint32_t a, uint32_t parity, volatile int *abort_flag)
 {
+    if (mbar_try_wait(a, parity)) return true;          // the common case costs no clock read
     const long long t0 = clock64();
     while (!mbar_try_wait(a, parity)) {
         if (*abort_flag) return false;
@@ -92,9 +96,9 @@ __device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t
     asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
                  ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
-__device__ __forceinline__ void tc_ld32(uint32_t taddr, float (&v)[32])
+// 32 consecutive fp32 columns of this thread's TMEM lane; asynchronous until tc_ld_wait()
+__device__ __forceinline__ void tc_ld32_issue(uint32_t taddr, uint32_t (&r)[32])
 {
-    uint32_t r[32];
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
         "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
@@ -104,9 +108,122 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, float (&v)[32])
           "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
           "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
         : "r"(taddr) : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+// Completes every load this thread has issued.  The registers pass through the statement so
+// that the compiler cannot move a use of them above it.
+__device__ __forceinline__ void tc_ld_wait(uint32_t (&r)[32])
+{
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+        : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+          "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
+          "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
+          "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+        :: "memory");
+}
+
+// Online max / sum-of-exp2 over one 32-column chunk of a row: arg = 2 s S + ct_j, computed
+// on column pairs with packed fp32 instructions.  The running reference mx is NOT updated on
+// the fast path: the exponentials are taken against the reference as it stands and only their
+// sum is tested.  A sum above 2^10 (some argument more than ~5 above the reference, which
+// would cost exponent accuracy; a reference of minus infinity gives an infinite sum) sends
+// the chunk through the exact path: maximum, integer-valued new reference, exact rescale.
+// The reference therefore is always the ceiling of a true argument of this row, so terms can
+// never all underflow.
+__device__ __forceinline__ void tc_reduce_chunk(const uint32_t (&r)[32], const float *gt, const float two_s,
+                                                float &mx, float &ts, double &sd)
+{
+    u64 v[16];
+    const u64 s2 = pack2(two_s, two_s);
+    const u64 nm = pack2(-mx, -mx);
+    u64 acc[2] = {0ull, 0ull};
 #pragma unroll
-    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+    for (int q = 0; q < 32; q += 4) {
+        const float4 g = *reinterpret_cast<const float4 *>(gt + q);
+        v[q / 2] = fma2(pack2(__uint_as_float(r[q]), __uint_as_float(r[q + 1])), s2, pack2(g.x, g.y));
+        v[q / 2 + 1] = fma2(pack2(__uint_as_float(r[q + 2]), __uint_as_float(r[q + 3])), s2, pack2(g.z, g.w));
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            float d0, d1;
+            unpack2(add2(v[q / 2 + h], nm), d0, d1);
+            acc[h] = add2(acc[h], pack2(ex2_fast(d0), ex2_fast(d1)));
+        }
+    }
+    float a0, a1, a2, a3;
+    unpack2(acc[0], a0, a1);
+    unpack2(acc[1], a2, a3);
+    float sc = (a0 + a1) + (a2 + a3);
+    if (!(sc <= 1024.f)) {
+        float m4[4] = {NEG_BIG, NEG_BIG, NEG_BIG, NEG_BIG};
+#pragma unroll
+        for (int q = 0; q < 16; q += 2) {
+            float x0, x1, x2, x3;
+            unpack2(v[q], x0, x1);
+            unpack2(v[q + 1], x2, x3);
+            m4[0] = fmaxf(m4[0], x0); m4[1] = fmaxf(m4[1], x1);
+            m4[2] = fmaxf(m4[2], x2); m4[3] = fmaxf(m4[3], x3);
+        }
+        const float mt = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
+        if (mt > mx) {                                  // always, unless the sum itself was not finite
+            const float mn = ceilf(mt);
+            const float fac = pow2i(mx - mn);
+            ts *= fac;
+            sd *= (double)fac;
+            mx = mn;
+        }
+        float s4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int q = 0; q < 16; q += 2) {
+            float x0, x1, x2, x3;
+            unpack2(v[q], x0, x1);
+            unpack2(v[q + 1], x2, x3);
+            s4[0] += ex2_fast(x0 - mx); s4[1] += ex2_fast(x1 - mx);
+            s4[2] += ex2_fast(x2 - mx); s4[3] += ex2_fast(x3 - mx);
+        }
+        sc = (s4[0] + s4[1]) + (s4[2] + s4[3]);
+    }
+    ts += sc;
+}
+
+// One accumulator tile of BN columns: this warp's half of the 32-column chunks (even or odd),
+// the next chunk's tensor-memory load in flight while the current one is reduced.
+template <int BN>
+__device__ __forceinline__ void tc_reduce_tile(const uint32_t taddr, const float *gt, const int half, const float two_s,
+                                               float &mx, float &ts, double &sd)
+{
+    constexpr int NCH = BN / 64;                   // chunks per warp
+    static_assert(NCH % 2 == 0, "chunks are processed in pairs");
+    uint32_t ra[32], rb[32];
+    tc_ld32_issue(taddr + (uint32_t)(half * 32), ra);
+    tc_ld_wait(ra);
+#pragma unroll
+    for (int i = 0; i < NCH; i += 2) {
+        const int c0 = (2 * i + half) * 32, c1 = c0 + 64;
+        tc_ld32_issue(taddr + (uint32_t)c1, rb);
+        tc_reduce_chunk(ra, gt + c0, two_s, mx, ts, sd);
+        tc_ld_wait(rb);
+        if (i + 2 < NCH) tc_ld32_issue(taddr + (uint32_t)(c1 + 64), ra);
+        tc_reduce_chunk(rb, gt + c1, two_s, mx, ts, sd);
+        if (i + 2 < NCH) tc_ld_wait(ra);
+    }
+}
+
+// Merges the two column halves of every row (warps 4-7 hand theirs to warps 0-3 through `xm`,
+// `xs`: 128 floats and 128 doubles of shared memory nobody else uses any more) and leaves the
+// row results where finish_rows expects them.  Called by all epilogue threads.
+__device__ __forceinline__ void tc_merge_halves(const int e, const float mx, const double sd, const bool ok,
+                                                float *xm, double *xs, float *row_m, double *row_s, float *row_h)
+{
+    const int row = e & 127;
+    if (e >= 128) { xm[row] = mx; xs[row] = ok ? sd : __longlong_as_double(0x7ff8000000000000LL); }
+    asm volatile("bar.sync 1, 256;" ::: "memory");     // also: every row is done with the column terms
+    if (e < 128) {
+        const float mo = xm[row];
+        const double so = xs[row];
+        const float mn = fmaxf(mx, mo);
+        row_m[row] = mn;
+        row_s[row] = ok ? sd * (double)pow2i(mx - mn) + so * (double)pow2i(mo - mn) : __longlong_as_double(0x7ff8000000000000LL);
+        row_h[row] = 0.f;
+    }
 }
 // shared-memory matrix descriptor: K-major tile, rows of 64 bf16 (128 B), 128-byte swizzle,
 // 8-row groups 1024 B apart
@@ -118,7 +235,7 @@ __device__ __forceinline__ uint64_t tc_desc(uint32_t saddr)
 __host__ __device__ constexpr uint32_t tc_idesc(int bn) { return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24); }
 
 template <int TC_STAGES, int TC_BN>
-__global__ void __launch_bounds__(TC_THREADS, 1)
+__global__ void __launch_bounds__(TC_THREADS, TC_BN == 128 ? 2 : 1)
 update_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUtensorMap tmy, const Dev P, const int leg)
 {
     extern __shared__ __align__(1024) unsigned char smem_tc[];
@@ -170,11 +287,11 @@ update_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant_
     if (tid == 0) {
         for (int s = 0; s < TC_STAGES; ++s) { mbar_init(b_full + 8 * s, 1); mbar_init(b_empty + 8 * s, 1); }
         mbar_init(b_a, 1);
-        for (int b = 0; b < 2; ++b) { mbar_init(b_tfull + 8 * b, 1); mbar_init(b_tempty + 8 * b, 128); }
+        for (int b = 0; b < 2; ++b) { mbar_init(b_tfull + 8 * b, 1); mbar_init(b_tempty + 8 * b, TC_EPI_THREADS); }
         abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 5) {
+    if (warp == TC_EPI_WARPS + 1) {
         if (TC_BN == 256) asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(&tmem_holder)) : "memory");
         else asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 256;" ::"r"(smem_u32(&tmem_holder)) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -191,7 +308,7 @@ update_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant_
     const long long dbg_t0 = clock64();
     (void)dbg_w0; (void)dbg_w1; (void)dbg_t0;
 
-    if (warp == 4) {
+    if (warp == TC_EPI_WARPS) {
         // ---------------- producer
         if (lane == 0) {
             // the row block rides on the first tile's ring barriers, chunk by chunk, so the first
@@ -215,7 +332,7 @@ update_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant_
                 }
             }
         }
-    } else if (warp == 5) {
+    } else if (warp == TC_EPI_WARPS + 1) {
         // ---------------- MMA issuer
         if (lane == 0) {
             bool ok = true;
@@ -243,50 +360,31 @@ update_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant_
             }
         }
     } else {
-        // ---------------- epilogue: thread e <-> row e <-> TMEM lane e
-        const int e = tid;
-        const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
+        // ---------------- epilogue: thread e <-> row (e & 127) <-> TMEM lane (e & 127); warps 0-3 take
+        // the even 32-column chunks of every tile, warps 4-7 the odd ones
+        const int e = tid, half = warp >> 2;
+        const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
         bool ok = true;
+        float ts = 0.f;
         for (int t = 0; t < ntiles && ok; ++t) {
             const int buf = t & 1;
-#pragma unroll
-            for (int h = 0; h < TC_BN / 128; ++h) {
-                const int j = t * TC_BN + h * 128 + e;
-                gts[buf][h * 128 + e] = (j < cp) ? colt[j] : NEG_BIG;
+            for (int q = e; q < TC_BN; q += TC_EPI_THREADS) {
+                const int j = t * TC_BN + q;
+                gts[buf][q] = (j < cp) ? colt[j] : NEG_BIG;
             }
-            asm volatile("bar.sync 1, 128;" ::: "memory");
+            asm volatile("bar.sync 1, 256;" ::: "memory");
             ok = TC_TIMED_WAIT(dbg_w0, mbar_wait(b_tfull + 8 * buf, (t >> 1) & 1, ab));
             if (!ok) break;
             tc_fence_after();
-            float ts = 0.f;
-#pragma unroll 1
-            for (int cb = 0; cb < TC_BN; cb += 32) {
-                float v[32];
-                tc_ld32(lane_base + (uint32_t)(buf * TC_BN + cb), v);
-                float mt = NEG_BIG;
-#pragma unroll
-                for (int q = 0; q < 32; ++q) {
-                    v[q] = fmaf(v[q], two_s, gts[buf][cb + q]);
-                    mt = fmaxf(mt, v[q]);
-                }
-                if (mt > mx + 8.0f) {
-                    const float mn = ceilf(mt);
-                    const float fac = pow2i(mx - mn);
-                    ts *= fac;
-                    sd *= (double)fac;
-                    mx = mn;
-                }
-#pragma unroll
-                for (int q = 0; q < 32; ++q) ts += ex2_fast(v[q] - mx);
-            }
+            tc_reduce_tile<TC_BN>(lane_base + (uint32_t)(buf * TC_BN), gts[buf], half, two_s, mx, ts, sd);
             sd += (double)ts;
+            ts = 0.f;
             tc_fence_before();
-            mbar_arrive(b_tempty + 8 * buf);                // all 128 rows have read this accumulator
+            mbar_arrive(b_tempty + 8 * buf);                // all rows have read this accumulator
         }
-        asm volatile("bar.sync 1, 128;" ::: "memory");     // every row is done with the column terms
-        row_m[e] = mx;
-        row_s[e] = ok ? sd : __longlong_as_double(0x7ff8000000000000LL);
-        row_h[e] = 0.f;
+        // the ring is idle by now: its first bytes carry the second half's partial results
+        tc_merge_halves(e, mx, sd, ok, reinterpret_cast<float *>(smem_tc + (sB - smem_u32(smem_tc)) + 1024),
+                        reinterpret_cast<double *>(smem_tc + (sB - smem_u32(smem_tc))), row_m, row_s, row_h);
     }
     if (abort_flag) {
         // a wait ran out: give copies that may still be in flight time to land in this CTA's
@@ -295,14 +393,14 @@ update_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant_
         while (clock64() - t0 < 200000LL) { }
     }
 #ifdef SKB_TC_DEBUG
-    if (blockIdx.x == 1 && blockIdx.y == 3 && leg == LEG_F && (lane == 0) && (warp == 0 || warp >= 4))
+    if (blockIdx.x == 1 && blockIdx.y == 3 && leg == LEG_F && (lane == 0) && (warp == 0 || warp == 4 || warp >= TC_EPI_WARPS))
         printf("[tc dbg] warp %d: total %lld clk, wait0 %lld, wait1 %lld (producer: empty; mma: full, tmem-empty; epilogue: tmem-full) tiles %d chunks/tile %d\n",
                warp, clock64() - dbg_t0, dbg_w0, dbg_w1, ntiles, nkc);
 #endif
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    if (warp == 5) {
+    if (warp == TC_EPI_WARPS + 1) {
         if (TC_BN == 256) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
         else asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 256;" ::"r"(tmem) : "memory");
     }
@@ -310,6 +408,329 @@ update_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant_
         if (tid == 0) atomicOr(&P.ctl->error, ERR_WAIT);
     }
     finish_rows<float, TC_BM, TC_THREADS>(P, c, leg, slot, (int)FORM_DOT, row_m, row_s, row_h, red, &is_last);
+}
+
+// ---------------------------------------------------------------- CTA-pair variant
+// Two CTAs of a cluster (two SMs) work on 256 consecutive row points of one lane with
+// tcgen05.mma.cta_group::2 (M = 256: 128 rows per CTA, N = 256).  Each CTA keeps its own 128-row
+// block resident and streams only ITS half of every 256-column tile (128 points x 64 dimensions
+// = 16 KB per ring stage); the tensor cores of both SMs read both halves.  Per SM that halves
+// the L2 -> shared-memory traffic of the column operand and leaves room for a deeper ring
+// (six stages beside a 128 KB row block), which is what the single-CTA kernel is short of.
+//
+// Barriers (same offsets in both CTAs):  full[s]  lives in the leader (cluster rank 0): one
+// arrival by the leader's producer, which expects the bytes of BOTH CTAs' copies; the peer's
+// copies complete on the leader's barrier.  empty[s] and tfull[b] are per CTA: the leader's MMA
+// thread commits to its own and to the peer's.  tempty[b] lives in the leader and counts the
+// 256 epilogue threads of the pair (the peer's arrive remotely).  Every wait is bounded as in
+// the single-CTA kernel; the two cluster-wide barriers are plain hardware barriers that every
+// thread of both CTAs reaches on every path (the early exits above them depend on the lane
+// only, which the pair shares).
+__device__ __forceinline__ uint32_t cluster_rank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_barrier()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// as tma_load_chunk, but the completion barrier may live in the peer CTA of the pair
+__device__ __forceinline__ void tma_load_chunk_pair(uint32_t dst, const CUtensorMap *tm, int row, uint32_t mbar_cluster)
+{
+    asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(0), "r"(row), "r"(mbar_cluster) : "memory");
+}
+__device__ __forceinline__ void tc_commit_pair(uint32_t mbar_cluster)
+{
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(mbar_cluster) : "memory");
+}
+__device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// instruction descriptor of the pair: D fp32, A and B bf16 K-major, M = 256 (two CTAs), N = 256
+__host__ __device__ constexpr uint32_t tc_idesc_pair() { return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(256 >> 3) << 17) | ((uint32_t)(256 >> 4) << 24); }
+
+constexpr int TC2_BN = 256;               // columns per accumulator tile
+constexpr int TC2_MAX_STAGES = 8;
+constexpr int TC2_FILE_WARPS = 4;               // one thread per row of an item for the float64 epilogue
+constexpr int TC2_THREADS = TC_THREADS + 32 * TC2_FILE_WARPS;
+
+// all-threads AND over the 256 epilogue threads (they must leave their loops together)
+__device__ __forceinline__ bool epi_all(const bool ok)
+{
+    uint32_t r;
+    asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.b32 p, %1, 0;\n\tbar.red.and.pred q, 3, 256, p;\n\tselp.u32 %0, 1, 0, q;\n\t}"
+                 : "=r"(r) : "r"((uint32_t)ok) : "memory");
+    return r != 0;
+}
+
+// The kernel is PERSISTENT: the grid holds one cluster per SM pair and every cluster walks the
+// work items (lane, pair of row blocks) cluster-index + k * cluster-count, so barrier set-up,
+// tensor-memory allocation, the first loads of an item, the exponentials of its last tile and
+// its float64 epilogue all overlap the MMAs of the neighbouring items.  The ring, the
+// accumulator buffers and their barrier phases simply run on across items.  A row-block chunk
+// of the NEXT item may overwrite the resident copy as soon as the ring stage it travels with
+// has been released, because MMAs retire in order and the ring (nstages <= d/64 stages) is not
+// longer than a tile: the release of that stage implies that the last tile's MMAs on the same
+// chunk have retired.
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TC2_THREADS, 1)
+update_tc_pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUtensorMap tmy, const Dev P, const int leg,
+                      const int nstages)
+{
+    extern __shared__ __align__(1024) unsigned char smem_tc[];
+    __shared__ __align__(8) unsigned long long bars[TC2_MAX_STAGES + TC2_MAX_STAGES / 2 + 6];
+    __shared__ uint32_t tmem_holder;
+    __shared__ int abort_flag;
+    __shared__ __align__(16) float gts[TC2_BN];            // column terms of the tile being reduced
+    __shared__ double xs[TC_BM];                           // second column half's partial results, then the merged
+    __shared__ float xm[TC_BM];                            // row results on their way to the filing warps
+    __shared__ double red[TC2_FILE_WARPS];
+
+    pdl_enter();
+    const Ctl c = *P.ctl;
+    if (c.done) return;
+    if (leg != LEG_V && c.static_final) return;
+    const bool rows_x = (leg == LEG_F);
+    const int nrows = rows_x ? P.n : P.m;
+    const int ncols = rows_x ? P.m : P.n, cp = rows_x ? P.mp : P.np;
+    const int nrt = (nrows + TC_BM - 1) / TC_BM;
+    const int npair = (nrt + 1) / 2;                       // row-block pairs per lane (the last may be half empty)
+    const int nitems = c.n_phys * npair;
+    const int ncl = (int)gridDim.x >> 1, cl = (int)blockIdx.x >> 1;
+    const uint32_t rank = cluster_rank();
+    const bool leader = (rank == 0);
+    const CUtensorMap *tm_row = rows_x ? &tmx : &tmy, *tm_col = rows_x ? &tmy : &tmx;
+    const int nkc = P.d / TC_BK;
+    const int ntiles = (ncols + TC2_BN - 1) / TC2_BN;
+    const int nct128 = (ncols + 127) / 128;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t sbase = (smem_u32(smem_tc) + 1023u) & ~1023u;
+    const uint32_t sA = sbase, sB = sbase + (uint32_t)nkc * TC_CHUNK;
+    const uint32_t b_full = smem_u32(&bars[0]), b_empty = smem_u32(&bars[TC2_MAX_STAGES]);
+    const uint32_t b_tfull = smem_u32(&bars[TC2_MAX_STAGES + TC2_MAX_STAGES / 2]), b_tempty = b_tfull + 16;
+    const uint32_t b_box_full = b_tfull + 32, b_box_empty = b_tfull + 40;
+    // the same barriers seen in the leader's / the peer's shared memory
+    const uint32_t b_full_leader = map_to_cta(b_full, 0);
+    const uint32_t b_tempty_leader = map_to_cta(b_tempty, 0);
+    const uint32_t b_empty_peer = map_to_cta(b_empty, 1);
+    const uint32_t b_tfull_peer = map_to_cta(b_tfull, 1);
+
+    if (tid == 0) {
+        for (int s = 0; s < nstages; ++s) mbar_init(b_full + 8 * s, 1);
+        for (int g = 0; g < nstages / 2; ++g) mbar_init(b_empty + 8 * g, 1);
+        for (int b = 0; b < 2; ++b) { mbar_init(b_tfull + 8 * b, 1); mbar_init(b_tempty + 8 * b, 2 * TC_EPI_WARPS); }
+        mbar_init(b_box_full, 1); mbar_init(b_box_empty, TC2_FILE_WARPS);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == TC_EPI_WARPS + 1) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(&tmem_holder)) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_barrier();                                  // both CTAs' barriers exist before anything remote touches them
+    tc_fence_after();
+    const uint32_t tmem = tmem_holder;
+    volatile int *ab = &abort_flag;
+    long long dbg_w0 = 0, dbg_w1 = 0;   // clocks spent in waits (debug builds)
+    const long long dbg_t0 = clock64();
+    (void)dbg_w0; (void)dbg_w1; (void)dbg_t0;
+
+    // every role walks the same items and skips the same ones
+#define TC2_FOR_ITEMS(item, slot, pb)                                                            \
+    for (int item = cl, slot, pb; item < nitems; item += ncl)                                    \
+        if (slot = item / npair, pb = item - slot * npair, leg == LEG_V && !(c.static_final || P.flag[slot])) continue; else
+
+    if (warp == TC_EPI_WARPS) {
+        // ---------------- producer (one per CTA): own row block once per item, own half of every column tile
+        if (lane == 0) {
+            int s = 0; uint32_t ph = 0;
+            bool first_round = true, go = true;
+            TC2_FOR_ITEMS(item, slot, pb) {
+                const int rb = 2 * pb + (int)rank;
+                const bool ghost = rb >= nrt;                  // odd number of row blocks: no rows for the pair's second CTA
+                const int row_tile0 = (slot * nrt + rb) * nkc;
+                const int col_tile0 = slot * nct128 * nkc;
+                for (int t = 0; t < ntiles && go; ++t) {
+                    for (int kc = 0; kc < nkc; ++kc) {
+                        // stages are released two at a time (one commit per eight MMAs)
+                        if (!first_round && (s & 1) == 0 && !TC_TIMED_WAIT(dbg_w0, mbar_wait(b_empty + 8 * (s >> 1), ph ^ 1u, ab))) { go = false; break; }
+                        if (leader) mbar_expect_tx(b_full + 8 * s, t == 0 ? 4 * TC_CHUNK : 2 * TC_CHUNK);
+                        if (t == 0)
+                            tma_load_chunk_pair(sA + kc * TC_CHUNK, tm_row, ghost ? 0x7fffff80 : (row_tile0 + kc) * TC_BM, b_full_leader + 8 * s);
+                        const int pt = t * 2 + (int)rank;              // this CTA's 128-point tile of the column operand
+                        tma_load_chunk_pair(sB + s * TC_CHUNK, tm_col, pt < nct128 ? (col_tile0 + pt * nkc + kc) * 128 : 0x7fffff80,
+                                            b_full_leader + 8 * s);
+                        if (++s == nstages) { s = 0; ph ^= 1u; first_round = false; }
+                    }
+                }
+                if (!go || *ab) break;
+            }
+        }
+    } else if (warp == TC_EPI_WARPS + 1) {
+        // ---------------- MMA issuer (leader only)
+        if (lane == 0 && leader) {
+            bool ok = true;
+            int s = 0; uint32_t ph = 0;
+            int tg = 0;                                         // tiles issued so far: accumulator buffer and phase
+            const uint64_t adesc0 = tc_desc(sA), bdesc0 = tc_desc(sB);   // the address field counts 16-byte units
+            TC2_FOR_ITEMS(item, slot, pb) {
+                for (int t = 0; t < ntiles && ok; ++t, ++tg) {
+                    const int buf = tg & 1;
+                    if (tg >= 2) ok = TC_TIMED_WAIT(dbg_w1, mbar_wait(b_tempty + 8 * buf, ((tg >> 1) - 1) & 1, ab));
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t d_tmem = tmem + (uint32_t)buf * TC2_BN;
+                    uint64_t ad = adesc0;
+                    for (int kc = 0; kc < nkc && ok; ++kc, ad += TC_CHUNK >> 4) {
+                        ok = TC_TIMED_WAIT(dbg_w0, mbar_wait(b_full + 8 * s, ph, ab));
+                        if (!ok) break;
+                        tc_fence_after();
+                        const uint64_t bd = bdesc0 + (uint64_t)(s * (TC_CHUNK >> 4));
+                        // four K = 16 slices of the 64-dimension chunk: 32 bytes apart inside the swizzle atom
+                        tc_mma_pair(d_tmem, ad, bd, tc_idesc_pair(), kc ? 1u : 0u);
+                        tc_mma_pair(d_tmem, ad + 2, bd + 2, tc_idesc_pair(), 1u);
+                        tc_mma_pair(d_tmem, ad + 4, bd + 4, tc_idesc_pair(), 1u);
+                        tc_mma_pair(d_tmem, ad + 6, bd + 6, tc_idesc_pair(), 1u);
+                        if (s & 1) {                            // both producers may refill this pair of stages
+                            tc_commit_pair(b_empty + 8 * (s >> 1));
+                            tc_commit_pair(b_empty_peer + 8 * (s >> 1));
+                        }
+                        if (++s == nstages) { s = 0; ph ^= 1u; }
+                    }
+                    if (ok) { tc_commit_pair(b_tfull + 8 * buf); tc_commit_pair(b_tfull_peer + 8 * buf); }
+                }
+                if (!ok) break;
+            }
+        }
+    } else if (warp >= TC_EPI_WARPS + 2) {
+        // ---------------- filing warps (one thread per row): take each item's merged row results
+        // (maximum, sum) from the epilogue warps and do everything that is slow and serial off
+        // their critical path: the float64 epilogue of the rows, the residual sum in a fixed
+        // order, and the lane's store / fence / ticket (its last block adds the parts up and sets
+        // the flags)
+        const int fw = warp - (TC_EPI_WARPS + 2), row = fw * 32 + lane;
+        int k = 0;
+        TC2_FOR_ITEMS(item, slot, pb) {
+            const int rb = 2 * pb + (int)rank;
+            if (rb >= nrt) continue;                                    // no rows, no message
+            int got = 0;
+            if (lane == 0) got = mbar_wait(b_box_full, k & 1, ab) ? 1 : 0;
+            got = __shfl_sync(0xffffffffu, got, 0);
+            __syncwarp();
+            if (!got) break;
+            const bool frozen = (P.mode == MODE_MASKED) && P.state[slot] != 0;
+            const int i = rb * TC_BM + row;
+            const float m = xm[row];
+            const double sm = xs[row];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(b_box_empty);                    // the row results may be overwritten
+            double term = 0.0;
+            if (i < nrows) term = finish_one_row<float>(P, c, leg, slot, (int)FORM_DOT, i, m, sm, 0.f, !frozen && leg != LEG_V);
+            if (leg != LEG_G) {
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) term += __shfl_down_sync(0xffffffffu, term, off);
+                if (lane == 0) red[fw] = term;
+                asm volatile("bar.sync 4, 128;" ::: "memory");
+                if (row == 0) finish_lane_residual(P, c, leg, slot, nrt, rb, ((red[0] + red[1]) + red[2]) + red[3], frozen);
+                asm volatile("bar.sync 4, 128;" ::: "memory");          // red[] is free again
+            }
+            ++k;
+        }
+    } else {
+        // ---------------- epilogue: thread e <-> row (e & 127) of this CTA's block <-> TMEM lane (e & 127);
+        // warps 0-3 take the even 32-column chunks of every tile, warps 4-7 the odd ones
+        const int e = tid, half = warp >> 2, row = e & 127;
+        const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+        bool ok = true;
+        int tg = 0, nbox = 0;
+        TC2_FOR_ITEMS(item, slot, pb) {
+            const int rb = 2 * pb + (int)rank;
+            const bool ghost = rb >= nrt;
+            const float *colt = rows_x ? reinterpret_cast<const float *>(P.gt) + (size_t)slot * cp
+                                       : reinterpret_cast<const float *>(P.ft[c.parity]) + (size_t)slot * cp;
+            const float two_s = (float)(2.0 * P.scale[slot]);
+            float mx = NEG_BIG, ts = 0.f;
+            double sd = 0.0;
+            float g_next = (e < cp) ? colt[e] : NEG_BIG;                // column term of the tile to come, one tile ahead
+            for (int t = 0; t < ntiles; ++t, ++tg) {
+                const int buf = tg & 1;
+                asm volatile("bar.sync 1, 256;" ::: "memory");          // everyone is done with the previous tile's column terms
+                gts[e] = g_next;
+                {
+                    const int j = (t + 1) * TC2_BN + e;
+                    g_next = (t + 1 < ntiles && j < cp) ? colt[j] : NEG_BIG;
+                }
+                ok = TC_TIMED_WAIT(dbg_w0, mbar_wait(b_tfull + 8 * buf, (tg >> 1) & 1, ab));
+                ok = epi_all(ok);                                       // also publishes the column terms
+                if (!ok) break;
+                tc_fence_after();
+                tc_reduce_tile<TC2_BN>(lane_base + (uint32_t)(buf * TC2_BN), gts, half, two_s, mx, ts, sd);
+                sd += (double)ts;
+                ts = 0.f;
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) {                                        // one arrival per warp: this accumulator is read
+                    if (leader) mbar_arrive(b_tempty + 8 * buf);
+                    else mbar_arrive_remote(b_tempty_leader + 8 * buf);
+                }
+            }
+            if (!ok) break;
+            // merge the two column halves of every row and hand the results to the filing warp
+            if (!ghost) {
+                if (nbox > 0 && !mbar_wait(b_box_empty, (nbox - 1) & 1, ab)) ok = false;   // previous item's results still being read
+                if (half) { xm[row] = mx; xs[row] = sd; }
+            }
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+            if (!half) {
+                if (!ghost) {
+                    const float mo = xm[row];
+                    const float mn = fmaxf(mx, mo);
+                    xs[row] = sd * (double)pow2i(mx - mn) + xs[row] * (double)pow2i(mo - mn);
+                    xm[row] = mn;
+                }
+                asm volatile("bar.sync 2, 128;" ::: "memory");
+                if (e == 0 && !ghost) mbar_arrive(b_box_full);
+            }
+            if (!ghost) ++nbox;
+        }
+    }
+#undef TC2_FOR_ITEMS
+    if (abort_flag) {
+        // a wait ran out: give copies that may still be in flight time to land in this CTA's
+        // shared memory before it is released (bounded: ~0.1 ms)
+        const long long t0 = clock64();
+        while (clock64() - t0 < 200000LL) { }
+    }
+#ifdef SKB_TC_DEBUG
+    if (blockIdx.x < 2 && leg == LEG_F && (lane == 0) && (warp == 0 || warp == 4 || warp >= TC_EPI_WARPS))
+        printf("[tc2 dbg] rank %u warp %d: total %lld clk, wait0 %lld, wait1 %lld (producer: empty; mma: full, tmem-empty; epilogue: tmem-full) tiles %d chunks/tile %d stages %d items %d clusters %d\n",
+               rank, warp, clock64() - dbg_t0, dbg_w0, dbg_w1, ntiles, nkc, nstages, nitems, ncl);
+#endif
+    tc_fence_before();
+    __syncthreads();
+    cluster_barrier();                                  // the pair is done with each other's memory
+    tc_fence_after();
+    if (warp == TC_EPI_WARPS + 1) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
+    if (abort_flag) {
+        if (tid == 0) atomicOr(&P.ctl->error, ERR_WAIT);
+    }
 }
 
 // Self-test of the bounded wait: one thread waits on a barrier that nothing will ever complete
@@ -351,7 +772,10 @@ bool tc_eligible(int d, bool bf16) { return bf16 && d >= 64 && d <= 512 && d % 6
 // d <= 256: 128-column tiles, two ring stages, small enough for two CTAs per SM (the second CTA's MMAs
 // cover this CTA's prologue and epilogue).  d > 256: 256-column tiles (the tensor pipe runs 128x256 MMAs
 // about twice as efficiently as 128x128 ones), three 32 KB stages beside the 128 KB row block.
-static bool tc_wide(int d) { return d > 256; }
+#ifndef SKB_TC_WIDE_FROM
+#define SKB_TC_WIDE_FROM 257
+#endif
+static bool tc_wide(int d) { return d >= SKB_TC_WIDE_FROM && d >= 2 * TC_BK; }   // the pair kernel's ring needs two stages <= d/64
 size_t tc_smem_bytes(int d) { return (size_t)(d / TC_BK + (tc_wide(d) ? 6 : 2)) * TC_CHUNK; }
 
 // Tensor map of one tiled operand copy: rows of 64 bf16 (128 B, contiguous), 128-row boxes.
@@ -401,23 +825,48 @@ void launch_retile(const void *src, void *dst, int W, int npts, int d, cudaStrea
 void launch_update_tc(const Dev &P, const void *maps, int leg, int width, cudaStream_t st)
 {
     // dynamic shared memory: the tiles, plus what it takes to start them on a 1024-byte boundary
-    static size_t pad[2] = {0, 0};
+    static size_t pad[3] = {0, 0, 0};
+    static size_t pair_static = 0;
     static bool attr_set = false;
+    static bool use_pair = true;
     if (!attr_set) {
         cudaFuncAttributes fa;
         cudaFuncGetAttributes(&fa, update_tc_kernel<2, 128>);
         pad[0] = (1024 - fa.sharedSizeBytes % 1024) % 1024;
         cudaFuncGetAttributes(&fa, update_tc_kernel<3, 256>);
         pad[1] = (1024 - fa.sharedSizeBytes % 1024) % 1024;
+        cudaFuncGetAttributes(&fa, update_tc_pair_kernel);
+        pad[2] = (1024 - fa.sharedSizeBytes % 1024) % 1024;
+        pair_static = fa.sharedSizeBytes;
         cudaFuncSetAttribute(update_tc_kernel<2, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(tc_smem_bytes(256) + pad[0]));
         cudaFuncSetAttribute(update_tc_kernel<3, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(tc_smem_bytes(512) + pad[1]));
+        cudaFuncSetAttribute(update_tc_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(232448 - pair_static));
+        const char *e = getenv("SKB_TC_PAIR");
+        if (e && e[0] == '0') use_pair = false;
         attr_set = true;
     }
     const CUtensorMap *tm = reinterpret_cast<const CUtensorMap *>(maps);
     const int nrows = (leg == LEG_F) ? P.n : P.m;
-    dim3 grid((nrows + TC_BM - 1) / TC_BM, width < 1 ? 1 : width);
-    if (!tc_wide(P.d)) launch_pdl(update_tc_kernel<2, 128>, grid, dim3(TC_THREADS), tc_smem_bytes(P.d) + pad[0], st, tm[0], tm[1], P, leg);
-    else launch_pdl(update_tc_kernel<3, 256>, grid, dim3(TC_THREADS), tc_smem_bytes(P.d) + pad[1], st, tm[0], tm[1], P, leg);
+    const int nrt = (nrows + TC_BM - 1) / TC_BM;
+    dim3 grid(nrt, width < 1 ? 1 : width);
+    if (!tc_wide(P.d)) {
+        launch_pdl(update_tc_kernel<2, 128>, grid, dim3(TC_THREADS), tc_smem_bytes(P.d) + pad[0], st, tm[0], tm[1], P, leg);
+    } else if (use_pair) {
+        // as many 16 KB ring stages as fit beside the resident row block (six at d = 512), an even
+        // number (released in pairs) and no more than a tile has chunks (see the kernel's header)
+        const size_t room = 232448 - pair_static - pad[2] - (size_t)(P.d / TC_BK) * TC_CHUNK;
+        int nst = (int)(room / TC_CHUNK);
+        if (nst > TC2_MAX_STAGES) nst = TC2_MAX_STAGES;
+        if (nst > P.d / TC_BK) nst = P.d / TC_BK;
+        nst &= ~1;
+        static int sm_count = 0;
+        if (!sm_count) { int dev = 0; cudaGetDevice(&dev); cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev); }
+        const int items = (width < 1 ? 1 : width) * ((nrt + 1) / 2);
+        const int ncl = items < sm_count / 2 ? items : sm_count / 2;
+        launch_pdl(update_tc_pair_kernel, dim3(2 * ncl), dim3(TC2_THREADS), (size_t)(P.d / TC_BK + nst) * TC_CHUNK + pad[2], st, tm[0], tm[1], P, leg, nst);
+    } else {
+        launch_pdl(update_tc_kernel<3, 256>, grid, dim3(TC_THREADS), tc_smem_bytes(P.d) + pad[1], st, tm[0], tm[1], P, leg);
+    }
 }
 
 }  // namespace skb
