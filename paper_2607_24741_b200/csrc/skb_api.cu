@@ -118,6 +118,8 @@ static size_t carve(const skb_config *c, const Variant *var, bool tensor, char *
     d.res_row = (double *)take(W * 8); d.res_col = (double *)take(W * 8);
     d.rrow = (double *)take(W * 8); d.rcol = (double *)take(W * 8);
     d.widths = (int *)take(((size_t)c->max_iter + 2) * 4);
+    const size_t nblk128 = ((n > m ? n : m) + 127) / 128;
+    d.tc_cnt = (unsigned *)take(W * nblk128 * 4);     // in every layout, so that the zeroed range is the same for all
     const size_t zero_end = off;
     d.scale = (double *)take(W * 8); d.lane_id = (int *)take(W * 4);
     d.center = (double *)take(W * DP * 8); d.form = (int *)take(W * 4);
@@ -128,6 +130,8 @@ static size_t carve(const skb_config *c, const Variant *var, bool tensor, char *
     d.tensor = tensor ? 1 : 0;
     if (tensor) {
         d.xb = take(tc_tiled_bytes(c->W, c->n, c->d)); d.yb = take(tc_tiled_bytes(c->W, c->m, c->d));
+        d.tc_pm = (float *)take(W * nblk128 * TC_MAX_SPLIT * 128 * 4);
+        d.tc_ps = (double *)take(W * nblk128 * TC_MAX_SPLIT * 128 * 8);
     } else {
         d.xs = take(W * DP * np * ts); d.ys = take(W * DP * mp * ts);
     }

@@ -26,6 +26,7 @@ enum Form : int { FORM_DOT = 0, FORM_DIFF = 1 };
 
 constexpr float NEG_BIG = -1.0e30f;   // "minus infinity" for padded columns (finite: no NaNs)
 constexpr int UPD_THREADS = 128;
+constexpr int TC_MAX_SPLIT = 8;      // a row block's columns go to at most this many clusters
 constexpr int MAX_PARTS = 1024;       // upper bound on row blocks per lane (residual partials)
 
 // Device-resident control block.  Written by the plan kernel (one CTA), read by all.
@@ -74,6 +75,11 @@ struct Dev {
     double *rrow, *rcol;      // residuals of the audited state
     unsigned *cnt_row, *cnt_col;
     double *part_row, *part_col;   // [W][MAX_PARTS] per-CTA partial sums (scratch)
+    // tensor path, row blocks whose columns were shared out among clusters: arrival word and the
+    // parts' row results [W][row block][TC_MAX_SPLIT][128]
+    unsigned *tc_cnt;
+    float *tc_pm;
+    double *tc_ps;
     // retire / move lists (plan -> emit_move)
     int *ret_slot, *ret_lane, *ret_src;
     double *ret_scale;

@@ -485,8 +485,15 @@ __device__ __forceinline__ bool finish_lane_residual(const Dev &P, const Ctl &c,
     const unsigned ticket = atomicAdd(cnt, 1u);
     if (ticket != (unsigned)(nblk - 1)) return false;
     __threadfence();
+    // block order, eight loads in flight at a time (one memory latency per eight parts, not eight)
     double tot = 0.0;
-    for (int b = 0; b < nblk; ++b) tot += reinterpret_cast<volatile double *>(parts)[b];
+    for (int b0 = 0; b0 < nblk; b0 += 8) {
+        double v[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) v[j] = (b0 + j < nblk) ? reinterpret_cast<volatile double *>(parts)[b0 + j] : 0.0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) if (b0 + j < nblk) tot += v[j];
+    }
     *cnt = 0u;
     const bool finite = isfinite(tot);
     if (leg == LEG_F) {

@@ -478,15 +478,49 @@ __device__ __forceinline__ bool epi_all(const bool ok)
     return r != 0;
 }
 
-// The kernel is PERSISTENT: the grid holds one cluster per SM pair and every cluster walks the
-// work items (lane, pair of row blocks) cluster-index + k * cluster-count, so barrier set-up,
-// tensor-memory allocation, the first loads of an item, the exponentials of its last tile and
-// its float64 epilogue all overlap the MMAs of the neighbouring items.  The ring, the
-// accumulator buffers and their barrier phases simply run on across items.  A row-block chunk
-// of the NEXT item may overwrite the resident copy as soon as the ring stage it travels with
-// has been released, because MMAs retire in order and the ring (nstages <= d/64 stages) is not
-// longer than a tile: the release of that stage implies that the last tile's MMAs on the same
-// chunk have retired.
+// the same over the 128 threads of the filing warps
+__device__ __forceinline__ bool file_all(const bool ok)
+{
+    uint32_t r;
+    asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.b32 p, %1, 0;\n\tbar.red.and.pred q, 5, 128, p;\n\tselp.u32 %0, 1, 0, q;\n\t}"
+                 : "=r"(r) : "r"((uint32_t)ok) : "memory");
+    return r != 0;
+}
+
+// The kernel is PERSISTENT and TILE-BALANCED.  The work of a launch is the sequence of units
+// (lane, pair of row blocks, group of column tiles), `upi` units per row-block pair; the grid
+// holds one cluster per SM pair and cluster c takes the units [c U / C, (c+1) U / C).  A run
+// of units of one row-block pair is a SEGMENT: the cluster loads the pair's row blocks once and
+// reduces the segment's column tiles.  Barrier set-up, tensor-memory allocation, the first
+// loads of a segment, the exponentials of its last tile and its float64 epilogue all overlap
+// the MMAs of the neighbouring segments; the ring, the accumulator buffers and their barrier
+// phases simply run on.  A row-block chunk of the NEXT segment may overwrite the resident copy
+// as soon as the ring stage it travels with has been released, because MMAs retire in order
+// and the ring (nstages <= d/64 stages) is not longer than a tile: the release of that stage
+// implies that the last tile's MMAs on the same chunk have retired.
+//
+// A row-block pair whose units went to several clusters is finished by whichever of them
+// arrives last: every part stores its rows' (maximum, sum) in global scratch and adds its unit
+// count and a start-unit bit to the block's arrival word; the last arrival merges the parts in
+// unit order (so the result does not depend on who was last) and runs the float64 epilogue.
+struct Seg { int slot, pb, t0, t1, fu, nu; };
+struct SegIter {
+    int u, u_end, upi, g, npair, ntiles;
+    __device__ __forceinline__ bool next(Seg &s)
+    {
+        if (u >= u_end) return false;
+        const int item = u / upi;
+        s.fu = u - item * upi;
+        s.nu = min(upi - s.fu, u_end - u);
+        u += s.nu;
+        s.slot = item / npair;
+        s.pb = item - s.slot * npair;
+        s.t0 = s.fu * g;
+        s.t1 = min(ntiles, (s.fu + s.nu) * g);
+        return true;
+    }
+};
+
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TC2_THREADS, 1)
 update_tc_pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUtensorMap tmy, const Dev P, const int leg,
                       const int nstages)
@@ -495,6 +529,7 @@ update_tc_pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_cons
     __shared__ __align__(8) unsigned long long bars[TC2_MAX_STAGES + TC2_MAX_STAGES / 2 + 6];
     __shared__ uint32_t tmem_holder;
     __shared__ int abort_flag;
+    __shared__ unsigned arrival;                           // filing warps: the arrival word before this part's add
     __shared__ __align__(16) float gts[TC2_BN];            // column terms of the tile being reduced
     __shared__ double xs[TC_BM];                           // second column half's partial results, then the merged
     __shared__ float xm[TC_BM];                            // row results on their way to the filing warps
@@ -509,14 +544,21 @@ update_tc_pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_cons
     const int ncols = rows_x ? P.m : P.n, cp = rows_x ? P.mp : P.np;
     const int nrt = (nrows + TC_BM - 1) / TC_BM;
     const int npair = (nrt + 1) / 2;                       // row-block pairs per lane (the last may be half empty)
-    const int nitems = c.n_phys * npair;
-    const int ncl = (int)gridDim.x >> 1, cl = (int)blockIdx.x >> 1;
     const uint32_t rank = cluster_rank();
     const bool leader = (rank == 0);
     const CUtensorMap *tm_row = rows_x ? &tmx : &tmy, *tm_col = rows_x ? &tmy : &tmx;
     const int nkc = P.d / TC_BK;
     const int ntiles = (ncols + TC2_BN - 1) / TC2_BN;
     const int nct128 = (ncols + 127) / 128;
+    // units: groups of g column tiles, at most TC_MAX_SPLIT per row-block pair
+    const int g = (ntiles + TC_MAX_SPLIT - 1) / TC_MAX_SPLIT;
+    const int upi = (ntiles + g - 1) / g;
+    const int U = c.n_phys * npair * upi;
+    const int ncl_grid = (int)gridDim.x >> 1, ncl = ncl_grid < U ? ncl_grid : U, cl = (int)blockIdx.x >> 1;
+    SegIter it0;
+    it0.upi = upi; it0.g = g; it0.npair = npair; it0.ntiles = ntiles;
+    it0.u = cl < ncl ? (int)((long long)cl * U / ncl) : 0;
+    it0.u_end = cl < ncl ? (int)((long long)(cl + 1) * U / ncl) : 0;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t sbase = (smem_u32(smem_tc) + 1023u) & ~1023u;
@@ -532,7 +574,7 @@ update_tc_pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_cons
 
     if (tid == 0) {
         for (int s = 0; s < nstages; ++s) mbar_init(b_full + 8 * s, 1);
-        for (int g = 0; g < nstages / 2; ++g) mbar_init(b_empty + 8 * g, 1);
+        for (int q = 0; q < nstages / 2; ++q) mbar_init(b_empty + 8 * q, 1);
         for (int b = 0; b < 2; ++b) { mbar_init(b_tfull + 8 * b, 1); mbar_init(b_tempty + 8 * b, 2 * TC_EPI_WARPS); }
         mbar_init(b_box_full, 1); mbar_init(b_box_empty, TC2_FILE_WARPS);
         abort_flag = 0;
@@ -552,27 +594,29 @@ update_tc_pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_cons
     const long long dbg_t0 = clock64();
     (void)dbg_w0; (void)dbg_w1; (void)dbg_t0;
 
-    // every role walks the same items and skips the same ones
-#define TC2_FOR_ITEMS(item, slot, pb)                                                            \
-    for (int item = cl, slot, pb; item < nitems; item += ncl)                                    \
-        if (slot = item / npair, pb = item - slot * npair, leg == LEG_V && !(c.static_final || P.flag[slot])) continue; else
+    // every role walks the same segments and skips the same ones (the column check only
+    // visits lanes that the screen flagged)
+    SegIter it = it0;
+    Seg sg;
+#define TC2_SKIP(slot) (leg == LEG_V && !(c.static_final || P.flag[slot]))
 
     if (warp == TC_EPI_WARPS) {
-        // ---------------- producer (one per CTA): own row block once per item, own half of every column tile
+        // ---------------- producer (one per CTA): own row block once per segment, own half of every column tile
         if (lane == 0) {
             int s = 0; uint32_t ph = 0;
             bool first_round = true, go = true;
-            TC2_FOR_ITEMS(item, slot, pb) {
-                const int rb = 2 * pb + (int)rank;
+            while (go && it.next(sg)) {
+                if (TC2_SKIP(sg.slot)) continue;
+                const int rb = 2 * sg.pb + (int)rank;
                 const bool ghost = rb >= nrt;                  // odd number of row blocks: no rows for the pair's second CTA
-                const int row_tile0 = (slot * nrt + rb) * nkc;
-                const int col_tile0 = slot * nct128 * nkc;
-                for (int t = 0; t < ntiles && go; ++t) {
+                const int row_tile0 = (sg.slot * nrt + rb) * nkc;
+                const int col_tile0 = sg.slot * nct128 * nkc;
+                for (int t = sg.t0; t < sg.t1 && go; ++t) {
                     for (int kc = 0; kc < nkc; ++kc) {
                         // stages are released two at a time (one commit per eight MMAs)
                         if (!first_round && (s & 1) == 0 && !TC_TIMED_WAIT(dbg_w0, mbar_wait(b_empty + 8 * (s >> 1), ph ^ 1u, ab))) { go = false; break; }
-                        if (leader) mbar_expect_tx(b_full + 8 * s, t == 0 ? 4 * TC_CHUNK : 2 * TC_CHUNK);
-                        if (t == 0)
+                        if (leader) mbar_expect_tx(b_full + 8 * s, t == sg.t0 ? 4 * TC_CHUNK : 2 * TC_CHUNK);
+                        if (t == sg.t0)
                             tma_load_chunk_pair(sA + kc * TC_CHUNK, tm_row, ghost ? 0x7fffff80 : (row_tile0 + kc) * TC_BM, b_full_leader + 8 * s);
                         const int pt = t * 2 + (int)rank;              // this CTA's 128-point tile of the column operand
                         tma_load_chunk_pair(sB + s * TC_CHUNK, tm_col, pt < nct128 ? (col_tile0 + pt * nkc + kc) * 128 : 0x7fffff80,
@@ -580,7 +624,7 @@ update_tc_pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_cons
                         if (++s == nstages) { s = 0; ph ^= 1u; first_round = false; }
                     }
                 }
-                if (!go || *ab) break;
+                if (*ab) go = false;
             }
         }
     } else if (warp == TC_EPI_WARPS + 1) {
@@ -590,8 +634,9 @@ update_tc_pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_cons
             int s = 0; uint32_t ph = 0;
             int tg = 0;                                         // tiles issued so far: accumulator buffer and phase
             const uint64_t adesc0 = tc_desc(sA), bdesc0 = tc_desc(sB);   // the address field counts 16-byte units
-            TC2_FOR_ITEMS(item, slot, pb) {
-                for (int t = 0; t < ntiles && ok; ++t, ++tg) {
+            while (ok && it.next(sg)) {
+                if (TC2_SKIP(sg.slot)) continue;
+                for (int t = sg.t0; t < sg.t1 && ok; ++t, ++tg) {
                     const int buf = tg & 1;
                     if (tg >= 2) ok = TC_TIMED_WAIT(dbg_w1, mbar_wait(b_tempty + 8 * buf, ((tg >> 1) - 1) & 1, ab));
                     if (!ok) break;
@@ -616,31 +661,58 @@ update_tc_pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_cons
                     }
                     if (ok) { tc_commit_pair(b_tfull + 8 * buf); tc_commit_pair(b_tfull_peer + 8 * buf); }
                 }
-                if (!ok) break;
             }
         }
     } else if (warp >= TC_EPI_WARPS + 2) {
-        // ---------------- filing warps (one thread per row): take each item's merged row results
+        // ---------------- filing warps (one thread per row): take each segment's merged row results
         // (maximum, sum) from the epilogue warps and do everything that is slow and serial off
-        // their critical path: the float64 epilogue of the rows, the residual sum in a fixed
-        // order, and the lane's store / fence / ticket (its last block adds the parts up and sets
-        // the flags)
+        // their critical path: the hand-over between the parts of a shared row block, the float64
+        // epilogue of the rows, the residual sum in a fixed order, and the lane's store / fence /
+        // ticket (its last block adds the parts up and sets the flags)
         const int fw = warp - (TC_EPI_WARPS + 2), row = fw * 32 + lane;
         int k = 0;
-        TC2_FOR_ITEMS(item, slot, pb) {
-            const int rb = 2 * pb + (int)rank;
+        while (it.next(sg)) {
+            if (TC2_SKIP(sg.slot)) continue;
+            const int slot = sg.slot, rb = 2 * sg.pb + (int)rank;
             if (rb >= nrt) continue;                                    // no rows, no message
             int got = 0;
             if (lane == 0) got = mbar_wait(b_box_full, k & 1, ab) ? 1 : 0;
             got = __shfl_sync(0xffffffffu, got, 0);
-            __syncwarp();
-            if (!got) break;
-            const bool frozen = (P.mode == MODE_MASKED) && P.state[slot] != 0;
-            const int i = rb * TC_BM + row;
-            const float m = xm[row];
-            const double sm = xs[row];
+            if (!file_all(got != 0)) break;                             // all four warps leave together
+            ++k;
+            float m = xm[row];
+            double sm = xs[row];
             __syncwarp();
             if (lane == 0) mbar_arrive(b_box_empty);                    // the row results may be overwritten
+            if (sg.nu != upi) {
+                // this cluster reduced only some of the row block's column tiles
+                const size_t blk = (size_t)slot * nrt + rb;
+                const size_t o = (blk * TC_MAX_SPLIT + sg.fu) * TC_BM + row;
+                P.tc_pm[o] = m;
+                P.tc_ps[o] = sm;
+                __threadfence();
+                asm volatile("bar.sync 4, 128;" ::: "memory");
+                if (row == 0) arrival = atomicAdd(&P.tc_cnt[blk], (unsigned)sg.nu + (1u << (8 + sg.fu)));
+                asm volatile("bar.sync 4, 128;" ::: "memory");
+                const unsigned before = arrival;
+                asm volatile("bar.sync 4, 128;" ::: "memory");          // `arrival` is free again
+                if ((int)(before & 0xffu) + sg.nu != upi) continue;     // not the last part: done
+                if (row == 0) P.tc_cnt[blk] = 0u;
+                __threadfence();
+                const unsigned starts = (before >> 8) | (1u << sg.fu);
+                m = NEG_BIG; sm = 0.0;
+                for (int f = 0; f < upi; ++f) {
+                    if (!((starts >> f) & 1u)) continue;
+                    const size_t q = (blk * TC_MAX_SPLIT + f) * TC_BM + row;
+                    const float mo = reinterpret_cast<volatile float *>(P.tc_pm)[q];
+                    const double so = reinterpret_cast<volatile double *>(P.tc_ps)[q];
+                    const float mn = fmaxf(m, mo);
+                    sm = sm * (double)pow2i(m - mn) + so * (double)pow2i(mo - mn);
+                    m = mn;
+                }
+            }
+            const bool frozen = (P.mode == MODE_MASKED) && P.state[slot] != 0;
+            const int i = rb * TC_BM + row;
             double term = 0.0;
             if (i < nrows) term = finish_one_row<float>(P, c, leg, slot, (int)FORM_DOT, i, m, sm, 0.f, !frozen && leg != LEG_V);
             if (leg != LEG_G) {
@@ -651,7 +723,6 @@ update_tc_pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_cons
                 if (row == 0) finish_lane_residual(P, c, leg, slot, nrt, rb, ((red[0] + red[1]) + red[2]) + red[3], frozen);
                 asm volatile("bar.sync 4, 128;" ::: "memory");          // red[] is free again
             }
-            ++k;
         }
     } else {
         // ---------------- epilogue: thread e <-> row (e & 127) of this CTA's block <-> TMEM lane (e & 127);
@@ -660,22 +731,23 @@ update_tc_pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_cons
         const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
         bool ok = true;
         int tg = 0, nbox = 0;
-        TC2_FOR_ITEMS(item, slot, pb) {
-            const int rb = 2 * pb + (int)rank;
+        while (ok && it.next(sg)) {
+            if (TC2_SKIP(sg.slot)) continue;
+            const int slot = sg.slot, rb = 2 * sg.pb + (int)rank;
             const bool ghost = rb >= nrt;
             const float *colt = rows_x ? reinterpret_cast<const float *>(P.gt) + (size_t)slot * cp
                                        : reinterpret_cast<const float *>(P.ft[c.parity]) + (size_t)slot * cp;
             const float two_s = (float)(2.0 * P.scale[slot]);
             float mx = NEG_BIG, ts = 0.f;
             double sd = 0.0;
-            float g_next = (e < cp) ? colt[e] : NEG_BIG;                // column term of the tile to come, one tile ahead
-            for (int t = 0; t < ntiles; ++t, ++tg) {
+            float g_next = (sg.t0 * TC2_BN + e < cp) ? colt[sg.t0 * TC2_BN + e] : NEG_BIG;   // column term, one tile ahead
+            for (int t = sg.t0; t < sg.t1; ++t, ++tg) {
                 const int buf = tg & 1;
                 asm volatile("bar.sync 1, 256;" ::: "memory");          // everyone is done with the previous tile's column terms
                 gts[e] = g_next;
                 {
                     const int j = (t + 1) * TC2_BN + e;
-                    g_next = (t + 1 < ntiles && j < cp) ? colt[j] : NEG_BIG;
+                    g_next = (t + 1 < sg.t1 && j < cp) ? colt[j] : NEG_BIG;
                 }
                 ok = TC_TIMED_WAIT(dbg_w0, mbar_wait(b_tfull + 8 * buf, (tg >> 1) & 1, ab));
                 ok = epi_all(ok);                                       // also publishes the column terms
@@ -692,9 +764,11 @@ update_tc_pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_cons
                 }
             }
             if (!ok) break;
-            // merge the two column halves of every row and hand the results to the filing warp
+            // merge the two column halves of every row and hand the results to the filing warps
             if (!ghost) {
-                if (nbox > 0 && !mbar_wait(b_box_empty, (nbox - 1) & 1, ab)) ok = false;   // previous item's results still being read
+                // the previous segment's results may still be being read; a wait that runs out raises
+                // the abort flag, which the next tile's vote turns into a common exit
+                if (nbox > 0) mbar_wait(b_box_empty, (nbox - 1) & 1, ab);
                 if (half) { xm[row] = mx; xs[row] = sd; }
             }
             asm volatile("bar.sync 1, 256;" ::: "memory");
@@ -711,7 +785,7 @@ update_tc_pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_cons
             if (!ghost) ++nbox;
         }
     }
-#undef TC2_FOR_ITEMS
+#undef TC2_SKIP
     if (abort_flag) {
         // a wait ran out: give copies that may still be in flight time to land in this CTA's
         // shared memory before it is released (bounded: ~0.1 ms)
@@ -720,8 +794,8 @@ update_tc_pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_cons
     }
 #ifdef SKB_TC_DEBUG
     if (blockIdx.x < 2 && leg == LEG_F && (lane == 0) && (warp == 0 || warp == 4 || warp >= TC_EPI_WARPS))
-        printf("[tc2 dbg] rank %u warp %d: total %lld clk, wait0 %lld, wait1 %lld (producer: empty; mma: full, tmem-empty; epilogue: tmem-full) tiles %d chunks/tile %d stages %d items %d clusters %d\n",
-               rank, warp, clock64() - dbg_t0, dbg_w0, dbg_w1, ntiles, nkc, nstages, nitems, ncl);
+        printf("[tc2 dbg] rank %u warp %d: total %lld clk, wait0 %lld, wait1 %lld (producer: empty; mma: full, tmem-empty; epilogue: tmem-full) tiles %d chunks/tile %d stages %d units %d clusters %d\n",
+               rank, warp, clock64() - dbg_t0, dbg_w0, dbg_w1, ntiles, nkc, nstages, U, ncl);
 #endif
     tc_fence_before();
     __syncthreads();
@@ -861,8 +935,10 @@ void launch_update_tc(const Dev &P, const void *maps, int leg, int width, cudaSt
         nst &= ~1;
         static int sm_count = 0;
         if (!sm_count) { int dev = 0; cudaGetDevice(&dev); cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev); }
-        const int items = (width < 1 ? 1 : width) * ((nrt + 1) / 2);
-        const int ncl = items < sm_count / 2 ? items : sm_count / 2;
+        const int ncolsh = (leg == LEG_F) ? P.m : P.n;
+        const int ntl = (ncolsh + TC2_BN - 1) / TC2_BN, gg = (ntl + TC_MAX_SPLIT - 1) / TC_MAX_SPLIT;
+        const long long units = (long long)(width < 1 ? 1 : width) * ((nrt + 1) / 2) * ((ntl + gg - 1) / gg);
+        const int ncl = units < sm_count / 2 ? (int)units : sm_count / 2;
         launch_pdl(update_tc_pair_kernel, dim3(2 * ncl), dim3(TC2_THREADS), (size_t)(P.d / TC_BK + nst) * TC_CHUNK + pad[2], st, tm[0], tm[1], P, leg, nst);
     } else {
         launch_pdl(update_tc_kernel<3, 256>, grid, dim3(TC_THREADS), tc_smem_bytes(P.d) + pad[1], st, tm[0], tm[1], P, leg);
