@@ -130,8 +130,8 @@ static size_t carve(const skb_config *c, const Variant *var, bool tensor, char *
     d.tensor = tensor ? 1 : 0;
     if (tensor) {
         d.xb = take(tc_tiled_bytes(c->W, c->n, c->d)); d.yb = take(tc_tiled_bytes(c->W, c->m, c->d));
-        d.tc_pm = (float *)take(W * nblk128 * TC_MAX_SPLIT * 128 * 4);
-        d.tc_ps = (double *)take(W * nblk128 * TC_MAX_SPLIT * 128 * 8);
+        d.tc_pm = (float *)take(W * nblk128 * 2 * TC_MAX_SPLIT * 128 * 4);
+        d.tc_ps = (double *)take(W * nblk128 * 2 * TC_MAX_SPLIT * 128 * 8);
     } else {
         d.xs = take(W * DP * np * ts); d.ys = take(W * DP * mp * ts);
     }

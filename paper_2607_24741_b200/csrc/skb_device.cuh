@@ -75,8 +75,8 @@ struct Dev {
     double *rrow, *rcol;      // residuals of the audited state
     unsigned *cnt_row, *cnt_col;
     double *part_row, *part_col;   // [W][MAX_PARTS] per-CTA partial sums (scratch)
-    // tensor path, row blocks whose columns were shared out among clusters: arrival word and the
-    // parts' row results [W][row block][TC_MAX_SPLIT][128]
+    // tensor path for d > 256: arrival word of a row block whose column tiles were shared out among
+    // clusters, and every unit's row results [W][row block][TC_MAX_SPLIT][column half][128]
     unsigned *tc_cnt;
     float *tc_pm;
     double *tc_ps;

@@ -1,33 +1,33 @@
-// Tensor-core variant of the update kernel for bf16 point clouds with a deep cross term
+// Tensor-core variants of the update kernel for bf16 point clouds with a deep cross term
 // (d a multiple of 64, 64 <= d <= 512): the only place on the path that is a dense
 // contraction.
 //
-// For a block of 128 row points the CTA computes S = R . C^T against column tiles of 128
-// points with tcgen05.mma (bf16 operands straight from the caller's layout, fp32
-// accumulators in tensor memory), then log2 pi_ij = 2 s S_ij + ct_j and the same online
-// max / sum-of-exp2 reduction and float64 epilogue as the SIMT kernels (dot form).
+// For a block of 128 row points a CTA computes S = R . C^T against tiles of column points
+// with tcgen05.mma (bf16 operands, fp32 accumulators in tensor memory), then
+// log2 pi_ij = 2 s S_ij + ct_j and the same online max / sum-of-exp2 reduction and float64
+// epilogue as the SIMT kernels (dot form).  Operands come from pre-tiled copies (every
+// 128-point x 64-dimension chunk is one contiguous 16 KB block in the workspace, which TMA
+// streams at about twice the rate of 1 KB-strided rows; 128-byte swizzle; points past the end
+// are stored as zeros).
 //
-// Warp roles (192 threads):
-//   warps 0-3  epilogue: thread e owns row e = TMEM lane e; tcgen05.ld 32 columns at a time,
-//              fma with the column term, online logsumexp entirely in registers (no shuffles)
-//   warp 4     producer: one lane issues TMA loads of pre-tiled operand copies (every
-//              128-point x 64-dimension chunk is one contiguous 16 KB block in the workspace,
-//              which TMA streams at about twice the rate of 1 KB-strided rows; 128-byte
-//              swizzle; points past the end are stored as zeros): the row block once
-//              (d/64 chunks of 16 KB, riding on the first tile's barriers), and column
-//              chunks through a ring of 2 (d <= 256, 128-column tiles, two CTAs per SM) or
-//              3 stages (d > 256, 256-column tiles of two chunks each)
-//   warp 5     allocates the TMEM columns of two accumulators (2 x 128 or 2 x 256); one lane issues
-//              the MMAs (4 x K=16 per 64-wide chunk) and commits to the ring's empty barriers and
-//              to the accumulator-full barrier, so the next tile's MMAs overlap this tile's
-//              exponentials.
+// Two kernels:
+//   update_tc_kernel        d <= 256: one CTA per row block, 128-column tiles, a two-stage ring,
+//                           small enough for two CTAs per SM
+//   update_tc_pair_kernel   d > 256: persistent clusters of two CTAs (tcgen05 cta_group::2, M = 256,
+//                           N = 256), described at its definition
+// Warp roles of both: warps 0-7 epilogue (thread <-> row <-> TMEM lane; warps 0-3 take the even
+// 32-column chunks of a tile, warps 4-7 the odd ones; tcgen05.ld one chunk ahead, packed fp32
+// arithmetic, no shuffles), one producer warp (one lane issues the TMA loads: the row block
+// once, riding on the first tile's barriers, then column chunks through the ring), one MMA
+// warp (allocates tensor memory for two accumulators; one lane issues 4 x K=16 MMAs per
+// 64-dimension chunk and commits to the ring's empty barriers and to the accumulator-full
+// barrier, so the next tile's MMAs overlap this tile's exponentials).
 // Every mbarrier wait is bounded by a clock budget; on expiry the kernel raises ERR_WAIT in
 // the control block, all roles leave their loops, tensor memory is freed and the kernel
 // returns (the host reports SKB_ERR_CUDA).
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <cstdio>
-#include <cstdlib>
 
 #include "skb_update.cuh"
 #include "skb_host.h"
@@ -292,8 +292,7 @@ update_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant_
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == TC_EPI_WARPS + 1) {
-        if (TC_BN == 256) asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(&tmem_holder)) : "memory");
-        else asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 256;" ::"r"(smem_u32(&tmem_holder)) : "memory");
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 256;" ::"r"(smem_u32(&tmem_holder)) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
@@ -401,8 +400,7 @@ update_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant_
     __syncthreads();
     tc_fence_after();
     if (warp == TC_EPI_WARPS + 1) {
-        if (TC_BN == 256) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
-        else asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 256;" ::"r"(tmem) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 256;" ::"r"(tmem) : "memory");
     }
     if (abort_flag) {
         if (tid == 0) atomicOr(&P.ctl->error, ERR_WAIT);
@@ -499,10 +497,19 @@ __device__ __forceinline__ bool file_all(const bool ok)
 // and the ring (nstages <= d/64 stages) is not longer than a tile: the release of that stage
 // implies that the last tile's MMAs on the same chunk have retired.
 //
-// A row-block pair whose units went to several clusters is finished by whichever of them
-// arrives last: every part stores its rows' (maximum, sum) in global scratch and adds its unit
-// count and a start-unit bit to the block's arrival word; the last arrival merges the parts in
-// unit order (so the result does not depend on who was last) and runs the float64 epilogue.
+// Every unit's row results (maximum, sum; one pair per column half) go to global scratch, and
+// a row block is finished by merging ALL its units' results in unit order: the value does not
+// depend on how the units were shared out, so every mode and every width gives the same bits.
+// A row block whose units went to several clusters is finished by whichever of them arrives
+// last (each adds its unit count to the block's arrival word after a fence).
+// column tiles per unit: at most TC_MAX_SPLIT units per row-block pair, and two tiles per unit
+// where there are that many (every unit starts its reduction cold, which costs one exact-path
+// chunk per warp)
+__host__ __device__ constexpr int tc_unit_tiles(int ntiles)
+{
+    const int g = (ntiles + TC_MAX_SPLIT - 1) / TC_MAX_SPLIT;
+    return g < 2 && ntiles >= 2 ? 2 : g;
+}
 struct Seg { int slot, pb, t0, t1, fu, nu; };
 struct SegIter {
     int u, u_end, upi, g, npair, ntiles;
@@ -531,8 +538,6 @@ update_tc_pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_cons
     __shared__ int abort_flag;
     __shared__ unsigned arrival;                           // filing warps: the arrival word before this part's add
     __shared__ __align__(16) float gts[TC2_BN];            // column terms of the tile being reduced
-    __shared__ double xs[TC_BM];                           // second column half's partial results, then the merged
-    __shared__ float xm[TC_BM];                            // row results on their way to the filing warps
     __shared__ double red[TC2_FILE_WARPS];
 
     pdl_enter();
@@ -551,7 +556,7 @@ update_tc_pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_cons
     const int ntiles = (ncols + TC2_BN - 1) / TC2_BN;
     const int nct128 = (ncols + 127) / 128;
     // units: groups of g column tiles, at most TC_MAX_SPLIT per row-block pair
-    const int g = (ntiles + TC_MAX_SPLIT - 1) / TC_MAX_SPLIT;
+    const int g = tc_unit_tiles(ntiles);
     const int upi = (ntiles + g - 1) / g;
     const int U = c.n_phys * npair * upi;
     const int ncl_grid = (int)gridDim.x >> 1, ncl = ncl_grid < U ? ncl_grid : U, cl = (int)blockIdx.x >> 1;
@@ -680,36 +685,29 @@ update_tc_pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_cons
             got = __shfl_sync(0xffffffffu, got, 0);
             if (!file_all(got != 0)) break;                             // all four warps leave together
             ++k;
-            float m = xm[row];
-            double sm = xs[row];
-            __syncwarp();
-            if (lane == 0) mbar_arrive(b_box_empty);                    // the row results may be overwritten
+            if (lane == 0) mbar_arrive(b_box_empty);                    // the epilogue may announce its next segment
+            const size_t blk = (size_t)slot * nrt + rb;
             if (sg.nu != upi) {
-                // this cluster reduced only some of the row block's column tiles
-                const size_t blk = (size_t)slot * nrt + rb;
-                const size_t o = (blk * TC_MAX_SPLIT + sg.fu) * TC_BM + row;
-                P.tc_pm[o] = m;
-                P.tc_ps[o] = sm;
+                // this cluster reduced only some of the row block's column tiles: the last to arrive finishes
                 __threadfence();
                 asm volatile("bar.sync 4, 128;" ::: "memory");
-                if (row == 0) arrival = atomicAdd(&P.tc_cnt[blk], (unsigned)sg.nu + (1u << (8 + sg.fu)));
+                if (row == 0) arrival = atomicAdd(&P.tc_cnt[blk], (unsigned)sg.nu);
                 asm volatile("bar.sync 4, 128;" ::: "memory");
                 const unsigned before = arrival;
                 asm volatile("bar.sync 4, 128;" ::: "memory");          // `arrival` is free again
-                if ((int)(before & 0xffu) + sg.nu != upi) continue;     // not the last part: done
+                if ((int)before + sg.nu != upi) continue;
                 if (row == 0) P.tc_cnt[blk] = 0u;
                 __threadfence();
-                const unsigned starts = (before >> 8) | (1u << sg.fu);
-                m = NEG_BIG; sm = 0.0;
-                for (int f = 0; f < upi; ++f) {
-                    if (!((starts >> f) & 1u)) continue;
-                    const size_t q = (blk * TC_MAX_SPLIT + f) * TC_BM + row;
-                    const float mo = reinterpret_cast<volatile float *>(P.tc_pm)[q];
-                    const double so = reinterpret_cast<volatile double *>(P.tc_ps)[q];
-                    const float mn = fmaxf(m, mo);
-                    sm = sm * (double)pow2i(m - mn) + so * (double)pow2i(mo - mn);
-                    m = mn;
-                }
+            }
+            float m = NEG_BIG;
+            double sm = 0.0;
+            for (int f = 0; f < 2 * upi; ++f) {                         // units in order, even chunks before odd ones
+                const size_t q = (blk * (2 * TC_MAX_SPLIT) + f) * TC_BM + row;
+                const float mo = reinterpret_cast<volatile float *>(P.tc_pm)[q];
+                const double so = reinterpret_cast<volatile double *>(P.tc_ps)[q];
+                const float mn = fmaxf(m, mo);
+                sm = sm * (double)pow2i(m - mn) + so * (double)pow2i(mo - mn);
+                m = mn;
             }
             const bool frozen = (P.mode == MODE_MASKED) && P.state[slot] != 0;
             const int i = rb * TC_BM + row;
@@ -762,26 +760,22 @@ update_tc_pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_cons
                     if (leader) mbar_arrive(b_tempty + 8 * buf);
                     else mbar_arrive_remote(b_tempty_leader + 8 * buf);
                 }
+                if ((t + 1) % g == 0 || t + 1 == ntiles) {
+                    // a unit is complete: its row results go to scratch and the reduction starts afresh
+                    if (!ghost) {
+                        const size_t q = ((((size_t)slot * nrt + rb) * TC_MAX_SPLIT + t / g) * 2 + half) * TC_BM + row;
+                        P.tc_pm[q] = mx;
+                        P.tc_ps[q] = sd;
+                    }
+                    mx = NEG_BIG;
+                    sd = 0.0;
+                }
             }
             if (!ok) break;
-            // merge the two column halves of every row and hand the results to the filing warps
-            if (!ghost) {
-                // the previous segment's results may still be being read; a wait that runs out raises
-                // the abort flag, which the next tile's vote turns into a common exit
-                if (nbox > 0) mbar_wait(b_box_empty, (nbox - 1) & 1, ab);
-                if (half) { xm[row] = mx; xs[row] = sd; }
-            }
+            // tell the filing warps that this segment's units are in scratch (at most one announcement ahead)
+            if (!ghost && nbox > 0) mbar_wait(b_box_empty, (nbox - 1) & 1, ab);
             asm volatile("bar.sync 1, 256;" ::: "memory");
-            if (!half) {
-                if (!ghost) {
-                    const float mo = xm[row];
-                    const float mn = fmaxf(mx, mo);
-                    xs[row] = sd * (double)pow2i(mx - mn) + xs[row] * (double)pow2i(mo - mn);
-                    xm[row] = mn;
-                }
-                asm volatile("bar.sync 2, 128;" ::: "memory");
-                if (e == 0 && !ghost) mbar_arrive(b_box_full);
-            }
+            if (e == 0 && !ghost) mbar_arrive(b_box_full);
             if (!ghost) ++nbox;
         }
     }
@@ -840,17 +834,12 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
 
 bool tc_eligible(int d, bool bf16) { return bf16 && d >= 64 && d <= 512 && d % 64 == 0; }
 
-// two ring stages when that lets two CTAs share an SM (d <= 256: the second CTA's MMAs cover
-// this CTA's prologue and epilogue), four otherwise
-// beyond d = 256 the row block lives in tensor memory, which leaves shared memory to a 12-stage ring
-// d <= 256: 128-column tiles, two ring stages, small enough for two CTAs per SM (the second CTA's MMAs
-// cover this CTA's prologue and epilogue).  d > 256: 256-column tiles (the tensor pipe runs 128x256 MMAs
-// about twice as efficiently as 128x128 ones), three 32 KB stages beside the 128 KB row block.
-#ifndef SKB_TC_WIDE_FROM
-#define SKB_TC_WIDE_FROM 257
-#endif
-static bool tc_wide(int d) { return d >= SKB_TC_WIDE_FROM && d >= 2 * TC_BK; }   // the pair kernel's ring needs two stages <= d/64
-size_t tc_smem_bytes(int d) { return (size_t)(d / TC_BK + (tc_wide(d) ? 6 : 2)) * TC_CHUNK; }
+// d <= 256: 128-column tiles and two ring stages, small enough for two CTAs per SM (the second
+// CTA's MMAs cover this CTA's prologue and epilogue).  d > 256: the persistent CTA-pair kernel
+// (its ring needs two stages and no more than d/64).
+constexpr size_t TC_SMEM_LIMIT = 232448;                  // 227 KB: static + dynamic shared memory of one CTA
+static bool tc_wide(int d) { return d > 256; }
+size_t tc_smem_bytes(int d) { return (size_t)(d / TC_BK + 2) * TC_CHUNK; }   // the two-CTAs-per-SM kernel
 
 // Tensor map of one tiled operand copy: rows of 64 bf16 (128 B, contiguous), 128-row boxes.
 const char *tc_make_map(void *out_map, void *base, int W, int npts, int d)
@@ -899,50 +888,45 @@ void launch_retile(const void *src, void *dst, int W, int npts, int d, cudaStrea
 void launch_update_tc(const Dev &P, const void *maps, int leg, int width, cudaStream_t st)
 {
     // dynamic shared memory: the tiles, plus what it takes to start them on a 1024-byte boundary
-    static size_t pad[3] = {0, 0, 0};
+    static size_t pad[2] = {0, 0};
     static size_t pair_static = 0;
+    static int sm_count = 0;
     static bool attr_set = false;
-    static bool use_pair = true;
     if (!attr_set) {
         cudaFuncAttributes fa;
         cudaFuncGetAttributes(&fa, update_tc_kernel<2, 128>);
         pad[0] = (1024 - fa.sharedSizeBytes % 1024) % 1024;
-        cudaFuncGetAttributes(&fa, update_tc_kernel<3, 256>);
-        pad[1] = (1024 - fa.sharedSizeBytes % 1024) % 1024;
         cudaFuncGetAttributes(&fa, update_tc_pair_kernel);
-        pad[2] = (1024 - fa.sharedSizeBytes % 1024) % 1024;
+        pad[1] = (1024 - fa.sharedSizeBytes % 1024) % 1024;
         pair_static = fa.sharedSizeBytes;
         cudaFuncSetAttribute(update_tc_kernel<2, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(tc_smem_bytes(256) + pad[0]));
-        cudaFuncSetAttribute(update_tc_kernel<3, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(tc_smem_bytes(512) + pad[1]));
-        cudaFuncSetAttribute(update_tc_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(232448 - pair_static));
-        const char *e = getenv("SKB_TC_PAIR");
-        if (e && e[0] == '0') use_pair = false;
+        cudaFuncSetAttribute(update_tc_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(TC_SMEM_LIMIT - pair_static));
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
         attr_set = true;
     }
     const CUtensorMap *tm = reinterpret_cast<const CUtensorMap *>(maps);
-    const int nrows = (leg == LEG_F) ? P.n : P.m;
+    const int nrows = (leg == LEG_F) ? P.n : P.m, ncols = (leg == LEG_F) ? P.m : P.n;
     const int nrt = (nrows + TC_BM - 1) / TC_BM;
-    dim3 grid(nrt, width < 1 ? 1 : width);
+    const int lanes = width < 1 ? 1 : width;
     if (!tc_wide(P.d)) {
-        launch_pdl(update_tc_kernel<2, 128>, grid, dim3(TC_THREADS), tc_smem_bytes(P.d) + pad[0], st, tm[0], tm[1], P, leg);
-    } else if (use_pair) {
-        // as many 16 KB ring stages as fit beside the resident row block (six at d = 512), an even
-        // number (released in pairs) and no more than a tile has chunks (see the kernel's header)
-        const size_t room = 232448 - pair_static - pad[2] - (size_t)(P.d / TC_BK) * TC_CHUNK;
-        int nst = (int)(room / TC_CHUNK);
-        if (nst > TC2_MAX_STAGES) nst = TC2_MAX_STAGES;
-        if (nst > P.d / TC_BK) nst = P.d / TC_BK;
-        nst &= ~1;
-        static int sm_count = 0;
-        if (!sm_count) { int dev = 0; cudaGetDevice(&dev); cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev); }
-        const int ncolsh = (leg == LEG_F) ? P.m : P.n;
-        const int ntl = (ncolsh + TC2_BN - 1) / TC2_BN, gg = (ntl + TC_MAX_SPLIT - 1) / TC_MAX_SPLIT;
-        const long long units = (long long)(width < 1 ? 1 : width) * ((nrt + 1) / 2) * ((ntl + gg - 1) / gg);
-        const int ncl = units < sm_count / 2 ? (int)units : sm_count / 2;
-        launch_pdl(update_tc_pair_kernel, dim3(2 * ncl), dim3(TC2_THREADS), (size_t)(P.d / TC_BK + nst) * TC_CHUNK + pad[2], st, tm[0], tm[1], P, leg, nst);
-    } else {
-        launch_pdl(update_tc_kernel<3, 256>, grid, dim3(TC_THREADS), tc_smem_bytes(P.d) + pad[1], st, tm[0], tm[1], P, leg);
+        launch_pdl(update_tc_kernel<2, 128>, dim3(nrt, lanes), dim3(TC_THREADS), tc_smem_bytes(P.d) + pad[0], st, tm[0], tm[1], P, leg);
+        return;
     }
+    // as many 16 KB ring stages as fit beside the resident row block (six at d = 512), an even
+    // number (released in pairs) and no more than a tile has chunks (see the kernel's header)
+    const int nkc = P.d / TC_BK;
+    const size_t room = TC_SMEM_LIMIT - pair_static - pad[1] - (size_t)nkc * TC_CHUNK;
+    int nst = (int)(room / TC_CHUNK);
+    if (nst > TC2_MAX_STAGES) nst = TC2_MAX_STAGES;
+    if (nst > nkc) nst = nkc;
+    nst &= ~1;
+    // one cluster per SM pair, fewer if there are fewer units of work
+    const int ntl = (ncols + TC2_BN - 1) / TC2_BN, g = tc_unit_tiles(ntl);
+    const long long units = (long long)lanes * ((nrt + 1) / 2) * ((ntl + g - 1) / g);
+    const int ncl = units < sm_count / 2 ? (int)units : sm_count / 2;
+    launch_pdl(update_tc_pair_kernel, dim3(2 * ncl), dim3(TC2_THREADS), (size_t)(nkc + nst) * TC_CHUNK + pad[1], st, tm[0], tm[1], P, leg, nst);
 }
 
 }  // namespace skb

@@ -328,6 +328,28 @@ def test_tensor_core_modes_and_compaction(oracle):
     assert pot_err(ra["f"], ra["g"], ref.f, ref.g, w.eps.astype(np.float64)).max() <= POT_TOL_F32
 
 
+@pytest.mark.parametrize("kw", [dict(W=5, n=300, m=520, d=320), dict(W=2, n=140, m=2400, d=512)])
+def test_tensor_core_pair_kernel_shapes_and_modes(oracle, kw):
+    # d > 256 runs the persistent CTA-pair kernel.  These shapes give it an odd number of row blocks
+    # (one CTA of the last pair has no rows), a ring shorter than six stages (d = 320), more column
+    # tiles than units (2400 columns) and, with so few lanes, row blocks whose column tiles are shared
+    # out among many clusters.  Whatever the split, the bits must not depend on it: ACTIVE (shrinking
+    # batch) and MASKED (fixed batch) must agree exactly.
+    w = wl.make("feature", **kw)
+    W = w.shape[0]
+    ra = run_gpu(w, mode="active", compute="tensor")
+    rm = run_gpu(w, mode="masked", compute="tensor")
+    np.testing.assert_array_equal(ra["depth"], rm["depth"])
+    np.testing.assert_array_equal(ra["f"], rm["f"]); np.testing.assert_array_equal(ra["g"], rm["g"])
+    misses = check_against_oracle(oracle, w, ra, range(W), pot_tol=POT_TOL_F32, exact_depth=False)
+    for t, dg, do, margin, decay in misses:
+        assert miss_allowed(margin, decay, MARGIN_F32)
+    check_accounting(oracle, ra, W, "active")
+    rs = run_gpu(w, mode="static", compute="tensor")
+    np.testing.assert_array_equal(ra["depth"], rs["depth"])
+    check_accounting(oracle, rs, W, "static")
+
+
 def test_tensor_core_request_on_ineligible_input_is_refused():
     import torch
     from paper_2607_24741_b200 import binding as B
