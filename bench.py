@@ -34,7 +34,7 @@ UNIT = "lane*n*m updates/s"
 # DRAM bytes (read + write) of ONE full-width f-leg launch of the dominant kernel, taken from ncu
 # captures of `bench.py --workload <name> --kernel-only` (one launch each; they equal the lanes'
 # operands read once)
-NCU_TRAFFIC_BYTES = {"sensor": 20.5e6, "registration": 13.7e6, "sweep": 42.0e6, "feature": 140.8e6}
+NCU_TRAFFIC_BYTES = {"sensor": 20.5e6, "registration": 13.7e6, "sweep": 42.0e6, "feature": 193.3e6}
 
 # nominal unit counts (148 SMs, 128 FP32 lanes and 16 special-function lanes per SM per clock,
 # 64 FP64 lanes) at the maximum SM clock; the fraction reported is against these
@@ -377,7 +377,7 @@ def main():
             # the cross term is a dense bf16 contraction: 2*d flops per pair against the measured
             # cuBLAS bf16 burst throughput (kernel timed alone)
             tf = 2.0 * d * pairs / (k_ms * 1e-3) / 1e12
-            line["roofline"] = {"bound": "tensor", "kernel": "update_tc_kernel (f-leg, full width)",
+            line["roofline"] = {"bound": "tensor", "kernel": "update_tc_pair_kernel (f-leg, full width)",
                                 "arithmetic": arith, "achieved": tf, "peak": pk["bf16_tflops"], "unit": "TFLOP/s",
                                 "frac": tf / pk["bf16_tflops"], "exp_frac": achieved_exp / mufu_peak,
                                 "ms_per_launch": k_ms, "pairs_per_launch": pairs,
