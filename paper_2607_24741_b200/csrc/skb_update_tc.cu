@@ -741,14 +741,26 @@ update_tc_pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_cons
             float g_next = (sg.t0 * TC2_BN + e < cp) ? colt[sg.t0 * TC2_BN + e] : NEG_BIG;   // column term, one tile ahead
             for (int t = sg.t0; t < sg.t1; ++t, ++tg) {
                 const int buf = tg & 1;
+#ifdef SKB_TC_DEBUG
+                const long long tb0 = clock64();
+#endif
                 asm volatile("bar.sync 1, 256;" ::: "memory");          // everyone is done with the previous tile's column terms
+#ifdef SKB_TC_DEBUG
+                dbg_w1 += clock64() - tb0;
+#endif
                 gts[e] = g_next;
                 {
                     const int j = (t + 1) * TC2_BN + e;
                     g_next = (t + 1 < sg.t1 && j < cp) ? colt[j] : NEG_BIG;
                 }
                 ok = TC_TIMED_WAIT(dbg_w0, mbar_wait(b_tfull + 8 * buf, (tg >> 1) & 1, ab));
+#ifdef SKB_TC_DEBUG
+                const long long tb1 = clock64();
+#endif
                 ok = epi_all(ok);                                       // also publishes the column terms
+#ifdef SKB_TC_DEBUG
+                dbg_w1 += clock64() - tb1;
+#endif
                 if (!ok) break;
                 tc_fence_after();
                 tc_reduce_tile<TC2_BN>(lane_base + (uint32_t)(buf * TC2_BN), gts, half, two_s, mx, ts, sd);
@@ -838,7 +850,7 @@ bool tc_eligible(int d, bool bf16) { return bf16 && d >= 64 && d <= 512 && d % 6
 // CTA's MMAs cover this CTA's prologue and epilogue).  d > 256: the persistent CTA-pair kernel
 // (its ring needs two stages and no more than d/64).
 constexpr size_t TC_SMEM_LIMIT = 232448;                  // 227 KB: static + dynamic shared memory of one CTA
-static bool tc_wide(int d) { return d > 256; }
+static bool tc_wide(int d) { return d > 256; }             // measured: the two kernels break even at d = 256
 size_t tc_smem_bytes(int d) { return (size_t)(d / TC_BK + 2) * TC_CHUNK; }   // the two-CTAs-per-SM kernel
 
 // Tensor map of one tiled operand copy: rows of 64 bf16 (128 B, contiguous), 128-row boxes.
