@@ -160,6 +160,9 @@ def main():
     ap.add_argument("--width-sweep", action="store_true",
                     help="width report: W in {1,2,4,8,16} lanes of the registration law at n = 4096, solved "
                          "one lane at a time (width-one), static-packed and active-packed (one JSON line)")
+    ap.add_argument("--audit-arms", action="store_true",
+                    help="time the audit policies on --workload: fused row screen + column check of flagged lanes "
+                         "(default) against a full two-sided check of every lane, each at every cycle and every 4th")
     ap.add_argument("--kernel-only", action="store_true",
                     help="only create the batch and time the update kernel (few launches; for profiler captures)")
     args = ap.parse_args()
@@ -252,6 +255,33 @@ def main():
             rows.append(row)
         print(json.dumps({"report": "tol-sweep", "workload": args.workload, "W": W, "n": n, "m": m, "d": d,
                           "rows": rows}), flush=True)
+        return
+    if args.audit_arms:
+        rows, ref_depth = [], {}
+        for every in (1, 4):
+            for arm, screen in (("screen", 0.0), ("full_check", 1e30)):
+                best, info, depth = None, None, None
+                for rep in range(3):
+                    torch.cuda.synchronize()
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                    sb = B.SinkhornBatch(x, y, a, b, eps, w.tol, mode=args.mode, compute=args.compute, max_iter=w.max_iter,
+                                         audit_every=every, tol_screen=screen)
+                    sb.drain()
+                    e1.record(); torch.cuda.synchronize()
+                    ms_ = e0.elapsed_time(e1)
+                    best = ms_ if best is None or ms_ < best else best
+                    depth, status = sb.depths(); st = sb.stats()
+                    info = {"slots": st["slots"], "cycles": st["cycles"], "pair_terms": st["pair_terms"],
+                            "done": int((status == 1).sum().item())}
+                    sb.close()
+                ref_depth.setdefault(every, depth)
+                # pair terms beyond the two legs of every slot are the column checks
+                check_terms = info["pair_terms"] - 2 * info["slots"] * n * m
+                rows.append({"audit_every": every, "arm": arm, "ms": best, **info, "column_check_pair_terms": check_terms,
+                             "depths_equal_to_screen_arm": bool((depth == ref_depth[every]).all().item())})
+        print(json.dumps({"report": "audit-arms", "workload": args.workload, "mode": args.mode, "W": W, "n": n, "m": m,
+                          "d": d, "tol": w.tol, "rows": rows}), flush=True)
         return
     if args.kernel_only:
         sb = B.SinkhornBatch(x, y, a, b, eps, w.tol, mode="static", compute=args.compute, max_iter=w.max_iter)
