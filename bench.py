@@ -149,7 +149,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="sensor", choices=["tiny", "sensor", "feature", "registration", "sweep"])
-    ap.add_argument("--mode", default="active", choices=["active", "masked", "static"])
+    ap.add_argument("--mode", default="active", choices=["active", "masked", "static", "masked_exit"])
     ap.add_argument("--compute", default="auto", choices=["auto", "f32", "mixed", "f64", "tensor"])
     ap.add_argument("--no-controls", action="store_true", help="skip the static / masked control timings")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -231,7 +231,7 @@ def main():
         rows = []
         for tol in wlmod.SWEEP_TOLS:
             row = {"tol": tol}
-            for mode in ("static", "masked", "active"):
+            for mode in ("static", "masked", "masked_exit", "active"):
                 best, info = None, None
                 for rep in range(3):
                     torch.cuda.synchronize()
@@ -252,6 +252,7 @@ def main():
             row["removed_slots"] = row["static"]["slots"] - row["active"]["slots"]
             row["static_over_active"] = row["static"]["ms"] / row["active"]["ms"]
             row["masked_over_active"] = row["masked"]["ms"] / row["active"]["ms"]
+            row["masked_exit_over_active"] = row["masked_exit"]["ms"] / row["active"]["ms"]
             rows.append(row)
         print(json.dumps({"report": "tol-sweep", "workload": args.workload, "W": W, "n": n, "m": m, "d": d,
                           "rows": rows}), flush=True)

@@ -51,7 +51,12 @@ typedef enum {
 typedef enum {
     SKB_ACTIVE = 0, /* retire and physically compact: later kernels run at survivor width A_k */
     SKB_MASKED = 1, /* freeze its potentials, keep it in place: kernels stay at width W        */
-    SKB_STATIC = 2  /* keep updating every lane until the deepest lane passes (l_max)          */
+    SKB_STATIC = 2, /* keep updating every lane until the deepest lane passes (l_max)          */
+    SKB_MASKED_EXIT = 3 /* as MASKED, but the thread blocks of a frozen lane return at once: a     */
+                        /* launch slot per lane, no pair work.  NOT the paper's logical-mask       */
+                        /* control (which keeps W * l_max slots of work, Section "controls"); an   */
+                        /* extra arm that asks whether physically moving survivors still pays on a  */
+                        /* kernel that can skip lanes.  Results are bit-identical to MASKED.        */
 } skb_mode;
 
 typedef enum { SKB_F32 = 0, SKB_BF16 = 1 } skb_dtype;           /* storage type of x and y only */

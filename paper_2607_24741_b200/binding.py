@@ -17,7 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libsinkhorn_batch.so")
 SKB_OK = 0
 STATUS_NAMES = {0: "SKB_OK", 1: "SKB_ERR_NULL", 2: "SKB_ERR_SHAPE", 3: "SKB_ERR_VALUE",
                 4: "SKB_ERR_WORKSPACE", 5: "SKB_ERR_STATE", 6: "SKB_ERR_CUDA"}
-MODES = {"active": 0, "masked": 1, "static": 2}
+MODES = {"active": 0, "masked": 1, "static": 2, "masked_exit": 3}
 COMPUTE = {"auto": 0, "f32": 1, "mixed": 2, "f64": 3, "tensor": 4}
 LANE_RUNNING, LANE_DONE, LANE_ITER_LIMIT, LANE_NONFINITE = 0, 1, 2, 3
 

@@ -79,7 +79,7 @@ static bool config_ok(const skb_config *c, std::string &why)
     if (!c) { why = "config is null"; return false; }
     if (c->W < 1 || c->n < 1 || c->m < 1 || c->d < 1) { why = "W, n, m, d must be >= 1"; return false; }
     if (c->xy_dtype != SKB_F32 && c->xy_dtype != SKB_BF16) { why = "bad xy_dtype"; return false; }
-    if (c->mode < SKB_ACTIVE || c->mode > SKB_STATIC) { why = "bad mode"; return false; }
+    if (c->mode < SKB_ACTIVE || c->mode > SKB_MASKED_EXIT) { why = "bad mode"; return false; }
     if (c->compute < SKB_COMPUTE_AUTO || c->compute > SKB_COMPUTE_TENSOR) { why = "bad compute type"; return false; }
     if (c->max_iter < 1 || c->audit_every < 1) { why = "max_iter and audit_every must be >= 1"; return false; }
     if (c->cost_form < 0 || c->cost_form > 2) { why = "cost_form must be 0 (automatic), 1 (expanded) or 2 (difference)"; return false; }
@@ -104,7 +104,9 @@ static size_t carve(const skb_config *c, const Variant *var, bool tensor, char *
     Dev d;
     memset(&d, 0, sizeof(d));
     d.W = c->W; d.n = c->n; d.m = c->m; d.d = c->d; d.np = (int)np; d.mp = (int)mp; d.DP = (int)DP;
-    d.mode = c->mode; d.max_iter = c->max_iter; d.audit_every = c->audit_every;
+    d.mode = c->mode == SKB_MASKED_EXIT ? (int)MODE_MASKED : (int)c->mode;
+    d.early_exit = c->mode == SKB_MASKED_EXIT;
+    d.max_iter = c->max_iter; d.audit_every = c->audit_every;
     d.xy_bf16 = c->xy_dtype == SKB_BF16; d.compute_f64 = var->f64;
     d.cost_form = c->d > 32 ? 1 : c->cost_form;      // the large-d kernels only have the expanded form
     // fp32: above this scaled squared radius the expanded cost loses more than ~4e-6 per term

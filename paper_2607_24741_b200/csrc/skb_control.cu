@@ -250,7 +250,9 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_kernel(const Dev P)
         Ctl *g = P.ctl;
         g->n_retire = (P.mode == MODE_STATIC) ? 0 : nret;
         g->emit_parity = c.parity;
-        g->pair_terms += (long long)A * P.n * P.m              // the f-leg that produced this screen
+        // lanes whose pair terms were really evaluated (the early-exit arm skips frozen lanes)
+        const int worked = P.early_exit ? c.n_running : A;
+        g->pair_terms += (long long)worked * P.n * P.m         // the f-leg that produced this screen
                          + (long long)nflagged * P.n * P.m;    // column checks
         bool go_on;
         if (P.mode == MODE_ACTIVE) {
@@ -263,7 +265,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_kernel(const Dev P)
             if (!go_on) g->static_final = 1;
         }
         if (go_on) {
-            const int width = (P.mode == MODE_ACTIVE) ? Anew : P.W;
+            const int width = (P.mode == MODE_ACTIVE) ? Anew : (P.early_exit ? g->n_running : P.W);
             g->cycle = k + 1;
             g->parity = c.parity ^ 1;
             g->slots += width;

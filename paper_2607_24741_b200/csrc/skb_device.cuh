@@ -50,6 +50,7 @@ struct Ctl {
 struct Dev {
     int W, n, m, d, np, mp, DP;
     int mode, max_iter, audit_every, xy_bf16, compute_f64, cost_form, tensor;
+    int early_exit;           // MASKED only: CTAs of a frozen lane return at once (an extra arm, not the paper's mask control)
     double form_threshold;    // scaled squared radius above which a lane uses the difference form
     double tol_screen, tol_stop;
     // slabs by slot

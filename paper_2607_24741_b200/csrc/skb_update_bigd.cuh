@@ -46,6 +46,7 @@ __global__ void __launch_bounds__(UPD_THREADS) update_bigd_kernel(const Dev P, c
     if (c.done) return;
     const int slot = blockIdx.y;
     if (slot >= c.n_phys) return;
+    if (P.early_exit && P.state[slot] != 0) return;     // early-exit mask arm: a frozen lane costs a launch slot only
     if (leg != LEG_V && c.static_final) return;
     if (leg == LEG_V && !(c.static_final || P.flag[slot])) return;
     const bool rows_x = (leg == LEG_F);

@@ -257,6 +257,7 @@ update_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant_
     if (c.done) return;
     const int slot = blockIdx.y;
     if (slot >= c.n_phys) return;
+    if (P.early_exit && P.state[slot] != 0) return;     // early-exit mask arm: a frozen lane costs a launch slot only
     if (leg != LEG_V && c.static_final) return;
     if (leg == LEG_V && !(c.static_final || P.flag[slot])) return;
     const bool rows_x = (leg == LEG_F);
@@ -603,7 +604,7 @@ update_tc_pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_cons
     // visits lanes that the screen flagged)
     SegIter it = it0;
     Seg sg;
-#define TC2_SKIP(slot) (leg == LEG_V && !(c.static_final || P.flag[slot]))
+#define TC2_SKIP(slot) ((leg == LEG_V && !(c.static_final || P.flag[slot])) || (P.early_exit && P.state[slot] != 0))
 
     if (warp == TC_EPI_WARPS) {
         // ---------------- producer (one per CTA): own row block once per segment, own half of every column tile

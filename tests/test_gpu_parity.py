@@ -117,6 +117,20 @@ def test_masked_equals_active_bitwise_and_static_matches_fixed_depth(oracle, cas
     assert rs["stats"]["slots"] - ra["stats"]["slots"] == W * lmax - int(ra["depth"].sum())
 
 
+@pytest.mark.parametrize("case,compute", [("sensor_ragged", "f32"), ("sweep_small", "mixed"), ("tiny", "f64")])
+def test_early_exit_mask_arm_equals_the_mask_control_bitwise(oracle, case, compute):
+    # the extra arm skips the pair work of frozen lanes: same bits as MASKED, but only the slots of ACTIVE
+    w = _make(case)
+    W = w.shape[0]
+    rm = run_gpu(w, mode="masked", compute=compute)
+    re = run_gpu(w, mode="masked_exit", compute=compute)
+    np.testing.assert_array_equal(rm["depth"], re["depth"]); np.testing.assert_array_equal(rm["status"], re["status"])
+    np.testing.assert_array_equal(rm["f"], re["f"]); np.testing.assert_array_equal(rm["g"], re["g"])
+    np.testing.assert_array_equal(rm["r_row"], re["r_row"]); np.testing.assert_array_equal(rm["r_col"], re["r_col"])
+    assert re["stats"]["slots"] == int(re["depth"].sum()) and rm["stats"]["slots"] == W * int(rm["depth"].max())
+    np.testing.assert_array_equal(np.array(re["stats"]["widths"]), oracle.slot_counts(re["depth"].astype(np.int64))["widths"])
+
+
 def test_packing_commutes_with_the_per_lane_map(oracle):
     # Eq. 2: a W-lane batch gives each lane what a one-lane batch gives it, bit for bit
     # (the arithmetic is fixed here: the automatic choice looks at the whole batch)
@@ -348,6 +362,9 @@ def test_tensor_core_pair_kernel_shapes_and_modes(oracle, kw):
     rs = run_gpu(w, mode="static", compute="tensor")
     np.testing.assert_array_equal(ra["depth"], rs["depth"])
     check_accounting(oracle, rs, W, "static")
+    rx = run_gpu(w, mode="masked_exit", compute="tensor")           # frozen lanes skipped, same bits
+    np.testing.assert_array_equal(rx["f"], rm["f"]); np.testing.assert_array_equal(rx["g"], rm["g"])
+    assert rx["stats"]["slots"] == ra["stats"]["slots"]
 
 
 def test_tensor_core_request_on_ineligible_input_is_refused():
