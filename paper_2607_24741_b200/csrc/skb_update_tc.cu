@@ -534,7 +534,7 @@ update_tc_pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_cons
                       const int nstages)
 {
     extern __shared__ __align__(1024) unsigned char smem_tc[];
-    __shared__ __align__(8) unsigned long long bars[TC2_MAX_STAGES + TC2_MAX_STAGES / 2 + 6];
+    __shared__ __align__(8) unsigned long long bars[2 * TC2_MAX_STAGES + 6];
     __shared__ uint32_t tmem_holder;
     __shared__ int abort_flag;
     __shared__ unsigned arrival;                           // filing warps: the arrival word before this part's add
@@ -570,7 +570,7 @@ update_tc_pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_cons
     const uint32_t sbase = (smem_u32(smem_tc) + 1023u) & ~1023u;
     const uint32_t sA = sbase, sB = sbase + (uint32_t)nkc * TC_CHUNK;
     const uint32_t b_full = smem_u32(&bars[0]), b_empty = smem_u32(&bars[TC2_MAX_STAGES]);
-    const uint32_t b_tfull = smem_u32(&bars[TC2_MAX_STAGES + TC2_MAX_STAGES / 2]), b_tempty = b_tfull + 16;
+    const uint32_t b_tfull = smem_u32(&bars[2 * TC2_MAX_STAGES]), b_tempty = b_tfull + 16;
     const uint32_t b_box_full = b_tfull + 32, b_box_empty = b_tfull + 40;
     // the same barriers seen in the leader's / the peer's shared memory
     const uint32_t b_full_leader = map_to_cta(b_full, 0);
@@ -580,7 +580,7 @@ update_tc_pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_cons
 
     if (tid == 0) {
         for (int s = 0; s < nstages; ++s) mbar_init(b_full + 8 * s, 1);
-        for (int q = 0; q < nstages / 2; ++q) mbar_init(b_empty + 8 * q, 1);
+        for (int q = 0; q < nstages; ++q) mbar_init(b_empty + 8 * q, 1);
         for (int b = 0; b < 2; ++b) { mbar_init(b_tfull + 8 * b, 1); mbar_init(b_tempty + 8 * b, 2 * TC_EPI_WARPS); }
         mbar_init(b_box_full, 1); mbar_init(b_box_empty, TC2_FILE_WARPS);
         abort_flag = 0;
@@ -619,8 +619,7 @@ update_tc_pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_cons
                 const int col_tile0 = sg.slot * nct128 * nkc;
                 for (int t = sg.t0; t < sg.t1 && go; ++t) {
                     for (int kc = 0; kc < nkc; ++kc) {
-                        // stages are released two at a time (one commit per eight MMAs)
-                        if (!first_round && (s & 1) == 0 && !TC_TIMED_WAIT(dbg_w0, mbar_wait(b_empty + 8 * (s >> 1), ph ^ 1u, ab))) { go = false; break; }
+                        if (!first_round && !TC_TIMED_WAIT(dbg_w0, mbar_wait(b_empty + 8 * s, ph ^ 1u, ab))) { go = false; break; }
                         if (leader) mbar_expect_tx(b_full + 8 * s, t == sg.t0 ? 4 * TC_CHUNK : 2 * TC_CHUNK);
                         if (t == sg.t0)
                             tma_load_chunk_pair(sA + kc * TC_CHUNK, tm_row, ghost ? 0x7fffff80 : (row_tile0 + kc) * TC_BM, b_full_leader + 8 * s);
@@ -659,10 +658,8 @@ update_tc_pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_cons
                         tc_mma_pair(d_tmem, ad + 2, bd + 2, tc_idesc_pair(), 1u);
                         tc_mma_pair(d_tmem, ad + 4, bd + 4, tc_idesc_pair(), 1u);
                         tc_mma_pair(d_tmem, ad + 6, bd + 6, tc_idesc_pair(), 1u);
-                        if (s & 1) {                            // both producers may refill this pair of stages
-                            tc_commit_pair(b_empty + 8 * (s >> 1));
-                            tc_commit_pair(b_empty_peer + 8 * (s >> 1));
-                        }
+                        tc_commit_pair(b_empty + 8 * s);        // both producers may refill this stage
+                        tc_commit_pair(b_empty_peer + 8 * s);
                         if (++s == nstages) { s = 0; ph ^= 1u; }
                     }
                     if (ok) { tc_commit_pair(b_tfull + 8 * buf); tc_commit_pair(b_tfull_peer + 8 * buf); }
@@ -927,14 +924,13 @@ void launch_update_tc(const Dev &P, const void *maps, int leg, int width, cudaSt
         launch_pdl(update_tc_kernel<2, 128>, dim3(nrt, lanes), dim3(TC_THREADS), tc_smem_bytes(P.d) + pad[0], st, tm[0], tm[1], P, leg);
         return;
     }
-    // as many 16 KB ring stages as fit beside the resident row block (six at d = 512), an even
-    // number (released in pairs) and no more than a tile has chunks (see the kernel's header)
+    // as many 16 KB ring stages as fit beside the resident row block (six at d = 512), at least
+    // two and no more than a tile has chunks (see the kernel's header)
     const int nkc = P.d / TC_BK;
     const size_t room = TC_SMEM_LIMIT - pair_static - pad[1] - (size_t)nkc * TC_CHUNK;
     int nst = (int)(room / TC_CHUNK);
     if (nst > TC2_MAX_STAGES) nst = TC2_MAX_STAGES;
     if (nst > nkc) nst = nkc;
-    nst &= ~1;
     // one cluster per SM pair, fewer if there are fewer units of work
     const int ntl = (ncols + TC2_BN - 1) / TC2_BN, g = tc_unit_tiles(ntl);
     const long long units = (long long)lanes * ((nrt + 1) / 2) * ((ntl + g - 1) / g);
