@@ -367,6 +367,20 @@ def test_tensor_core_pair_kernel_shapes_and_modes(oracle, kw):
     assert rx["stats"]["slots"] == ra["stats"]["slots"]
 
 
+def test_tensor_core_pair_kernel_many_small_lanes(oracle):
+    # many more work units than clusters: every cluster walks several segments of different lanes,
+    # retirements move the tiled operand copies, and the column check visits a few flagged lanes
+    w = wl.make("feature", W=150, n=130, m=140, d=320)
+    r = run_gpu(w, mode="active", compute="tensor")
+    lanes = [0, 1, 73, 74, 75, 148, 149] + list(range(9, 150, 29))
+    misses = check_against_oracle(oracle, w, r, lanes, pot_tol=POT_TOL_F32, exact_depth=False)
+    for t, dg, do, margin, decay in misses:
+        assert miss_allowed(margin, decay, MARGIN_F32)
+    check_accounting(oracle, r, 150, "active")
+    rm = run_gpu(w, mode="masked", compute="tensor")
+    np.testing.assert_array_equal(rm["depth"], r["depth"]); np.testing.assert_array_equal(rm["f"], r["f"])
+
+
 def test_tensor_core_request_on_ineligible_input_is_refused():
     import torch
     from paper_2607_24741_b200 import binding as B
