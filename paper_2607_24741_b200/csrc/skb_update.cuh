@@ -254,33 +254,12 @@ __device__ __forceinline__ void stream_f32(float *sm, const float *colc, const f
 #pragma unroll
                     for (int p = 0; p < NP; ++p) acc[r][p] = add2(add2(phd[r], ct[p]), sub2(cl[p], acc[r][p]));
             }
-            // running maxima: one rarely taken branch per step covers all rows
-            float mt[R];
+            // Exponentials against the reference as it stands; only their sum is tested.  A sum
+            // above 2^10 (an argument more than ~8 above the reference, which would cost exponent
+            // accuracy; a reference of minus infinity gives an infinite sum) sends the step
+            // through the exact path: maxima, integer-valued new references, exact rescale.
+            u64 es[R];
             bool grow = false;
-#pragma unroll
-            for (int r = 0; r < R; ++r) {
-                float a[CW];
-#pragma unroll
-                for (int p = 0; p < NP; ++p) unpack2(acc[r][p], a[2 * p], a[2 * p + 1]);
-                mt[r] = fmaxf(a[0], a[1]);
-#pragma unroll
-                for (int e = 2; e < CW; ++e) mt[r] = fmaxf(mt[r], a[e]);
-                grow = grow || (mt[r] > mx[r] + 8.0f);
-            }
-            if (grow) {                                        // lazy rescale: terms stay below 2^9
-#pragma unroll
-                for (int r = 0; r < R; ++r) {
-                    if (mt[r] > mx[r] + 8.0f) {
-                        const float mn = ceilf(mt[r]);
-                        const float fac = pow2i(mx[r] - mn);
-                        float t0, t1;
-                        unpack2(ts[r], t0, t1);
-                        ts[r] = pack2(t0 * fac, t1 * fac);
-                        sd[r] *= (double)fac;
-                        mx[r] = mn;
-                    }
-                }
-            }
 #pragma unroll
             for (int r = 0; r < R; ++r) {
                 const u64 mm = pack2(mx[r], mx[r]);
@@ -291,11 +270,39 @@ __device__ __forceinline__ void stream_f32(float *sm, const float *colc, const f
                     unpack2(sub2(acc[r][p], mm), lo, hi);
                     e[p] = pack2(ex2_fast(lo), ex2_fast(hi));
                 }
-                u64 es = add2(e[0], e[1]);
+                es[r] = add2(e[0], e[1]);
 #pragma unroll
-                for (int p = 2; p < NP; p += 2) es = add2(es, add2(e[p], e[p + 1]));
-                ts[r] = add2(ts[r], es);
+                for (int p = 2; p < NP; p += 2) es[r] = add2(es[r], add2(e[p], e[p + 1]));
+                float s0, s1;
+                unpack2(es[r], s0, s1);
+                grow = grow || !(s0 + s1 <= 1024.f);
             }
+            if (grow) {                                        // rare: lazy rescale, terms stay below 2^10
+#pragma unroll
+                for (int r = 0; r < R; ++r) {
+                    float a[CW];
+#pragma unroll
+                    for (int p = 0; p < NP; ++p) unpack2(acc[r][p], a[2 * p], a[2 * p + 1]);
+                    float mt = fmaxf(a[0], a[1]);
+#pragma unroll
+                    for (int e = 2; e < CW; ++e) mt = fmaxf(mt, a[e]);
+                    if (mt > mx[r] + 8.0f) {
+                        const float mn = ceilf(mt);
+                        const float fac = pow2i(mx[r] - mn);
+                        float t0, t1;
+                        unpack2(ts[r], t0, t1);
+                        ts[r] = pack2(t0 * fac, t1 * fac);
+                        sd[r] *= (double)fac;
+                        mx[r] = mn;
+                        float q = 0.f;
+#pragma unroll
+                        for (int e = 0; e < CW; ++e) q += ex2_fast(a[e] - mn);
+                        es[r] = pack2(q, 0.f);
+                    }
+                }
+            }
+#pragma unroll
+            for (int r = 0; r < R; ++r) ts[r] = add2(ts[r], es[r]);
         }
 #pragma unroll
         for (int r = 0; r < R; ++r) {
