@@ -115,7 +115,7 @@ static size_t carve(const skb_config *c, const Variant *var, bool tensor, char *
     d.ctl = (Ctl *)take(sizeof(Ctl));
     d.state = (int *)take(W * 4); d.flag = (int *)take(W * 4); d.verdict = (int *)take(W * 4);
     d.nonfinite = (int *)take(W * 4);
-    d.cnt_row = (unsigned *)take(W * 4); d.cnt_col = (unsigned *)take(W * 4);
+    d.rsum_row = (unsigned long long *)take(W * 8); d.rsum_col = (unsigned long long *)take(W * 8);
     d.depth = (int *)take(W * 4); d.status = (int *)take(W * 4); d.emitted = (int *)take(W * 4);
     d.res_row = (double *)take(W * 8); d.res_col = (double *)take(W * 8);
     d.rrow = (double *)take(W * 8); d.rcol = (double *)take(W * 8);
@@ -128,7 +128,6 @@ static size_t carve(const skb_config *c, const Variant *var, bool tensor, char *
     d.ret_slot = (int *)take(W * 4); d.ret_lane = (int *)take(W * 4); d.ret_src = (int *)take(W * 4);
     d.ret_scale = (double *)take(W * 8);
     d.hole_list = (int *)take(W * 4); d.fill_list = (int *)take(W * 4);
-    d.part_row = (double *)take(W * MAX_PARTS * 8); d.part_col = (double *)take(W * MAX_PARTS * 8);
     d.tensor = tensor ? 1 : 0;
     if (tensor) {
         d.xb = take(tc_tiled_bytes(c->W, c->n, c->d)); d.yb = take(tc_tiled_bytes(c->W, c->m, c->d));

@@ -160,6 +160,21 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_kernel(const Dev P)
     const int A = c.n_phys;
     const bool limit = k >= P.max_iter;
 
+    // the legs left each lane's residuals as exact fixed-point sums: turn them into the values,
+    // the screen flag and the two-sided verdict (Eq. 5) everything below works with, and clear
+    // the sums for the next cycle
+    for (int s = tid; s < A; s += NT) {
+        const int fl = lane_flag(P, c, s) ? 1 : 0;
+        const double rr = (double)P.rsum_row[s] * (1.0 / RSUM_SCALE);
+        const double rc = (double)P.rsum_col[s] * (1.0 / RSUM_SCALE);
+        P.rsum_row[s] = 0ull; P.rsum_col[s] = 0ull;
+        if (!c.static_final) P.rrow[s] = rr;         // STATIC's closing column check runs no f-leg: keep the last screen's value
+        P.rcol[s] = rc;
+        P.flag[s] = fl;
+        P.verdict[s] = (!P.nonfinite[s] && fmax(rr, rc) <= P.tol_stop) ? 1 : 0;
+    }
+    __syncthreads();
+
     if (P.mode == MODE_STATIC && c.static_final) {   // emit every lane at the common boundary
         for (int s = tid; s < P.W; s += NT) {
             P.ret_slot[s] = s; P.ret_lane[s] = s; P.ret_src[s] = -1; P.ret_scale[s] = P.scale[s];

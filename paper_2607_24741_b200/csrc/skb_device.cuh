@@ -27,7 +27,9 @@ enum Form : int { FORM_DOT = 0, FORM_DIFF = 1 };
 constexpr float NEG_BIG = -1.0e30f;   // "minus infinity" for padded columns (finite: no NaNs)
 constexpr int UPD_THREADS = 128;
 constexpr int TC_MAX_SPLIT = 8;      // a row block's columns go to at most this many clusters
-constexpr int MAX_PARTS = 1024;       // upper bound on row blocks per lane (residual partials)
+constexpr int MAX_PARTS = 1024;       // upper bound on row blocks per lane (their clamped fixed-point parts cannot overflow 64 bits)
+constexpr double RSUM_SCALE = 1125899906842624.0;   // 2^50
+constexpr double RSUM_PART_MAX = 4.0;                // a row block's part is clamped here (an L1 residual never exceeds 2 near convergence)
 
 // Device-resident control block.  Written by the plan kernel (one CTA), read by all.
 struct Ctl {
@@ -74,8 +76,10 @@ struct Dev {
     int *verdict;             // two-sided check passed
     int *nonfinite;
     double *rrow, *rcol;      // residuals of the audited state
-    unsigned *cnt_row, *cnt_col;
-    double *part_row, *part_col;   // [W][MAX_PARTS] per-CTA partial sums (scratch)
+    // marginal residuals of the audited state as fixed-point sums (units of 2^-50): every row block
+    // adds its part with one integer atomic, so the total is exact and independent of the order
+    // of arrival; the plan kernel turns them into rrow / rcol / flag / verdict and clears them
+    unsigned long long *rsum_row, *rsum_col;
     // tensor path for d > 256: arrival word of a row block whose column tiles were shared out among
     // clusters, and every unit's row results [W][row block][TC_MAX_SPLIT][column half][128]
     unsigned *tc_cnt;
@@ -92,6 +96,16 @@ struct Dev {
     int *widths;              // [max_iter + 2]
     Ctl *ctl;
 };
+
+// Screen verdict of a lane from its accumulated row residual: the same predicate for the column
+// check (which lanes to visit) and for the planner (which lanes may retire).
+__device__ __forceinline__ bool lane_flag(const Dev &P, const Ctl &c, const int slot)
+{
+    const bool passed = P.state[slot] != 0;                  // MASKED: frozen; STATIC: already passed
+    const bool audited = c.cycle >= 1 && (c.cycle % P.audit_every) == 0;
+    const bool live = !(passed && (P.mode == MODE_MASKED || P.mode == MODE_STATIC));
+    return audited && live && !P.nonfinite[slot] && (double)P.rsum_row[slot] * (1.0 / RSUM_SCALE) <= P.tol_screen;
+}
 
 __device__ __forceinline__ float ex2_fast(float x)
 {

@@ -322,7 +322,7 @@ __device__ __forceinline__ void stream_f64(double *sm, const double *colc, const
                                            const int cp, const int ncols,
                                            const double (&xr)[Tune<double, DP>::R][DP],
                                            const int tid, const int cs,
-                                           const float (&m0)[Tune<double, DP>::R],
+                                           const double (&est)[Tune<double, DP>::R],
                                            float (&mx)[Tune<double, DP>::R], double (&sd)[Tune<double, DP>::R])
 {
     constexpr int R = Tune<double, DP>::R, CW = Tune<double, DP>::CW;
@@ -333,12 +333,15 @@ __device__ __forceinline__ void stream_f64(double *sm, const double *colc, const
 
     float ts[R];
     double md[R];
-#pragma unroll
-    for (int r = 0; r < R; ++r) { mx[r] = m0[r]; md[r] = (double)m0[r]; ts[r] = 0.f; sd[r] = 0.0; }
-
     const int ntiles = (ncols + TJ - 1) / TJ;
     load_tile<double, DP, TJ, NR>(sm, colc, colt, colt, cp, 0, tid);
     cp_async_commit();
+    // the reference points only now: the loads behind `est` have been in flight beside the tile's
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+        mx[r] = (fabs(est[r]) < 1.0e7) ? ceilf((float)est[r]) : NEG_BIG;
+        md[r] = (double)mx[r]; ts[r] = 0.f; sd[r] = 0.0;
+    }
     for (int t = 0; t < ntiles; ++t) {
         if (t + 1 < ntiles) {
             load_tile<double, DP, TJ, NR>(sm + ((t + 1) & 1) * STAGE, colc, colt, colt, cp, (t + 1) * TJ, tid);
@@ -479,43 +482,18 @@ __device__ __forceinline__ double finish_one_row(const Dev &P, const Ctl &c, con
     return term;
 }
 
-// One thread per row block hands in its block's residual sum; the last block of the lane to
-// arrive adds all of them in block order (fixed summation order) and sets the lane's flags.
-// Returns true for that last block.
-__device__ __forceinline__ bool finish_lane_residual(const Dev &P, const Ctl &c, const int leg, const int slot,
-                                                     const int nblk, const int blk, const double block_sum, const bool frozen)
+// One thread per row block hands in its block's residual sum: one integer atomic on the lane's
+// fixed-point total (exact, so the total does not depend on the order of arrival; nobody has to
+// arrive last).  A part that is not finite marks the lane instead.
+__device__ __forceinline__ void finish_lane_residual(const Dev &P, const int leg, const int slot,
+                                                     const double block_sum, const bool frozen)
 {
-    double *parts = (leg == LEG_F ? P.part_row : P.part_col) + (size_t)slot * MAX_PARTS;
-    unsigned *cnt = (leg == LEG_F ? P.cnt_row : P.cnt_col) + slot;
-    parts[blk] = block_sum;
-    __threadfence();
-    const unsigned ticket = atomicAdd(cnt, 1u);
-    if (ticket != (unsigned)(nblk - 1)) return false;
-    __threadfence();
-    // block order, eight loads in flight at a time (one memory latency per eight parts, not eight)
-    double tot = 0.0;
-    for (int b0 = 0; b0 < nblk; b0 += 8) {
-        double v[8];
-#pragma unroll
-        for (int j = 0; j < 8; ++j) v[j] = (b0 + j < nblk) ? reinterpret_cast<volatile double *>(parts)[b0 + j] : 0.0;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) if (b0 + j < nblk) tot += v[j];
+    if (!isfinite(block_sum)) {
+        if (leg != LEG_F || !frozen) P.nonfinite[slot] = 1;
+        return;
     }
-    *cnt = 0u;
-    const bool finite = isfinite(tot);
-    if (leg == LEG_F) {
-        P.rrow[slot] = tot;
-        const bool audited = c.cycle >= 1 && (c.cycle % P.audit_every) == 0;
-        const bool live = !frozen && !(P.mode == MODE_STATIC && P.state[slot] != 0);
-        P.flag[slot] = (audited && live && finite && tot <= P.tol_screen) ? 1 : 0;
-        if (!finite && !frozen) P.nonfinite[slot] = 1;
-    } else {
-        P.rcol[slot] = tot;
-        const double two = fmax(P.rrow[slot], tot);
-        P.verdict[slot] = (finite && two <= P.tol_stop) ? 1 : 0;
-        if (!finite) P.nonfinite[slot] = 1;
-    }
-    return true;
+    const unsigned long long part = __double2ull_rn(fmin(block_sum, RSUM_PART_MAX) * RSUM_SCALE);
+    atomicAdd((leg == LEG_F ? P.rsum_row : P.rsum_col) + slot, part);
 }
 
 // Float64 epilogue of a CTA's RB rows (one thread per row) and the fused residual reduction.
@@ -524,7 +502,7 @@ __device__ __forceinline__ bool finish_lane_residual(const Dev &P, const Ctl &c,
 template <typename T, int RB, int THREADS = UPD_THREADS>
 __device__ __forceinline__ void finish_rows(const Dev &P, const Ctl &c, const int leg, const int slot,
                                             const int form, const float *row_m, const double *row_s,
-                                            const float *row_h, double *red, int *is_last)
+                                            const float *row_h, double *red)
 {
     constexpr int NWARP = THREADS / 32;
     const int nrows = (leg == LEG_F) ? P.n : P.m;
@@ -548,9 +526,8 @@ __device__ __forceinline__ void finish_rows(const Dev &P, const Ctl &c, const in
         double s = 0.0;
 #pragma unroll
         for (int w = 0; w < NWARP; ++w) s += red[w];
-        finish_lane_residual(P, c, leg, slot, (nrows + RB - 1) / RB, blockIdx.x, s, frozen);
+        finish_lane_residual(P, leg, slot, s, frozen);
     }
-    (void)is_last;
 }
 
 template <typename T, int DP, int CS, int XF>
@@ -568,7 +545,6 @@ __global__ void __launch_bounds__(UPD_THREADS) update_kernel(const Dev P, const 
     __shared__ float row_m[RB];
     __shared__ float row_h[RB];
     __shared__ double red[NWARP];
-    __shared__ int is_last;
 
     pdl_enter();
     const Ctl c = *P.ctl;
@@ -577,7 +553,7 @@ __global__ void __launch_bounds__(UPD_THREADS) update_kernel(const Dev P, const 
     if (slot >= c.n_phys) return;
     if (P.early_exit && P.state[slot] != 0) return;     // early-exit mask arm: a frozen lane costs a launch slot only
     if (leg != LEG_V && c.static_final) return;
-    if (leg == LEG_V && !(c.static_final || P.flag[slot])) return;
+    if (leg == LEG_V && !(c.static_final || lane_flag(P, c, slot))) return;
 
     // roles: rows are x-points for the f-leg, y-points otherwise
     const bool rows_x = (leg == LEG_F);
@@ -622,16 +598,15 @@ __global__ void __launch_bounds__(UPD_THREADS) update_kernel(const Dev P, const 
     // a fraction of a unit of the truth, so the rescale branch of the streaming loop stays cold.
     // A reference far too HIGH would push every term towards the flush-to-zero range: such a CTA
     // repeats the pass from "minus infinity", as the other arithmetic modes always do.
-    float m0[R];
+    double m0[R];                                        // |m0| >= 1e7 stands for "no estimate"
 #pragma unroll
-    for (int r = 0; r < R; ++r) m0[r] = NEG_BIG;
+    for (int r = 0; r < R; ++r) m0[r] = (double)NEG_BIG;
     if constexpr (sizeof(T) == 8 && XF != 0) {
 #pragma unroll
         for (int r = 0; r < R; ++r) {
             if (row0 + r < nrows) {
                 const size_t o = (size_t)slot * rp + row0 + r;
-                const double est = (rows_x ? P.la2 : P.lb2)[o] + (rows_x ? P.sqx : P.sqy)[o] - prow[row0 + r];
-                if (fabs(est) < 1.0e7) m0[r] = ceilf((float)est);
+                m0[r] = (rows_x ? P.la2 : P.lb2)[o] + (rows_x ? P.sqx : P.sqy)[o] - prow[row0 + r];
             }
         }
     }
@@ -661,10 +636,10 @@ __global__ void __launch_bounds__(UPD_THREADS) update_kernel(const Dev P, const 
                 bool low = false;
 #pragma unroll
                 for (int r = 0; r < R; ++r)
-                    low = low || (row0 + r < nrows && m0[r] != NEG_BIG && !(sd[r] >= 0x1p-20));
+                    low = low || (row0 + r < nrows && fabs(m0[r]) < 1.0e7 && !(sd[r] >= 0x1p-20));
                 if (!__syncthreads_or(low ? 1 : 0)) break;
 #pragma unroll
-                for (int r = 0; r < R; ++r) m0[r] = NEG_BIG;
+                for (int r = 0; r < R; ++r) m0[r] = (double)NEG_BIG;
                 continue;
             }
         }
@@ -679,7 +654,7 @@ __global__ void __launch_bounds__(UPD_THREADS) update_kernel(const Dev P, const 
         }
     }
     __syncthreads();
-    finish_rows<T, RB>(P, c, leg, slot, form, row_m, row_s, row_h, red, &is_last);
+    finish_rows<T, RB>(P, c, leg, slot, form, row_m, row_s, row_h, red);
 }
 
 }  // namespace skb

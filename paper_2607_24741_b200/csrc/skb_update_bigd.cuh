@@ -39,7 +39,6 @@ __global__ void __launch_bounds__(UPD_THREADS) update_bigd_kernel(const Dev P, c
     __shared__ float row_m[RB];
     __shared__ float row_h[RB];
     __shared__ double red[UPD_THREADS / 32];
-    __shared__ int is_last;
 
     pdl_enter();
     const Ctl c = *P.ctl;
@@ -48,7 +47,7 @@ __global__ void __launch_bounds__(UPD_THREADS) update_bigd_kernel(const Dev P, c
     if (slot >= c.n_phys) return;
     if (P.early_exit && P.state[slot] != 0) return;     // early-exit mask arm: a frozen lane costs a launch slot only
     if (leg != LEG_V && c.static_final) return;
-    if (leg == LEG_V && !(c.static_final || P.flag[slot])) return;
+    if (leg == LEG_V && !(c.static_final || lane_flag(P, c, slot))) return;
     const bool rows_x = (leg == LEG_F);
     const int nrows = rows_x ? P.n : P.m, rp = rows_x ? P.np : P.mp;
     const int ncols = rows_x ? P.m : P.n, cp = rows_x ? P.mp : P.np;
@@ -178,7 +177,7 @@ __global__ void __launch_bounds__(UPD_THREADS) update_bigd_kernel(const Dev P, c
         for (int r = 0; r < R; ++r) { row_m[lrow0 + r] = mx[r]; row_s[lrow0 + r] = sd[r]; row_h[lrow0 + r] = 0.f; }
     }
     __syncthreads();
-    finish_rows<T, RB>(P, c, leg, slot, (int)FORM_DOT, row_m, row_s, row_h, red, &is_last);
+    finish_rows<T, RB>(P, c, leg, slot, (int)FORM_DOT, row_m, row_s, row_h, red);
 }
 
 }  // namespace skb

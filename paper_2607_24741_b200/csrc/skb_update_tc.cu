@@ -250,7 +250,6 @@ update_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant_
     float *row_h = reinterpret_cast<float *>(small_buf + 1536);
     constexpr uint32_t STAGE_BYTES = (TC_BN / 128) * TC_CHUNK;     // one or two 128-point chunks per stage
     __shared__ double red[TC_THREADS / 32];
-    __shared__ int is_last;
 
     pdl_enter();
     const Ctl c = *P.ctl;
@@ -259,7 +258,7 @@ update_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant_
     if (slot >= c.n_phys) return;
     if (P.early_exit && P.state[slot] != 0) return;     // early-exit mask arm: a frozen lane costs a launch slot only
     if (leg != LEG_V && c.static_final) return;
-    if (leg == LEG_V && !(c.static_final || P.flag[slot])) return;
+    if (leg == LEG_V && !(c.static_final || lane_flag(P, c, slot))) return;
     const bool rows_x = (leg == LEG_F);
     const int nrows = rows_x ? P.n : P.m;
     const int ncols = rows_x ? P.m : P.n, cp = rows_x ? P.mp : P.np;
@@ -406,7 +405,7 @@ update_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant_
     if (abort_flag) {
         if (tid == 0) atomicOr(&P.ctl->error, ERR_WAIT);
     }
-    finish_rows<float, TC_BM, TC_THREADS>(P, c, leg, slot, (int)FORM_DOT, row_m, row_s, row_h, red, &is_last);
+    finish_rows<float, TC_BM, TC_THREADS>(P, c, leg, slot, (int)FORM_DOT, row_m, row_s, row_h, red);
 }
 
 // ---------------------------------------------------------------- CTA-pair variant
@@ -596,15 +595,16 @@ update_tc_pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_cons
     tc_fence_after();
     const uint32_t tmem = tmem_holder;
     volatile int *ab = &abort_flag;
-    long long dbg_w0 = 0, dbg_w1 = 0;   // clocks spent in waits (debug builds)
+#ifdef SKB_TC_DEBUG
+    long long dbg_w0 = 0, dbg_w1 = 0;   // clocks spent in waits
     const long long dbg_t0 = clock64();
-    (void)dbg_w0; (void)dbg_w1; (void)dbg_t0;
+#endif
 
     // every role walks the same segments and skips the same ones (the column check only
     // visits lanes that the screen flagged)
     SegIter it = it0;
     Seg sg;
-#define TC2_SKIP(slot) ((leg == LEG_V && !(c.static_final || P.flag[slot])) || (P.early_exit && P.state[slot] != 0))
+#define TC2_SKIP(slot) ((leg == LEG_V && !(c.static_final || lane_flag(P, c, slot))) || (P.early_exit && P.state[slot] != 0))
 
     if (warp == TC_EPI_WARPS) {
         // ---------------- producer (one per CTA): own row block once per segment, own half of every column tile
@@ -716,7 +716,7 @@ update_tc_pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_cons
                 for (int off = 16; off > 0; off >>= 1) term += __shfl_down_sync(0xffffffffu, term, off);
                 if (lane == 0) red[fw] = term;
                 asm volatile("bar.sync 4, 128;" ::: "memory");
-                if (row == 0) finish_lane_residual(P, c, leg, slot, nrt, rb, ((red[0] + red[1]) + red[2]) + red[3], frozen);
+                if (row == 0) finish_lane_residual(P, leg, slot, ((red[0] + red[1]) + red[2]) + red[3], frozen);
                 asm volatile("bar.sync 4, 128;" ::: "memory");          // red[] is free again
             }
         }
