@@ -160,25 +160,12 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_kernel(const Dev P)
     const int A = c.n_phys;
     const bool limit = k >= P.max_iter;
 
-    // the legs left each lane's residuals as exact fixed-point sums: turn them into the values,
-    // the screen flag and the two-sided verdict (Eq. 5) everything below works with, and clear
-    // the sums for the next cycle
-    for (int s = tid; s < A; s += NT) {
-        const int fl = lane_flag(P, c, s) ? 1 : 0;
-        const double rr = (double)P.rsum_row[s] * (1.0 / RSUM_SCALE);
-        const double rc = (double)P.rsum_col[s] * (1.0 / RSUM_SCALE);
-        P.rsum_row[s] = 0ull; P.rsum_col[s] = 0ull;
-        if (!c.static_final) P.rrow[s] = rr;         // STATIC's closing column check runs no f-leg: keep the last screen's value
-        P.rcol[s] = rc;
-        P.flag[s] = fl;
-        P.verdict[s] = (!P.nonfinite[s] && fmax(rr, rc) <= P.tol_stop) ? 1 : 0;
-    }
-    __syncthreads();
-
     if (P.mode == MODE_STATIC && c.static_final) {   // emit every lane at the common boundary
         for (int s = tid; s < P.W; s += NT) {
             P.ret_slot[s] = s; P.ret_lane[s] = s; P.ret_src[s] = -1; P.ret_scale[s] = P.scale[s];
-            P.res_row[s] = P.rrow[s]; P.res_col[s] = P.rcol[s];
+            // the closing column check ran no f-leg: r_row is the last screen's value
+            P.res_row[s] = P.rrow[s]; P.res_col[s] = (double)P.rsum_col[s] * (1.0 / RSUM_SCALE);
+            P.rsum_col[s] = 0ull;
             if (P.nonfinite[s]) P.status[s] = LANE_NONFINITE;
         }
         if (tid == 0) {
@@ -190,21 +177,37 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_kernel(const Dev P)
     }
 
     // which running lanes leave at this audit
+    auto decide_vals = [&](bool held, int nf, int fl, int vd, int &ret, int &st) {
+        ret = 0; st = LANE_RUNNING;
+        if (held) return;
+        if (nf) { ret = 1; st = LANE_NONFINITE; }
+        else if (fl && vd) { ret = 1; st = LANE_DONE; }
+        else if (limit) { ret = 1; st = LANE_ITER_LIMIT; }
+    };
     auto decide = [&](int s, int &ret, int &st) {
         ret = 0; st = LANE_RUNNING;
         if (s >= A) return;
         const bool held = (P.mode != MODE_ACTIVE) && P.state[s] != 0;   // frozen / already passed
-        if (held) return;
-        if (P.nonfinite[s]) { ret = 1; st = LANE_NONFINITE; }
-        else if (P.flag[s] && P.verdict[s]) { ret = 1; st = LANE_DONE; }
-        else if (limit) { ret = 1; st = LANE_ITER_LIMIT; }
+        decide_vals(held, P.nonfinite[s], P.flag[s], P.verdict[s], ret, st);
     };
 
-    // pass 1: count retirees and screen-positive lanes
+    // pass 1.  The legs left each lane's residuals as exact fixed-point sums: turn them into the
+    // values, the screen flag and the two-sided verdict (Eq. 5), clear the sums for the next
+    // cycle, and count retirees and screen-positive lanes on the way.
     int cnt = 0, nflag = 0;
     for (int s = tid; s < A; s += NT) {
-        int r, st; decide(s, r, st); cnt += r;
-        nflag += (P.flag[s] != 0);
+        const int fl = lane_flag(P, c, s) ? 1 : 0;
+        const int nf = P.nonfinite[s];
+        const bool held = (P.mode != MODE_ACTIVE) && P.state[s] != 0;
+        const double rr = (double)P.rsum_row[s] * (1.0 / RSUM_SCALE);
+        const double rc = (double)P.rsum_col[s] * (1.0 / RSUM_SCALE);
+        const int vd = (!nf && fmax(rr, rc) <= P.tol_stop) ? 1 : 0;
+        P.rsum_row[s] = 0ull; P.rsum_col[s] = 0ull;
+        P.rrow[s] = rr; P.rcol[s] = rc;
+        P.flag[s] = fl; P.verdict[s] = vd;
+        int r, st; decide_vals(held, nf, fl, vd, r, st);
+        cnt += r;
+        nflag += fl;
     }
     for (int off = 16; off > 0; off >>= 1) {
         cnt += __shfl_down_sync(0xffffffffu, cnt, off);
