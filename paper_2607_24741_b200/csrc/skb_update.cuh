@@ -65,8 +65,15 @@ template <int DP> struct Tune<double, DP> {
     static constexpr int CW = DP <= 8 ? SKB_F64_CW : 4;
 };
 
+// Columns per shared-memory tile: at least two steps, and enough of them between the two barriers
+// of a tile that the warps of a CTA drift apart (the special-function unit idles when they all do
+// FMAs at once); bounded by the shared memory the double-buffered tile may take.
+#ifndef SKB_TJ_SMALL
+#define SKB_TJ_SMALL 512
+#endif
 template <typename T, int DP, int CS> struct TileCols {
-    static constexpr int value = (Tune<T, DP>::CW * CS * 2 > 128) ? Tune<T, DP>::CW * CS * 2 : 128;   // >= 2 steps per tile
+    static constexpr int wish = sizeof(T) == 8 ? 128 : (DP <= 4 ? SKB_TJ_SMALL : (DP <= 16 ? 256 : 128));
+    static constexpr int value = (Tune<T, DP>::CW * CS * 2 > wish) ? Tune<T, DP>::CW * CS * 2 : wish;
 };
 
 __device__ __forceinline__ u64 pack2(float lo, float hi)
