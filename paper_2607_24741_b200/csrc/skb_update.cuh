@@ -584,6 +584,20 @@ __global__ void __launch_bounds__(UPD_THREADS) update_kernel(const Dev P, const 
     const int lrow0 = warp * RW + rg * R;                // this thread's R consecutive CTA-local rows
     const int row0 = blockIdx.x * RB + lrow0;
 
+    // the float64 epilogue's operands (one thread per row, much later): start them on their way to
+    // L1 now, so that the epilogue does not begin with a round trip to L2 (the column tiles
+    // stream through cp.async and leave L1 alone)
+    for (int lr = tid; lr < RB; lr += UPD_THREADS) {
+        const int i = blockIdx.x * RB + lr;
+        if (i < nrows) {
+            const size_t o = (size_t)slot * rp + i;
+            asm volatile("prefetch.global.L1 [%0];" ::"l"((rows_x ? P.la2 : P.lb2) + o));
+            asm volatile("prefetch.global.L1 [%0];" ::"l"((rows_x ? P.sqx : P.sqy) + o));
+            asm volatile("prefetch.global.L1 [%0];" ::"l"(prow + i));
+            if (leg != LEG_G) asm volatile("prefetch.global.L1 [%0];" ::"l"((rows_x ? P.wa : P.wb) + o));
+        }
+    }
+
     // R consecutive rows of one dimension are one aligned vector load (padding rows hold zeros)
     T xr[R][DP];
     T ph[R];
