@@ -382,17 +382,18 @@ __device__ __forceinline__ void stream_f64(double *sm, const double *colc, const
                 }
             }
             if (XF) {
-                // shifted arguments in fp32 (needed for ex2 anyway); their maximum steers the rescale
-                float v[R][CW];
+                // shifted arguments in fp32, their exponentials against the reference as it stands;
+                // only a step whose sum exceeds 2^10 (or is not finite) moves the reference
+                float v[R][CW], e2[R];
                 bool grow = false;
 #pragma unroll
                 for (int r = 0; r < R; ++r) {
 #pragma unroll
                     for (int e = 0; e < CW; ++e) v[r][e] = (float)(acc[r][e] - md[r]);
-                    float vm = v[r][0];
+                    e2[r] = 0.f;
 #pragma unroll
-                    for (int e = 1; e < CW; ++e) vm = fmaxf(vm, v[r][e]);
-                    grow = grow || (vm > 8.0f);
+                    for (int e = 0; e < CW; ++e) e2[r] += ex2_fast(v[r][e]);
+                    grow = grow || !(e2[r] <= 1024.f);
                 }
                 if (grow) {                                   // rare: move the reference point up
 #pragma unroll
@@ -407,18 +408,14 @@ __device__ __forceinline__ void stream_f64(double *sm, const double *colc, const
                             sd[r] *= (double)fac;
                             mx[r] = mn;
                             md[r] = (double)mn;
+                            e2[r] = 0.f;
 #pragma unroll
-                            for (int e = 0; e < CW; ++e) v[r][e] = (float)(acc[r][e] - md[r]);
+                            for (int e = 0; e < CW; ++e) e2[r] += ex2_fast((float)(acc[r][e] - md[r]));
                         }
                     }
                 }
 #pragma unroll
-                for (int r = 0; r < R; ++r) {
-                    float e2 = 0.f;
-#pragma unroll
-                    for (int e = 0; e < CW; ++e) e2 += ex2_fast(v[r][e]);
-                    ts[r] += e2;
-                }
+                for (int r = 0; r < R; ++r) ts[r] += e2[r];
             } else {
 #pragma unroll
                 for (int r = 0; r < R; ++r) {
