@@ -365,11 +365,14 @@ update_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant_
         const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
         bool ok = true;
         float ts = 0.f;
+        static_assert(TC_BN <= TC_EPI_THREADS, "one column term per epilogue thread and tile");
+        float g_next = (e < TC_BN && e < cp) ? colt[e] : NEG_BIG;       // column term, one tile ahead
         for (int t = 0; t < ntiles && ok; ++t) {
             const int buf = t & 1;
-            for (int q = e; q < TC_BN; q += TC_EPI_THREADS) {
-                const int j = t * TC_BN + q;
-                gts[buf][q] = (j < cp) ? colt[j] : NEG_BIG;
+            if (e < TC_BN) {
+                gts[buf][e] = g_next;
+                const int j = (t + 1) * TC_BN + e;
+                g_next = (t + 1 < ntiles && j < cp) ? colt[j] : NEG_BIG;
             }
             asm volatile("bar.sync 1, 256;" ::: "memory");
             ok = TC_TIMED_WAIT(dbg_w0, mbar_wait(b_tfull + 8 * buf, (t >> 1) & 1, ab));
