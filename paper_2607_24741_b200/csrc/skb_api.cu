@@ -306,11 +306,12 @@ static void enqueue_cycle(skb_batch *h)
     const int w = h->known_width;
     launch_leg(h, LEG_F, w);
     launch_leg(h, LEG_V, w);
-    launch_plan(h->dev, w, h->stream);
-    launch_emit_move(h->dev, w, h->stream);
+    int nk = 3;
+    nk += launch_plan(h->dev, w, h->stream);
+    nk += launch_emit_move(h->dev, w, h->stream);
     launch_leg(h, LEG_G, w);
     h->enqueued++;
-    h->launches += 5;
+    h->launches += nk;
 }
 
 static skb_status absorb(skb_batch *h, const Ctl &c)

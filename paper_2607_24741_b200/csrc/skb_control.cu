@@ -149,6 +149,11 @@ __device__ __forceinline__ void block_scan3(int f0, int f1, int f2, int (&ex)[3]
     tot[0] = run[0]; tot[1] = run[1]; tot[2] = run[2];
 }
 
+template <typename T>
+__device__ __forceinline__ void emit_move_one(const Dev &P, const Ctl &c, const int r);
+
+// FUSE: the same block also emits and moves the lanes it retires (see launch_plan).
+template <typename T, bool FUSE>
 __global__ void __launch_bounds__(PLAN_THREADS) plan_kernel(const Dev P)
 {
     __shared__ int wsum[PLAN_THREADS / 32][3];
@@ -170,8 +175,14 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_kernel(const Dev P)
         }
         if (tid == 0) {
             Ctl *g = P.ctl;
-            g->n_retire = P.W; g->emit_parity = c.parity; g->n_running = 0; g->done = 1;
+            g->n_retire = FUSE ? 0 : P.W; g->emit_parity = c.parity; g->n_running = 0; g->done = 1;
             g->pair_terms += (long long)P.W * P.n * P.m;      // the final column check
+        }
+        if (FUSE) {
+            __syncthreads();
+            Ctl cc = c;
+            cc.emit_parity = c.parity;
+            for (int r = 0; r < P.W; ++r) emit_move_one<T>(P, cc, r);
         }
         return;
     }
@@ -266,7 +277,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_kernel(const Dev P)
     }
     if (tid == 0) {
         Ctl *g = P.ctl;
-        g->n_retire = (P.mode == MODE_STATIC) ? 0 : nret;
+        g->n_retire = (P.mode == MODE_STATIC || FUSE) ? 0 : nret;      // what is left for the emit/move kernel
         g->emit_parity = c.parity;
         // lanes whose pair terms were really evaluated (the early-exit arm skips frozen lanes)
         const int worked = P.early_exit ? c.n_running : A;
@@ -293,12 +304,15 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_kernel(const Dev P)
             g->done = 1;
         }
     }
+    if (FUSE && P.mode != MODE_STATIC && nret > 0) {
+        __syncthreads();                                  // the lists and per-slot scalars above are this block's own writes
+        Ctl cc = c;
+        cc.emit_parity = c.parity;
+        for (int r = 0; r < nret; ++r) emit_move_one<T>(P, cc, r);
+    }
 }
 
 // ---------------------------------------------------------------- emit + move
-template <typename T>
-__device__ __forceinline__ void emit_move_one(const Dev &P, const Ctl &c, const int r);
-
 template <typename T>
 __global__ void __launch_bounds__(256) emit_move_kernel(const Dev P)
 {
@@ -397,15 +411,40 @@ void launch_prep(const Dev &P, const void *x, const void *y, const float *a, con
     if (P.compute_f64) prep_kernel<double><<<grid, 128, 0, st>>>(P, x, y, a, b);
     else prep_kernel<float><<<grid, 128, 0, st>>>(P, x, y, a, b);
 }
-void launch_plan(const Dev &P, int width, cudaStream_t st)
+// Bytes one retirement can move (a survivor's whole state into the hole) plus what it emits.
+static size_t lane_state_bytes(const Dev &P)
+{
+    const size_t ts = P.compute_f64 ? 8 : 4;
+    size_t coords = (size_t)P.DP * (P.np + P.mp) * ts;
+    if (P.tensor) coords = ((size_t)((P.n + 127) / 128) + (size_t)((P.m + 127) / 128)) * P.d * 256;
+    return coords + (size_t)(P.np + P.mp) * (4 * 8 + 2 * ts + 8);
+}
+// When even the retirement of every lane at once would move little (narrow batches of small
+// lanes), the planner's own block emits and moves, and the emit/move kernel is not launched:
+// one kernel less in the chain of dependent launches that bounds a narrow cycle.  Same device
+// functions either way, so the results do not depend on the choice.
+static bool plan_fuses_move(const Dev &P, int width)
+{
+    const int lanes = (P.mode == MODE_STATIC) ? P.W : (width < 1 ? 1 : width);
+    return (size_t)lanes * lane_state_bytes(P) <= ((size_t)512 << 10);
+}
+int launch_plan(const Dev &P, int width, cudaStream_t st)
 {
     int nt = (width + 31) / 32 * 32;
     if (P.mode == MODE_STATIC) nt = (P.W + 31) / 32 * 32;
-    nt = nt < 128 ? 128 : (nt > PLAN_THREADS ? PLAN_THREADS : nt);
-    launch_pdl(plan_kernel, dim3(1), dim3(nt), 0, st, P);
+    const bool fuse = plan_fuses_move(P, width);
+    nt = nt < (fuse ? 256 : 128) ? (fuse ? 256 : 128) : (nt > PLAN_THREADS ? PLAN_THREADS : nt);
+    if (fuse) {
+        if (P.compute_f64) launch_pdl(plan_kernel<double, true>, dim3(1), dim3(nt), 0, st, P);
+        else launch_pdl(plan_kernel<float, true>, dim3(1), dim3(nt), 0, st, P);
+    } else {
+        launch_pdl(plan_kernel<float, false>, dim3(1), dim3(nt), 0, st, P);
+    }
+    return 1;
 }
-void launch_emit_move(const Dev &P, int width, cudaStream_t st)
+int launch_emit_move(const Dev &P, int width, cudaStream_t st)
 {
+    if (plan_fuses_move(P, width)) return 0;
     if (width < 1) width = 1;
     const size_t bytes = (size_t)P.DP * (P.np + P.mp) * (P.compute_f64 ? 8 : 4);
     int gx = (int)(bytes / (256 * 16 * 4)) + 1;
@@ -413,6 +452,7 @@ void launch_emit_move(const Dev &P, int width, cudaStream_t st)
     dim3 grid(gx, width > 128 ? 128 : width);
     if (P.compute_f64) launch_pdl(emit_move_kernel<double>, grid, dim3(256), 0, st, P);
     else launch_pdl(emit_move_kernel<float>, grid, dim3(256), 0, st, P);
+    return 1;
 }
 void launch_gather(const Dev &P, void *f, void *g, bool f64, cudaStream_t st)
 {

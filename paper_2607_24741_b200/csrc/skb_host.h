@@ -32,7 +32,7 @@ int padded_dim(int d);
 
 void launch_lane_stats(const Dev &P, const void *x, const void *y, const float *eps, double *max_radius, cudaStream_t st);
 void launch_prep(const Dev &P, const void *x, const void *y, const float *a, const float *b, cudaStream_t st);
-void launch_plan(const Dev &P, int width, cudaStream_t st);
+int launch_plan(const Dev &P, int width, cudaStream_t st);        // both return the number of kernels launched
 // tensor-core update kernel (bf16 inputs, d a multiple of 64 up to 512)
 bool tc_eligible(int d, bool bf16);
 const char *tc_make_map(void *out_map, void *base, int W, int npts, int d);
@@ -40,7 +40,7 @@ size_t tc_tiled_bytes(int W, int npts, int d);
 void launch_retile(const void *src, void *dst, int W, int npts, int d, cudaStream_t st);
 void launch_wait_probe(int *out, long long budget_clocks, cudaStream_t st);
 void launch_update_tc(const Dev &P, const void *maps, int leg, int width, cudaStream_t st);
-void launch_emit_move(const Dev &P, int width, cudaStream_t st);
+int launch_emit_move(const Dev &P, int width, cudaStream_t st);
 void launch_gather(const Dev &P, void *f, void *g, bool f64, cudaStream_t st);
 void launch_gather_small(const Dev &P, int *depth, int *status, float *rrow, float *rcol, cudaStream_t st);
 
