@@ -15,10 +15,28 @@ static void launch_update(const Dev &P, int leg, int width, cudaStream_t st)
         cudaFuncSetAttribute(update_kernel<T, DP, CS, XF>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         attr_set = true;
     }
-    const int rb = (UPD_THREADS / 32) * Tune<T, DP>::R * (32 / CS);
     const int nrows = (leg == LEG_F) ? P.n : P.m;
-    dim3 grid((nrows + rb - 1) / rb, width < 1 ? 1 : width);
-    launch_pdl(update_kernel<T, DP, CS, XF>, grid, dim3(UPD_THREADS), smem, st, P, leg);
+    const int lanes = width < 1 ? 1 : width;
+    if constexpr (sizeof(T) == 8 && XF == 1 && DP <= 8) {
+        // Float64 arguments with few dimensions: four rows per thread halve the shared-memory
+        // loads per multiply-add (faster when the grid fills the GPU), two rows give twice the
+        // blocks (lower latency when it does not).  Same bits either way, so the choice may follow
+        // the width from launch to launch.
+        constexpr int RW = 4;
+        static bool attr_wide = false;
+        if (!attr_wide) {
+            cudaFuncSetAttribute(update_kernel<T, DP, CS, XF, RW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            attr_wide = true;
+        }
+        const int rbw = (UPD_THREADS / 32) * RW * (32 / CS);
+        const long long ctas = (long long)((nrows + rbw - 1) / rbw) * lanes;
+        if (ctas >= 2 * 148 * 4) {
+            launch_pdl(update_kernel<T, DP, CS, XF, RW>, dim3((nrows + rbw - 1) / rbw, lanes), dim3(UPD_THREADS), smem, st, P, leg);
+            return;
+        }
+    }
+    const int rb = (UPD_THREADS / 32) * Tune<T, DP>::R * (32 / CS);
+    launch_pdl(update_kernel<T, DP, CS, XF>, dim3((nrows + rb - 1) / rb, lanes), dim3(UPD_THREADS), smem, st, P, leg);
 }
 
 #define SKB_V(T, F64, XF, DP, CS) \

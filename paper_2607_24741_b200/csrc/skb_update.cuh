@@ -324,15 +324,15 @@ __device__ __forceinline__ void stream_f32(float *sm, const float *colc, const f
 
 // ------------------------------------------------------------------ float64 arguments
 // XF = 1: exponentials on the fp32 special-function unit; XF = 0: software exp2 in float64.
-template <int DP, int CS, int XF>
+template <int DP, int CS, int XF, int R>
 __device__ __forceinline__ void stream_f64(double *sm, const double *colc, const double *colt,
                                            const int cp, const int ncols,
-                                           const double (&xr)[Tune<double, DP>::R][DP],
+                                           const double (&xr)[R][DP],
                                            const int tid, const int cs,
-                                           const double (&est)[Tune<double, DP>::R],
-                                           float (&mx)[Tune<double, DP>::R], double (&sd)[Tune<double, DP>::R])
+                                           const double (&est)[R],
+                                           float (&mx)[R], double (&sd)[R])
 {
-    constexpr int R = Tune<double, DP>::R, CW = Tune<double, DP>::CW;
+    constexpr int CW = Tune<double, DP>::CW;
     constexpr int TJ = TileCols<double, DP, CS>::value;
     constexpr int STEPS = TJ / (CW * CS);
     constexpr int NR = DP + 1;
@@ -486,18 +486,22 @@ __device__ __forceinline__ double finish_one_row(const Dev &P, const Ctl &c, con
     return term;
 }
 
-// One thread per row block hands in its block's residual sum: one integer atomic on the lane's
-// fixed-point total (exact, so the total does not depend on the order of arrival; nobody has to
-// arrive last).  A part that is not finite marks the lane instead.
-__device__ __forceinline__ void finish_lane_residual(const Dev &P, const int leg, const int slot,
-                                                     const double block_sum, const bool frozen)
+// A row's term of the marginal residual in fixed point.  Terms are summed as integers from here
+// on (registers, shuffles, shared memory, one atomic per row block on the lane's total), so the
+// total is exact and does not depend on how rows are grouped into threads and blocks nor on
+// the order in which blocks arrive.  A term that is not finite marks the lane instead.
+__device__ __forceinline__ unsigned long long residual_fixed(const Dev &P, const int leg, const int slot,
+                                                             const double term, const bool frozen)
 {
-    if (!isfinite(block_sum)) {
+    if (!isfinite(term)) {
         if (leg != LEG_F || !frozen) P.nonfinite[slot] = 1;
-        return;
+        return 0ull;
     }
-    const unsigned long long part = __double2ull_rn(fmin(block_sum, RSUM_PART_MAX) * RSUM_SCALE);
-    atomicAdd((leg == LEG_F ? P.rsum_row : P.rsum_col) + slot, part);
+    return __double2ull_rn(fmin(term, RSUM_ROW_MAX) * RSUM_SCALE);
+}
+__device__ __forceinline__ void finish_lane_residual(const Dev &P, const int leg, const int slot, const unsigned long long block_sum)
+{
+    atomicAdd((leg == LEG_F ? P.rsum_row : P.rsum_col) + slot, block_sum);
 }
 
 // Float64 epilogue of a CTA's RB rows (one thread per row) and the fused residual reduction.
@@ -513,31 +517,35 @@ __device__ __forceinline__ void finish_rows(const Dev &P, const Ctl &c, const in
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const bool frozen = (P.mode == MODE_MASKED) && P.state[slot] != 0;
     const bool writes = !frozen && leg != LEG_V;
-    double term_sum = 0.0;
+    unsigned long long term_sum = 0ull;
     for (int lr = tid; lr < RB; lr += THREADS) {
         const int i = blockIdx.x * RB + lr;
         if (i >= nrows) continue;
-        term_sum += finish_one_row<T>(P, c, leg, slot, form, i, row_m[lr], row_s[lr], row_h[lr], writes);
+        const double term = finish_one_row<T>(P, c, leg, slot, form, i, row_m[lr], row_s[lr], row_h[lr], writes);
+        if (leg != LEG_G) term_sum += residual_fixed(P, leg, slot, term, frozen);
     }
     if (leg == LEG_G) return;
 
-    // fused marginal-residual reduction -> one flag per lane
+    // fused marginal-residual reduction -> one exact total per lane
+    unsigned long long *redu = reinterpret_cast<unsigned long long *>(red);
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) term_sum += __shfl_down_sync(0xffffffffu, term_sum, off);
-    if (lane == 0) red[warp] = term_sum;
+    if (lane == 0) redu[warp] = term_sum;
     __syncthreads();
     if (tid == 0) {
-        double s = 0.0;
+        unsigned long long s = 0ull;
 #pragma unroll
-        for (int w = 0; w < NWARP; ++w) s += red[w];
-        finish_lane_residual(P, leg, slot, s, frozen);
+        for (int w = 0; w < NWARP; ++w) s += redu[w];
+        finish_lane_residual(P, leg, slot, s);
     }
 }
 
-template <typename T, int DP, int CS, int XF>
+// RR: rows per thread, 0 = the type's default.  Rows are independent and a row's arithmetic does
+// not depend on which thread holds it, so launches with different RR give the same bits.
+template <typename T, int DP, int CS, int XF, int RR = 0>
 __global__ void __launch_bounds__(UPD_THREADS) update_kernel(const Dev P, const int leg)
 {
-    constexpr int R = Tune<T, DP>::R;
+    constexpr int R = RR ? RR : Tune<T, DP>::R;
     constexpr int RG = 32 / CS;                  // row groups per warp
     constexpr int RW = R * RG;                   // rows per warp
     constexpr int NWARP = UPD_THREADS / 32;
@@ -634,7 +642,7 @@ __global__ void __launch_bounds__(UPD_THREADS) update_kernel(const Dev P, const 
             if (form == FORM_DOT) stream_f32<DP, CS, FORM_DOT>(sm, colc, colt, coll, cp, ncols, xr, ph, tid, cs, mx, sd);
             else stream_f32<DP, CS, FORM_DIFF>(sm, colc, colt, coll, cp, ncols, xr, ph, tid, cs, mx, sd);
         } else {
-            stream_f64<DP, CS, XF>(sm, colc, colt, cp, ncols, xr, tid, cs, m0, mx, sd);
+            stream_f64<DP, CS, XF, R>(sm, colc, colt, cp, ncols, xr, tid, cs, m0, mx, sd);
         }
 
         // merge the CS column splits of each row: maxima are integers, so the scalings are exact

@@ -541,7 +541,7 @@ update_tc_pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_cons
     __shared__ int abort_flag;
     __shared__ unsigned arrival;                           // filing warps: the arrival word before this part's add
     __shared__ __align__(16) float gts[TC2_BN];            // column terms of the tile being reduced
-    __shared__ double red[TC2_FILE_WARPS];
+    __shared__ unsigned long long red[TC2_FILE_WARPS];
 
     pdl_enter();
     const Ctl c = *P.ctl;
@@ -712,14 +712,17 @@ update_tc_pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_cons
             }
             const bool frozen = (P.mode == MODE_MASKED) && P.state[slot] != 0;
             const int i = rb * TC_BM + row;
-            double term = 0.0;
-            if (i < nrows) term = finish_one_row<float>(P, c, leg, slot, (int)FORM_DOT, i, m, sm, 0.f, !frozen && leg != LEG_V);
+            unsigned long long term = 0ull;
+            if (i < nrows) {
+                const double tr = finish_one_row<float>(P, c, leg, slot, (int)FORM_DOT, i, m, sm, 0.f, !frozen && leg != LEG_V);
+                if (leg != LEG_G) term = residual_fixed(P, leg, slot, tr, frozen);
+            }
             if (leg != LEG_G) {
 #pragma unroll
                 for (int off = 16; off > 0; off >>= 1) term += __shfl_down_sync(0xffffffffu, term, off);
                 if (lane == 0) red[fw] = term;
                 asm volatile("bar.sync 4, 128;" ::: "memory");
-                if (row == 0) finish_lane_residual(P, leg, slot, ((red[0] + red[1]) + red[2]) + red[3], frozen);
+                if (row == 0) finish_lane_residual(P, leg, slot, ((red[0] + red[1]) + red[2]) + red[3]);
                 asm volatile("bar.sync 4, 128;" ::: "memory");          // red[] is free again
             }
         }

@@ -131,6 +131,19 @@ def test_early_exit_mask_arm_equals_the_mask_control_bitwise(oracle, case, compu
     np.testing.assert_array_equal(np.array(re["stats"]["widths"]), oracle.slot_counts(re["depth"].astype(np.int64))["widths"])
 
 
+def test_rows_per_thread_follow_the_width_without_changing_bits():
+    # Mixed arithmetic launches four rows per thread while the grid fills the GPU and two rows once the
+    # batch has shrunk; MASKED never shrinks, so it stays on four.  A row's arithmetic does not depend on
+    # the thread that holds it and residual terms are summed as integers, so the two modes must agree
+    # bit for bit at the bench size (1024 lanes, where ACTIVE crosses the switch).
+    w = wl.make("sweep")
+    ra = run_gpu(w, mode="active", compute="mixed", widths_cap=10)
+    rm = run_gpu(w, mode="masked", compute="mixed", widths_cap=10)
+    np.testing.assert_array_equal(ra["depth"], rm["depth"])
+    np.testing.assert_array_equal(ra["f"], rm["f"]); np.testing.assert_array_equal(ra["g"], rm["g"])
+    np.testing.assert_array_equal(ra["r_row"], rm["r_row"]); np.testing.assert_array_equal(ra["r_col"], rm["r_col"])
+
+
 def test_packing_commutes_with_the_per_lane_map(oracle):
     # Eq. 2: a W-lane batch gives each lane what a one-lane batch gives it, bit for bit
     # (the arithmetic is fixed here: the automatic choice looks at the whole batch)
