@@ -10,7 +10,8 @@
 // layout; a thread keeps R rows in registers and walks a group of adjacent columns per
 // step; with CS > 1 the column groups of a tile are dealt round-robin to CS neighbouring
 // lanes of the warp and the (max, sum) pairs are merged by xor-shuffles at the end.
-// The running maximum is kept integer-valued, so every rescale is an exact power of two.
+// The reference point (running maximum) is kept integer-valued, so every rescale is an exact
+// power of two; it only moves when a step's sum of exponentials says it must.
 //
 // Arithmetic of arg_ij:
 //   fp32, dot form   arg = ct_j + r_i . c_j, packed two columns at a time (fma.rn.f32x2);
@@ -29,8 +30,9 @@
 //   LEG_G  gam_new from L  (after it the column marginal equals b, Eq. 4).
 //   LEG_V  column marginal of the audited state for screen-positive lanes only,
 //          the second half of the two-sided check (Eq. 5).
-// The per-CTA L1 partial sums go to scratch; the last CTA of a lane adds them in a fixed
-// order and writes the lane's residual and its one flag (screen-positive / verdict).
+// The rows' L1 terms are summed in fixed point (exactly, whatever the grouping and order) into one
+// total per lane; the plan kernel turns the totals into the lane's residual, its one flag
+// (screen-positive) and the verdict, and the column-check leg reads the same flag predicate.
 #pragma once
 #include "skb_device.cuh"
 

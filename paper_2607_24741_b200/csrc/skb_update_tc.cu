@@ -672,9 +672,8 @@ update_tc_pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_cons
     } else if (warp >= TC_EPI_WARPS + 2) {
         // ---------------- filing warps (one thread per row): take each segment's merged row results
         // (maximum, sum) from the epilogue warps and do everything that is slow and serial off
-        // their critical path: the hand-over between the parts of a shared row block, the float64
-        // epilogue of the rows, the residual sum in a fixed order, and the lane's store / fence /
-        // ticket (its last block adds the parts up and sets the flags)
+        // their critical path: the hand-over between the parts of a shared row block, the merge of
+        // all units in unit order, the float64 epilogue of the rows and their residual terms
         const int fw = warp - (TC_EPI_WARPS + 2), row = fw * 32 + lane;
         int k = 0;
         while (it.next(sg)) {
