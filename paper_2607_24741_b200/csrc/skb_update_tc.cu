@@ -543,34 +543,12 @@ update_tc_pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_cons
     __shared__ __align__(16) float gts[TC2_BN];            // column terms of the tile being reduced
     __shared__ unsigned long long red[TC2_FILE_WARPS];
 
-    pdl_enter();
-    const Ctl c = *P.ctl;
-    if (c.done) return;
-    if (leg != LEG_V && c.static_final) return;
-    const bool rows_x = (leg == LEG_F);
-    const int nrows = rows_x ? P.n : P.m;
-    const int ncols = rows_x ? P.m : P.n, cp = rows_x ? P.mp : P.np;
-    const int nrt = (nrows + TC_BM - 1) / TC_BM;
-    const int npair = (nrt + 1) / 2;                       // row-block pairs per lane (the last may be half empty)
+    // Set-up that touches nothing an earlier kernel writes comes BEFORE the wait for that kernel:
+    // with programmatic dependent launch it overlaps the predecessor's tail (on SMs that are free).
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t rank = cluster_rank();
     const bool leader = (rank == 0);
-    const CUtensorMap *tm_row = rows_x ? &tmx : &tmy, *tm_col = rows_x ? &tmy : &tmx;
-    const int nkc = P.d / TC_BK;
-    const int ntiles = (ncols + TC2_BN - 1) / TC2_BN;
-    const int nct128 = (ncols + 127) / 128;
-    // units: groups of g column tiles, at most TC_MAX_SPLIT per row-block pair
-    const int g = tc_unit_tiles(ntiles);
-    const int upi = (ntiles + g - 1) / g;
-    const int U = c.n_phys * npair * upi;
-    const int ncl_grid = (int)gridDim.x >> 1, ncl = ncl_grid < U ? ncl_grid : U, cl = (int)blockIdx.x >> 1;
-    SegIter it0;
-    it0.upi = upi; it0.g = g; it0.npair = npair; it0.ntiles = ntiles;
-    it0.u = cl < ncl ? (int)((long long)cl * U / ncl) : 0;
-    it0.u_end = cl < ncl ? (int)((long long)(cl + 1) * U / ncl) : 0;
-
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const uint32_t sbase = (smem_u32(smem_tc) + 1023u) & ~1023u;
-    const uint32_t sA = sbase, sB = sbase + (uint32_t)nkc * TC_CHUNK;
     const uint32_t b_full = smem_u32(&bars[0]), b_empty = smem_u32(&bars[TC2_MAX_STAGES]);
     const uint32_t b_tfull = smem_u32(&bars[2 * TC2_MAX_STAGES]), b_tempty = b_tfull + 16;
     const uint32_t b_box_full = b_tfull + 32, b_box_empty = b_tfull + 40;
@@ -579,7 +557,6 @@ update_tc_pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_cons
     const uint32_t b_tempty_leader = map_to_cta(b_tempty, 0);
     const uint32_t b_empty_peer = map_to_cta(b_empty, 1);
     const uint32_t b_tfull_peer = map_to_cta(b_tfull, 1);
-
     if (tid == 0) {
         for (int s = 0; s < nstages; ++s) mbar_init(b_full + 8 * s, 1);
         for (int q = 0; q < nstages; ++q) mbar_init(b_empty + 8 * q, 1);
@@ -596,6 +573,33 @@ update_tc_pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_cons
     __syncthreads();
     cluster_barrier();                                  // both CTAs' barriers exist before anything remote touches them
     tc_fence_after();
+    asm volatile("griddepcontrol.wait;" ::: "memory");  // from here on: data of the kernels before this one
+
+    const Ctl c = *P.ctl;
+    // nothing to do (batch finished, or STATIC's closing pass, which runs the column check only):
+    // an empty unit range, and the common exit below
+    const bool idle = c.done || (leg != LEG_V && c.static_final);
+    const bool rows_x = (leg == LEG_F);
+    const int nrows = rows_x ? P.n : P.m;
+    const int ncols = rows_x ? P.m : P.n, cp = rows_x ? P.mp : P.np;
+    const int nrt = (nrows + TC_BM - 1) / TC_BM;
+    const int npair = (nrt + 1) / 2;                       // row-block pairs per lane (the last may be half empty)
+    const CUtensorMap *tm_row = rows_x ? &tmx : &tmy, *tm_col = rows_x ? &tmy : &tmx;
+    const int nkc = P.d / TC_BK;
+    const int ntiles = (ncols + TC2_BN - 1) / TC2_BN;
+    const int nct128 = (ncols + 127) / 128;
+    // units: groups of g column tiles, at most TC_MAX_SPLIT per row-block pair
+    const int g = tc_unit_tiles(ntiles);
+    const int upi = (ntiles + g - 1) / g;
+    const int U = idle ? 0 : c.n_phys * npair * upi;
+    const int ncl_grid = (int)gridDim.x >> 1, ncl = ncl_grid < U ? ncl_grid : U, cl = (int)blockIdx.x >> 1;
+    SegIter it0;
+    it0.upi = upi; it0.g = g; it0.npair = npair; it0.ntiles = ntiles;
+    it0.u = cl < ncl ? (int)((long long)cl * U / ncl) : 0;
+    it0.u_end = cl < ncl ? (int)((long long)(cl + 1) * U / ncl) : 0;
+
+    const uint32_t sbase = (smem_u32(smem_tc) + 1023u) & ~1023u;
+    const uint32_t sA = sbase, sB = sbase + (uint32_t)nkc * TC_CHUNK;
     const uint32_t tmem = tmem_holder;
     volatile int *ab = &abort_flag;
 #ifdef SKB_TC_DEBUG
