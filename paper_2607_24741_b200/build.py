@@ -44,7 +44,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
     with ThreadPoolExecutor(max_workers=len(SOURCES)) as ex:
         objs = list(ex.map(compile_one, SOURCES))
-    subprocess.run([nvcc, "-shared", "-o", LIB, *objs, "-lcudart"], check=True, stdout=sys.stderr, stderr=sys.stderr)
+    subprocess.run([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-o", LIB, *objs, "-lcudart"], check=True,
+                   stdout=sys.stderr, stderr=sys.stderr)
     return LIB
 
 
