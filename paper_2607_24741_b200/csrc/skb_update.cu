@@ -6,6 +6,8 @@
 
 namespace skb {
 
+constexpr long long NARROW_BLOCKS = 148 * 4;      // below this many blocks some SM has fewer than four
+
 template <typename T, int DP, int CS, int XF>
 static void launch_update(const Dev &P, int leg, int width, cudaStream_t st)
 {
@@ -32,6 +34,27 @@ static void launch_update(const Dev &P, int leg, int width, cudaStream_t st)
         const long long ctas = (long long)((nrows + rbw - 1) / rbw) * lanes;
         if (ctas >= 2 * 148 * 4) {
             launch_pdl(update_kernel<T, DP, CS, XF, RW>, dim3((nrows + rbw - 1) / rbw, lanes), dim3(UPD_THREADS), smem, st, P, leg);
+            return;
+        }
+    }
+    if constexpr (sizeof(T) == 4 && DP <= 4 && CS == 4) {
+        // Few dimensions, bound by the special-function unit: when a narrow batch would leave SMs
+        // without a block, fewer rows per thread give 2x or 4x the blocks (same bits, see above).
+        static bool attr_narrow = false;
+        if (!attr_narrow) {
+            cudaFuncSetAttribute(update_kernel<T, DP, CS, XF, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            cudaFuncSetAttribute(update_kernel<T, DP, CS, XF, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            attr_narrow = true;
+        }
+        const auto blocks = [&](int r) { const int rbr = (UPD_THREADS / 32) * r * (32 / CS); return (long long)((nrows + rbr - 1) / rbr) * lanes; };
+        if (blocks(Tune<T, DP>::R) < NARROW_BLOCKS) {
+            if (blocks(2) >= NARROW_BLOCKS) {
+                const int rbr = (UPD_THREADS / 32) * 2 * (32 / CS);
+                launch_pdl(update_kernel<T, DP, CS, XF, 2>, dim3((nrows + rbr - 1) / rbr, lanes), dim3(UPD_THREADS), smem, st, P, leg);
+            } else {
+                const int rbr = (UPD_THREADS / 32) * 1 * (32 / CS);
+                launch_pdl(update_kernel<T, DP, CS, XF, 1>, dim3((nrows + rbr - 1) / rbr, lanes), dim3(UPD_THREADS), smem, st, P, leg);
+            }
             return;
         }
     }
@@ -96,7 +119,11 @@ const Variant *choose_variant(int W, int n, int m, int d, bool f64, bool fast_ex
     double best = -1.0;
     for (int c : {1, 4, 32}) {
         const int rb = (UPD_THREADS / 32) * R * (32 / c);
-        const long long ctas = (long long)W * ((mn + rb - 1) / rb);
+        long long ctas = (long long)W * ((mn + rb - 1) / rb);
+        if (!f64 && DP <= 4 && c == 4) {             // the launcher may drop to one row per thread
+            const int rb1 = (UPD_THREADS / 32) * (32 / c);
+            ctas = (long long)W * ((mn + rb1 - 1) / rb1);
+        }
         const double util_n = (double)n / ((double)((n + rb - 1) / rb) * rb);
         const double util_m = (double)m / ((double)((m + rb - 1) / rb) * rb);
         const double fill = ctas >= 592 ? 1.0 : (double)ctas / 592.0;

@@ -123,7 +123,9 @@ __device__ __forceinline__ void load_rows(const T *p, const bool ok, T (&v)[R])
         for (int r = 0; r < R; ++r) v[r] = T(0);
         return;
     }
-    if constexpr (BYTES == 8) {
+    if constexpr (BYTES == 4) {
+        v[0] = p[0];
+    } else if constexpr (BYTES == 8) {
         const uint2 t = *reinterpret_cast<const uint2 *>(p);
         memcpy(v, &t, 8);
     } else if constexpr (BYTES == 16) {
@@ -163,14 +165,14 @@ __device__ __forceinline__ void load_tile(T *dst, const T *colc, const T *colt, 
 // ------------------------------------------------------------------ fp32, packed pairs
 // Leaves per row the integer-valued maximum mx[r] and sd[r] = sum 2^(arg - mx[r]) over the
 // columns this thread visited.
-template <int DP, int CS, int FORM>
+template <int DP, int CS, int FORM, int R>
 __device__ __forceinline__ void stream_f32(float *sm, const float *colc, const float *colt, const float *coll,
                                            const int cp, const int ncols,
-                                           const float (&xrow)[Tune<float, DP>::R][DP],
-                                           const float (&ph)[Tune<float, DP>::R], const int tid, const int cs,
-                                           float (&mx)[Tune<float, DP>::R], double (&sd)[Tune<float, DP>::R])
+                                           const float (&xrow)[R][DP],
+                                           const float (&ph)[R], const int tid, const int cs,
+                                           float (&mx)[R], double (&sd)[R])
 {
-    constexpr int R = Tune<float, DP>::R, CW = Tune<float, DP>::CW;
+    constexpr int CW = Tune<float, DP>::CW;
     constexpr int NP = CW / 2;                       // packed column pairs per step
     constexpr int TJ = TileCols<float, DP, CS>::value;
     constexpr int STEPS = TJ / (CW * CS);
@@ -641,8 +643,8 @@ __global__ void __launch_bounds__(UPD_THREADS) update_kernel(const Dev P, const 
 #pragma unroll 1
     for (int pass = 0; pass < 2; ++pass) {
         if constexpr (sizeof(T) == 4) {
-            if (form == FORM_DOT) stream_f32<DP, CS, FORM_DOT>(sm, colc, colt, coll, cp, ncols, xr, ph, tid, cs, mx, sd);
-            else stream_f32<DP, CS, FORM_DIFF>(sm, colc, colt, coll, cp, ncols, xr, ph, tid, cs, mx, sd);
+            if (form == FORM_DOT) stream_f32<DP, CS, FORM_DOT, R>(sm, colc, colt, coll, cp, ncols, xr, ph, tid, cs, mx, sd);
+            else stream_f32<DP, CS, FORM_DIFF, R>(sm, colc, colt, coll, cp, ncols, xr, ph, tid, cs, mx, sd);
         } else {
             stream_f64<DP, CS, XF, R>(sm, colc, colt, cp, ncols, xr, tid, cs, m0, mx, sd);
         }
