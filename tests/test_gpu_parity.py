@@ -350,6 +350,9 @@ def test_tensor_core_modes_and_compaction(oracle):
     np.testing.assert_array_equal(ra["f"], rm["f"]); np.testing.assert_array_equal(ra["g"], rm["g"])
     assert len(set(ra["depth"].tolist())) > 1                    # lanes really leave at different depths
     check_accounting(oracle, ra, 6, "active"); check_accounting(oracle, rs, 6, "static")
+    rx = run_gpu(w, mode="masked_exit", compute="tensor")         # frozen lanes' blocks return at once: same bits
+    np.testing.assert_array_equal(rx["f"], rm["f"]); np.testing.assert_array_equal(rx["depth"], rm["depth"])
+    assert rx["stats"]["slots"] == ra["stats"]["slots"]
     ref = oracle.solve_batch(w.x, w.y, w.a, w.b, w.eps, w.tol, max_iter=w.max_iter)
     np.testing.assert_array_equal(ra["depth"], ref.depth)
     assert pot_err(ra["f"], ra["g"], ref.f, ref.g, w.eps.astype(np.float64)).max() <= POT_TOL_F32
