@@ -562,7 +562,18 @@ __global__ void __launch_bounds__(UPD_THREADS) update_kernel(const Dev P, const 
     __shared__ float row_h[RB];
     __shared__ double red[NWARP];
 
-    pdl_enter();
+    // Programmatic dependent launch.  The f-leg follows the g-leg, which writes neither the control
+    // block nor coordinates nor the row potentials: its control block, row coordinates and epilogue
+    // operands are read while that g-leg is still finishing, and only the column terms wait.  The
+    // other legs wait first; the g-leg releases its dependent (the next f-leg) only AFTER its own
+    // wait, so that an early f-leg can rely on the planner and the move being complete.
+    const bool early = (leg == LEG_F);
+    if (early) {
+        asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    } else {
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    }
     const Ctl c = *P.ctl;
     if (c.done) return;
     const int slot = blockIdx.y;
@@ -619,6 +630,8 @@ __global__ void __launch_bounds__(UPD_THREADS) update_kernel(const Dev P, const 
     }
 #pragma unroll
     for (int r = 0; r < R; ++r) ph[r] = (row0 + r < nrows && form == FORM_DIFF) ? (T)prow[row0 + r] : T(0);
+
+    if (early) asm volatile("griddepcontrol.wait;" ::: "memory");
 
     float mx[R];
     double sd[R];
