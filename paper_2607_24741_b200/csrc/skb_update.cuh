@@ -567,14 +567,12 @@ __global__ void __launch_bounds__(UPD_THREADS) update_kernel(const Dev P, const 
     // operands are read while that g-leg is still finishing, and only the column terms wait.  The
     // other legs wait first; the g-leg releases its dependent (the next f-leg) only AFTER its own
     // wait, so that an early f-leg can rely on the planner and the move being complete.
+    // (The column check also reads the control block early, then waits for the f-leg's verdict.)
     const bool early = (leg == LEG_F);
-    if (early) {
-        asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    } else {
-        asm volatile("griddepcontrol.wait;" ::: "memory");
-        asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    }
+    if (leg == LEG_G) asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const Ctl c = *P.ctl;
+    if (leg == LEG_V) asm volatile("griddepcontrol.wait;" ::: "memory");
     if (c.done) return;
     const int slot = blockIdx.y;
     if (slot >= c.n_phys) return;
