@@ -128,9 +128,14 @@ def dual_value(C, f, g, eps, a, b) -> float:
 
 
 def solve_lane(x, y, a, b, eps, tol, *, tol_screen=0.0, max_iter=5000, audit_every=1,
-               fixed_cycles=0, neighbours=False, history=False, dual=False) -> LaneResult:
-    """Run one lane to its completion depth (or ``fixed_cycles`` cycles)."""
+               fixed_cycles=0, neighbours=False, history=False, dual=False, f0=None, g0=None,
+               audit_initial=False) -> LaneResult:
+    """Run one lane to its completion depth (or ``fixed_cycles`` cycles), from the cold
+    proposal f = g = 0 or from the warm proposal (f0, g0); with ``audit_initial`` the proposal
+    itself is audited first and a lane that already passes has depth 0."""
     x, y, a, b = _c64(x), _c64(y), _c64(a), _c64(b)
+    f0 = None if f0 is None else _c64(f0)
+    g0 = None if g0 is None else _c64(g0)
     n, d = x.shape
     m = y.shape[0]
     f, g = np.empty(n), np.empty(m)
@@ -149,7 +154,7 @@ def solve_lane(x, y, a, b, eps, tol, *, tol_screen=0.0, max_iter=5000, audit_eve
                            int(max_iter), int(audit_every), int(fixed_cycles), _d(f), _d(g),
                            _d(fp), _d(gp), _d(fn), _d(gn), ctypes.byref(depth),
                            ctypes.byref(status), ctypes.byref(rr), ctypes.byref(rc), _d(hr),
-                           _d(hc), _d(dh))
+                           _d(hc), _d(dh), _d(f0), _d(g0), int(bool(audit_initial)))
     if ret != 0:
         raise ValueError(f"oracle rejected the lane (code {ret})")
     return LaneResult(f, g, depth.value, status.value, rr.value, rc.value, fp, gp, fn, gn, hr, hc, dh)

@@ -133,8 +133,14 @@ double orc_dual(int n, int m, const double *C, const double *f, const double *g,
  *   fixed_cycles == 0: stop at the first audited cycle k with
  *     r_row <= tol_screen and max(r_row, r_col) <= tol_stop.
  *
+ *   f0, g0 (either may be NULL = zeros): the proposal the iteration starts from
+ *     (Section "Initialization and repeated couplings": cold proposals are f = g = 0,
+ *     warm ones carry potentials over from an earlier coupling).
+ *   audit_initial != 0: the proposal itself gets the audit of Eq. 5 before any update;
+ *     a lane whose proposal already passes needs no update and has depth 0.
+ *
  * Outputs (any may be NULL): f,g at the depth; f_prev,g_prev one cycle before
- * (zeros if depth == 1); f_next,g_next one cycle after; r_row,r_col at the
+ * (the proposal if depth <= 1); f_next,g_next one cycle after; r_row,r_col at the
  * depth; hist_row/hist_col[k-1] residuals at every audited cycle k (NaN where
  * not audited), length max_iter (+1 used when f_next is requested);
  * dual_hist[2(k-1)], [2(k-1)+1] dual value after the f-leg and g-leg of cycle k.
@@ -144,7 +150,7 @@ int orc_lane(int n, int m, int d, const double *x, const double *y, const double
              int audit_every, int fixed_cycles, double *f_out, double *g_out, double *f_prev,
              double *g_prev, double *f_next, double *g_next, int *depth_out, int *status_out,
              double *r_row_out, double *r_col_out, double *hist_row, double *hist_col,
-             double *dual_hist)
+             double *dual_hist, const double *f0, const double *g0, int audit_initial)
 {
     if (n < 1 || m < 1 || d < 1 || !(eps > 0.0) || max_iter < 1) return -1;
     if (audit_every < 1) audit_every = 1;
@@ -158,12 +164,25 @@ int orc_lane(int n, int m, int d, const double *x, const double *y, const double
     double *col = (double *)malloc(sizeof(double) * m);
     if (!C || !f || !g || !fp || !gp || !row || !col) return -2;
     orc_cost_matrix(n, m, d, x, y, C);
+    if (f0) memcpy(f, f0, sizeof(double) * n);
+    if (g0) memcpy(g, g0, sizeof(double) * m);
+    memcpy(fp, f, sizeof(double) * n);
+    memcpy(gp, g, sizeof(double) * m);
 
     int depth = 0, status = ORC_RUNNING;
     double rr_at = NAN, rc_at = NAN;
     int last = fixed_cycles > 0 ? fixed_cycles : max_iter;
     int k;
-    for (k = 1; k <= last; ++k) {
+    if (audit_initial) {                   /* the proposal may already satisfy Eq. 5 */
+        double rr, rc;
+        orc_residuals(n, m, C, f, g, eps, a, b, row, col, &rr, &rc);
+        if ((rr <= tol_screen) && (fmax(rr, rc) <= tol_stop)) {
+            status = ORC_DONE;
+            rr_at = rr;
+            rc_at = rc;
+        }
+    }
+    for (k = 1; k <= last && !(status == ORC_DONE && fixed_cycles == 0); ++k) {
         memcpy(fp, f, sizeof(double) * n);
         memcpy(gp, g, sizeof(double) * m);
         orc_f_leg(n, m, C, g, a, eps, f);
@@ -244,7 +263,8 @@ int orc_batch(int W, int n, int m, int d, const double *x, const double *y, cons
                           max_iter, audit_every, fixed_cycles, f ? f + (size_t)t * n : NULL,
                           g ? g + (size_t)t * m : NULL, NULL, NULL, NULL, NULL,
                           depth ? depth + t : NULL, status ? status + t : NULL,
-                          r_row ? r_row + t : NULL, r_col ? r_col + t : NULL, NULL, NULL, NULL);
+                          r_row ? r_row + t : NULL, r_col ? r_col + t : NULL, NULL, NULL, NULL,
+                          NULL, NULL, 0);
         if (rc != 0) {
 #ifdef _OPENMP
 #pragma omp atomic write

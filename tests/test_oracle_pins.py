@@ -244,3 +244,46 @@ def test_slot_identity_and_paper_counts(oracle):
         s = oracle.slot_counts(depths)
         assert s["S_static"] == s_static and s["S_active"] == s_static - (s_static - s_active - deficit)
         assert s["R"] == s_static - s["S_active"]
+
+
+def test_warm_proposal_is_the_same_iteration_started_later(oracle):
+    # Section "Initialization and repeated couplings": a proposal only replaces the starting point.
+    # Starting from the cold iteration's own state after j cycles must land on the cold run's states
+    # j cycles earlier (semigroup property of the fixed map F_t of Eq. 2) - checked against the cold
+    # run, not against the warm code path itself.
+    x, y, a, b = rand_instance(11, 9, 12, 2)
+    eps, tol = 0.2, 1e-7
+    cold = oracle.solve_lane(x, y, a, b, eps, tol)
+    assert cold.depth > 6
+    for j in (1, 4):
+        part = oracle.solve_lane(x, y, a, b, eps, tol, fixed_cycles=j)
+        warm = oracle.solve_lane(x, y, a, b, eps, tol, f0=part.f, g0=part.g)
+        assert warm.depth == cold.depth - j and warm.status == oracle.DONE
+        np.testing.assert_allclose(warm.f, cold.f, rtol=0, atol=1e-14)
+        np.testing.assert_allclose(warm.g, cold.g, rtol=0, atol=1e-14)
+    # zeros given explicitly are the cold proposal
+    z = oracle.solve_lane(x, y, a, b, eps, tol, f0=np.zeros(9), g0=np.zeros(12))
+    assert z.depth == cold.depth and np.array_equal(z.f, cold.f)
+
+
+def test_audit_of_the_proposal_is_eq5_at_the_proposal(oracle):
+    x, y, a, b = rand_instance(12, 7, 10, 3)
+    eps = 0.3
+    C = cdist(x, y, "sqeuclidean")
+    conv = oracle.solve_lane(x, y, a, b, eps, 1e-12)
+    g0 = conv.g + 0.01 * np.sin(np.arange(10))
+    P = plan(C, conv.f, g0, eps)
+    rr, rc = np.abs(P.sum(1) - a).sum(), np.abs(P.sum(0) - b).sum()
+    assert rr > 1e-3 and rc > 1e-3                        # neither marginal is current for this proposal
+    # thresholds above both residuals: the proposal passes as it is, depth 0, nothing is updated
+    r0 = oracle.solve_lane(x, y, a, b, eps, 2 * max(rr, rc), f0=conv.f, g0=g0, audit_initial=True)
+    assert r0.depth == 0 and r0.status == oracle.DONE
+    assert r0.r_row == pytest.approx(rr, rel=1e-12) and r0.r_col == pytest.approx(rc, rel=1e-12)
+    np.testing.assert_array_equal(r0.f, conv.f); np.testing.assert_array_equal(r0.g, g0)
+    # stop threshold between the two residuals, screen wide open: the two-sided test must fail on the larger one
+    lo, hi = min(rr, rc), max(rr, rc)
+    r1 = oracle.solve_lane(x, y, a, b, eps, 0.5 * (lo + hi), tol_screen=10.0, f0=conv.f, g0=g0, audit_initial=True)
+    assert r1.depth >= 1
+    # without the initial audit the same call never reports depth 0
+    r2 = oracle.solve_lane(x, y, a, b, eps, 2 * max(rr, rc), f0=conv.f, g0=g0)
+    assert r2.depth == 1
