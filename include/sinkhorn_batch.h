@@ -108,10 +108,14 @@ size_t sinkhorn_batch_workspace_bytes(const skb_config *cfg);
  *   b   [W, m] fp32, > 0, each lane sums to 1                    (device)
  *   eps [W]    fp32, > 0, per-lane regularisation                (device)
  *   tol        two-sided stopping tolerance tau_stop of Eq. 5    (> 0)
- * Potentials start cold, f = g = 0.  Inputs are copied into the workspace in the
- * kernels' own layout; they may be freed once the stream has passed this call.
- * Non-positive weights or eps and non-finite coordinates are detected on the
- * device and reported by the first step/drain as SKB_ERR_VALUE.
+ * Potentials start cold, f = g = 0 (sinkhorn_batch_warm_start replaces them).  Inputs are
+ * copied into the workspace in the kernels' own layout; they may be freed once the stream
+ * has passed this call.  Non-positive weights or eps and non-finite coordinates are
+ * detected on the device and reported as SKB_ERR_VALUE by drain, or by a later step once
+ * the control block it reads back asynchronously has arrived.
+ * The call waits for its set-up kernels (their time is SKB_PHASE_CREATE of
+ * sinkhorn_batch_stats); with SKB_COMPUTE_AUTO it first waits for the lanes' cost range to
+ * come back from the device, because the choice of arithmetic decides the layout.
  * On success *out holds the handle; the caller releases it with
  * sinkhorn_batch_destroy (the workspace stays the caller's).
  */
@@ -119,9 +123,26 @@ skb_status sinkhorn_batch_create(const void *x, const void *y, const float *a, c
                                  const float *eps, float tol, const skb_config *cfg,
                                  skb_batch **out);
 
+/*
+ * Warm proposal (Section "Initialization and repeated couplings"): start from the caller's
+ * potentials instead of f = g = 0.
+ *   f0 [W, n], g0 [W, m]  float64, device, the paper's convention pi = exp((f + g - C)/eps);
+ *                         either may be null (that side stays cold).  Non-finite values are
+ *                         reported as SKB_ERR_VALUE like bad inputs.
+ *   audit_initial != 0    the proposal itself is audited (row screen, two-sided check of
+ *                         Eq. 5) before any update: a lane whose proposal already passes
+ *                         retires at depth 0 with the proposal as its output and its
+ *                         measured residuals; the others go on from it.
+ * Valid only before the first step/drain (SKB_ERR_STATE afterwards).  Enqueues one kernel.
+ */
+skb_status sinkhorn_batch_warm_start(skb_batch *h, const double *f0, const double *g0, int audit_initial);
+
 /* Enqueue `cycles` full cycles (both legs of Eq. 3 plus screen, two-sided check and
- * retirement after every audited one).  Never synchronises.  Cycles past the point
- * where every lane is finished are no-ops. */
+ * retirement after every audited one).  Never synchronises: each call leaves an asynchronous
+ * copy of the device's control block behind and looks, without waiting, whether an earlier
+ * one has arrived; from it the launch width follows the survivors and device-side errors
+ * (bad input values, a bounded wait that ran out) are returned.  Cycles past the point where
+ * every lane is finished are no-ops. */
 skb_status sinkhorn_batch_step(skb_batch *h, int cycles);
 
 /* Run until every lane is retired (passed, hit max_iter, or went non-finite), then
@@ -148,15 +169,49 @@ skb_status sinkhorn_batch_depths(skb_batch *h, int *depth, int *lane_status);
 skb_status sinkhorn_batch_residuals(skb_batch *h, float *r_row, float *r_col);
 
 /*
- * Work accounting (Eq. 6-8), host outs, any may be null.  Synchronises.
+ * Phases of the time model T_active = sum_k c_k(A_k) + H_screen + H_check + H_compact
+ * (Section "Hardware realization and break-even", Eq. 11): the update legs are c_k (the row
+ * screen rides inside the f-leg, so H_screen has no time of its own), the column check is
+ * H_check, planning plus emission/compaction is H_compact.
+ */
+typedef enum {
+    SKB_PHASE_CREATE = 0,       /* set-up kernels of create (always measured)                 */
+    SKB_PHASE_F_LEG = 1,        /* f-leg launches, row screen included                        */
+    SKB_PHASE_COLUMN_CHECK = 2, /* column half of the two-sided check, flagged lanes only     */
+    SKB_PHASE_PLAN = 3,         /* flags -> retire list, hole/filler pairing, counters        */
+    SKB_PHASE_EMIT_MOVE = 4,    /* retirees' outputs written, survivors moved into holes       */
+    SKB_PHASE_G_LEG = 5,        /* g-leg launches                                             */
+    SKB_N_PHASES = 6
+} skb_phase;
+
+/*
+ * Phase timing on or off (off at creation), only before the first step/drain.  When on, every
+ * kernel of every cycle is bracketed by CUDA events on the batch's stream; the kernels of a
+ * cycle then run strictly one after the other (normally the next kernel's launch overlaps the
+ * current one), so a profiled solve is slower than a plain one and its phases add up to ITS
+ * duration.  Events are collected every 16 cycles with a stream synchronisation.
+ */
+skb_status sinkhorn_batch_set_profiling(skb_batch *h, int on);
+
+/*
+ * Work accounting (Eq. 6-8) and the cost record of Eq. 11, host outs, any may be null.
+ * Synchronises.
  *   slots      lane-cycles physically executed: sum_k A_k in ACTIVE mode, W*l_max otherwise
  *   cycles     complete cycles executed (l_max)
  *   widths     widths[k-1] = physical width of cycle k, for k = 1..min(cycles, widths_cap)
  *   pair_terms exp-terms evaluated by the update kernel, all passes (legs, look-ahead
  *              screen, column check)
+ *   phase_ms   [SKB_N_PHASES] milliseconds per skb_phase summed over the solve so far;
+ *              entries other than SKB_PHASE_CREATE are zero unless phase timing is on
  */
 skb_status sinkhorn_batch_stats(skb_batch *h, long long *slots, int *cycles, int *widths,
-                                int widths_cap, long long *pair_terms);
+                                int widths_cap, long long *pair_terms, float *phase_ms);
+
+/* Per-cycle update cost c_k of Eq. 11 from a profiled solve: update_ms[k-1] = f-leg + g-leg
+ * milliseconds of cycle k (host out, up to cap entries); *count = cycles recorded.  Together
+ * with widths[] of sinkhorn_batch_stats this is c_k as a function of the width A_k.
+ * Synchronises. */
+skb_status sinkhorn_batch_cycle_trace(skb_batch *h, float *update_ms, int cap, int *count);
 
 /* The arithmetic the batch actually runs (skb_compute, never AUTO): what an automatic
  * batch resolved to from its data.  Host out. */
@@ -172,15 +227,27 @@ skb_status sinkhorn_batch_arithmetic(skb_batch *h, int *compute);
  */
 skb_status sinkhorn_batch_selftest_bounded_wait(int *out3, float budget_ms, void *stream);
 
+/*
+ * Self-test: measured issue rates of the units that bound the update kernels, for quoting a
+ * roofline fraction against delivered rather than nominal rates.  Runs four short register-only
+ * loops (fp32 FMA, packed fp32x2 FMA, float64 FMA, fp32 ex2) and writes the operations per
+ * second of each to ops_per_second[0..3] (host out; an fp32x2 instruction counts as two FMAs).
+ * sink: any device float the caller owns (the loops need an address they might write to; they
+ * never do).  Synchronises the stream.
+ */
+skb_status sinkhorn_batch_selftest_unit_rates(double *ops_per_second, float *sink, void *stream);
+
 /* Number of kernels this handle has launched so far (host out). */
 skb_status sinkhorn_batch_launch_count(skb_batch *h, long long *launches);
 
 /*
  * Measurement aid: launches the update kernel for one leg (0 = f-leg, 1 = g-leg) `reps`
  * times at the batch's current width, bracketed by CUDA events on the batch's stream, and
- * returns the mean duration per launch in milliseconds (host out).  The f-leg only reads
- * the current state and rewrites the look-ahead buffers, so the solve is not disturbed;
- * the g-leg recomputes g from the current f.  Synchronises.
+ * returns the mean duration per launch in milliseconds (host out).  Call it between cycles
+ * (after step, before drain).  The launches are dry runs: all pair work and the row epilogue,
+ * but no potential is stored and no residual term added, so a solve continued afterwards
+ * gives the same bits as one that was never profiled.  Returns SKB_ERR_STATE when no lane is
+ * running any more (the launch would return at once).  Synchronises.
  */
 skb_status sinkhorn_batch_profile_update(skb_batch *h, int leg, int reps, float *ms_per_launch);
 
@@ -216,9 +283,14 @@ void sinkhorn_batch_destroy(skb_batch *h);
  * image (held by every GPU that loads the library until exit), so W <= SKB_STATIC_MAX_LANES
  * and n <= SKB_STATIC_MAX_ROWS; larger shapes return SKB_ERR_SHAPE.  The call performs no
  * cudaMalloc, cudaFree or other allocating call.  The first call on each device looks the
- * array's device address up (with that device current); make that first call before any
- * stream capture begins.  All calls share the one array: calls whose kernels could overlap
- * on the GPU (different streams, different threads) race and must be ordered by the caller.
+ * array's device address up (with that device current) and, where the CUDA runtime loads
+ * kernels lazily, is also the moment the runtime loads this library's device code onto that
+ * device (which reserves device memory for the code and may synchronise): make that first
+ * call during warm-up, before any stream capture begins and before memory is frozen.  All
+ * calls share the one array: calls whose kernels could overlap on the GPU (different
+ * streams, different threads) race and must be ordered by the caller.
+ * sinkhorn_row_residual_static_last_error() gives the text of the calling thread's last
+ * failed call (empty after a successful one).
  */
 #define SKB_STATIC_MAX_LANES 256
 #define SKB_STATIC_MAX_ROWS 8192
@@ -228,8 +300,9 @@ skb_status sinkhorn_row_residual_static(const float *x, const float *y, const fl
                                         int W, int n, int m, int d, float *r_row, void *stream);
 const char *sinkhorn_row_residual_static_last_error(void);
 
-/* Host string describing the last error on this handle (or of the last failed create
- * when h is null).  Valid until the next call on the same handle. */
+/* Host string describing the last error on this handle (or, when h is null, of the calling
+ * thread's last failed create or host-buffer solve).  Valid until the next call on the same
+ * handle (h null: the next failing create of the same thread). */
 const char *sinkhorn_batch_last_error(const skb_batch *h);
 
 #ifdef __cplusplus

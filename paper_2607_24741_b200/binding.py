@@ -28,8 +28,10 @@ EXPORTS = (
     "sinkhorn_batch_stats", "sinkhorn_batch_destroy", "sinkhorn_batch_last_error",
     "sinkhorn_batch_host_workspace_bytes", "sinkhorn_batch_solve_host",
     "sinkhorn_batch_launch_count", "sinkhorn_batch_profile_update", "sinkhorn_batch_arithmetic",
-    "sinkhorn_batch_selftest_bounded_wait",
+    "sinkhorn_batch_selftest_bounded_wait", "sinkhorn_batch_warm_start", "sinkhorn_batch_set_profiling",
+    "sinkhorn_batch_cycle_trace", "sinkhorn_batch_selftest_unit_rates",
 )
+PHASES = ("create", "f_leg", "column_check", "plan", "emit_move", "g_leg")
 # entry points outside the sinkhorn_batch_* family
 EXTRA_EXPORTS = ("sinkhorn_row_residual_static", "sinkhorn_row_residual_static_last_error")
 
@@ -69,8 +71,13 @@ def _load():
     lib.sinkhorn_batch_depths.argtypes = [vp, vp, vp]
     lib.sinkhorn_batch_residuals.argtypes = [vp, vp, vp]
     lib.sinkhorn_batch_stats.argtypes = [vp, ctypes.POINTER(ctypes.c_longlong), ctypes.POINTER(ctypes.c_int),
-                                         vp, ctypes.c_int, ctypes.POINTER(ctypes.c_longlong)]
+                                         vp, ctypes.c_int, ctypes.POINTER(ctypes.c_longlong),
+                                         ctypes.POINTER(ctypes.c_float)]
+    lib.sinkhorn_batch_warm_start.argtypes = [vp, vp, vp, ctypes.c_int]
+    lib.sinkhorn_batch_set_profiling.argtypes = [vp, ctypes.c_int]
+    lib.sinkhorn_batch_cycle_trace.argtypes = [vp, vp, ctypes.c_int, ctypes.POINTER(ctypes.c_int)]
     lib.sinkhorn_batch_selftest_bounded_wait.argtypes = [vp, ctypes.c_float, vp]
+    lib.sinkhorn_batch_selftest_unit_rates.argtypes = [ctypes.POINTER(ctypes.c_double), vp, vp]
     lib.sinkhorn_batch_arithmetic.argtypes = [vp, ctypes.POINTER(ctypes.c_int)]
     lib.sinkhorn_batch_launch_count.argtypes = [vp, ctypes.POINTER(ctypes.c_longlong)]
     lib.sinkhorn_batch_profile_update.argtypes = [vp, ctypes.c_int, ctypes.c_int, ctypes.POINTER(ctypes.c_float)]
@@ -163,6 +170,17 @@ def sinkhorn_row_residual_static(x, y, a, f, g, eps, stream=None):
     return out
 
 
+def unit_rates(device=None):
+    """Measured operations per second of the fp32 FMA, packed fp32x2 FMA, float64 FMA and fp32 ex2
+    units (the library's self-test loops)."""
+    dev = torch.device("cuda", torch.cuda.current_device()) if device is None else device
+    sink = torch.zeros(1, dtype=torch.float32, device=dev)
+    out = (ctypes.c_double * 4)()
+    with torch.cuda.device(dev):
+        _check(lib.sinkhorn_batch_selftest_unit_rates(out, _ptr(sink), torch.cuda.current_stream(dev).cuda_stream))
+    return dict(zip(("ffma", "ffma2", "dfma", "ex2"), list(out)))
+
+
 class SinkhornBatch:
     """One batch of W lanes on the current CUDA device (thin wrapper over the C calls)."""
 
@@ -226,14 +244,33 @@ class SinkhornBatch:
         _check(lib.sinkhorn_batch_residuals(self.h, _ptr(rr), _ptr(rc)), self.h)
         return rr, rc
 
+    def warm_start(self, f0=None, g0=None, audit_initial=False):
+        for t, shape in ((f0, (self.W, self.n)), (g0, (self.W, self.m))):
+            if t is not None and (t.dtype != torch.float64 or not t.is_cuda or tuple(t.shape) != shape
+                                  or not t.is_contiguous()):
+                raise ValueError("f0 [W,n] and g0 [W,m] must be contiguous float64 CUDA tensors")
+        _check(lib.sinkhorn_batch_warm_start(self.h, _ptr(f0), _ptr(g0), 1 if audit_initial else 0), self.h)
+        self._warm = (f0, g0)
+
+    def set_profiling(self, on=True):
+        _check(lib.sinkhorn_batch_set_profiling(self.h, 1 if on else 0), self.h)
+
     def stats(self, widths_cap=0):
         slots, terms, cycles = ctypes.c_longlong(0), ctypes.c_longlong(0), ctypes.c_int(0)
         buf = (ctypes.c_int * max(widths_cap, 1))()
+        ph = (ctypes.c_float * len(PHASES))()
         _check(lib.sinkhorn_batch_stats(self.h, ctypes.byref(slots), ctypes.byref(cycles),
-                                        ctypes.cast(buf, ctypes.c_void_p), widths_cap, ctypes.byref(terms)), self.h)
+                                        ctypes.cast(buf, ctypes.c_void_p), widths_cap, ctypes.byref(terms), ph), self.h)
         k = min(cycles.value, widths_cap)
         return {"slots": slots.value, "cycles": cycles.value, "pair_terms": terms.value,
-                "widths": list(buf[:k])}
+                "widths": list(buf[:k]), "phase_ms": dict(zip(PHASES, list(ph)))}
+
+    def cycle_trace(self):
+        n = ctypes.c_int(0)
+        _check(lib.sinkhorn_batch_cycle_trace(self.h, None, 0, ctypes.byref(n)), self.h)
+        buf = (ctypes.c_float * max(n.value, 1))()
+        _check(lib.sinkhorn_batch_cycle_trace(self.h, ctypes.cast(buf, ctypes.c_void_p), n.value, ctypes.byref(n)), self.h)
+        return list(buf[:n.value])
 
     def arithmetic(self) -> str:
         c = ctypes.c_int(0)

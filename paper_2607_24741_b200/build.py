@@ -9,7 +9,7 @@ from concurrent.futures import ThreadPoolExecutor
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsinkhorn_batch.so")
-SOURCES = ("skb_update.cu", "skb_control.cu", "skb_api.cu", "skb_noalloc.cu", "skb_update_tc.cu")
+SOURCES = ("skb_update.cu", "skb_control.cu", "skb_api.cu", "skb_noalloc.cu", "skb_update_tc.cu", "skb_selftest.cu")
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--use_fast_math=false"]
 

@@ -27,11 +27,23 @@ struct skb_batch {
     long long launches;    // kernels launched so far
     int res_device;        // device the pooled host resources belong to
     bool tensor;           // the tensor-core update kernel is in use
+    bool snap_pending;     // step() left a control-block snapshot in flight (ev[snap_idx])
+    int snap_idx;
+    // phase timing (Eq. 11's cost record): off unless sinkhorn_batch_set_profiling turned it on
+    bool profiling;
+    bool no_multi_cycle;   // measurement switch: keep one launch per leg even where several cycles per launch are possible
+    std::vector<cudaEvent_t> pev;      // timing events, PHASE_EVENTS_PER_CYCLE per enqueued cycle of a chunk + 1
+    int pev_used;                      // events recorded since the last harvest
+    float phase_ms[SKB_N_PHASES];
+    std::vector<float> cycle_update_ms;   // per cycle: f-leg + g-leg
     alignas(64) unsigned char maps[2 * 128];   // CUtensorMap of x and of y
     std::string err;
 };
 
-static std::string g_create_err;
+// Text of the last failed create (or host-buffer solve) of the calling thread.
+static thread_local std::string g_create_err;
+static const int PHASE_EVENTS_PER_CYCLE = 5;     // f-leg | column check | plan | emit/move | g-leg, boundaries shared
+static const int PROFILE_CHUNK = 16;             // cycles between two harvests of the timing events
 
 // Host-side resources of a handle (a pinned control-block pair and two events) are recycled
 // through a small per-device pool: allocating and freeing pinned memory costs hundreds of
@@ -52,8 +64,8 @@ static cudaError_t host_res_get(HostRes *r)
     }
     r->device = dev; r->pinned = nullptr; r->ev[0] = r->ev[1] = nullptr;
     if ((e = cudaHostAlloc((void **)&r->pinned, 2 * sizeof(Ctl), cudaHostAllocDefault)) != cudaSuccess) return e;
-    if ((e = cudaEventCreateWithFlags(&r->ev[0], cudaEventDisableTiming)) != cudaSuccess) return e;
-    return cudaEventCreateWithFlags(&r->ev[1], cudaEventDisableTiming);
+    if ((e = cudaEventCreate(&r->ev[0])) != cudaSuccess) return e;      // timing events: they also bracket create
+    return cudaEventCreate(&r->ev[1]);
 }
 
 static void host_res_put(const HostRes &r)
@@ -115,6 +127,7 @@ static size_t carve(const skb_config *c, const Variant *var, bool tensor, char *
     d.ctl = (Ctl *)take(sizeof(Ctl));
     d.state = (int *)take(W * 4); d.flag = (int *)take(W * 4); d.verdict = (int *)take(W * 4);
     d.nonfinite = (int *)take(W * 4);
+    d.ret_at = (int *)take(W * 4); d.n_checks = (int *)take(W * 4);
     d.rsum_row = (unsigned long long *)take(W * 8); d.rsum_col = (unsigned long long *)take(W * 8);
     d.depth = (int *)take(W * 4); d.status = (int *)take(W * 4); d.emitted = (int *)take(W * 4);
     d.res_row = (double *)take(W * 8); d.res_col = (double *)take(W * 8);
@@ -223,6 +236,8 @@ extern "C" skb_status sinkhorn_batch_create(const void *x, const void *y, const 
     h->known_width = cfg->W; h->finished = false; h->enqueued = 0; h->launches = 0; h->h_ctl = nullptr;
     h->ev[0] = h->ev[1] = nullptr;
     h->tensor = cfg->compute == SKB_COMPUTE_TENSOR;
+    h->snap_pending = false; h->snap_idx = 0; h->profiling = false; h->pev_used = 0; h->no_multi_cycle = false;
+    for (int i = 0; i < SKB_N_PHASES; ++i) h->phase_ms[i] = 0.f;
     carve(cfg, var, h->tensor, (char *)cfg->workspace, &h->dev);
     h->dev.tol_stop = (double)tol;
     h->dev.tol_screen = cfg->tol_screen > 0.0f ? (double)cfg->tol_screen : (double)tol;
@@ -240,6 +255,7 @@ extern "C" skb_status sinkhorn_batch_create(const void *x, const void *y, const 
     memset(&init, 0, sizeof(init));
     init.n_phys = cfg->W; init.n_running = cfg->W;
     h->h_ctl[0] = init;
+    cudaEventRecord(h->ev[1], h->stream);          // start of the set-up work (SKB_PHASE_CREATE)
     if ((e = cudaMemsetAsync(cfg->workspace, 0, zero_end, h->stream)) != cudaSuccess ||
         (e = cudaMemcpyAsync(h->dev.ctl, &h->h_ctl[0], sizeof(Ctl), cudaMemcpyHostToDevice, h->stream)) != cudaSuccess) {
         skb_status st = cuda_fail(nullptr, e, "create");
@@ -288,8 +304,38 @@ extern "C" skb_status sinkhorn_batch_create(const void *x, const void *y, const 
         sinkhorn_batch_destroy(h);
         return st;
     }
-    cudaEventSynchronize(h->ev[0]);
+    if ((e = cudaEventSynchronize(h->ev[0])) != cudaSuccess ||
+        (e = cudaEventElapsedTime(&h->phase_ms[SKB_PHASE_CREATE], h->ev[1], h->ev[0])) != cudaSuccess) {
+        skb_status st = cuda_fail(nullptr, e, "create");
+        sinkhorn_batch_destroy(h);
+        return st;
+    }
     *out = h;
+    return SKB_OK;
+}
+
+extern "C" skb_status sinkhorn_batch_warm_start(skb_batch *h, const double *f0, const double *g0, int audit_initial)
+{
+    if (!h) return SKB_ERR_NULL;
+    if (h->enqueued != 0) return fail(h, SKB_ERR_STATE, "a warm proposal must be given before the first step or drain");
+    if (f0 || g0) { launch_warm(h->dev, f0, g0, h->stream); h->launches += 1; }
+    h->dev.audit_initial = audit_initial ? 1 : 0;
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? SKB_OK : cuda_fail(h, e, "warm_start");
+}
+
+extern "C" skb_status sinkhorn_batch_set_profiling(skb_batch *h, int on)
+{
+    if (!h) return SKB_ERR_NULL;
+    if (h->enqueued != 0) return fail(h, SKB_ERR_STATE, "phase timing must be switched before the first step or drain");
+    if (on && h->pev.empty()) {
+        h->pev.resize(PROFILE_CHUNK * PHASE_EVENTS_PER_CYCLE + 1, nullptr);
+        for (cudaEvent_t &ev : h->pev) {
+            cudaError_t e = cudaEventCreate(&ev);
+            if (e != cudaSuccess) return cuda_fail(h, e, "set_profiling");
+        }
+    }
+    h->profiling = on != 0;
     return SKB_OK;
 }
 
@@ -301,17 +347,65 @@ static void launch_leg(skb_batch *h, int leg, int w)
     else h->var->launch(h->dev, leg, w, h->stream);
 }
 
-static void enqueue_cycle(skb_batch *h)
+// ACTIVE batches whose lanes have few row blocks run several whole cycles per launch, one
+// thread-block cluster per lane (lane_cycles_kernel), followed by one planner for all of them.
+static bool cycles_in_one_launch(const skb_batch *h)
+{
+    if (h->cfg.mode != SKB_ACTIVE || h->tensor || h->profiling || !h->var->launch_cycles || h->no_multi_cycle) return false;
+    const int mx = h->cfg.n > h->cfg.m ? h->cfg.n : h->cfg.m;
+    return (mx + h->var->rows_per_cta - 1) / h->var->rows_per_cta <= MAX_CLUSTER_BLOCKS;
+}
+
+// `cycles` cycles in one launch (1 <= cycles <= MAX_CYCLES_IN_LAUNCH): lanes that pass inside it write their own
+// outputs; the planner accounts for every cycle of the launch and fills the holes.
+static void enqueue_cycles_launch(skb_batch *h, int cycles)
 {
     const int w = h->known_width;
-    launch_leg(h, LEG_F, w);
-    launch_leg(h, LEG_V, w);
-    int nk = 3;
-    nk += launch_plan(h->dev, w, h->stream);
+    h->var->launch_cycles(h->dev, cycles, w, h->stream);
+    int nk = 1;
+    nk += launch_plan_cycles(h->dev, w, cycles, h->stream);
     nk += launch_emit_move(h->dev, w, h->stream);
-    launch_leg(h, LEG_G, w);
+    h->enqueued += cycles;
+    h->launches += nk;
+}
+
+static void enqueue_cycle(skb_batch *h)
+{
+    if (cycles_in_one_launch(h)) { enqueue_cycles_launch(h, 1); return; }
+    const int w = h->known_width;
+    // phase timing: an event between every two kernels of the cycle (which also keeps them from
+    // overlapping: a kernel launched after an event record waits for everything before it)
+    const bool prof = h->profiling && h->pev_used + PHASE_EVENTS_PER_CYCLE + (h->pev_used == 0 ? 1 : 0) <= (int)h->pev.size();
+    auto mark = [&]() { if (prof) cudaEventRecord(h->pev[h->pev_used++], h->stream); };
+    if (prof && h->pev_used == 0) mark();
+    launch_leg(h, LEG_F, w); mark();
+    launch_leg(h, LEG_V, w); mark();
+    int nk = 3;
+    nk += launch_plan(h->dev, w, h->stream); mark();
+    nk += launch_emit_move(h->dev, w, h->stream); mark();
+    launch_leg(h, LEG_G, w); mark();
     h->enqueued++;
     h->launches += nk;
+}
+
+// Waits for the timing events recorded so far and adds their intervals to the phase totals.
+static cudaError_t harvest_phases(skb_batch *h)
+{
+    if (h->pev_used < 2) { h->pev_used = 0; return cudaSuccess; }
+    cudaError_t e = cudaEventSynchronize(h->pev[h->pev_used - 1]);
+    static const int phase_of[PHASE_EVENTS_PER_CYCLE] = {SKB_PHASE_F_LEG, SKB_PHASE_COLUMN_CHECK, SKB_PHASE_PLAN,
+                                                         SKB_PHASE_EMIT_MOVE, SKB_PHASE_G_LEG};
+    float upd = 0.f;
+    for (int i = 0; i + 1 < h->pev_used && e == cudaSuccess; ++i) {
+        float ms = 0.f;
+        e = cudaEventElapsedTime(&ms, h->pev[i], h->pev[i + 1]);
+        const int ph = phase_of[i % PHASE_EVENTS_PER_CYCLE];
+        h->phase_ms[ph] += ms;
+        if (ph == SKB_PHASE_F_LEG || ph == SKB_PHASE_G_LEG) upd += ms;
+        if (ph == SKB_PHASE_G_LEG) { h->cycle_update_ms.push_back(upd); upd = 0.f; }
+    }
+    h->pev_used = 0;
+    return e;
 }
 
 static skb_status absorb(skb_batch *h, const Ctl &c)
@@ -324,12 +418,43 @@ static skb_status absorb(skb_batch *h, const Ctl &c)
     return SKB_OK;
 }
 
+// A snapshot of the control block that an earlier step() left in flight: absorb it if it has
+// arrived (wait == false: only look), so that device-side errors surface and the launch width
+// follows the survivors without any call ever blocking.
+static skb_status poll_snapshot(skb_batch *h, bool wait)
+{
+    if (!h->snap_pending) return SKB_OK;
+    cudaError_t e = wait ? cudaEventSynchronize(h->ev[h->snap_idx]) : cudaEventQuery(h->ev[h->snap_idx]);
+    if (e == cudaErrorNotReady) return SKB_OK;
+    h->snap_pending = false;
+    if (e != cudaSuccess) return cuda_fail(h, e, "snapshot");
+    return absorb(h, h->h_ctl[h->snap_idx]);
+}
+
 extern "C" skb_status sinkhorn_batch_step(skb_batch *h, int cycles)
 {
     if (!h) return SKB_ERR_NULL;
     if (cycles < 0) return fail(h, SKB_ERR_VALUE, "cycles must be >= 0");
-    for (int i = 0; i < cycles && !h->finished; ++i) enqueue_cycle(h);
-    cudaError_t e = cudaGetLastError();
+    skb_status st = poll_snapshot(h, false);
+    if (st != SKB_OK) return st;
+    cudaError_t e;
+    if (cycles_in_one_launch(h)) {
+        for (int left = cycles; left > 0 && !h->finished; left -= MAX_CYCLES_IN_LAUNCH)
+            enqueue_cycles_launch(h, left < MAX_CYCLES_IN_LAUNCH ? left : MAX_CYCLES_IN_LAUNCH);
+    } else {
+        for (int i = 0; i < cycles && !h->finished; ++i) {
+            enqueue_cycle(h);
+            if (h->profiling && h->pev_used + PHASE_EVENTS_PER_CYCLE > (int)h->pev.size() &&
+                (e = harvest_phases(h)) != cudaSuccess) return cuda_fail(h, e, "step (phase timing)");
+        }
+    }
+    if (!h->snap_pending && cycles > 0) {
+        h->snap_idx ^= 1;
+        if ((e = cudaMemcpyAsync(&h->h_ctl[h->snap_idx], h->dev.ctl, sizeof(Ctl), cudaMemcpyDeviceToHost, h->stream)) != cudaSuccess ||
+            (e = cudaEventRecord(h->ev[h->snap_idx], h->stream)) != cudaSuccess) return cuda_fail(h, e, "step");
+        h->snap_pending = true;
+    }
+    e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(h, e, "step");
     return SKB_OK;
 }
@@ -338,12 +463,20 @@ extern "C" skb_status sinkhorn_batch_drain(skb_batch *h, int *cycles_run)
 {
     if (!h) return SKB_ERR_NULL;
     cudaError_t e;
+    {
+        skb_status st0 = poll_snapshot(h, true);
+        if (st0 != SKB_OK) { cudaStreamSynchronize(h->stream); return st0; }
+    }
     int chunk = 2, snap = 0, rounds = 0;
     bool have_prev = false;
+    const bool multi = cycles_in_one_launch(h);
+    const int chunk_max = multi ? 32 : 16;
     // every lane is retired by the audit that follows cycle max_iter; STATIC needs one more pass
     const long long hard_cap = (long long)h->cfg.max_iter + 4;
     while (!h->finished) {
-        for (int i = 0; i < chunk; ++i) enqueue_cycle(h);
+        if (multi) enqueue_cycles_launch(h, chunk);
+        else for (int i = 0; i < chunk; ++i) enqueue_cycle(h);
+        if (h->profiling && (e = harvest_phases(h)) != cudaSuccess) return cuda_fail(h, e, "drain (phase timing)");
         if ((e = cudaMemcpyAsync(&h->h_ctl[snap], h->dev.ctl, sizeof(Ctl), cudaMemcpyDeviceToHost, h->stream)) != cudaSuccess)
             return cuda_fail(h, e, "drain");
         if ((e = cudaEventRecord(h->ev[snap], h->stream)) != cudaSuccess) return cuda_fail(h, e, "drain");
@@ -356,7 +489,7 @@ extern "C" skb_status sinkhorn_batch_drain(skb_batch *h, int *cycles_run)
         snap ^= 1;
         // grow the chunk every other round: cycles enqueued past completion are empty launches that
         // still have to drain, which matters for batches that finish within a dozen cycles
-        if (chunk < 16 && (++rounds & 1) == 0) chunk *= 2;
+        if (chunk < chunk_max && (++rounds & 1) == 0) chunk *= 2;
         if (h->enqueued > hard_cap + 64) break;
     }
     if ((e = cudaStreamSynchronize(h->stream)) != cudaSuccess) return cuda_fail(h, e, "drain");
@@ -422,12 +555,17 @@ extern "C" skb_status sinkhorn_batch_residuals(skb_batch *h, float *r_row, float
 }
 
 extern "C" skb_status sinkhorn_batch_stats(skb_batch *h, long long *slots, int *cycles, int *widths,
-                                           int widths_cap, long long *pair_terms)
+                                           int widths_cap, long long *pair_terms, float *phase_ms)
 {
     if (!h) return SKB_ERR_NULL;
     Ctl c;
     skb_status st = read_ctl(h, &c);
     if (st != SKB_OK) return st;
+    if (h->profiling) {
+        cudaError_t e = harvest_phases(h);
+        if (e != cudaSuccess) return cuda_fail(h, e, "stats (phase timing)");
+    }
+    if (phase_ms) for (int i = 0; i < SKB_N_PHASES; ++i) phase_ms[i] = h->phase_ms[i];
     if (slots) *slots = c.slots;
     if (cycles) *cycles = c.cycle;
     if (pair_terms) *pair_terms = c.pair_terms;
@@ -437,6 +575,20 @@ extern "C" skb_status sinkhorn_batch_stats(skb_batch *h, long long *slots, int *
         cudaError_t e = cudaMemcpy(widths, h->dev.widths, (size_t)k * sizeof(int), cudaMemcpyDeviceToHost);
         if (e != cudaSuccess) return cuda_fail(h, e, "stats");
     }
+    return SKB_OK;
+}
+
+extern "C" skb_status sinkhorn_batch_cycle_trace(skb_batch *h, float *update_ms, int cap, int *count)
+{
+    if (!h || !count) return SKB_ERR_NULL;
+    if (h->profiling) {
+        cudaError_t e = cudaStreamSynchronize(h->stream);
+        if (e == cudaSuccess) e = harvest_phases(h);
+        if (e != cudaSuccess) return cuda_fail(h, e, "cycle_trace");
+    }
+    const int n = (int)h->cycle_update_ms.size();
+    *count = n;
+    if (update_ms) for (int i = 0; i < n && i < cap; ++i) update_ms[i] = h->cycle_update_ms[i];
     return SKB_OK;
 }
 
@@ -467,14 +619,23 @@ extern "C" skb_status sinkhorn_batch_profile_update(skb_batch *h, int leg, int r
 {
     if (!h || !ms_per_launch) return SKB_ERR_NULL;
     if ((leg != LEG_F && leg != LEG_G) || reps < 1) return fail(h, SKB_ERR_VALUE, "leg must be 0 or 1 and reps >= 1");
+    Ctl now;
+    skb_status st0 = read_ctl(h, &now);
+    if (st0 != SKB_OK) return st0;
+    if (now.done || now.static_final) return fail(h, SKB_ERR_STATE, "no lane is running: an update launch would return at once");
     cudaEvent_t a, b;
     cudaError_t e;
     if ((e = cudaEventCreate(&a)) != cudaSuccess) return cuda_fail(h, e, "profile");
     if ((e = cudaEventCreate(&b)) != cudaSuccess) { cudaEventDestroy(a); return cuda_fail(h, e, "profile"); }
+    // dry-run launches: the leg does all of its pair work and its row epilogue but stores no potential
+    // and adds no residual term, so the batch's state is exactly what it was
+    const Dev saved = h->dev;
+    h->dev.dry_run = 1;
     launch_leg(h, leg, h->known_width);          // warm-up
     cudaEventRecord(a, h->stream);
     for (int i = 0; i < reps; ++i) launch_leg(h, leg, h->known_width);
     cudaEventRecord(b, h->stream);
+    h->dev = saved;
     e = cudaEventSynchronize(b);
     float ms = 0.f;
     if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, a, b);
@@ -550,7 +711,7 @@ extern "C" skb_status sinkhorn_batch_solve_host(const void *x, const void *y, co
         if (e == cudaSuccess) e = cudaStreamSynchronize(st);
         if (e != cudaSuccess) rc = cuda_fail(nullptr, e, "solve_host (copy out)");
     }
-    if (rc == SKB_OK && (slots || cycles)) rc = sinkhorn_batch_stats(h, slots, cycles, nullptr, 0, nullptr);
+    if (rc == SKB_OK && (slots || cycles)) rc = sinkhorn_batch_stats(h, slots, cycles, nullptr, 0, nullptr, nullptr);
     if (rc != SKB_OK && h) g_create_err = h->err;
     sinkhorn_batch_destroy(h);
     return rc;
@@ -560,6 +721,7 @@ extern "C" void sinkhorn_batch_destroy(skb_batch *h)
 {
     if (!h) return;
     if (h->stream || h->h_ctl) cudaStreamSynchronize(h->stream);
+    for (cudaEvent_t ev : h->pev) if (ev) cudaEventDestroy(ev);
     if (h->h_ctl && h->ev[0] && h->ev[1]) {
         HostRes r; r.pinned = h->h_ctl; r.ev[0] = h->ev[0]; r.ev[1] = h->ev[1]; r.device = h->res_device;
         host_res_put(r);

@@ -6,10 +6,12 @@
 //             ballot / prefix-sum scan, records depth, status and residuals of retirees
 //             (completion depth l_t, Eq. 6), pairs every hole left below the new width
 //             with a survivor from above it, and advances the counters of Eq. 7.
+//  warm       replaces the cold potentials by a caller's proposal (Section "Initialization and
+//             repeated couplings"), before the first cycle.
 //  emit_move  writes retirees' potentials to the result buffers in the caller's units and
-//             copies each paired survivor's state into its hole ("physically compacts all
-//             candidate-indexed state", Section "Screen, verify, and compact").  Holes and
-//             sources are disjoint slot sets, so the in-place copies cannot race.
+//             moves every slot-indexed array of a paired survivor into the hole it fills
+//             (Section "Screen, verify, and compact").  Holes and sources are disjoint slot
+//             sets, so the in-place copies cannot race.
 //  gather     potentials in original lane order (retired lanes from the result buffers,
 //             running lanes from their slots).
 #include "skb_device.cuh"
@@ -126,6 +128,36 @@ __global__ void prep_kernel(const Dev P, const void *xin, const void *yin, const
     }
 }
 
+// Warm proposal: potentials in the caller's units -> the kernels' representation of both buffers
+// (same formulas as the cold start in prep_kernel, with phi = s f0 and gam = s g0 instead of 0).
+// Runs before the first cycle, when slot t still holds lane t.
+template <typename T>
+__global__ void warm_kernel(const Dev P, const double *f0, const double *g0)
+{
+    const int slot = blockIdx.y, side = blockIdx.z;
+    const int npts = side ? P.m : P.n, pp = side ? P.mp : P.np;
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= npts) return;
+    const double *src = side ? g0 : f0;
+    if (!src) return;
+    const double v = src[(size_t)slot * npts + i];
+    if (!isfinite(v)) { atomicOr(&P.ctl->error, ERR_VALUE); return; }
+    const int form = (sizeof(T) == 8) ? (int)FORM_DOT : P.form[slot];
+    const size_t o = (size_t)slot * pp + i;
+    const double pot = P.scale[slot] * v;
+    T hi, lo;
+    if (form == FORM_DOT) { hi = (T)(pot - (side ? P.sqy : P.sqx)[o]); lo = T(0); }
+    else { hi = (T)pot; lo = (T)(pot - (double)hi); }
+    if (!side) {
+        P.phi[0][o] = pot; P.phi[1][o] = pot;
+        reinterpret_cast<T *>(P.ft[0])[o] = hi; reinterpret_cast<T *>(P.ft[1])[o] = hi;
+        reinterpret_cast<T *>(P.fl[0])[o] = lo; reinterpret_cast<T *>(P.fl[1])[o] = lo;
+    } else {
+        P.gam[o] = pot;
+        reinterpret_cast<T *>(P.gt)[o] = hi; reinterpret_cast<T *>(P.gl)[o] = lo;
+    }
+}
+
 // ---------------------------------------------------------------- plan
 constexpr int PLAN_THREADS = 1024;   // upper bound; the launch sizes the block to the width
 
@@ -150,7 +182,7 @@ __device__ __forceinline__ void block_scan3(int f0, int f1, int f2, int (&ex)[3]
 }
 
 template <typename T>
-__device__ __forceinline__ void emit_move_one(const Dev &P, const Ctl &c, const int r);
+__device__ __forceinline__ void emit_move_one(const Dev &P, const Ctl &c, const int r, const int tid, const int nth);
 
 // FUSE: the same block also emits and moves the lanes it retires (see launch_plan).
 template <typename T, bool FUSE>
@@ -182,7 +214,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_kernel(const Dev P)
             __syncthreads();
             Ctl cc = c;
             cc.emit_parity = c.parity;
-            for (int r = 0; r < P.W; ++r) emit_move_one<T>(P, cc, r);
+            for (int r = 0; r < P.W; ++r) emit_move_one<T>(P, cc, r, tid, NT);
         }
         return;
     }
@@ -308,7 +340,96 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_kernel(const Dev P)
         __syncthreads();                                  // the lists and per-slot scalars above are this block's own writes
         Ctl cc = c;
         cc.emit_parity = c.parity;
-        for (int r = 0; r < nret; ++r) emit_move_one<T>(P, cc, r);
+        for (int r = 0; r < nret; ++r) emit_move_one<T>(P, cc, r, tid, NT);
+    }
+}
+
+// Planner after a multi-cycle launch (lane_cycles_kernel): the lanes that passed inside the launch
+// have written their own depth, status, residuals and potentials; what is left is the accounting of
+// Eq. 6-8 for all `K` cycles of the launch at once - widths A_k, slots, pair terms - the pairing of
+// holes below the new width with survivors from above it, and the advance of the control block.
+template <typename T, bool FUSE>
+__global__ void __launch_bounds__(PLAN_THREADS) plan_cycles_kernel(const Dev P, const int K)
+{
+    __shared__ int wsum[PLAN_THREADS / 32][3];
+    __shared__ int left_at[MAX_CYCLES_IN_LAUNCH];   // lanes that left at the audit of the state after k0 + j cycles
+    __shared__ int checks_s;
+    pdl_enter();
+    const Ctl c = *P.ctl;
+    const int tid = threadIdx.x, NT = blockDim.x;
+    if (c.done) { if (tid == 0) P.ctl->n_retire = 0; return; }
+    const int k0 = c.cycle, A = c.n_phys;
+    for (int j = tid; j < K; j += NT) left_at[j] = 0;
+    if (tid == 0) checks_s = 0;
+    __syncthreads();
+    int nchk = 0;
+    for (int s = tid; s < A; s += NT) {
+        const int r = P.ret_at[s];
+        if (r > 0) atomicAdd(&left_at[r - 1 - k0], 1);
+        nchk += P.n_checks[s];
+        P.rsum_row[s] = 0ull; P.rsum_col[s] = 0ull;      // between launches the residual sums are zero
+    }
+    for (int off = 16; off > 0; off >>= 1) nchk += __shfl_down_sync(0xffffffffu, nchk, off);
+    if ((tid & 31) == 0 && nchk) atomicAdd(&checks_s, nchk);
+    __syncthreads();
+    int nret = 0;
+    for (int j = 0; j < K; ++j) nret += left_at[j];
+    const int Anew = A - nret;
+    const int parity_new = c.parity ^ (K & 1);       // survivors ran all K cycles
+    // ordered lists: holes below the new width, survivors at or above it
+    int base[3] = {0, 0, 0};
+    for (int s0 = 0; s0 < (nret > 0 ? A : 0); s0 += NT) {
+        const int s = s0 + tid;
+        const int r = (s < A && P.ret_at[s] > 0) ? 1 : 0;
+        const int hole = r && s < Anew;
+        const int fill = (s < A) && !r && s >= Anew;
+        int ex[3], tot[3];
+        block_scan3(r, hole, fill, ex, tot, wsum);
+        if (hole) P.hole_list[base[1] + ex[1]] = s;
+        if (fill) P.fill_list[base[2] + ex[2]] = s;
+        base[0] += tot[0]; base[1] += tot[1]; base[2] += tot[2];
+        __syncthreads();
+    }
+    __threadfence_block();
+    __syncthreads();
+    const int nholes = base[1];
+    for (int h = tid; h < nholes; h += NT) {
+        const int dst = P.hole_list[h], src = P.fill_list[h];
+        P.ret_slot[h] = dst; P.ret_lane[h] = -1; P.ret_src[h] = src; P.ret_scale[h] = 1.0;   // move only
+        P.lane_id[dst] = P.lane_id[src];
+        P.scale[dst] = P.scale[src];
+        P.form[dst] = P.form[src];
+        P.nonfinite[dst] = 0;
+    }
+    for (int s = tid; s < A; s += NT) { P.ret_at[s] = 0; P.n_checks[s] = 0; }
+    if (tid == 0) {
+        Ctl *g = P.ctl;
+        const long long nm = (long long)P.n * P.m;
+        long long slots = 0, terms = (long long)checks_s * nm;
+        int w = A, ran = 0;
+        for (int j = 0; j < K; ++j) {
+            terms += (long long)w * nm;              // the f-leg whose epilogue screened the state after k0 + j cycles
+            w -= left_at[j];
+            if (w == 0) break;
+            if (k0 + j < P.max_iter + 1) P.widths[k0 + j] = w;      // cycle k0 + j + 1 ran at width w
+            slots += w;
+            terms += (long long)w * nm;              // its g-leg
+            ++ran;
+        }
+        g->cycle = k0 + ran;
+        g->parity = parity_new;
+        g->emit_parity = parity_new ^ 1;             // the move copies the OTHER buffer: the survivors' current row potentials
+        g->n_phys = Anew; g->n_running = Anew;
+        g->n_retire = FUSE ? 0 : nholes;
+        g->slots += slots;
+        g->pair_terms += terms;
+        if (Anew == 0) g->done = 1;
+    }
+    if (FUSE && nholes > 0) {
+        __syncthreads();
+        Ctl cc = c;
+        cc.emit_parity = parity_new ^ 1;
+        for (int r = 0; r < nholes; ++r) emit_move_one<T>(P, cc, r, tid, NT);
     }
 }
 
@@ -318,32 +439,52 @@ __global__ void __launch_bounds__(256) emit_move_kernel(const Dev P)
 {
     pdl_enter();
     const Ctl c = *P.ctl;
-    for (int r = blockIdx.y; r < c.n_retire; r += gridDim.y) emit_move_one<T>(P, c, r);
+    const int nret = c.n_retire;
+    if (nret <= 0) return;
+    // The launch's blocks are dealt out among the retirees of this audit (usually one or two): a move
+    // is a plain copy of up to a few MB and should have the whole machine's loads in flight.
+    const int nb = gridDim.x, b = blockIdx.x;
+    const int per = nb / nret;
+    if (per >= 1) {
+        const int r = b / per;
+        if (r < nret) emit_move_one<T>(P, c, r, (b % per) * blockDim.x + threadIdx.x, per * blockDim.x);
+    } else {
+        for (int r = b; r < nret; r += nb) emit_move_one<T>(P, c, r, threadIdx.x, blockDim.x);
+    }
 }
 
+// Retiree r of the list: `nth` threads (this one is number `tid`) write its outputs and, if its slot
+// is a hole below the new width, copy the paired survivor's state into it.
 template <typename T>
-__device__ __forceinline__ void emit_move_one(const Dev &P, const Ctl &c, const int r)
+__device__ __forceinline__ void emit_move_one(const Dev &P, const Ctl &c, const int r, const int tid, const int nth)
 {
     const int slot = P.ret_slot[r], lane = P.ret_lane[r], src = P.ret_src[r];
     const double inv_s = 1.0 / P.ret_scale[r];
-    const int tid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
     const int ep = c.emit_parity;
-    // emit: potentials of the audited state in the caller's units (f = phi / s)
-    for (int i = tid; i < P.n; i += nth)
-        P.f_out[(size_t)lane * P.n + i] = P.phi[ep][(size_t)slot * P.np + i] * inv_s;
+    // emit: potentials of the audited state in the caller's units (f = phi / s); lane < 0: the lane
+    // in the hole wrote its own outputs when it left (multi-cycle launches), only the move is left
+    if (lane >= 0)
+        for (int i = tid; i < P.n; i += nth)
+            P.f_out[(size_t)lane * P.n + i] = P.phi[ep][(size_t)slot * P.np + i] * inv_s;
     for (int j = tid; j < P.m; j += nth) {
         // the hole's own g is read before the survivor's g is copied over it (same thread)
-        P.g_out[(size_t)lane * P.m + j] = P.gam[(size_t)slot * P.mp + j] * inv_s;
+        if (lane >= 0) P.g_out[(size_t)lane * P.m + j] = P.gam[(size_t)slot * P.mp + j] * inv_s;
         if (src >= 0) P.gam[(size_t)slot * P.mp + j] = P.gam[(size_t)src * P.mp + j];
     }
-    if (tid == 0) P.emitted[lane] = 1;
+    if (tid == 0 && lane >= 0) P.emitted[lane] = 1;
     if (src < 0) return;
     // move the survivor in slot `src` into the hole `slot` (16-byte vector copies)
     auto copy = [&](void *base, size_t bytes_per_lane) {
         const uint4 *s4 = reinterpret_cast<const uint4 *>((const char *)base + (size_t)src * bytes_per_lane);
         uint4 *d4 = reinterpret_cast<uint4 *>((char *)base + (size_t)slot * bytes_per_lane);
         const size_t nv = bytes_per_lane / 16;
-        for (size_t v = tid; v < nv; v += nth) d4[v] = s4[v];
+        for (size_t v = tid; v < nv; v += 4 * (size_t)nth) {       // four loads in flight per thread
+            uint4 a[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) if (v + (size_t)u * nth < nv) a[u] = s4[v + (size_t)u * nth];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) if (v + (size_t)u * nth < nv) d4[v + (size_t)u * nth] = a[u];
+        }
     };
     const int np_ = ep ^ 1;   // buffer that holds the survivors' current row potentials
     if (P.tensor) {
@@ -411,6 +552,13 @@ void launch_prep(const Dev &P, const void *x, const void *y, const float *a, con
     if (P.compute_f64) prep_kernel<double><<<grid, 128, 0, st>>>(P, x, y, a, b);
     else prep_kernel<float><<<grid, 128, 0, st>>>(P, x, y, a, b);
 }
+void launch_warm(const Dev &P, const double *f0, const double *g0, cudaStream_t st)
+{
+    const int pp = P.n > P.m ? P.n : P.m;
+    dim3 grid((pp + 127) / 128, P.W, 2);
+    if (P.compute_f64) warm_kernel<double><<<grid, 128, 0, st>>>(P, f0, g0);
+    else warm_kernel<float><<<grid, 128, 0, st>>>(P, f0, g0);
+}
 // Bytes one retirement can move (a survivor's whole state into the hole) plus what it emits.
 static size_t lane_state_bytes(const Dev &P)
 {
@@ -442,16 +590,30 @@ int launch_plan(const Dev &P, int width, cudaStream_t st)
     }
     return 1;
 }
+int launch_plan_cycles(const Dev &P, int width, int cycles, cudaStream_t st)
+{
+    int nt = (width + 31) / 32 * 32;
+    const bool fuse = plan_fuses_move(P, width);
+    nt = nt < (fuse ? 256 : 128) ? (fuse ? 256 : 128) : (nt > PLAN_THREADS ? PLAN_THREADS : nt);
+    if (fuse) {
+        if (P.compute_f64) launch_pdl(plan_cycles_kernel<double, true>, dim3(1), dim3(nt), 0, st, P, cycles);
+        else launch_pdl(plan_cycles_kernel<float, true>, dim3(1), dim3(nt), 0, st, P, cycles);
+    } else {
+        launch_pdl(plan_cycles_kernel<float, false>, dim3(1), dim3(nt), 0, st, P, cycles);
+    }
+    return 1;
+}
 int launch_emit_move(const Dev &P, int width, cudaStream_t st)
 {
     if (plan_fuses_move(P, width)) return 0;
     if (width < 1) width = 1;
-    const size_t bytes = (size_t)P.DP * (P.np + P.mp) * (P.compute_f64 ? 8 : 4);
-    int gx = (int)(bytes / (256 * 16 * 4)) + 1;
-    if (gx > 64) gx = 64;
-    dim3 grid(gx, width > 128 ? 128 : width);
-    if (P.compute_f64) launch_pdl(emit_move_kernel<double>, grid, dim3(256), 0, st, P);
-    else launch_pdl(emit_move_kernel<float>, grid, dim3(256), 0, st, P);
+    // one block per 16 KB of a lane's state (four 16-byte vectors per thread and pass), at least one
+    // block per lane that could retire at once, at most four blocks per SM
+    long long blocks = (long long)((lane_state_bytes(P) + 16383) / 16384);
+    if (blocks < (width > 128 ? 128 : width)) blocks = width > 128 ? 128 : width;
+    if (blocks > 148 * 4) blocks = 148 * 4;
+    if (P.compute_f64) launch_pdl(emit_move_kernel<double>, dim3((unsigned)blocks), dim3(256), 0, st, P);
+    else launch_pdl(emit_move_kernel<float>, dim3((unsigned)blocks), dim3(256), 0, st, P);
     return 1;
 }
 void launch_gather(const Dev &P, void *f, void *g, bool f64, cudaStream_t st)

@@ -54,6 +54,8 @@ struct Dev {
     int W, n, m, d, np, mp, DP;
     int mode, max_iter, audit_every, xy_bf16, compute_f64, cost_form, tensor;
     int early_exit;           // MASKED only: CTAs of a frozen lane return at once (an extra arm, not the paper's mask control)
+    int dry_run;              // measurement launches: a leg computes everything but stores no potential and adds no residual term
+    int audit_initial;        // warm proposals: the state before the first cycle is audited too (a lane may retire at depth 0)
     double form_threshold;    // scaled squared radius above which a lane uses the difference form
     double tol_screen, tol_stop;
     // slabs by slot
@@ -76,8 +78,11 @@ struct Dev {
     int *flag;                // screen-positive at this audit
     int *verdict;             // two-sided check passed
     int *nonfinite;
+    // multi-cycle launches: cycle count + 1 at which the lane in the slot left inside the launch
+    // (0 = still running), and the column checks it ran
+    int *ret_at, *n_checks;
     double *rrow, *rcol;      // residuals of the audited state
-    // marginal residuals of the audited state as fixed-point sums (units of 2^-50): every row block
+    // marginal residuals of the audited state as fixed-point sums (units of 2^-44): every row block
     // adds its part with one integer atomic, so the total is exact and independent of the order
     // of arrival; the plan kernel turns them into rrow / rcol / flag / verdict and clears them
     unsigned long long *rsum_row, *rsum_col;
@@ -103,7 +108,7 @@ struct Dev {
 __device__ __forceinline__ bool lane_flag(const Dev &P, const Ctl &c, const int slot)
 {
     const bool passed = P.state[slot] != 0;                  // MASKED: frozen; STATIC: already passed
-    const bool audited = c.cycle >= 1 && (c.cycle % P.audit_every) == 0;
+    const bool audited = (c.cycle >= 1 && (c.cycle % P.audit_every) == 0) || (c.cycle == 0 && P.audit_initial);
     const bool live = !(passed && (P.mode == MODE_MASKED || P.mode == MODE_STATIC));
     return audited && live && !P.nonfinite[slot] && (double)P.rsum_row[slot] * (1.0 / RSUM_SCALE) <= P.tol_screen;
 }

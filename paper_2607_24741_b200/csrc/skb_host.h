@@ -6,6 +6,20 @@
 namespace skb {
 
 // Launch with programmatic stream serialization allowed (the kernel must call pdl_enter()).
+//
+// Invariants the kernels of a cycle rely on (f-leg, column check, plan, emit/move, g-leg, in that
+// order on one stream):
+//  - every kernel executes griddepcontrol.wait in at least one block before it completes, so that
+//    "my predecessor has completed" implies "everything earlier in the stream has completed";
+//  - the control block is written by the plan kernel only, coordinates and the per-slot scalars by
+//    the plan and emit/move kernels only;
+//  - a kernel that reads state BEFORE its own wait (the SIMT f-leg: control block, row coordinates,
+//    row potentials; the column check: control block) may do so because the kernel that released it
+//    is a g-leg (of this batch or of another batch sharing the stream), and g-legs release their
+//    dependents only after their own wait: by then the plan and emit/move kernels before it are
+//    complete, and nothing between them and the early reader writes what it reads early;
+//  - kernels launched without the attribute (set-up, read-back, a caller's own kernels) neither
+//    start early nor release early, so they may sit anywhere in the stream.
 template <typename... KArgs, typename... Args>
 inline void launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args)
 {
@@ -24,7 +38,11 @@ struct Variant {
     int rows_per_cta;
     size_t smem;
     void (*launch)(const Dev &, int leg, int width, cudaStream_t);
+    // several whole cycles per launch, one thread-block cluster per lane; null where there is none
+    void (*launch_cycles)(const Dev &, int cycles, int width, cudaStream_t);
 };
+constexpr int MAX_CLUSTER_BLOCKS = 8;       // portable cluster size: a lane needs at most this many row blocks
+constexpr int MAX_CYCLES_IN_LAUNCH = 64;    // upper bound on the cycles one multi-cycle launch runs
 // Picks the variant for a shape (depends on the static shape only, so that every mode
 // and every run of the same batch uses the same reduction order).  Null if unsupported.
 const Variant *choose_variant(int W, int n, int m, int d, bool f64, bool fast_exp, int force_cs);
@@ -32,6 +50,7 @@ int padded_dim(int d);
 
 void launch_lane_stats(const Dev &P, const void *x, const void *y, const float *eps, double *max_radius, cudaStream_t st);
 void launch_prep(const Dev &P, const void *x, const void *y, const float *a, const float *b, cudaStream_t st);
+void launch_warm(const Dev &P, const double *f0, const double *g0, cudaStream_t st);
 int launch_plan(const Dev &P, int width, cudaStream_t st);        // both return the number of kernels launched
 // tensor-core update kernel (bf16 inputs, d a multiple of 64 up to 512)
 bool tc_eligible(int d, bool bf16);
@@ -41,6 +60,7 @@ void launch_retile(const void *src, void *dst, int W, int npts, int d, cudaStrea
 void launch_wait_probe(int *out, long long budget_clocks, cudaStream_t st);
 void launch_update_tc(const Dev &P, const void *maps, int leg, int width, cudaStream_t st);
 int launch_emit_move(const Dev &P, int width, cudaStream_t st);
+int launch_plan_cycles(const Dev &P, int width, int cycles, cudaStream_t st);
 void launch_gather(const Dev &P, void *f, void *g, bool f64, cudaStream_t st);
 void launch_gather_small(const Dev &P, int *depth, int *status, float *rrow, float *rcol, cudaStream_t st);
 

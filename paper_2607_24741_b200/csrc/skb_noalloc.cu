@@ -40,7 +40,7 @@ static __device__ __align__(256) unsigned char g_scratch[SKB_STATIC_SCRATCH_BYTE
 
 std::mutex g_mu;
 Scratch *g_dev_scratch[NA_MAX_DEVICES] = {};
-std::string g_err;
+thread_local std::string g_err;       // text of the calling thread's last failure; empty after a success
 
 __global__ void __launch_bounds__(NA_THREADS) row_residual_kernel(
     Scratch *sc, const float *x, const float *y, const float *a, const double *f, const double *g,
@@ -127,5 +127,6 @@ extern "C" skb_status sinkhorn_row_residual_static(const float *x, const float *
     row_residual_kernel<<<grid, NA_THREADS, 0, st>>>(sc, x, y, a, f, g, eps, n, m, d, r_row);
     e = cudaGetLastError();
     if (e != cudaSuccess) return fail(SKB_ERR_CUDA, std::string("launch: ") + cudaGetErrorString(e));
+    g_err.clear();
     return SKB_OK;
 }

@@ -62,9 +62,36 @@ static void launch_update(const Dev &P, int leg, int width, cudaStream_t st)
     launch_pdl(update_kernel<T, DP, CS, XF>, dim3((nrows + rb - 1) / rb, lanes), dim3(UPD_THREADS), smem, st, P, leg);
 }
 
+// Several whole cycles per launch: grid.x = row blocks of the larger cloud = one thread-block
+// cluster per lane (the caller has checked that a lane has at most MAX_CLUSTER_BLOCKS of them).
+template <typename T, int DP, int CS, int XF>
+static void launch_cycles(const Dev &P, int cycles, int width, cudaStream_t st)
+{
+    static bool attr_set = false;
+    const size_t smem = 2 * (size_t)(DP + 2) * TileCols<T, DP, CS>::value * sizeof(T);
+    if (!attr_set) {
+        cudaFuncSetAttribute(lane_cycles_kernel<T, DP, CS, XF>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        attr_set = true;
+    }
+    const int rb = (UPD_THREADS / 32) * Tune<T, DP>::R * (32 / CS);
+    const int mx = P.n > P.m ? P.n : P.m;
+    const int nc = (mx + rb - 1) / rb;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(nc, width < 1 ? 1 : width); cfg.blockDim = dim3(UPD_THREADS);
+    cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = nc; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 2;
+    cudaLaunchKernelEx(&cfg, lane_cycles_kernel<T, DP, CS, XF>, P, cycles);
+}
+
 #define SKB_V(T, F64, XF, DP, CS) \
     { F64, XF, DP, Tune<T, DP>::R, CS, (UPD_THREADS / 32) * Tune<T, DP>::R * (32 / CS), \
-      2 * (size_t)(DP + 2) * TileCols<T, DP, CS>::value * sizeof(T), &launch_update<T, DP, CS, XF> }
+      2 * (size_t)(DP + 2) * TileCols<T, DP, CS>::value * sizeof(T), &launch_update<T, DP, CS, XF>, \
+      &launch_cycles<T, DP, CS, XF> }
 #define SKB_ROW(DP) \
     SKB_V(float, 0, 0, DP, 1), SKB_V(float, 0, 0, DP, 4), SKB_V(float, 0, 0, DP, 32), \
     SKB_V(double, 1, 0, DP, 1), SKB_V(double, 1, 0, DP, 4), SKB_V(double, 1, 0, DP, 32), \
@@ -88,9 +115,9 @@ static void launch_bigd(const Dev &P, int leg, int width, cudaStream_t st)
 
 // DP = 0 marks the large-d kernels: the padded dimension is d rounded up to the chunk size
 static const Variant g_bigd[] = {
-    {0, 0, 0, 4, 4, BIGD_RB, 2 * (size_t)BIGD_KC * (BIGD_RB + BIGD_TJ) * 4, &launch_bigd<float, 0>},
-    {1, 0, 0, 4, 4, BIGD_RB, 2 * (size_t)BIGD_KC * (BIGD_RB + BIGD_TJ) * 8, &launch_bigd<double, 0>},
-    {1, 1, 0, 4, 4, BIGD_RB, 2 * (size_t)BIGD_KC * (BIGD_RB + BIGD_TJ) * 8, &launch_bigd<double, 1>},
+    {0, 0, 0, 4, 4, BIGD_RB, 2 * (size_t)BIGD_KC * (BIGD_RB + BIGD_TJ) * 4, &launch_bigd<float, 0>, nullptr},
+    {1, 0, 0, 4, 4, BIGD_RB, 2 * (size_t)BIGD_KC * (BIGD_RB + BIGD_TJ) * 8, &launch_bigd<double, 0>, nullptr},
+    {1, 1, 0, 4, 4, BIGD_RB, 2 * (size_t)BIGD_KC * (BIGD_RB + BIGD_TJ) * 8, &launch_bigd<double, 1>, nullptr},
 };
 
 int padded_dim(int d)

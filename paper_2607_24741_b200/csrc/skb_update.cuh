@@ -297,7 +297,11 @@ __device__ __forceinline__ void stream_f32(float *sm, const float *colc, const f
                     float mt = fmaxf(a[0], a[1]);
 #pragma unroll
                     for (int e = 2; e < CW; ++e) mt = fmaxf(mt, a[e]);
-                    if (mt > mx[r] + 8.0f) {
+                    // the row's OWN sum decides (not a sibling row's that happened to trip the branch): a
+                    // row's bits must not depend on which rows share its thread
+                    float q0, q1;
+                    unpack2(es[r], q0, q1);
+                    if (!(q0 + q1 <= 1024.f)) {
                         const float mn = ceilf(mt);
                         const float fac = pow2i(mx[r] - mn);
                         float t0, t1;
@@ -405,7 +409,7 @@ __device__ __forceinline__ void stream_f64(double *sm, const double *colc, const
                         double mt = acc[r][0];
 #pragma unroll
                         for (int e = 1; e < CW; ++e) mt = fmax(mt, acc[r][e]);
-                        if (mt > md[r] + 8.0) {
+                        if (!(e2[r] <= 1024.f)) {                         // the row's own sum decides, never a sibling's
                             const float mn = ceilf((float)mt) + 1.0f;      // +1: the fp32 copy may round down
                             const float fac = pow2i(mx[r] - mn);
                             ts[r] *= fac;
@@ -520,7 +524,7 @@ __device__ __forceinline__ void finish_rows(const Dev &P, const Ctl &c, const in
     const int nrows = (leg == LEG_F) ? P.n : P.m;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const bool frozen = (P.mode == MODE_MASKED) && P.state[slot] != 0;
-    const bool writes = !frozen && leg != LEG_V;
+    const bool writes = !frozen && leg != LEG_V && !P.dry_run;
     unsigned long long term_sum = 0ull;
     for (int lr = tid; lr < RB; lr += THREADS) {
         const int i = blockIdx.x * RB + lr;
@@ -528,7 +532,7 @@ __device__ __forceinline__ void finish_rows(const Dev &P, const Ctl &c, const in
         const double term = finish_one_row<T>(P, c, leg, slot, form, i, row_m[lr], row_s[lr], row_h[lr], writes);
         if (leg != LEG_G) term_sum += residual_fixed(P, leg, slot, term, frozen);
     }
-    if (leg == LEG_G) return;
+    if (leg == LEG_G || P.dry_run) return;
 
     // fused marginal-residual reduction -> one exact total per lane
     unsigned long long *redu = reinterpret_cast<unsigned long long *>(red);
@@ -544,41 +548,30 @@ __device__ __forceinline__ void finish_rows(const Dev &P, const Ctl &c, const in
     }
 }
 
-// RR: rows per thread, 0 = the type's default.  Rows are independent and a row's arithmetic does
-// not depend on which thread holds it, so launches with different RR give the same bits.
-template <typename T, int DP, int CS, int XF, int RR = 0>
-__global__ void __launch_bounds__(UPD_THREADS) update_kernel(const Dev P, const int leg)
+// Shared-memory scratch of one leg besides the column tiles.
+template <int RB>
+struct LegScratch {
+    double row_s[RB];
+    float row_m[RB];
+    float row_h[RB];
+    double red[UPD_THREADS / 32];
+};
+
+// One leg for the row block blockIdx.x of the lane in `slot`: row operands, streaming reduction over
+// all columns, float64 epilogue, residual terms.  `c` supplies the cycle count and the buffer parity
+// of the state the leg starts from.  PDL_EARLY: this is an f-leg launched as a kernel of its own,
+// which reads its row operands while the kernel before it is still finishing and waits for it only
+// before the column terms.  A row's arithmetic does not depend on the thread that holds it, nor on
+// whether the leg runs as its own launch or inside the multi-cycle kernel below, so every way of
+// running it gives the same bits.
+template <typename T, int DP, int CS, int XF, int R, bool PDL_EARLY>
+__device__ __forceinline__ void run_leg(const Dev &P, const Ctl &c, const int leg, const int slot, T *sm,
+                                        LegScratch<(UPD_THREADS / 32) * R * (32 / CS)> &sc)
 {
-    constexpr int R = RR ? RR : Tune<T, DP>::R;
     constexpr int RG = 32 / CS;                  // row groups per warp
     constexpr int RW = R * RG;                   // rows per warp
     constexpr int NWARP = UPD_THREADS / 32;
     constexpr int RB = NWARP * RW;               // rows per CTA
-
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    T *sm = reinterpret_cast<T *>(smem_raw);
-    __shared__ double row_s[RB];
-    __shared__ float row_m[RB];
-    __shared__ float row_h[RB];
-    __shared__ double red[NWARP];
-
-    // Programmatic dependent launch.  The f-leg follows the g-leg, which writes neither the control
-    // block nor coordinates nor the row potentials: its control block, row coordinates and epilogue
-    // operands are read while that g-leg is still finishing, and only the column terms wait.  The
-    // other legs wait first; the g-leg releases its dependent (the next f-leg) only AFTER its own
-    // wait, so that an early f-leg can rely on the planner and the move being complete.
-    // (The column check also reads the control block early, then waits for the f-leg's verdict.)
-    const bool early = (leg == LEG_F);
-    if (leg == LEG_G) asm volatile("griddepcontrol.wait;" ::: "memory");
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    const Ctl c = *P.ctl;
-    if (leg == LEG_V) asm volatile("griddepcontrol.wait;" ::: "memory");
-    if (c.done) return;
-    const int slot = blockIdx.y;
-    if (slot >= c.n_phys) return;
-    if (P.early_exit && P.state[slot] != 0) return;     // early-exit mask arm: a frozen lane costs a launch slot only
-    if (leg != LEG_V && c.static_final) return;
-    if (leg == LEG_V && !(c.static_final || lane_flag(P, c, slot))) return;
 
     // roles: rows are x-points for the f-leg, y-points otherwise
     const bool rows_x = (leg == LEG_F);
@@ -629,7 +622,7 @@ __global__ void __launch_bounds__(UPD_THREADS) update_kernel(const Dev P, const 
 #pragma unroll
     for (int r = 0; r < R; ++r) ph[r] = (row0 + r < nrows && form == FORM_DIFF) ? (T)prow[row0 + r] : T(0);
 
-    if (early) asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (PDL_EARLY && leg == LEG_F) asm volatile("griddepcontrol.wait;" ::: "memory");
 
     float mx[R];
     double sd[R];
@@ -679,8 +672,12 @@ __global__ void __launch_bounds__(UPD_THREADS) update_kernel(const Dev P, const 
                 for (int r = 0; r < R; ++r)
                     low = low || (row0 + r < nrows && fabs(m0[r]) < 1.0e7 && !(sd[r] >= 0x1p-20));
                 if (!__syncthreads_or(low ? 1 : 0)) break;
+                // only the rows whose estimate failed start over from "minus infinity"; the others
+                // repeat the very same pass (same bits), so that a row's result does not depend on
+                // which rows share its block
 #pragma unroll
-                for (int r = 0; r < R; ++r) m0[r] = (double)NEG_BIG;
+                for (int r = 0; r < R; ++r)
+                    if (row0 + r < nrows && fabs(m0[r]) < 1.0e7 && !(sd[r] >= 0x1p-20)) m0[r] = (double)NEG_BIG;
                 continue;
             }
         }
@@ -689,13 +686,166 @@ __global__ void __launch_bounds__(UPD_THREADS) update_kernel(const Dev P, const 
     if (cs == 0) {
 #pragma unroll
         for (int r = 0; r < R; ++r) {
-            row_m[lrow0 + r] = mx[r];
-            row_s[lrow0 + r] = sd[r];
-            row_h[lrow0 + r] = (float)ph[r];
+            sc.row_m[lrow0 + r] = mx[r];
+            sc.row_s[lrow0 + r] = sd[r];
+            sc.row_h[lrow0 + r] = (float)ph[r];
         }
     }
     __syncthreads();
-    finish_rows<T, RB>(P, c, leg, slot, form, row_m, row_s, row_h, red);
+    finish_rows<T, RB>(P, c, leg, slot, form, sc.row_m, sc.row_s, sc.row_h, sc.red);
+}
+
+// RR: rows per thread, 0 = the type's default.  Rows are independent and a row's arithmetic does
+// not depend on which thread holds it, so launches with different RR give the same bits.
+template <typename T, int DP, int CS, int XF, int RR = 0>
+__global__ void __launch_bounds__(UPD_THREADS) update_kernel(const Dev P, const int leg)
+{
+    constexpr int R = RR ? RR : Tune<T, DP>::R;
+    constexpr int RB = (UPD_THREADS / 32) * R * (32 / CS);   // rows per CTA
+
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    T *sm = reinterpret_cast<T *>(smem_raw);
+    __shared__ LegScratch<RB> sc;
+
+    // Programmatic dependent launch.  The f-leg follows the g-leg, which writes neither the control
+    // block nor coordinates nor the row potentials: its control block, row coordinates and epilogue
+    // operands are read while that g-leg is still finishing, and only the column terms wait.  The
+    // other legs wait first; the g-leg releases its dependent (the next f-leg) only AFTER its own
+    // wait, so that an early f-leg can rely on the planner and the move being complete.
+    // (The column check also reads the control block early, then waits for the f-leg's verdict.)
+    const bool early = (leg == LEG_F);
+    if (leg == LEG_G) asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const Ctl c = *P.ctl;
+    if (leg == LEG_V) asm volatile("griddepcontrol.wait;" ::: "memory");
+    const int slot = blockIdx.y;
+    const bool idle = c.done || slot >= c.n_phys
+                      || (P.early_exit && P.state[slot] != 0)   // early-exit mask arm: a frozen lane costs a launch slot only
+                      || (leg != LEG_V && c.static_final)
+                      || (leg == LEG_V && !(c.static_final || lane_flag(P, c, slot)))
+                      || (int)blockIdx.x * RB >= (leg == LEG_F ? P.n : P.m);
+    if (idle) {
+        // Every kernel of the chain must wait at least once before it completes: a kernel's wait
+        // covers its immediate predecessor only, and "everything earlier in the stream has finished"
+        // follows from it only if that predecessor waited too.  An f-leg with nothing to do has not
+        // waited yet, so its first block does so here (a batch that is finished, or another batch's
+        // kernels in the same stream, would otherwise let later kernels overtake a running g-leg).
+        if (early && blockIdx.x == 0 && blockIdx.y == 0) asm volatile("griddepcontrol.wait;" ::: "memory");
+        return;
+    }
+    run_leg<T, DP, CS, XF, R, true>(P, c, leg, slot, sm, sc);
+}
+
+// ------------------------------------------------------------------ several cycles per launch
+// One thread-block CLUSTER per lane: block r of the cluster owns row block r of both clouds and the
+// cluster walks the lane through up to `cycles` whole cycles inside one launch -
+//     f-leg (with the row screen of the state before it) -> [column check if screen-positive] ->
+//     verdict -> retire, or g-leg and on to the next cycle
+// - so that a cycle costs two or three cluster barriers instead of a chain of five dependent
+// launches.  Lanes are independent problems (Eq. 2): clusters never wait for one another, and
+// inside a cluster the only synchronisation is the hardware cluster barrier, which every thread of
+// every block reaches on every path (all blocks of a cluster take the same decisions from the same
+// values).  Blocks hand the potentials to one another through global memory (the column terms are
+// read by cp.async, which bypasses L1, after the barrier's release/acquire).
+// A lane that passes the two-sided check (Eq. 5) writes its own outputs and leaves; the planner that
+// follows the launch does the accounting of Eq. 6-8 for all cycles of the launch at once and fills
+// the holes (Section "Screen, verify, and compact").  The legs are run_leg, so the bits are those
+// of the one-launch-per-leg path.
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ unsigned long long ld_cg_u64(const unsigned long long *p)
+{
+    unsigned long long v;
+    asm volatile("ld.global.cg.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ int ld_cg_s32(const int *p)
+{
+    int v;
+    asm volatile("ld.global.cg.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+template <typename T, int DP, int CS, int XF, int RR = 0>
+__global__ void __launch_bounds__(UPD_THREADS) lane_cycles_kernel(const Dev P, const int cycles)
+{
+    constexpr int R = RR ? RR : Tune<T, DP>::R;
+    constexpr int RB = (UPD_THREADS / 32) * R * (32 / CS);
+
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    T *sm = reinterpret_cast<T *>(smem_raw);
+    __shared__ LegScratch<RB> sc;
+
+    pdl_enter();
+    Ctl c = *P.ctl;                              // private copy: cycle and parity advance per lane below
+    const int slot = blockIdx.y;
+    if (c.done || slot >= c.n_phys) return;      // the whole cluster takes this exit together
+    const int tid = threadIdx.x;
+    const int lane_id = P.lane_id[slot];
+    const double inv_s = 1.0 / P.scale[slot];
+    unsigned long long seen_row = 0ull, seen_col = 0ull;     // totals already accounted for (the sums are only cleared at the end)
+    int checks = 0, retired_at = 0;
+
+    for (int it = 0; it < cycles; ++it) {
+        // f-leg of cycle k+1; its epilogue also yields the row residual of the state after k cycles
+        run_leg<T, DP, CS, XF, R, false>(P, c, LEG_F, slot, sm, sc);
+        cluster_sync_all();
+        const unsigned long long tot_row = ld_cg_u64(P.rsum_row + slot);
+        const double rr = (double)(tot_row - seen_row) * (1.0 / RSUM_SCALE);
+        seen_row = tot_row;
+        int nf = ld_cg_s32(P.nonfinite + slot);
+        const int k = c.cycle;
+        const bool audited = (k >= 1 && (k % P.audit_every) == 0) || (k == 0 && P.audit_initial);
+        const bool fl = audited && !nf && rr <= P.tol_screen;
+        double rc = 0.0;
+        if (fl) {                                // two-sided check: the column marginal, genuinely measured
+            run_leg<T, DP, CS, XF, R, false>(P, c, LEG_V, slot, sm, sc);
+            cluster_sync_all();
+            const unsigned long long tot_col = ld_cg_u64(P.rsum_col + slot);
+            rc = (double)(tot_col - seen_col) * (1.0 / RSUM_SCALE);
+            seen_col = tot_col;
+            nf = ld_cg_s32(P.nonfinite + slot);
+            ++checks;
+        }
+        const bool vd = !nf && fmax(rr, rc) <= P.tol_stop;
+        const bool limit = k >= P.max_iter;
+        int st = LANE_RUNNING;
+        if (nf) st = LANE_NONFINITE;
+        else if (fl && vd) st = LANE_DONE;
+        else if (limit) st = LANE_ITER_LIMIT;
+        if (st != LANE_RUNNING) {
+            // retire: this block's rows of the potentials of the audited state, in the caller's units
+            const double *phi = P.phi[c.parity] + (size_t)slot * P.np;
+            const double *gam = P.gam + (size_t)slot * P.mp;
+            for (int lr = tid; lr < RB; lr += UPD_THREADS) {
+                const int i = blockIdx.x * RB + lr;
+                if (i < P.n) P.f_out[(size_t)lane_id * P.n + i] = phi[i] * inv_s;
+                if (i < P.m) P.g_out[(size_t)lane_id * P.m + i] = gam[i] * inv_s;
+            }
+            if (blockIdx.x == 0 && tid == 0) {
+                P.res_row[lane_id] = rr;
+                P.res_col[lane_id] = fl ? rc : __longlong_as_double(0x7ff8000000000000LL);
+                P.depth[lane_id] = (limit && st != LANE_DONE) ? P.max_iter : k;
+                P.status[lane_id] = st;
+                P.emitted[lane_id] = 1;
+            }
+            retired_at = k + 1;
+            break;
+        }
+        c.cycle = k + 1;
+        c.parity ^= 1;
+        run_leg<T, DP, CS, XF, R, false>(P, c, LEG_G, slot, sm, sc);
+        cluster_sync_all();
+    }
+    // hand over to the planner: when the lane left (0 = still running) and how many column checks
+    // it ran.  The residual sums are left as they are (another block of the cluster may still be
+    // reading them); the planner clears them.
+    if (blockIdx.x == 0 && tid == 0) {
+        P.ret_at[slot] = retired_at;
+        P.n_checks[slot] = checks;
+    }
 }
 
 }  // namespace skb

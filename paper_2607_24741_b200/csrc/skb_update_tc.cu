@@ -717,7 +717,7 @@ update_tc_pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_cons
             const int i = rb * TC_BM + row;
             unsigned long long term = 0ull;
             if (i < nrows) {
-                const double tr = finish_one_row<float>(P, c, leg, slot, (int)FORM_DOT, i, m, sm, 0.f, !frozen && leg != LEG_V);
+                const double tr = finish_one_row<float>(P, c, leg, slot, (int)FORM_DOT, i, m, sm, 0.f, !frozen && leg != LEG_V && !P.dry_run);
                 if (leg != LEG_G) term = residual_fixed(P, leg, slot, tr, frozen);
             }
             if (leg != LEG_G) {
@@ -725,7 +725,7 @@ update_tc_pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_cons
                 for (int off = 16; off > 0; off >>= 1) term += __shfl_down_sync(0xffffffffu, term, off);
                 if (lane == 0) red[fw] = term;
                 asm volatile("bar.sync 4, 128;" ::: "memory");
-                if (row == 0) finish_lane_residual(P, leg, slot, ((red[0] + red[1]) + red[2]) + red[3]);
+                if (row == 0 && !P.dry_run) finish_lane_residual(P, leg, slot, ((red[0] + red[1]) + red[2]) + red[3]);
                 asm volatile("bar.sync 4, 128;" ::: "memory");          // red[] is free again
             }
         }

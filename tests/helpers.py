@@ -1,12 +1,32 @@
 """Shared helpers for the GPU parity tests: run a workload through the C-ABI binding and
-through the CPU oracle on the same arrays, and compare the way the acceptance bar says."""
+through the CPU oracle on the same arrays, and compare the way the acceptance bar says.
+
+Every comparison adds one entry to LEDGER: how many lanes were compared, how many stopped one
+audit away from the oracle (each with the oracle's margin at the disputed audit), the largest
+potential error and the largest residual deviations.  tests/test_yy_parity_ledger.py bounds
+the totals and writes the table out, so that no near-threshold lane goes unreported."""
 from __future__ import annotations
+
+import os
+from concurrent.futures import ThreadPoolExecutor
 
 import numpy as np
 
+LEDGER: list[dict] = []
+
+# The band inside which the acceptance bar itself allows a lane to stop one audit away.
+NORTH_STAR_BAND = 1e-6
+
+# |r_col reported by the GPU - float64 column residual of the potentials it emitted|.  After a
+# g-leg the column marginal is current (Eq. 4), so both are pure arithmetic error: the column
+# check repeats the g-leg's sums in the GPU's arithmetic and finds (almost) nothing, while the
+# float64 evaluation sees the g-leg's own error: 2^-22 per fp32 exponential, plus half an ulp of
+# the scaled cost (up to 512, i.e. 2^-15 in the exponent) when the exponents are fp32 too.
+RCOL_ABS = {"f64": 1e-10, "mixed": 2e-6, "f32": 5e-5, "tensor": 5e-5}
+
 
 def run_gpu(w, mode="active", compute="auto", column_split=0, audit_every=1, tol_screen=0.0,
-            max_iter=None, tol=None, widths_cap=200000, cost_form=0):
+            max_iter=None, tol=None, widths_cap=200000, cost_form=0, warm=None, audit_initial=False):
     import torch
     from paper_2607_24741_b200 import binding as B
     dev = torch.device("cuda:0")
@@ -20,6 +40,9 @@ def run_gpu(w, mode="active", compute="auto", column_split=0, audit_every=1, tol
                          audit_every=audit_every, tol_screen=tol_screen, column_split=column_split,
                          cost_form=cost_form)
     try:
+        if warm is not None:
+            sb.warm_start(torch.from_numpy(warm[0]).to(dev), torch.from_numpy(warm[1]).to(dev),
+                          audit_initial=audit_initial)
         cycles = sb.drain()
         f, g = sb.potentials(f64=True)
         f32, g32 = sb.potentials()
@@ -27,11 +50,12 @@ def run_gpu(w, mode="active", compute="auto", column_split=0, audit_every=1, tol
         rr, rc = sb.residuals()
         stats = sb.stats(widths_cap=widths_cap)
         left = sb.active()
+        arith = sb.arithmetic()
     finally:
         sb.close()
     return dict(f=f.cpu().numpy(), g=g.cpu().numpy(), f32=f32.cpu().numpy(), g32=g32.cpu().numpy(),
                 depth=depth.cpu().numpy(), status=status.cpu().numpy(), r_row=rr.cpu().numpy(),
-                r_col=rc.cpu().numpy(), stats=stats, cycles=cycles, left=left)
+                r_col=rc.cpu().numpy(), stats=stats, cycles=cycles, left=left, arith=arith)
 
 
 def pot_err(f, g, fo, go, eps):
@@ -41,55 +65,23 @@ def pot_err(f, g, fo, go, eps):
     return num / den
 
 
-def oracle_lanes(oracle, w, lanes, tol=None, max_iter=None, audit_every=1, tol_screen=0.0):
-    """Per-lane oracle results with the neighbouring states (depth-1, depth, depth+1)."""
-    out = {}
-    for t in lanes:
-        out[t] = oracle.solve_lane(w.x[t], w.y[t], w.a[t], w.b[t], float(w.eps[t]),
-                                   w.tol if tol is None else tol,
-                                   max_iter=w.max_iter if max_iter is None else max_iter,
-                                   audit_every=audit_every, tol_screen=tol_screen,
-                                   neighbours=True, history=True)
-    return out
+def oracle_lanes(oracle, w, lanes, tol=None, max_iter=None, audit_every=1, tol_screen=0.0, warm=None,
+                 audit_initial=False):
+    """Per-lane oracle results with the neighbouring states (depth-1, depth, depth+1); lanes are
+    independent problems (Eq. 2), so they are spread over the host cores, one whole lane each."""
+    lanes = list(lanes)
 
-
-def check_against_oracle(oracle, w, r, lanes, *, pot_tol, exact_depth, tol=None, max_iter=None,
-                         audit_every=1, tol_screen=0.0):
-    """Acceptance bar on the given lanes.  Depths must be equal; where exact_depth is False a
-    lane may be off by one audit, and every such lane is returned with the oracle's margin
-    |r - tol|/tol at the two candidate depths so that the caller can bound and report it.
-    Potentials are compared at the GPU's own depth (the oracle also emits its neighbours)."""
-    tol = w.tol if tol is None else tol
-    ref = oracle_lanes(oracle, w, lanes, tol, max_iter, audit_every, tol_screen)
-    misses = []
-    for t in lanes:
-        o = ref[t]
-        dg = int(r["depth"][t]); do = o.depth
-        assert r["status"][t] == o.status, (t, r["status"][t], o.status)
-        if dg == do:
-            fo, go = o.f, o.g
-        else:
-            assert not exact_depth, f"lane {t}: depth {dg} != oracle {do}"
-            assert abs(dg - do) == audit_every, f"lane {t}: depth {dg} vs oracle {do}"
-            fo, go = (o.f_prev, o.g_prev) if dg < do else (o.f_next, o.g_next)
-            if audit_every == 1:
-                hist = np.maximum(o.hist_row, o.hist_col)
-                k = min(dg, do)                       # the audit the two sides disagree on
-                margin = abs(hist[k - 1] - tol) / tol
-                # relative decay of the oracle residual per cycle around that audit: an error injected
-                # every cycle is remembered for about 1/decay cycles
-                decay = abs(hist[max(k - 2, 0)] - hist[k - 1]) / tol if k >= 2 else 1.0
-                misses.append((t, dg, do, margin, decay))
-        if dg == do or audit_every == 1:
-            e = pot_err(r["f"][t][None], r["g"][t][None], fo[None], go[None], float(w.eps[t]))[0]
-            assert e <= pot_tol, f"lane {t}: potential error {e:.3e} > {pot_tol}"
-        if o.status == oracle.DONE:
-            # the achieved two-sided residual, evaluated in float64 from the emitted potentials
-            rr, rc = oracle.residuals(w.x[t], w.y[t], w.a[t], w.b[t], float(w.eps[t]), r["f"][t], r["g"][t])
-            assert max(rr, rc) <= tol * (1 + 5e-3), (t, rr, rc)
-            assert r["r_row"][t] <= tol
-            assert abs(r["r_row"][t] - rr) <= 2e-2 * tol
-    return misses
+    def one(t):
+        kw = {}
+        if warm is not None:
+            kw = dict(f0=warm[0][t], g0=warm[1][t], audit_initial=audit_initial)
+        return oracle.solve_lane(w.x[t], w.y[t], w.a[t], w.b[t], float(w.eps[t]),
+                                 w.tol if tol is None else tol,
+                                 max_iter=w.max_iter if max_iter is None else max_iter,
+                                 audit_every=audit_every, tol_screen=tol_screen,
+                                 neighbours=True, history=True, **kw)
+    with ThreadPoolExecutor(max_workers=min(len(lanes), os.cpu_count() or 1) or 1) as ex:
+        return dict(zip(lanes, ex.map(one, lanes)))
 
 
 def miss_allowed(margin, decay, floor):
@@ -97,6 +89,94 @@ def miss_allowed(margin, decay, floor):
     arithmetic's residual error: a floor, or for slowly converging lanes the fp32 exponential
     error 2^-22 accumulated over the ~1/decay cycles the iteration remembers (factor 4 slack)."""
     return margin <= max(floor, 4.0 * 2.0 ** -22 / max(decay, 1e-12))
+
+
+def compare_lane(oracle, w, r, t, o, *, pot_tol, exact_depth, tol, audit_every=1, report_tol=None, entry=None):
+    """One lane of the acceptance bar against an oracle result `o` (anything with depth, status, f, g,
+    f_prev, g_prev, f_next, g_next and the history of max(r_row, r_col) in `hist`).  Returns the miss
+    record of a lane that stopped one audit away, else None."""
+    dg = int(r["depth"][t]); do = int(o.depth)
+    assert r["status"][t] == o.status, (t, r["status"][t], o.status)
+    miss = None
+    if dg == do:
+        fo, go = o.f, o.g
+    else:
+        assert not exact_depth, f"lane {t}: depth {dg} != oracle {do}"
+        assert abs(dg - do) == audit_every, f"lane {t}: depth {dg} vs oracle {do}"
+        fo, go = (o.f_prev, o.g_prev) if dg < do else (o.f_next, o.g_next)
+        if audit_every == 1:
+            hist = o.hist
+            k = min(dg, do)                       # the audit the two sides disagree on
+            margin = abs(hist[k - 1] - tol) / tol
+            # relative decay of the oracle residual per cycle around that audit: an error injected
+            # every cycle is remembered for about 1/decay cycles
+            decay = abs(hist[max(k - 2, 0)] - hist[k - 1]) / tol if k >= 2 else 1.0
+            miss = (t, dg, do, float(margin), float(decay))
+    e = None
+    if dg == do or audit_every == 1:
+        e = pot_err(r["f"][t][None], r["g"][t][None], np.asarray(fo, np.float64)[None],
+                    np.asarray(go, np.float64)[None], float(w.eps[t]))[0]
+        assert e <= pot_tol, f"lane {t}: potential error {e:.3e} > {pot_tol}"
+    if o.status == oracle.DONE:
+        # the achieved two-sided residual, evaluated in float64 from the emitted potentials
+        rr, rc = oracle.residuals(w.x[t], w.y[t], w.a[t], w.b[t], float(w.eps[t]), r["f"][t], r["g"][t])
+        if report_tol is not None:
+            # guard arm: the solve ran with a stricter threshold, the reported tolerance holds with no slack
+            assert max(rr, rc) <= report_tol, (t, rr, rc)
+        else:
+            assert max(rr, rc) <= tol * (1 + 5e-3), (t, rr, rc)
+        assert r["r_row"][t] <= tol
+        assert abs(r["r_row"][t] - rr) <= 2e-2 * tol
+        # the column half of the two-sided check (Eq. 5) as the GPU measured it
+        assert np.isfinite(r["r_col"][t]) and r["r_col"][t] >= 0.0
+        assert abs(float(r["r_col"][t]) - rc) <= RCOL_ABS[r["arith"]], (t, float(r["r_col"][t]), rc)
+        if entry is not None:
+            entry["max_residual_over_tol"] = float(max(entry["max_residual_over_tol"], max(rr, rc) / (report_tol or tol)))
+            entry["max_rrow_dev_over_tol"] = float(max(entry["max_rrow_dev_over_tol"], abs(float(r["r_row"][t]) - rr) / tol))
+            entry["max_rcol_dev"] = float(max(entry["max_rcol_dev"], abs(float(r["r_col"][t]) - rc)))
+    if entry is not None and e is not None:
+        entry["max_pot_err"] = max(entry["max_pot_err"], float(e))
+    return miss
+
+
+def new_entry(label, w, r, lanes, tol, floor):
+    return dict(label=label, workload=w.name, shape=[int(v) for v in w.shape], arith=r["arith"], tol=float(tol), lanes=len(lanes),
+                equal=0, misses=[], floor=floor, max_pot_err=0.0, max_residual_over_tol=0.0,
+                max_rrow_dev_over_tol=0.0, max_rcol_dev=0.0)
+
+
+def close_entry(entry, misses, floor):
+    for (t, dg, do, margin, decay) in misses:
+        entry["misses"].append(dict(lane=int(t), gpu=dg, oracle=do, margin=margin, decay=decay,
+                                    inside_1e6_band=bool(margin <= NORTH_STAR_BAND)))
+        if floor is not None:
+            assert miss_allowed(margin, decay, floor), \
+                f"{entry['label']} lane {t}: gpu {dg} oracle {do} margin {margin:.2e} decay {decay:.2e}"
+    entry["equal"] = entry["lanes"] - len(misses)
+    LEDGER.append(entry)
+
+
+def check_against_oracle(oracle, w, r, lanes, *, pot_tol, exact_depth, tol=None, max_iter=None,
+                         audit_every=1, tol_screen=0.0, floor=None, label="", report_tol=None, warm=None,
+                         audit_initial=False):
+    """Acceptance bar on the given lanes.  Depths must be equal; where exact_depth is False a
+    lane may be off by one audit, and every such lane is returned with the oracle's margin
+    |r - tol|/tol at the two candidate depths (and, when `floor` is given, held to miss_allowed).
+    Potentials are compared at the GPU's own depth (the oracle also emits its neighbours)."""
+    tol = w.tol if tol is None else tol
+    lanes = list(lanes)
+    ref = oracle_lanes(oracle, w, lanes, tol, max_iter, audit_every, tol_screen, warm, audit_initial)
+    entry = new_entry(label, w, r, lanes, tol, floor)
+    misses = []
+    for t in lanes:
+        o = ref[t]
+        o.hist = np.maximum(o.hist_row, o.hist_col)
+        m = compare_lane(oracle, w, r, t, o, pot_tol=pot_tol, exact_depth=exact_depth, tol=tol,
+                         audit_every=audit_every, report_tol=report_tol, entry=entry)
+        if m is not None:
+            misses.append(m)
+    close_entry(entry, misses, floor)
+    return misses
 
 
 def check_accounting(oracle, r, W, mode):

@@ -3,15 +3,19 @@ same seeded inputs.  Bar: completion depths equal; potentials within 1e-4 relati
 oracle state at the same depth; achieved two-sided residual <= tol; slot counts exactly those
 of Eq. 6-8.  Float64 arithmetic must meet it with no exception.  The default arithmetic
 (fp32, or float64 exponents with fp32 exponentials when a lane's cost/eps range is beyond
-fp32) may sit one audit away only when the oracle's own residual at the disputed audit is
-within 1e-5 relative of tol; every such lane is printed.  Pure fp32 arithmetic is held to the
+fp32, or the tensor-core cross term for bf16 inputs) may sit one audit away only when the
+oracle's own residual at the disputed audit is within 1e-5 relative of tol (or the decay-scaled
+bound of helpers.miss_allowed for very slow lanes); every such lane goes into the ledger that
+tests/test_yy_parity_ledger.py bounds and writes out.  Pure fp32 arithmetic is held to the
 same bar where its error model says it can meet it, and to its documented limits elsewhere."""
+import os
 import ctypes
 
 import numpy as np
 import pytest
 
-from helpers import check_accounting, check_against_oracle, miss_allowed, pot_err, run_gpu
+from helpers import (LEDGER, check_accounting, check_against_oracle, close_entry, compare_lane, new_entry,
+                     pot_err, run_gpu)
 from paper_2607_24741_b200 import workloads as wl
 
 pytestmark = pytest.mark.gpu
@@ -51,10 +55,8 @@ def test_default_arithmetic_meets_the_bar(oracle, case):
     w = _make(case)
     W = w.shape[0]
     r = run_gpu(w, mode="active")
-    misses = check_against_oracle(oracle, w, r, range(W), pot_tol=POT_TOL_F32, exact_depth=False)
-    for t, dg, do, margin, decay in misses:
-        print(f"[depth miss] {case} lane {t}: gpu {dg} oracle {do} oracle margin {margin:.2e} decay/cycle {decay:.2e}")
-        assert miss_allowed(margin, decay, MARGIN_AUTO)
+    check_against_oracle(oracle, w, r, range(W), pot_tol=POT_TOL_F32, exact_depth=False, floor=MARGIN_AUTO,
+                         label=f"default arithmetic, {case}")
     check_accounting(oracle, r, W, "active")
     # the float getter is the float64 one rounded
     np.testing.assert_array_equal(r["f32"], r["f"].astype(np.float32))
@@ -67,10 +69,8 @@ def test_pure_fp32_arithmetic_where_it_suffices(oracle, case, cost_form):
     w = _make(case)
     W = w.shape[0]
     r = run_gpu(w, mode="active", compute="f32", cost_form=cost_form)
-    misses = check_against_oracle(oracle, w, r, range(W), pot_tol=POT_TOL_F32, exact_depth=False)
-    for t, dg, do, margin, decay in misses:
-        print(f"[depth miss] {case} form {cost_form} lane {t}: gpu {dg} oracle {do} margin {margin:.2e} decay/cycle {decay:.2e}")
-        assert miss_allowed(margin, decay, MARGIN_F32)
+    misses = check_against_oracle(oracle, w, r, range(W), pot_tol=POT_TOL_F32, exact_depth=False, floor=MARGIN_F32,
+                                  label=f"pure fp32 (forced), {case}, cost form {cost_form}")
     assert len(misses) <= max(1, W // 8)
 
 
@@ -167,7 +167,8 @@ def test_every_column_split_agrees_with_the_oracle(oracle, cs):
     assert check_against_oracle(oracle, w, r, range(5), pot_tol=POT_TOL_F64, exact_depth=True) == []
     w3 = wl.make("registration", W=3, n=700)
     r3 = run_gpu(w3, mode="active", column_split=cs)
-    check_against_oracle(oracle, w3, r3, range(3), pot_tol=POT_TOL_F32, exact_depth=False)
+    check_against_oracle(oracle, w3, r3, range(3), pot_tol=POT_TOL_F32, exact_depth=False, floor=MARGIN_AUTO,
+                         label=f"registration n=700, column split {cs}")
 
 
 def test_audit_grid_screen_threshold_and_iteration_limit(oracle):
@@ -271,25 +272,24 @@ def test_host_buffer_call_matches_device_call(oracle):
     np.testing.assert_array_equal(g, r["g32"]); assert slots.value == r["stats"]["slots"]
 
 
-# ---- BASELINE sizes, in the launch configuration bench.py times (ACTIVE, default arithmetic) ----
+# ---- the five workloads at their full sizes, in the launch configuration the benchmark times
+#      (ACTIVE, default arithmetic); the oracle runs one whole lane per host core
 FULL = {
-    "tiny": (range(8), {}),
-    "sensor": ([0, 1, 17, 63, 100, 128, 200, 255], {}),
-    "feature": ([0, 21, 63], {}),
-    "sweep": ([0, 3, 5, 8, 100, 511, 777, 1023], {}),
+    "tiny": range(8),
+    "sensor": range(256),                       # every lane: the oracle needs well under a second for all of them
+    "feature": list(range(0, 64, 4)),
+    "sweep": list(range(0, 1024, 4)),
 }
 
 
 @pytest.mark.parametrize("name", list(FULL))
-def test_full_size_sampled_lanes_against_oracle(oracle, name):
-    lanes, kw = FULL[name]
-    w = wl.make(name, **kw)
+def test_full_size_lanes_against_oracle(oracle, name):
+    lanes = FULL[name]
+    w = wl.make(name)
     W = w.shape[0]
     r = run_gpu(w, mode="active")
-    misses = check_against_oracle(oracle, w, r, lanes, pot_tol=POT_TOL_F32, exact_depth=False)
-    for t, dg, do, margin, decay in misses:
-        print(f"[depth miss] {name} lane {t}: gpu {dg} oracle {do} oracle margin {margin:.2e} decay/cycle {decay:.2e}")
-        assert miss_allowed(margin, decay, MARGIN_AUTO)
+    check_against_oracle(oracle, w, r, lanes, pot_tol=POT_TOL_F32, exact_depth=False, floor=MARGIN_AUTO,
+                         label=f"full size, {name}")
     # properties that hold at any size
     depth = r["depth"].astype(np.int64)
     assert np.all(r["status"] == 1) and np.all(r["r_row"] <= w.tol)
@@ -297,44 +297,77 @@ def test_full_size_sampled_lanes_against_oracle(oracle, name):
     np.testing.assert_array_equal(np.array(r["stats"]["widths"]), oracle.survivor_widths(depth))
 
 
-def test_full_size_registration_properties(oracle):
-    # one oracle lane would take ~15 core-minutes here: check what can be computed one by one
+class _Stored:
+    """One lane of tests/golden/registration_n8192.npz in the shape compare_lane expects."""
+    def __init__(self, z, i):
+        self.depth = int(z["depth"][i]); self.status = int(z["status"][i])
+        self.f, self.g = z["f"][i], z["g"][i]
+        self.f_prev, self.g_prev = z["f_prev"][i], z["g_prev"][i]
+        self.f_next, self.g_next = z["f_next"][i], z["g_next"][i]
+        tail = z["hist"][i]
+        self.hist = np.full(self.depth, np.nan)
+        k = min(len(tail), self.depth)
+        self.hist[self.depth - k:] = tail[len(tail) - k:]
+        self.r_row = float(z["r_row"][i])
+
+
+def test_full_size_registration_against_stored_oracle(oracle):
+    # One oracle lane at n = m = 8192 takes a quarter of an hour, so the oracle's results for six lanes
+    # are stored (tests/golden/make_registration_golden.py wrote them, calling the oracle only); the
+    # float64 residual evaluation of the emitted state is cheap enough to run here.
+    z = np.load(os.path.join(os.path.dirname(__file__), "golden", "registration_n8192.npz"))
     w = wl.make("registration")
     W, n, m, d = w.shape
+    assert int(z["n"]) == n and float(z["tol"]) == w.tol
     r = run_gpu(w, mode="active")
     depth = r["depth"].astype(np.int64)
     assert np.all(r["status"] == 1) and np.all(r["r_row"] <= w.tol) and np.all(depth > 50)
     assert r["stats"]["slots"] == depth.sum() and r["cycles"] == depth.max()
     np.testing.assert_array_equal(np.array(r["stats"]["widths"]), oracle.survivor_widths(depth))
-    for t in (0, 31):
-        # the achieved two-sided residual of the emitted state, evaluated by the oracle in float64
-        rr, rc = oracle.residuals(w.x[t], w.y[t], w.a[t], w.b[t], float(w.eps[t]), r["f"][t], r["g"][t])
-        assert max(rr, rc) <= w.tol * (1 + 5e-3) and abs(rr - r["r_row"][t]) <= 2e-2 * w.tol
-        # the emitted g is the g-leg of the emitted f (Eq. 4): the column marginal is current
-        assert rc <= 1e-5
-        # one more oracle cycle from the emitted state still passes and lowers the row residual
-        C = oracle.cost_matrix(w.x[t], w.y[t])
-        f1 = oracle.f_leg(C, r["g"][t], w.a[t], float(w.eps[t])); g1 = oracle.g_leg(C, f1, w.b[t], float(w.eps[t]))
-        row, col = oracle.marginals(C, f1, g1, float(w.eps[t]))
-        assert np.abs(row - w.a[t]).sum() < rr
-        # and one cycle BACK did not pass: undo is impossible, but the screen value of the state before
-        # the last cycle is bounded below by the monotone decay: r(l-1) >= r(l)
-        assert rr > 0.5 * w.tol            # the lane stopped at its first passing audit, not long after
+    lanes = [int(t) for t in z["lanes"]]
+    entry = new_entry("full size, registration (stored oracle)", w, r, lanes, w.tol, MARGIN_AUTO)
+    misses = []
+    for i, t in enumerate(lanes):
+        o = _Stored(z, i)
+        assert abs(o.r_row - o.hist[-1]) <= 1e-15
+        miss = compare_lane(oracle, w, r, t, o, pot_tol=POT_TOL_F32, exact_depth=False, tol=w.tol, entry=entry)
+        if miss is not None:
+            misses.append(miss)
+    close_entry(entry, misses, MARGIN_AUTO)
+    t = lanes[0]
+    # one more oracle cycle from the emitted state still passes and lowers the row residual
+    C = oracle.cost_matrix(w.x[t], w.y[t])
+    f1 = oracle.f_leg(C, r["g"][t], w.a[t], float(w.eps[t])); g1 = oracle.g_leg(C, f1, w.b[t], float(w.eps[t]))
+    row, col = oracle.marginals(C, f1, g1, float(w.eps[t]))
+    rr0, _ = oracle.residuals(w.x[t], w.y[t], w.a[t], w.b[t], float(w.eps[t]), r["f"][t], r["g"][t])
+    assert np.abs(row - w.a[t]).sum() < rr0
+
+
+# ---- the paper's guard: a stricter threshold inside, the reported tolerance outside ----------------
+@pytest.mark.parametrize("case", list(CASES))
+def test_guarded_thresholds_meet_the_reported_tolerance_without_slack(oracle, case):
+    # Section "Screen, verify, and compact": screen and check run at 9.5e-4, the output is reported at
+    # 1e-3.  Both sides get the guarded threshold; the float64 residual of every emitted state must then
+    # be within the REPORTED tolerance with no allowance for the GPU's arithmetic.
+    w = _make(case)
+    W = w.shape[0]
+    guard, reported = 9.5e-4, 1e-3
+    r = run_gpu(w, mode="active", tol=guard)
+    check_against_oracle(oracle, w, r, range(W), pot_tol=POT_TOL_F32, exact_depth=False, tol=guard, floor=MARGIN_AUTO,
+                         label=f"guard arm 9.5e-4 -> 1e-3, {case}", report_tol=reported)
+    check_accounting(oracle, r, W, "active")
 
 
 # ---- tensor-core cross term (bf16 inputs, d a multiple of 64) ------------------------------------
-POT_TOL_BF16 = 5e-3     # acceptance bar for bf16 inputs; measured errors are ~1e-6
-
-
+# (bf16 products are exact in fp32 and accumulate in fp32, so the error model is the default
+# arithmetic's: same margin, same potential bar; the acceptance bar for bf16 inputs, 5e-3, is far looser.)
 @pytest.mark.parametrize("kw", [dict(W=3, n=200, m=333, d=64), dict(W=2, n=256, d=128), dict(W=2, n=129, m=640, d=512)])
 def test_tensor_core_path_against_oracle(oracle, kw):
     w = wl.make("feature", **kw)
     W = w.shape[0]
     r = run_gpu(w, mode="active", compute="tensor")
-    misses = check_against_oracle(oracle, w, r, range(W), pot_tol=POT_TOL_F32, exact_depth=False)
-    for t, dg, do, margin, decay in misses:
-        print(f"[depth miss] tensor {kw} lane {t}: gpu {dg} oracle {do} oracle margin {margin:.2e} decay/cycle {decay:.2e}")
-        assert miss_allowed(margin, decay, MARGIN_F32)
+    check_against_oracle(oracle, w, r, range(W), pot_tol=POT_TOL_F32, exact_depth=False, floor=MARGIN_AUTO,
+                         label=f"tensor cores, {kw}")
     check_accounting(oracle, r, W, "active")
     # what AUTO picks for such inputs is this very path: bit-identical results
     ra = run_gpu(w, mode="active")
@@ -371,9 +404,8 @@ def test_tensor_core_pair_kernel_shapes_and_modes(oracle, kw):
     rm = run_gpu(w, mode="masked", compute="tensor")
     np.testing.assert_array_equal(ra["depth"], rm["depth"])
     np.testing.assert_array_equal(ra["f"], rm["f"]); np.testing.assert_array_equal(ra["g"], rm["g"])
-    misses = check_against_oracle(oracle, w, ra, range(W), pot_tol=POT_TOL_F32, exact_depth=False)
-    for t, dg, do, margin, decay in misses:
-        assert miss_allowed(margin, decay, MARGIN_F32)
+    check_against_oracle(oracle, w, ra, range(W), pot_tol=POT_TOL_F32, exact_depth=False, floor=MARGIN_AUTO,
+                         label=f"tensor cores (CTA pairs), {kw}")
     check_accounting(oracle, ra, W, "active")
     rs = run_gpu(w, mode="static", compute="tensor")
     np.testing.assert_array_equal(ra["depth"], rs["depth"])
@@ -389,9 +421,8 @@ def test_tensor_core_pair_kernel_many_small_lanes(oracle):
     w = wl.make("feature", W=150, n=130, m=140, d=320)
     r = run_gpu(w, mode="active", compute="tensor")
     lanes = [0, 1, 73, 74, 75, 148, 149] + list(range(9, 150, 29))
-    misses = check_against_oracle(oracle, w, r, lanes, pot_tol=POT_TOL_F32, exact_depth=False)
-    for t, dg, do, margin, decay in misses:
-        assert miss_allowed(margin, decay, MARGIN_F32)
+    check_against_oracle(oracle, w, r, lanes, pot_tol=POT_TOL_F32, exact_depth=False, floor=MARGIN_AUTO,
+                         label="tensor cores (CTA pairs), 150 small lanes")
     check_accounting(oracle, r, 150, "active")
     rm = run_gpu(w, mode="masked", compute="tensor")
     np.testing.assert_array_equal(rm["depth"], r["depth"]); np.testing.assert_array_equal(rm["f"], r["f"])
@@ -412,10 +443,8 @@ def test_other_tolerances_of_the_sweep_grid(oracle, tol):
     # the disagreement sweep runs the same lanes at five tolerances: depths, slots and potentials at each
     w = wl.make("sweep", W=24, n=100, m=77, max_iter=50000)
     r = run_gpu(w, mode="active", tol=tol)
-    misses = check_against_oracle(oracle, w, r, range(24), pot_tol=POT_TOL_F32, exact_depth=False, tol=tol)
-    for t, dg, do, margin, decay in misses:
-        print(f"[depth miss] tol {tol} lane {t}: gpu {dg} oracle {do} oracle margin {margin:.2e} decay/cycle {decay:.2e}")
-        assert miss_allowed(margin, decay, MARGIN_AUTO)
+    check_against_oracle(oracle, w, r, range(24), pot_tol=POT_TOL_F32, exact_depth=False, tol=tol, floor=MARGIN_AUTO,
+                         label=f"sweep grid, tol {tol}")
     check_accounting(oracle, r, 24, "active")
     rs = run_gpu(w, mode="static", tol=tol)
     np.testing.assert_array_equal(rs["depth"], r["depth"])
@@ -474,6 +503,192 @@ def test_mixed_arithmetic_with_a_useless_reference_estimate(oracle):
     for mode in ("active", "static"):
         r = run_gpu(w, mode=mode, compute="mixed")
         assert (r["status"] == oracle.DONE).all()
-        misses = check_against_oracle(oracle, w, r, range(W), pot_tol=POT_TOL_F32, exact_depth=False)
-        for t, dg, do, margin, decay in misses:
-            assert miss_allowed(margin, decay, MARGIN_AUTO)
+        check_against_oracle(oracle, w, r, range(W), pot_tol=POT_TOL_F32, exact_depth=False, floor=MARGIN_AUTO,
+                             label=f"clouds far apart, {mode}")
+
+
+# ---- warm proposals and the audit of the proposal itself -------------------------------------------
+@pytest.mark.parametrize("compute", ["f64", "auto"])
+def test_warm_proposal_continues_a_cold_solve(oracle, compute):
+    # Section "Initialization and repeated couplings".  A proposal that is the cold iteration's state after
+    # j cycles must finish l_t - j cycles later at the same potentials (both sides get the same proposal).
+    w = wl.make("sensor", W=6, n=150, m=170)
+    j = 2
+    part = oracle.solve_batch(w.x, w.y, w.a, w.b, w.eps, w.tol, fixed_cycles=j)
+    warm = (part.f, part.g)
+    r = run_gpu(w, compute=compute, warm=warm)
+    tolp = POT_TOL_F64 if compute == "f64" else POT_TOL_F32
+    check_against_oracle(oracle, w, r, range(6), pot_tol=tolp, exact_depth=compute == "f64", warm=warm,
+                         floor=None if compute == "f64" else MARGIN_AUTO, label=f"warm proposal, {compute}")
+    cold = run_gpu(w, compute=compute)
+    np.testing.assert_array_equal(r["depth"] + j, cold["depth"])
+    check_accounting(oracle, r, 6, "active")
+
+
+@pytest.mark.parametrize("compute", ["f64", "mixed", "f32"])
+@pytest.mark.parametrize("mode", ["active", "masked"])
+def test_audit_of_the_proposal_measures_both_marginals(oracle, compute, mode):
+    # With audit_initial the proposal itself gets the screen and the two-sided check.  Here the proposal
+    # is a converged state whose g has been perturbed, so NEITHER marginal is current: the column residual
+    # is far from rounding level and the column-check leg has to measure it.  Thresholds are chosen so
+    # that some lanes pass at depth 0 (their output is the proposal, with the measured residuals) and the
+    # others go on.
+    w = wl.make("sensor", W=8, n=130, m=150)
+    conv = oracle.solve_batch(w.x, w.y, w.a, w.b, w.eps, 1e-9, max_iter=2000)
+    rng = np.random.default_rng(5)
+    amp = np.linspace(0.002, 0.05, 8)[:, None] * w.eps[:, None].astype(np.float64)
+    warm = (conv.f.copy(), conv.g + amp * rng.standard_normal(conv.g.shape))
+    tol = 2e-2
+    r = run_gpu(w, mode=mode, compute=compute, warm=warm, audit_initial=True, tol=tol)
+    ref = {t: oracle.solve_lane(w.x[t], w.y[t], w.a[t], w.b[t], float(w.eps[t]), tol, f0=warm[0][t], g0=warm[1][t],
+                                audit_initial=True) for t in range(8)}
+    np.testing.assert_array_equal(r["depth"], [ref[t].depth for t in range(8)])
+    zero = [t for t in range(8) if ref[t].depth == 0]
+    assert 2 <= len(zero) <= 6                                   # the case really has both kinds of lane
+    rel = {"f64": 1e-9, "mixed": 1e-5, "f32": 2e-4}[compute]
+    for t in zero:
+        # the proposal comes back as it went in (up to the rounding of scaling by 1/eps and back)
+        np.testing.assert_allclose(r["f"][t], warm[0][t], rtol=1e-14, atol=0)
+        np.testing.assert_allclose(r["g"][t], warm[1][t], rtol=1e-14, atol=0)
+        assert ref[t].r_col > 1e-3 and ref[t].r_row > 1e-4       # both far above rounding level
+        assert abs(r["r_col"][t] - ref[t].r_col) <= rel * ref[t].r_col + 1e-7
+        assert abs(r["r_row"][t] - ref[t].r_row) <= rel * ref[t].r_row + 1e-7
+    e = pot_err(r["f"], r["g"], np.stack([ref[t].f for t in range(8)]), np.stack([ref[t].g for t in range(8)]),
+                w.eps.astype(np.float64))
+    assert e.max() <= (POT_TOL_F64 if compute == "f64" else POT_TOL_F32)
+    assert r["stats"]["slots"] == (int(r["depth"].sum()) if mode == "active" else 8 * int(r["depth"].max()))
+
+
+def test_warm_start_is_refused_after_the_first_cycle():
+    import torch
+    from paper_2607_24741_b200 import binding as B
+    w = wl.make("tiny")
+    t = lambda v: torch.from_numpy(v).to("cuda:0")
+    sb = B.SinkhornBatch(t(w.x), t(w.y), t(w.a), t(w.b), t(w.eps), w.tol)
+    sb.step(1)
+    z = torch.zeros(8, 64, dtype=torch.float64, device="cuda:0")
+    with pytest.raises(B.SkbError) as e:
+        sb.warm_start(z, z)
+    assert e.value.code == 5
+    sb.close()
+    sb = B.SinkhornBatch(t(w.x), t(w.y), t(w.a), t(w.b), t(w.eps), w.tol)
+    bad = z.clone(); bad[3, 7] = float("nan")
+    sb.warm_start(bad, z)
+    with pytest.raises(B.SkbError) as e:
+        sb.drain()
+    assert e.value.code == 3
+    sb.close()
+
+
+# ---- measurement aids must not disturb the solve ----------------------------------------------------
+def _solve_plain(w, compute, mode="active"):
+    r = run_gpu(w, mode=mode, compute=compute)
+    return r
+
+
+@pytest.mark.parametrize("case,compute", [("tiny", "auto"), ("sensor_ragged", "f32"), ("feature_small", "auto")])
+def test_profiling_an_update_leg_leaves_the_solve_bit_identical(case, compute):
+    import torch
+    from paper_2607_24741_b200 import binding as B
+    w = _make(case)
+    plain = run_gpu(w, compute=compute)
+    dev = torch.device("cuda:0")
+    t = lambda v: torch.from_numpy(v).to(dev)
+    x, y = t(w.x), t(w.y)
+    if w.xy_dtype == "bf16":
+        x, y = x.bfloat16(), y.bfloat16()
+    sb = B.SinkhornBatch(x, y, t(w.a), t(w.b), t(w.eps), w.tol, compute=compute, max_iter=w.max_iter)
+    sb.step(3)
+    assert sb.profile_update(leg=0, reps=5) > 0.0
+    assert sb.profile_update(leg=1, reps=2) > 0.0
+    sb.drain()
+    f, g = sb.potentials(f64=True); depth, status = sb.depths(); rr, rc = sb.residuals(); st = sb.stats()
+    np.testing.assert_array_equal(depth.cpu().numpy(), plain["depth"])
+    np.testing.assert_array_equal(f.cpu().numpy(), plain["f"]); np.testing.assert_array_equal(g.cpu().numpy(), plain["g"])
+    np.testing.assert_array_equal(rr.cpu().numpy(), plain["r_row"])
+    assert st["slots"] == plain["stats"]["slots"]
+    with pytest.raises(B.SkbError) as e:                      # nothing is running any more
+        sb.profile_update(leg=0, reps=1)
+    assert e.value.code == 5
+    sb.close()
+
+
+@pytest.mark.parametrize("case,mode", [("sweep_small", "active"), ("sensor_ragged", "static"), ("registration_small", "active")])
+def test_phase_timing_adds_up_and_changes_no_bit(case, mode):
+    # Eq. 11: update legs (c_k), column check (H_check), planning and emission/compaction (H_compact)
+    import torch
+    from paper_2607_24741_b200 import binding as B
+    w = _make(case)
+    plain = run_gpu(w, mode=mode)
+    dev = torch.device("cuda:0")
+    t = lambda v: torch.from_numpy(v).to(dev)
+    sb = B.SinkhornBatch(t(w.x), t(w.y), t(w.a), t(w.b), t(w.eps), w.tol, mode=mode, max_iter=w.max_iter)
+    sb.set_profiling(True)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(); sb.drain(); e1.record(); torch.cuda.synchronize()
+    wall = e0.elapsed_time(e1)
+    st = sb.stats(widths_cap=100000)
+    trace = sb.cycle_trace()
+    f, g = sb.potentials(f64=True); depth, _ = sb.depths()
+    sb.close()
+    np.testing.assert_array_equal(depth.cpu().numpy(), plain["depth"])
+    np.testing.assert_array_equal(f.cpu().numpy(), plain["f"]); np.testing.assert_array_equal(g.cpu().numpy(), plain["g"])
+    ph = st["phase_ms"]
+    assert ph["create"] > 0 and ph["f_leg"] > 0 and ph["g_leg"] > 0 and ph["plan"] > 0
+    cyc = sum(ph[k] for k in ("f_leg", "column_check", "plan", "emit_move", "g_leg"))
+    assert 0.5 * wall <= cyc <= wall                     # the rest is the gaps between the harvested chunks
+    assert len(trace) >= st["cycles"] and abs(sum(trace) - ph["f_leg"] - ph["g_leg"]) <= 1e-3 * cyc + 1e-3
+    assert plain["stats"]["phase_ms"]["f_leg"] == 0.0 and plain["stats"]["phase_ms"]["create"] > 0
+
+
+def test_step_alone_follows_the_width_and_reports_device_errors():
+    import time
+    import torch
+    from paper_2607_24741_b200 import binding as B
+    w = wl.make("tiny")
+    t = lambda v: torch.from_numpy(v).to("cuda:0")
+    a = w.a.copy(); a[2, 5] = -1.0
+    sb = B.SinkhornBatch(t(w.x), t(w.y), t(a), t(w.b), t(w.eps), w.tol)
+    code = None
+    for _ in range(200):                                  # no drain, no synchronising call
+        try:
+            sb.step(1)
+        except B.SkbError as e:
+            code = e.code
+            break
+        time.sleep(0.001)
+    assert code == 3
+    sb.close()
+    # a good batch stepped to the end: the launches stop growing once the host has seen it finish
+    ref = run_gpu(w)
+    sb = B.SinkhornBatch(t(w.x), t(w.y), t(w.a), t(w.b), t(w.eps), w.tol)
+    for _ in range(int(ref["depth"].max()) // 10 + 3):
+        sb.step(10); time.sleep(0.002)
+    torch.cuda.synchronize(); sb.step(1)
+    before = sb.launch_count(); sb.step(50)
+    assert sb.launch_count() == before                     # finished: further steps enqueue nothing
+    depth, _ = sb.depths(); f, _g = sb.potentials(f64=True)
+    np.testing.assert_array_equal(depth.cpu().numpy(), ref["depth"]); np.testing.assert_array_equal(f.cpu().numpy(), ref["f"])
+    sb.close()
+
+
+def test_two_batches_interleaved_on_one_stream(oracle):
+    # Two handles sharing a stream, stepped alternately; one finishes long before the other.  An f-leg then
+    # follows the OTHER batch's (possibly empty) kernels: every kernel of a cycle must still see complete
+    # predecessors.
+    import torch
+    from paper_2607_24741_b200 import binding as B
+    wa = wl.make("tiny"); wb = wl.make("sensor", W=12, n=300, m=260)
+    t = lambda v: torch.from_numpy(v).to("cuda:0")
+    ra, rb = run_gpu(wa), run_gpu(wb)
+    sa = B.SinkhornBatch(t(wa.x), t(wa.y), t(wa.a), t(wa.b), t(wa.eps), wa.tol)
+    sb = B.SinkhornBatch(t(wb.x), t(wb.y), t(wb.a), t(wb.b), t(wb.eps), wb.tol)
+    for _ in range(int(ra["depth"].max()) + 2):
+        sa.step(1); sb.step(1)
+    torch.cuda.synchronize()
+    for s, r in ((sa, ra), (sb, rb)):
+        assert s.active() == 0
+        f, g = s.potentials(f64=True); depth, _ = s.depths()
+        np.testing.assert_array_equal(depth.cpu().numpy(), r["depth"])
+        np.testing.assert_array_equal(f.cpu().numpy(), r["f"]); np.testing.assert_array_equal(g.cpu().numpy(), r["g"])
+        s.close()
