@@ -490,6 +490,16 @@ def workload_entry(name, args, dev, flush, unit_rates, local_rank, headline=None
                                  "frac_binding": roof["frac"], "binding": roof.get("binding_unit", roof["bound"]),
                                  "frac_of_measured_unit_rates": roof.get("frac_of_measured_unit_rates")},
              "phases": R.phases("active"), "clocks": clk.summary()}
+    # break-even condition of the time model (Eq. 12): the update time saved by running at the survivor
+    # width A_k instead of W must exceed what screening, checking and compaction cost
+    c_w = roof["ms_per_launch"] + roof["g_leg_ms_per_launch"]
+    mdl = entry["phases"]["model"]
+    saved = info["cycles"] * c_w - mdl["sum_c_k"]
+    overhead = mdl["H_screen"] + mdl["H_check"] + mdl["H_compact"]
+    entry["break_even"] = {"c_W_ms_per_cycle": c_w, "cycles": info["cycles"], "sum_k_c_W_minus_c_Ak_ms": saved,
+                           "H_screen_plus_H_check_plus_H_compact_ms": overhead, "holds": bool(saved > overhead),
+                           "note": "c_k(A_k) and the H terms from the profiled solve (one launch per leg, no overlap); "
+                                   "c_k(W) = f-leg + g-leg at full width, timed alone"}
     if name == "registration":
         entry["parity"] = R.parity_stored()
     elif name == "feature":
@@ -510,7 +520,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=HEADLINE, choices=list(ALL))
-    ap.add_argument("--mode", default="active", choices=["active", "masked", "static", "masked_exit"])
+    ap.add_argument("--mode", default=None, choices=["active", "masked", "static", "masked_exit"])
     ap.add_argument("--compute", default="auto", choices=["auto", "f32", "mixed", "f64", "tensor"])
     ap.add_argument("--only", action="store_true", help="measure --workload only (no `workloads` object)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -525,14 +535,20 @@ def main():
                     help="time the audit policies on --workload: fused row screen + column check of flagged lanes "
                          "(default) against a full two-sided check of every lane, each at every cycle and every 4th")
     ap.add_argument("--kernel-only", action="store_true",
-                    help="only create the batch and time the update kernel (few launches; for profiler captures)")
+                    help="only create the batch and time the update kernel (few launches; for profiler captures); "
+                         "with --mode active: three 32-cycle launches of the multi-cycle kernel instead")
     ap.add_argument("--move-only", action="store_true",
                     help="a short ACTIVE solve of the first --lanes lanes with phase timing: emission/compaction "
                          "bytes, time and GB/s (few launches; for profiler captures of the compaction kernel)")
     ap.add_argument("--lanes", type=int, default=0, help="with --move-only / --kernel-only: use the first LANES lanes only")
     ap.add_argument("--unit-rates", action="store_true", help="only run the unit-rate self-test (one JSON line)")
+    ap.add_argument("--shadow-replay", action="store_true",
+                    help="replay a solve of the first --lanes lanes (default 256) cycle by cycle and compare, at every audit, "
+                         "the fused row screen with the row residual computed directly from the potentials")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.mode is None:
+        args.mode = "static" if args.kernel_only else "active"   # --kernel-only times the per-leg kernel unless --mode active is given
 
     rank = int(os.environ.get("RANK", "0")); world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -594,6 +610,8 @@ def main():
 
     R = Runner(args.workload, args, dev, tol=args.tol)
     w = R.w
+    if args.shadow_replay and not args.lanes:
+        args.lanes = min(256, w.shape[0])
     if args.lanes:
         L = args.lanes
         R.x, R.y, R.a, R.b, R.eps = R.x[:L].contiguous(), R.y[:L].contiguous(), R.a[:L].contiguous(), R.b[:L].contiguous(), R.eps[:L].contiguous()
@@ -628,6 +646,20 @@ def main():
                              "depths_equal_to_screen_arm": bool((depth == ref_depth[every]).all().item())})
         print(json.dumps({"report": "audit-arms", "workload": args.workload, "mode": args.mode, "W": W, "n": n, "m": m,
                           "d": d, "tol": w.tol, "rows": rows}), flush=True)
+        return
+    if args.shadow_replay:
+        print(json.dumps(shadow_replay(R, args)), flush=True)
+        return
+    if args.kernel_only and args.mode == "active":
+        # a few multi-cycle launches of the ACTIVE path (for profiler captures of the cluster kernels)
+        sb = R.batch("active")
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        sb.step(32); torch.cuda.synchronize()
+        e0.record(); sb.step(32); sb.step(32); e1.record(); torch.cuda.synchronize()
+        out = {"workload": args.workload, "arithmetic": sb.arithmetic(), "cycles": 64,
+               "us_per_cycle": 1e3 * e0.elapsed_time(e1) / 64, "lanes_left": sb.active()}
+        sb.close()
+        print(json.dumps(out), flush=True)
         return
     if args.kernel_only:
         sb = R.batch("static")
@@ -705,6 +737,55 @@ def main():
     if world > 1:
         dist.barrier()
         dist.destroy_process_group()
+
+
+def shadow_replay(R, args, max_cycles=4000):
+    """Shadow replay of the audit (the paper's attribution campaign counts screen-negative audits that a
+    full check would already have released, and the largest gap between the screen and the full row
+    residual).  Lanes stay in place (MASKED), one cycle per step; after every cycle the row residual of the
+    current state is computed DIRECTLY from its potentials (a float64 pass over all pairs,
+    sinkhorn_row_residual_static), and one cycle later the library reports what its fused screen made of
+    that same state."""
+    torch, B, w = R.torch, R.B, R.w
+    W, n, m, d = w.shape
+    if W > 256 or n > 8192:
+        raise SystemExit("--shadow-replay: at most 256 lanes (use --lanes) of at most 8192 points")
+    x32, y32 = R.x.float(), R.y.float()
+    sb = R.batch("masked")
+    tol = w.tol
+    negatives = missed_ready = early_ready = events = 0
+    worst, worst_rel = 0.0, 0.0
+    direct_prev = None
+    running = torch.ones(W, dtype=torch.bool, device=R.dev)
+    for k in range(1, max_cycles + 1):
+        sb.step(1)
+        if direct_prev is not None:
+            screen, _, _ = sb.last_audit()                   # the screen of the state after k-1 cycles
+            sel = running & ~torch.isnan(screen)
+            dp, sc = direct_prev[sel].double(), screen[sel].double()
+            events += int(sel.sum().item())
+            neg = sc > tol
+            negatives += int(neg.sum().item())
+            missed_ready += int((neg & (dp <= tol)).sum().item())
+            early_ready += int((~neg & (dp > tol)).sum().item())
+            if dp.numel():
+                gap = (sc - dp).abs()
+                worst = max(worst, float(gap.max().item()))
+                worst_rel = max(worst_rel, float((gap / dp.clamp_min(1e-300)).max().item()))
+        depth, status = sb.depths()
+        running = status == 0
+        if not bool(running.any().item()):
+            break
+        f, g = sb.potentials(f64=True)
+        direct_prev = B.sinkhorn_row_residual_static(x32, y32, R.a, f, g, R.eps)
+    cycles = sb.stats()["cycles"]
+    arith = sb.arithmetic()
+    sb.close()
+    return {"report": "shadow-replay", "workload": args.workload, "W": W, "n": n, "m": m, "d": d, "tol": tol,
+            "arithmetic": arith, "cycles": cycles, "lane_audits_compared": events, "screen_negative": negatives,
+            "missed_ready": missed_ready, "screen_positive_but_direct_above_tol": early_ready,
+            "max_abs_screen_minus_direct": worst, "max_rel_screen_minus_direct": worst_rel,
+            "paper_in_kind": {"screen_negative": 1488, "missed_ready": 0, "max_discrepancy": 1.86e-7}}
 
 
 def move_accounting(w, widths, depth, R):

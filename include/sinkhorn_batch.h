@@ -169,6 +169,18 @@ skb_status sinkhorn_batch_depths(skb_batch *h, int *depth, int *lane_status);
 skb_status sinkhorn_batch_residuals(skb_batch *h, float *r_row, float *r_col);
 
 /*
+ * What the most recent audit measured, per lane still held in a slot (device outs [W], original
+ * lane order, any may be null; entries of lanes that have left are not touched): the fused row
+ * screen's value r_row, the column residual r_col of screen-positive lanes (NaN otherwise) and
+ * whether the lane was screen-positive.  After step(k) these belong to the state after k-1
+ * cycles: the screen of a state is a by-product of the NEXT f-leg.  For shadow replays of the
+ * audit (Section 5's attribution: does the screen ever hold back a lane the full check would
+ * release?).  Kept by the one-launch-per-leg path only: MASKED, STATIC, tensor-core or profiled
+ * batches (SKB_ERR_STATE otherwise).  Enqueues one kernel.
+ */
+skb_status sinkhorn_batch_last_audit(skb_batch *h, float *r_row, float *r_col, int *flagged);
+
+/*
  * Phases of the time model T_active = sum_k c_k(A_k) + H_screen + H_check + H_compact
  * (Section "Hardware realization and break-even", Eq. 11): the update legs are c_k (the row
  * screen rides inside the f-leg, so H_screen has no time of its own), the column check is

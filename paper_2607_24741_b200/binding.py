@@ -29,7 +29,7 @@ EXPORTS = (
     "sinkhorn_batch_host_workspace_bytes", "sinkhorn_batch_solve_host",
     "sinkhorn_batch_launch_count", "sinkhorn_batch_profile_update", "sinkhorn_batch_arithmetic",
     "sinkhorn_batch_selftest_bounded_wait", "sinkhorn_batch_warm_start", "sinkhorn_batch_set_profiling",
-    "sinkhorn_batch_cycle_trace", "sinkhorn_batch_selftest_unit_rates",
+    "sinkhorn_batch_cycle_trace", "sinkhorn_batch_selftest_unit_rates", "sinkhorn_batch_last_audit",
 )
 PHASES = ("create", "f_leg", "column_check", "plan", "emit_move", "g_leg")
 # entry points outside the sinkhorn_batch_* family
@@ -73,6 +73,7 @@ def _load():
     lib.sinkhorn_batch_stats.argtypes = [vp, ctypes.POINTER(ctypes.c_longlong), ctypes.POINTER(ctypes.c_int),
                                          vp, ctypes.c_int, ctypes.POINTER(ctypes.c_longlong),
                                          ctypes.POINTER(ctypes.c_float)]
+    lib.sinkhorn_batch_last_audit.argtypes = [vp, vp, vp, vp]
     lib.sinkhorn_batch_warm_start.argtypes = [vp, vp, vp, ctypes.c_int]
     lib.sinkhorn_batch_set_profiling.argtypes = [vp, ctypes.c_int]
     lib.sinkhorn_batch_cycle_trace.argtypes = [vp, vp, ctypes.c_int, ctypes.POINTER(ctypes.c_int)]
@@ -251,6 +252,14 @@ class SinkhornBatch:
                 raise ValueError("f0 [W,n] and g0 [W,m] must be contiguous float64 CUDA tensors")
         _check(lib.sinkhorn_batch_warm_start(self.h, _ptr(f0), _ptr(g0), 1 if audit_initial else 0), self.h)
         self._warm = (f0, g0)
+
+    def last_audit(self):
+        """Row screen value, column residual (NaN where not checked) and screen flag of the most recent audit."""
+        rr = torch.full((self.W,), float("nan"), dtype=torch.float32, device=self.device)
+        rc = torch.full((self.W,), float("nan"), dtype=torch.float32, device=self.device)
+        fl = torch.full((self.W,), -1, dtype=torch.int32, device=self.device)
+        _check(lib.sinkhorn_batch_last_audit(self.h, _ptr(rr), _ptr(rc), _ptr(fl)), self.h)
+        return rr, rc, fl
 
     def set_profiling(self, on=True):
         _check(lib.sinkhorn_batch_set_profiling(self.h, 1 if on else 0), self.h)

@@ -213,9 +213,9 @@ extern "C" skb_status sinkhorn_batch_create(const void *x, const void *y, const 
     const Variant *var_big = variant_for(cfg, automatic ? SKB_COMPUTE_MIXED : cfg->compute);
     if (!var || !var_big) return fail(nullptr, SKB_ERR_SHAPE, "dimension d is not supported by any update kernel");
     const int mx = cfg->n > cfg->m ? cfg->n : cfg->m;
-    if ((mx + var->rows_per_cta - 1) / var->rows_per_cta > MAX_PARTS ||
-        (mx + var_big->rows_per_cta - 1) / var_big->rows_per_cta > MAX_PARTS)
-        return fail(nullptr, SKB_ERR_SHAPE, "n or m too large for the residual scratch");
+    // a lane's residual is a 64-bit fixed-point sum of per-row terms clamped at RSUM_ROW_MAX
+    if ((double)mx * RSUM_ROW_MAX * RSUM_SCALE >= 18446744073709551616.0)
+        return fail(nullptr, SKB_ERR_SHAPE, "n and m must be at most 262143 (fixed-point residual sums)");
     if (cfg->W > 65535) return fail(nullptr, SKB_ERR_SHAPE, "W must be <= 65535");
     const bool can_tensor = tc_eligible(cfg->d, cfg->xy_dtype == SKB_BF16);
     if (cfg->compute == SKB_COMPUTE_TENSOR && !can_tensor)
@@ -552,6 +552,15 @@ extern "C" skb_status sinkhorn_batch_residuals(skb_batch *h, float *r_row, float
     launch_gather_small(h->dev, nullptr, nullptr, r_row, r_col, h->stream);
     cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? SKB_OK : cuda_fail(h, e, "residuals");
+}
+
+extern "C" skb_status sinkhorn_batch_last_audit(skb_batch *h, float *r_row, float *r_col, int *flagged)
+{
+    if (!h) return SKB_ERR_NULL;
+    if (cycles_in_one_launch(h)) return fail(h, SKB_ERR_STATE, "per-audit values are kept by the one-launch-per-leg path only (MASKED, STATIC, tensor or profiled batches)");
+    launch_gather_audit(h->dev, r_row, r_col, flagged, h->stream);
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? SKB_OK : cuda_fail(h, e, "last_audit");
 }
 
 extern "C" skb_status sinkhorn_batch_stats(skb_batch *h, long long *slots, int *cycles, int *widths,

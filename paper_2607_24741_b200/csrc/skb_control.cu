@@ -540,6 +540,22 @@ __global__ void gather_small_kernel(const Dev P, int *depth, int *status, float 
     if (rcol) rcol[t] = (float)P.res_col[t];
 }
 
+// What the most recent audit measured for the lanes still held in a slot (one-launch-per-leg path).
+__global__ void gather_audit_kernel(const Dev P, float *rrow, float *rcol, int *flagged)
+{
+    const Ctl c = *P.ctl;
+    const int s = blockIdx.x * blockDim.x + threadIdx.x;
+    if (s >= P.W || s >= c.n_phys) return;
+    const int lane = P.lane_id[s];
+    if (rrow) rrow[lane] = (float)P.rrow[s];
+    if (rcol) rcol[lane] = P.flag[s] ? (float)P.rcol[s] : __int_as_float(0x7fc00000);
+    if (flagged) flagged[lane] = P.flag[s];
+}
+void launch_gather_audit(const Dev &P, float *rrow, float *rcol, int *flagged, cudaStream_t st)
+{
+    gather_audit_kernel<<<(P.W + 255) / 256, 256, 0, st>>>(P, rrow, rcol, flagged);
+}
+
 // ---------------------------------------------------------------- launchers
 void launch_lane_stats(const Dev &P, const void *x, const void *y, const float *eps, double *, cudaStream_t st)
 {

@@ -27,10 +27,10 @@ enum Form : int { FORM_DOT = 0, FORM_DIFF = 1 };
 constexpr float NEG_BIG = -1.0e30f;   // "minus infinity" for padded columns (finite: no NaNs)
 constexpr int UPD_THREADS = 128;
 constexpr int TC_MAX_SPLIT = 8;      // a row block's columns go to at most this many clusters
-constexpr int MAX_PARTS = 1024;       // upper bound on row blocks per lane
+constexpr int MAX_CLUSTER_RANKS = 8;  // blocks per cluster (portable limit): row blocks of a lane in the multi-cycle kernels
 constexpr double RSUM_SCALE = 17592186044416.0;     // 2^44: unit of the fixed-point residual sums
 constexpr double RSUM_ROW_MAX = 4.0;                 // one row's term is clamped here (a whole L1 residual never exceeds 2 near
-                                                     // convergence), so 65536 rows cannot overflow 64 bits
+                                                     // convergence), so fewer than 2^18 rows cannot overflow 64 bits
 
 // Device-resident control block.  Written by the plan kernel (one CTA), read by all.
 struct Ctl {

@@ -41,7 +41,7 @@ struct Variant {
     // several whole cycles per launch, one thread-block cluster per lane; null where there is none
     void (*launch_cycles)(const Dev &, int cycles, int width, cudaStream_t);
 };
-constexpr int MAX_CLUSTER_BLOCKS = 8;       // portable cluster size: a lane needs at most this many row blocks
+constexpr int MAX_CLUSTER_BLOCKS = MAX_CLUSTER_RANKS;   // a lane needs at most this many row blocks
 constexpr int MAX_CYCLES_IN_LAUNCH = 64;    // upper bound on the cycles one multi-cycle launch runs
 // Picks the variant for a shape (depends on the static shape only, so that every mode
 // and every run of the same batch uses the same reduction order).  Null if unsupported.
@@ -62,6 +62,7 @@ void launch_update_tc(const Dev &P, const void *maps, int leg, int width, cudaSt
 int launch_emit_move(const Dev &P, int width, cudaStream_t st);
 int launch_plan_cycles(const Dev &P, int width, int cycles, cudaStream_t st);
 void launch_gather(const Dev &P, void *f, void *g, bool f64, cudaStream_t st);
+void launch_gather_audit(const Dev &P, float *rrow, float *rcol, int *flagged, cudaStream_t st);
 void launch_gather_small(const Dev &P, int *depth, int *status, float *rrow, float *rcol, cudaStream_t st);
 
 }  // namespace skb

@@ -6,6 +6,8 @@
 
 namespace skb {
 
+constexpr size_t RESIDENT_SMEM_LIMIT = 52 * 1024; // shared memory of a block of the resident multi-cycle kernel: four blocks fit an SM
+
 constexpr long long NARROW_BLOCKS = 148 * 4;      // below this many blocks some SM has fewer than four
 
 template <typename T, int DP, int CS, int XF>
@@ -39,22 +41,16 @@ static void launch_update(const Dev &P, int leg, int width, cudaStream_t st)
     }
     if constexpr (sizeof(T) == 4 && DP <= 4 && CS == 4) {
         // Few dimensions, bound by the special-function unit: when a narrow batch would leave SMs
-        // without a block, fewer rows per thread give 2x or 4x the blocks (same bits, see above).
+        // without a block, one row per thread gives twice the blocks (same bits, see above).
         static bool attr_narrow = false;
         if (!attr_narrow) {
-            cudaFuncSetAttribute(update_kernel<T, DP, CS, XF, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
             cudaFuncSetAttribute(update_kernel<T, DP, CS, XF, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
             attr_narrow = true;
         }
-        const auto blocks = [&](int r) { const int rbr = (UPD_THREADS / 32) * r * (32 / CS); return (long long)((nrows + rbr - 1) / rbr) * lanes; };
-        if (blocks(Tune<T, DP>::R) < NARROW_BLOCKS) {
-            if (blocks(2) >= NARROW_BLOCKS) {
-                const int rbr = (UPD_THREADS / 32) * 2 * (32 / CS);
-                launch_pdl(update_kernel<T, DP, CS, XF, 2>, dim3((nrows + rbr - 1) / rbr, lanes), dim3(UPD_THREADS), smem, st, P, leg);
-            } else {
-                const int rbr = (UPD_THREADS / 32) * 1 * (32 / CS);
-                launch_pdl(update_kernel<T, DP, CS, XF, 1>, dim3((nrows + rbr - 1) / rbr, lanes), dim3(UPD_THREADS), smem, st, P, leg);
-            }
+        const int rb2 = (UPD_THREADS / 32) * Tune<T, DP>::R * (32 / CS);
+        if ((long long)((nrows + rb2 - 1) / rb2) * lanes < NARROW_BLOCKS) {
+            const int rbr = (UPD_THREADS / 32) * 1 * (32 / CS);
+            launch_pdl(update_kernel<T, DP, CS, XF, 1>, dim3((nrows + rbr - 1) / rbr, lanes), dim3(UPD_THREADS), smem, st, P, leg);
             return;
         }
     }
@@ -76,16 +72,27 @@ static void launch_cycles(const Dev &P, int cycles, int width, cudaStream_t st)
     const int rb = (UPD_THREADS / 32) * Tune<T, DP>::R * (32 / CS);
     const int mx = P.n > P.m ? P.n : P.m;
     const int nc = (mx + rb - 1) / rb;
+    // a lane small enough to live in shared memory for the whole launch (at four blocks per SM)
+    const size_t res_smem = ResidentLayout<T, DP, CS>::bytes(P.n, P.m);
+    const bool resident = res_smem <= RESIDENT_SMEM_LIMIT;
+    if (resident) {
+        static bool res_attr_set = false;
+        if (!res_attr_set) {
+            cudaFuncSetAttribute(lane_resident_kernel<T, DP, CS, XF>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)RESIDENT_SMEM_LIMIT);
+            res_attr_set = true;
+        }
+    }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(nc, width < 1 ? 1 : width); cfg.blockDim = dim3(UPD_THREADS);
-    cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cfg.dynamicSmemBytes = resident ? res_smem : smem; cfg.stream = st;
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     attr[1].id = cudaLaunchAttributeClusterDimension;
     attr[1].val.clusterDim.x = nc; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
     cfg.attrs = attr; cfg.numAttrs = 2;
-    cudaLaunchKernelEx(&cfg, lane_cycles_kernel<T, DP, CS, XF>, P, cycles);
+    if (resident) cudaLaunchKernelEx(&cfg, lane_resident_kernel<T, DP, CS, XF>, P, cycles);
+    else cudaLaunchKernelEx(&cfg, lane_cycles_kernel<T, DP, CS, XF>, P, cycles);
 }
 
 #define SKB_V(T, F64, XF, DP, CS) \

@@ -52,8 +52,11 @@ template <typename T, int DP> struct Tune;
 #ifndef SKB_UNROLL_Q
 #define SKB_UNROLL_Q 1
 #endif
+// (fp32, d <= 4: two rows measured faster than four at every width of the registration workload -
+// f-leg 609 against 628 us at 32 lanes, 319 against 331 us at 16 - because twice the blocks balance
+// better over the SMs, which outweighs the extra shared-memory loads per pair.)
 template <int DP> struct Tune<float, DP> {
-    static constexpr int R = DP <= 8 ? 4 : (DP == 16 ? SKB_F32_R16 : 2);
+    static constexpr int R = DP <= 4 ? 2 : (DP <= 8 ? 4 : (DP == 16 ? SKB_F32_R16 : 2));
     static constexpr int CW = DP <= 8 ? 8 : (DP == 16 ? SKB_F32_CW16 : 4);
 };
 #ifndef SKB_F64_R
@@ -165,12 +168,16 @@ __device__ __forceinline__ void load_tile(T *dst, const T *colc, const T *colt, 
 // ------------------------------------------------------------------ fp32, packed pairs
 // Leaves per row the integer-valued maximum mx[r] and sd[r] = sum 2^(arg - mx[r]) over the
 // columns this thread visited.
-template <int DP, int CS, int FORM, int R>
+// RES = 1: every column tile of the lane is already resident in shared memory (tile t at
+// sm + t * res_stride, its term rows at row res_trow and res_trow + 1 of the tile); nothing is
+// loaded and no block-wide barrier is needed.  Same steps in the same order, same bits.
+template <int DP, int CS, int FORM, int R, int RES = 0>
 __device__ __forceinline__ void stream_f32(float *sm, const float *colc, const float *colt, const float *coll,
                                            const int cp, const int ncols,
                                            const float (&xrow)[R][DP],
                                            const float (&ph)[R], const int tid, const int cs,
-                                           float (&mx)[R], double (&sd)[R])
+                                           float (&mx)[R], double (&sd)[R],
+                                           const int res_stride = 0, const int res_trow = 0)
 {
     constexpr int CW = Tune<float, DP>::CW;
     constexpr int NP = CW / 2;                       // packed column pairs per step
@@ -192,18 +199,23 @@ __device__ __forceinline__ void stream_f32(float *sm, const float *colc, const f
     for (int r = 0; r < R; ++r) { mx[r] = NEG_BIG; ts[r] = 0ull; sd[r] = 0.0; }
 
     const int ntiles = (ncols + TJ - 1) / TJ;
-    load_tile<float, DP, TJ, NR>(sm, colc, colt, coll, cp, 0, tid);
-    cp_async_commit();
+    const int ctoff = RES ? res_trow * TJ : DP * TJ, cloff = ctoff + TJ;
+    if constexpr (!RES) {
+        load_tile<float, DP, TJ, NR>(sm, colc, colt, coll, cp, 0, tid);
+        cp_async_commit();
+    }
     for (int t = 0; t < ntiles; ++t) {
-        if (t + 1 < ntiles) {
-            load_tile<float, DP, TJ, NR>(sm + ((t + 1) & 1) * STAGE, colc, colt, coll, cp, (t + 1) * TJ, tid);
-            cp_async_commit();
-            cp_async_wait<1>();
-        } else {
-            cp_async_wait<0>();
+        if constexpr (!RES) {
+            if (t + 1 < ntiles) {
+                load_tile<float, DP, TJ, NR>(sm + ((t + 1) & 1) * STAGE, colc, colt, coll, cp, (t + 1) * TJ, tid);
+                cp_async_commit();
+                cp_async_wait<1>();
+            } else {
+                cp_async_wait<0>();
+            }
+            __syncthreads();
         }
-        __syncthreads();
-        const float *st = sm + (t & 1) * STAGE;
+        const float *st = RES ? sm + t * res_stride : sm + (t & 1) * STAGE;
         constexpr int UQ = SKB_UNROLL_Q;
 #pragma unroll UQ
         for (int q = 0; q < STEPS; ++q) {
@@ -212,7 +224,7 @@ __device__ __forceinline__ void stream_f32(float *sm, const float *colc, const f
             u64 ct[NP];
 #pragma unroll
             for (int h = 0; h < NP / 2; ++h) {
-                const ulonglong2 c = *reinterpret_cast<const ulonglong2 *>(st + DP * TJ + jj + 4 * h);
+                const ulonglong2 c = *reinterpret_cast<const ulonglong2 *>(st + ctoff + jj + 4 * h);
                 ct[2 * h] = c.x; ct[2 * h + 1] = c.y;
             }
             if (FORM == FORM_DOT) {
@@ -257,7 +269,7 @@ __device__ __forceinline__ void stream_f32(float *sm, const float *colc, const f
                 u64 cl[NP];
 #pragma unroll
                 for (int h = 0; h < NP / 2; ++h) {
-                    const ulonglong2 v = *reinterpret_cast<const ulonglong2 *>(st + (DP + 1) * TJ + jj + 4 * h);
+                    const ulonglong2 v = *reinterpret_cast<const ulonglong2 *>(st + cloff + jj + 4 * h);
                     cl[2 * h] = v.x; cl[2 * h + 1] = v.y;
                 }
 #pragma unroll
@@ -326,19 +338,20 @@ __device__ __forceinline__ void stream_f32(float *sm, const float *colc, const f
             sd[r] += (double)(t0 + t1);
             ts[r] = 0ull;
         }
-        __syncthreads();
+        if constexpr (!RES) __syncthreads();
     }
 }
 
 // ------------------------------------------------------------------ float64 arguments
 // XF = 1: exponentials on the fp32 special-function unit; XF = 0: software exp2 in float64.
-template <int DP, int CS, int XF, int R>
+template <int DP, int CS, int XF, int R, int RES = 0>
 __device__ __forceinline__ void stream_f64(double *sm, const double *colc, const double *colt,
                                            const int cp, const int ncols,
                                            const double (&xr)[R][DP],
                                            const int tid, const int cs,
                                            const double (&est)[R],
-                                           float (&mx)[R], double (&sd)[R])
+                                           float (&mx)[R], double (&sd)[R],
+                                           const int res_stride = 0, const int res_trow = 0)
 {
     constexpr int CW = Tune<double, DP>::CW;
     constexpr int TJ = TileCols<double, DP, CS>::value;
@@ -349,8 +362,11 @@ __device__ __forceinline__ void stream_f64(double *sm, const double *colc, const
     float ts[R];
     double md[R];
     const int ntiles = (ncols + TJ - 1) / TJ;
-    load_tile<double, DP, TJ, NR>(sm, colc, colt, colt, cp, 0, tid);
-    cp_async_commit();
+    const int ctoff = RES ? res_trow * TJ : DP * TJ;
+    if constexpr (!RES) {
+        load_tile<double, DP, TJ, NR>(sm, colc, colt, colt, cp, 0, tid);
+        cp_async_commit();
+    }
     // the reference points only now: the loads behind `est` have been in flight beside the tile's
 #pragma unroll
     for (int r = 0; r < R; ++r) {
@@ -358,22 +374,24 @@ __device__ __forceinline__ void stream_f64(double *sm, const double *colc, const
         md[r] = (double)mx[r]; ts[r] = 0.f; sd[r] = 0.0;
     }
     for (int t = 0; t < ntiles; ++t) {
-        if (t + 1 < ntiles) {
-            load_tile<double, DP, TJ, NR>(sm + ((t + 1) & 1) * STAGE, colc, colt, colt, cp, (t + 1) * TJ, tid);
-            cp_async_commit();
-            cp_async_wait<1>();
-        } else {
-            cp_async_wait<0>();
+        if constexpr (!RES) {
+            if (t + 1 < ntiles) {
+                load_tile<double, DP, TJ, NR>(sm + ((t + 1) & 1) * STAGE, colc, colt, colt, cp, (t + 1) * TJ, tid);
+                cp_async_commit();
+                cp_async_wait<1>();
+            } else {
+                cp_async_wait<0>();
+            }
+            __syncthreads();
         }
-        __syncthreads();
-        const double *st = sm + (t & 1) * STAGE;
+        const double *st = RES ? sm + t * res_stride : sm + (t & 1) * STAGE;
 #pragma unroll 1
         for (int q = 0; q < STEPS; ++q) {
             const int jj = (q * CS + cs) * CW;
             double acc[R][CW];
 #pragma unroll
             for (int h = 0; h < CW / 2; ++h) {
-                const double2 c0 = *reinterpret_cast<const double2 *>(st + DP * TJ + jj + 2 * h);
+                const double2 c0 = *reinterpret_cast<const double2 *>(st + ctoff + jj + 2 * h);
 #pragma unroll
                 for (int r = 0; r < R; ++r) { acc[r][2 * h] = c0.x; acc[r][2 * h + 1] = c0.y; }
             }
@@ -445,8 +463,36 @@ __device__ __forceinline__ void stream_f64(double *sm, const double *colc, const
 #pragma unroll
             for (int r = 0; r < R; ++r) { sd[r] += (double)ts[r]; ts[r] = 0.f; }
         }
-        __syncthreads();
+        if constexpr (!RES) __syncthreads();
     }
+}
+
+// The arithmetic of one row's epilogue.  m: integer-valued maximum, s: sum of 2^(arg - m) over all
+// columns, h: the fp32 shift a difference-form row carried, pold: the potential the leg started
+// from.  Gives the updated potential that makes the row's marginal equal to its weight (Eq. 3) and,
+// where asked, the row's term w |marginal/weight - 1| of the L1 residual of the state before the leg.
+__device__ __forceinline__ void row_math(const int form, const bool want_term, const double lw, const double sq,
+                                         const double w, const double pold, const float m, const double s,
+                                         const float h, double &pnew, double &term)
+{
+    const double L = (double)m + log2(s);
+    double lmarg;                          // log2 of the row's marginal under the potentials the leg started from
+    if (form == FORM_DOT) {
+        pnew = lw + sq - L;
+        lmarg = lw + pold - pnew;
+    } else {
+        lmarg = L - ((double)h - pold);
+        pnew = pold + (lw - lmarg);
+    }
+    term = want_term ? w * fabs(expm1((lmarg - lw) * 0.6931471805599453)) : 0.0;
+}
+// The per-point term the opposite leg streams: high part (expanded form: potential minus the scaled
+// squared norm) and low part (difference form only).
+template <typename T>
+__device__ __forceinline__ void split_potential(const int form, const double pnew, const double sq, T &hi, T &lo)
+{
+    if (form == FORM_DOT) { hi = (T)(pnew - sq); lo = T(0); }
+    else { hi = (T)pnew; lo = (T)(pnew - (double)hi); }
 }
 
 // Float64 epilogue of ONE row of a leg: `m` is the integer-valued maximum and `s` the sum of
@@ -464,23 +510,11 @@ __device__ __forceinline__ double finish_one_row(const Dev &P, const Ctl &c, con
     const double lw = (rows_x ? P.la2 : P.lb2)[o];
     const double sq = (rows_x ? P.sqx : P.sqy)[o];
     const double pold = prow[i];
-    const double L = (double)m + log2(s);
-    // log2 of this row's marginal under the potentials the leg started from, and the
-    // updated potential that makes the marginal equal to the weight (Eq. 3)
-    double lmarg, pnew;
-    if (form == FORM_DOT) {
-        pnew = lw + sq - L;
-        lmarg = lw + pold - pnew;
-    } else {
-        lmarg = L - ((double)h - pold);
-        pnew = pold + (lw - lmarg);
-    }
-    double term = 0.0;
-    if (leg != LEG_G) term = (rows_x ? P.wa : P.wb)[o] * fabs(expm1((lmarg - lw) * 0.6931471805599453));
+    double pnew, term;
+    row_math(form, leg != LEG_G, lw, sq, leg != LEG_G ? (rows_x ? P.wa : P.wb)[o] : 0.0, pold, m, s, h, pnew, term);
     if (writes) {
         T hi, lo;
-        if (form == FORM_DOT) { hi = (T)(pnew - sq); lo = T(0); }
-        else { hi = (T)pnew; lo = (T)(pnew - (double)hi); }
+        split_potential<T>(form, pnew, sq, hi, lo);
         if (leg == LEG_F) {
             P.phi[c.parity ^ 1][o] = pnew;
             reinterpret_cast<T *>(P.ft[c.parity ^ 1])[o] = hi;
@@ -518,7 +552,7 @@ __device__ __forceinline__ void finish_lane_residual(const Dev &P, const int leg
 template <typename T, int RB, int THREADS = UPD_THREADS>
 __device__ __forceinline__ void finish_rows(const Dev &P, const Ctl &c, const int leg, const int slot,
                                             const int form, const float *row_m, const double *row_s,
-                                            const float *row_h, double *red)
+                                            const float *row_h, double *red, const int row_base)
 {
     constexpr int NWARP = THREADS / 32;
     const int nrows = (leg == LEG_F) ? P.n : P.m;
@@ -527,7 +561,7 @@ __device__ __forceinline__ void finish_rows(const Dev &P, const Ctl &c, const in
     const bool writes = !frozen && leg != LEG_V && !P.dry_run;
     unsigned long long term_sum = 0ull;
     for (int lr = tid; lr < RB; lr += THREADS) {
-        const int i = blockIdx.x * RB + lr;
+        const int i = row_base + lr;
         if (i >= nrows) continue;
         const double term = finish_one_row<T>(P, c, leg, slot, form, i, row_m[lr], row_s[lr], row_h[lr], writes);
         if (leg != LEG_G) term_sum += residual_fixed(P, leg, slot, term, frozen);
@@ -548,6 +582,25 @@ __device__ __forceinline__ void finish_rows(const Dev &P, const Ctl &c, const in
     }
 }
 
+// Merge of the CS column splits of each row (lanes RG = 32 / CS apart hold the same rows): maxima are
+// integers, so the scalings are exact powers of two and each sum is rounded once.
+template <int CS, int R>
+__device__ __forceinline__ void merge_splits(float (&mx)[R], double (&sd)[R])
+{
+    constexpr int RG = 32 / CS;
+#pragma unroll
+    for (int off = 1; off < CS; off <<= 1) {
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            const float mo = __shfl_xor_sync(0xffffffffu, mx[r], off * RG);
+            const double so = __shfl_xor_sync(0xffffffffu, sd[r], off * RG);
+            const float mn = fmaxf(mx[r], mo);
+            sd[r] = sd[r] * (double)pow2i(mx[r] - mn) + so * (double)pow2i(mo - mn);
+            mx[r] = mn;
+        }
+    }
+}
+
 // Shared-memory scratch of one leg besides the column tiles.
 template <int RB>
 struct LegScratch {
@@ -557,17 +610,18 @@ struct LegScratch {
     double red[UPD_THREADS / 32];
 };
 
-// One leg for the row block blockIdx.x of the lane in `slot`: row operands, streaming reduction over
+// One leg for the RB rows from `row_base` on of the lane in `slot`: row operands, streaming reduction over
 // all columns, float64 epilogue, residual terms.  `c` supplies the cycle count and the buffer parity
 // of the state the leg starts from.  PDL_EARLY: this is an f-leg launched as a kernel of its own,
 // which reads its row operands while the kernel before it is still finishing and waits for it only
 // before the column terms.  A row's arithmetic does not depend on the thread that holds it, nor on
 // whether the leg runs as its own launch or inside the multi-cycle kernel below, so every way of
 // running it gives the same bits.
-template <typename T, int DP, int CS, int XF, int R, bool PDL_EARLY>
+template <typename T, int DP, int CS, int XF, int R, bool PDL_EARLY, int RBS = (UPD_THREADS / 32) * R * (32 / CS)>
 __device__ __forceinline__ void run_leg(const Dev &P, const Ctl &c, const int leg, const int slot, T *sm,
-                                        LegScratch<(UPD_THREADS / 32) * R * (32 / CS)> &sc)
+                                        LegScratch<RBS> &sc, const int row_base)
 {
+    static_assert(RBS >= (UPD_THREADS / 32) * R * (32 / CS), "scratch smaller than the row block");
     constexpr int RG = 32 / CS;                  // row groups per warp
     constexpr int RW = R * RG;                   // rows per warp
     constexpr int NWARP = UPD_THREADS / 32;
@@ -577,7 +631,7 @@ __device__ __forceinline__ void run_leg(const Dev &P, const Ctl &c, const int le
     const bool rows_x = (leg == LEG_F);
     const int nrows = rows_x ? P.n : P.m, rp = rows_x ? P.np : P.mp;
     const int ncols = rows_x ? P.m : P.n, cp = rows_x ? P.mp : P.np;
-    if ((int)blockIdx.x * RB >= nrows) return;
+    if (row_base >= nrows) return;
     const int form = (sizeof(T) == 8) ? (int)FORM_DOT : P.form[slot];   // float64 arguments never need the difference form
     const T *rowc = reinterpret_cast<const T *>(rows_x ? P.xs : P.ys) + (size_t)slot * DP * rp;
     const T *colc = reinterpret_cast<const T *>(rows_x ? P.ys : P.xs) + (size_t)slot * DP * cp;
@@ -593,13 +647,13 @@ __device__ __forceinline__ void run_leg(const Dev &P, const Ctl &c, const int le
     // shared-memory address per load when CS <= 4 (a broadcast, the cheapest access pattern)
     const int cs = lane / RG, rg = lane % RG;
     const int lrow0 = warp * RW + rg * R;                // this thread's R consecutive CTA-local rows
-    const int row0 = blockIdx.x * RB + lrow0;
+    const int row0 = row_base + lrow0;
 
     // the float64 epilogue's operands (one thread per row, much later): start them on their way to
     // L1 now, so that the epilogue does not begin with a round trip to L2 (the column tiles
     // stream through cp.async and leave L1 alone)
     for (int lr = tid; lr < RB; lr += UPD_THREADS) {
-        const int i = blockIdx.x * RB + lr;
+        const int i = row_base + lr;
         if (i < nrows) {
             const size_t o = (size_t)slot * rp + i;
             asm volatile("prefetch.global.L1 [%0];" ::"l"((rows_x ? P.la2 : P.lb2) + o));
@@ -653,18 +707,7 @@ __device__ __forceinline__ void run_leg(const Dev &P, const Ctl &c, const int le
             stream_f64<DP, CS, XF, R>(sm, colc, colt, cp, ncols, xr, tid, cs, m0, mx, sd);
         }
 
-        // merge the CS column splits of each row: maxima are integers, so the scalings are exact
-#pragma unroll
-        for (int off = 1; off < CS; off <<= 1) {
-#pragma unroll
-            for (int r = 0; r < R; ++r) {
-                const float mo = __shfl_xor_sync(0xffffffffu, mx[r], off * RG);
-                const double so = __shfl_xor_sync(0xffffffffu, sd[r], off * RG);
-                const float mn = fmaxf(mx[r], mo);
-                sd[r] = sd[r] * (double)pow2i(mx[r] - mn) + so * (double)pow2i(mo - mn);
-                mx[r] = mn;
-            }
-        }
+        merge_splits<CS, R>(mx, sd);
         if constexpr (sizeof(T) == 8 && XF != 0) {
             if (pass == 0) {
                 bool low = false;
@@ -692,11 +735,12 @@ __device__ __forceinline__ void run_leg(const Dev &P, const Ctl &c, const int le
         }
     }
     __syncthreads();
-    finish_rows<T, RB>(P, c, leg, slot, form, sc.row_m, sc.row_s, sc.row_h, sc.red);
+    finish_rows<T, RB>(P, c, leg, slot, form, sc.row_m, sc.row_s, sc.row_h, sc.red, row_base);
 }
 
-// RR: rows per thread, 0 = the type's default.  Rows are independent and a row's arithmetic does
-// not depend on which thread holds it, so launches with different RR give the same bits.
+// One leg as a launch of its own.  RR: rows per thread, 0 = the type's default.  Rows are independent
+// and a row's arithmetic does not depend on which thread holds it, so launches with different RR
+// give the same bits.
 template <typename T, int DP, int CS, int XF, int RR = 0>
 __global__ void __launch_bounds__(UPD_THREADS) update_kernel(const Dev P, const int leg)
 {
@@ -719,11 +763,12 @@ __global__ void __launch_bounds__(UPD_THREADS) update_kernel(const Dev P, const 
     const Ctl c = *P.ctl;
     if (leg == LEG_V) asm volatile("griddepcontrol.wait;" ::: "memory");
     const int slot = blockIdx.y;
+    const int row_base = (int)blockIdx.x * RB;
     const bool idle = c.done || slot >= c.n_phys
                       || (P.early_exit && P.state[slot] != 0)   // early-exit mask arm: a frozen lane costs a launch slot only
                       || (leg != LEG_V && c.static_final)
                       || (leg == LEG_V && !(c.static_final || lane_flag(P, c, slot)))
-                      || (int)blockIdx.x * RB >= (leg == LEG_F ? P.n : P.m);
+                      || row_base >= (leg == LEG_F ? P.n : P.m);
     if (idle) {
         // Every kernel of the chain must wait at least once before it completes: a kernel's wait
         // covers its immediate predecessor only, and "everything earlier in the stream has finished"
@@ -733,7 +778,7 @@ __global__ void __launch_bounds__(UPD_THREADS) update_kernel(const Dev P, const 
         if (early && blockIdx.x == 0 && blockIdx.y == 0) asm volatile("griddepcontrol.wait;" ::: "memory");
         return;
     }
-    run_leg<T, DP, CS, XF, R, true>(P, c, leg, slot, sm, sc);
+    run_leg<T, DP, CS, XF, R, true>(P, c, leg, slot, sm, sc, row_base);
 }
 
 // ------------------------------------------------------------------ several cycles per launch
@@ -785,24 +830,34 @@ __global__ void __launch_bounds__(UPD_THREADS) lane_cycles_kernel(const Dev P, c
     const int tid = threadIdx.x;
     const int lane_id = P.lane_id[slot];
     const double inv_s = 1.0 / P.scale[slot];
-    unsigned long long seen_row = 0ull, seen_col = 0ull;     // totals already accounted for (the sums are only cleared at the end)
+    unsigned long long seen_row = 0ull, seen_col = 0ull;     // totals already accounted for (the planner clears the sums)
     int checks = 0, retired_at = 0;
 
-    for (int it = 0; it < cycles; ++it) {
-        // f-leg of cycle k+1; its epilogue also yields the row residual of the state after k cycles
-        run_leg<T, DP, CS, XF, R, false>(P, c, LEG_F, slot, sm, sc);
+    // One call site for the three kinds of leg (the leg is a run-time value), so that the streaming
+    // loops are instantiated once.  leg F: f-leg of cycle k+1, whose epilogue also yields the row
+    // residual of the state after k cycles; leg V: column check of that state; leg G: g-leg.
+    int leg = LEG_F, it = 0, nf = 0;
+    double rr = 0.0, rc = 0.0;
+    bool fl = false;
+    for (;;) {
+        run_leg<T, DP, CS, XF, R, false>(P, c, leg, slot, sm, sc, (int)blockIdx.x * RB);
         cluster_sync_all();
-        const unsigned long long tot_row = ld_cg_u64(P.rsum_row + slot);
-        const double rr = (double)(tot_row - seen_row) * (1.0 / RSUM_SCALE);
-        seen_row = tot_row;
-        int nf = ld_cg_s32(P.nonfinite + slot);
+        if (leg == LEG_G) {
+            if (++it >= cycles) break;
+            leg = LEG_F;
+            continue;
+        }
         const int k = c.cycle;
-        const bool audited = (k >= 1 && (k % P.audit_every) == 0) || (k == 0 && P.audit_initial);
-        const bool fl = audited && !nf && rr <= P.tol_screen;
-        double rc = 0.0;
-        if (fl) {                                // two-sided check: the column marginal, genuinely measured
-            run_leg<T, DP, CS, XF, R, false>(P, c, LEG_V, slot, sm, sc);
-            cluster_sync_all();
+        if (leg == LEG_F) {
+            const unsigned long long tot_row = ld_cg_u64(P.rsum_row + slot);
+            rr = (double)(tot_row - seen_row) * (1.0 / RSUM_SCALE);
+            seen_row = tot_row;
+            nf = ld_cg_s32(P.nonfinite + slot);
+            const bool audited = (k >= 1 && (k % P.audit_every) == 0) || (k == 0 && P.audit_initial);
+            fl = audited && !nf && rr <= P.tol_screen;
+            rc = 0.0;
+            if (fl) { leg = LEG_V; continue; }     // two-sided check: the column marginal, genuinely measured
+        } else {
             const unsigned long long tot_col = ld_cg_u64(P.rsum_col + slot);
             rc = (double)(tot_col - seen_col) * (1.0 / RSUM_SCALE);
             seen_col = tot_col;
@@ -836,8 +891,7 @@ __global__ void __launch_bounds__(UPD_THREADS) lane_cycles_kernel(const Dev P, c
         }
         c.cycle = k + 1;
         c.parity ^= 1;
-        run_leg<T, DP, CS, XF, R, false>(P, c, LEG_G, slot, sm, sc);
-        cluster_sync_all();
+        leg = LEG_G;
     }
     // hand over to the planner: when the lane left (0 = still running) and how many column checks
     // it ran.  The residual sums are left as they are (another block of the cluster may still be
@@ -845,6 +899,305 @@ __global__ void __launch_bounds__(UPD_THREADS) lane_cycles_kernel(const Dev P, c
     if (blockIdx.x == 0 && tid == 0) {
         P.ret_at[slot] = retired_at;
         P.n_checks[slot] = checks;
+    }
+}
+
+
+// ------------------------------------------------------------------ several cycles per launch, lane in shared memory
+// The same walk as lane_cycles_kernel, with the lane's whole state resident in the cluster's shared
+// memory for the length of the launch: every block holds ALL column tiles of both clouds
+// (coordinates and per-point terms, in the streaming kernels' tile layout) and the float64
+// potentials and constants of its OWN rows.  A leg streams from shared memory; its epilogue
+// writes each new per-point term into the tile copies of every block of the cluster (distributed
+// shared memory) and the block's part of the residual into every block's table, and ONE cluster
+// barrier per leg makes them visible.  Inside the loop nothing touches global memory but the
+// (constant, L1-resident) row coordinates; the state is loaded once and written back once.
+// Tile t of the y cloud: rows 0..DP-1 coordinates, row DP term, row DP+1 low part.
+// Tile t of the x cloud: coordinates, then (term, low part) of buffer parity 0 and of parity 1: the
+// f-leg writes the look-ahead potentials into the other parity while the column check may still
+// need the current one.
+template <typename V>
+__device__ __forceinline__ void st_cluster(V *local, const unsigned rank, const V v)
+{
+    const unsigned laddr = (unsigned)__cvta_generic_to_shared(local);
+    unsigned raddr;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(raddr) : "r"(laddr), "r"(rank));
+    if constexpr (sizeof(V) == 8) {
+        unsigned long long bits;
+        memcpy(&bits, &v, 8);
+        asm volatile("st.shared::cluster.b64 [%0], %1;" ::"r"(raddr), "l"(bits) : "memory");
+    } else {
+        unsigned bits;
+        memcpy(&bits, &v, 4);
+        asm volatile("st.shared::cluster.b32 [%0], %1;" ::"r"(raddr), "r"(bits) : "memory");
+    }
+}
+
+template <typename T, int DP, int CS>
+struct ResidentLayout {
+    static constexpr int R = Tune<T, DP>::R;
+    static constexpr int RB = (UPD_THREADS / 32) * R * (32 / CS);
+    static constexpr int TJ = TileCols<T, DP, CS>::value;
+    static constexpr int STY = (DP + 2) * TJ;
+    static constexpr int STX = (DP + 4) * TJ;
+    static constexpr int NDBL = 9;                     // float64 arrays of RB own rows each
+    static size_t bytes(const int n, const int m)
+    {
+        const size_t ntx = (n + TJ - 1) / TJ, nty = (m + TJ - 1) / TJ;
+        return sizeof(T) * (nty * STY + ntx * STX) + (size_t)NDBL * RB * sizeof(double);
+    }
+};
+
+template <typename T, int DP, int CS, int XF>
+__global__ void __launch_bounds__(UPD_THREADS) lane_resident_kernel(const Dev P, const int cycles)
+{
+    typedef ResidentLayout<T, DP, CS> L;
+    constexpr int R = L::R, RB = L::RB, TJ = L::TJ, STY = L::STY, STX = L::STX;
+    constexpr int RG = 32 / CS, RW = R * RG;
+
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    __shared__ LegScratch<RB> sc;
+    __shared__ unsigned long long part[2][MAX_CLUSTER_RANKS];    // [row | column residual][block of the cluster]
+    __shared__ int part_nf[2][MAX_CLUSTER_RANKS];
+
+    pdl_enter();
+    Ctl c = *P.ctl;
+    const int slot = blockIdx.y;
+    if (c.done || slot >= c.n_phys) return;      // the whole cluster takes this exit together
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int b = blockIdx.x, NC = gridDim.x;
+    const int ntY = (P.m + TJ - 1) / TJ, ntX = (P.n + TJ - 1) / TJ;
+    T *colsY = reinterpret_cast<T *>(smem_raw);
+    T *colsX = colsY + (size_t)ntY * STY;
+    double *own = reinterpret_cast<double *>(colsX + (size_t)ntX * STX);
+    double *lwx = own, *sqx = own + RB, *wax = own + 2 * RB, *lwy = own + 3 * RB, *sqy = own + 4 * RB, *wby = own + 5 * RB;
+    double *potx[2] = {own + 6 * RB, own + 7 * RB};
+    double *poty = own + 8 * RB;
+
+    // ---- the lane comes in: all column tiles of both clouds, this block's rows of everything else
+    const T *xs = reinterpret_cast<const T *>(P.xs) + (size_t)slot * DP * P.np;
+    const T *ys = reinterpret_cast<const T *>(P.ys) + (size_t)slot * DP * P.mp;
+    for (int t = 0; t < ntY; ++t)
+        load_tile<T, DP, TJ, DP + 2>(colsY + (size_t)t * STY, ys, reinterpret_cast<const T *>(P.gt) + (size_t)slot * P.mp,
+                                     reinterpret_cast<const T *>(P.gl) + (size_t)slot * P.mp, P.mp, t * TJ, tid);
+    for (int t = 0; t < ntX; ++t) {
+        load_tile<T, DP, TJ, DP + 2>(colsX + (size_t)t * STX, xs, reinterpret_cast<const T *>(P.ft[0]) + (size_t)slot * P.np,
+                                     reinterpret_cast<const T *>(P.fl[0]) + (size_t)slot * P.np, P.np, t * TJ, tid);
+        load_tile<T, 0, TJ, 2>(colsX + (size_t)t * STX + (DP + 2) * TJ, xs, reinterpret_cast<const T *>(P.ft[1]) + (size_t)slot * P.np,
+                               reinterpret_cast<const T *>(P.fl[1]) + (size_t)slot * P.np, P.np, t * TJ, tid);
+    }
+    cp_async_commit();
+    for (int lr = tid; lr < RB; lr += UPD_THREADS) {
+        const int i = b * RB + lr;
+        if (i < P.n) {
+            const size_t o = (size_t)slot * P.np + i;
+            lwx[lr] = P.la2[o]; sqx[lr] = P.sqx[o]; wax[lr] = P.wa[o];
+            potx[0][lr] = P.phi[0][o]; potx[1][lr] = P.phi[1][o];
+        }
+        if (i < P.m) {
+            const size_t o = (size_t)slot * P.mp + i;
+            lwy[lr] = P.lb2[o]; sqy[lr] = P.sqy[o]; wby[lr] = P.wb[o];
+            poty[lr] = P.gam[o];
+        }
+    }
+    cp_async_wait<0>();
+    const int form = (sizeof(T) == 8) ? (int)FORM_DOT : P.form[slot];
+    const int lane_id = P.lane_id[slot];
+    const double inv_s = 1.0 / P.scale[slot];
+    cluster_sync_all();                          // every block's tables exist before anyone writes into them
+
+    // one leg on the resident state; leaves this block's part of the residual in every block's table
+    auto leg_resident = [&](const int leg, const int parity) {
+        const bool rows_x = (leg == LEG_F);
+        const int nrows = rows_x ? P.n : P.m, rp = rows_x ? P.np : P.mp;
+        const int ncols = rows_x ? P.m : P.n, cp = rows_x ? P.mp : P.np;
+        unsigned long long block_sum = 0ull;
+        int block_nf = 0;
+        if (b * RB < nrows) {
+            const T *rowc = rows_x ? xs : ys;
+            T *cols = rows_x ? colsY : colsX;
+            const int stride = rows_x ? STY : STX;
+            const int trow = rows_x ? DP : DP + 2 * parity;       // the g-leg and the column check read f of `parity`
+            const double *prow = rows_x ? potx[parity] : poty;    // indexed by the block-local row
+            const double *lw = rows_x ? lwx : lwy, *sq = rows_x ? sqx : sqy, *wt = rows_x ? wax : wby;
+            const int cs = lane / RG, rg = lane % RG;
+            const int lrow0 = warp * RW + rg * R;
+            const int row0 = b * RB + lrow0;
+            T xr[R][DP];
+            T ph[R];
+#pragma unroll
+            for (int k = 0; k < DP; ++k) {
+                T v[R];
+                load_rows<T, R>(rowc + (size_t)k * rp + row0, row0 < rp, v);
+#pragma unroll
+                for (int r = 0; r < R; ++r) xr[r][k] = v[r];
+            }
+#pragma unroll
+            for (int r = 0; r < R; ++r) ph[r] = (row0 + r < nrows && form == FORM_DIFF) ? (T)prow[lrow0 + r] : T(0);
+            float mx[R];
+            double sd[R];
+            double m0[R];
+#pragma unroll
+            for (int r = 0; r < R; ++r) m0[r] = (double)NEG_BIG;
+            if constexpr (sizeof(T) == 8 && XF != 0) {
+#pragma unroll
+                for (int r = 0; r < R; ++r)
+                    if (row0 + r < nrows) m0[r] = lw[lrow0 + r] + sq[lrow0 + r] - prow[lrow0 + r];
+            }
+#pragma unroll 1
+            for (int pass = 0; pass < 2; ++pass) {
+                if constexpr (sizeof(T) == 4) {
+                    if (form == FORM_DOT) stream_f32<DP, CS, FORM_DOT, R, 1>(cols, nullptr, nullptr, nullptr, cp, ncols, xr, ph, tid, cs, mx, sd, stride, trow);
+                    else stream_f32<DP, CS, FORM_DIFF, R, 1>(cols, nullptr, nullptr, nullptr, cp, ncols, xr, ph, tid, cs, mx, sd, stride, trow);
+                } else {
+                    stream_f64<DP, CS, XF, R, 1>(cols, nullptr, nullptr, cp, ncols, xr, tid, cs, m0, mx, sd, stride, trow);
+                }
+                merge_splits<CS, R>(mx, sd);
+                if constexpr (sizeof(T) == 8 && XF != 0) {
+                    if (pass == 0) {
+                        bool low = false;
+#pragma unroll
+                        for (int r = 0; r < R; ++r)
+                            low = low || (row0 + r < nrows && fabs(m0[r]) < 1.0e7 && !(sd[r] >= 0x1p-20));
+                        if (!__syncthreads_or(low ? 1 : 0)) break;
+#pragma unroll
+                        for (int r = 0; r < R; ++r)
+                            if (row0 + r < nrows && fabs(m0[r]) < 1.0e7 && !(sd[r] >= 0x1p-20)) m0[r] = (double)NEG_BIG;
+                        continue;
+                    }
+                }
+                break;
+            }
+            if (cs == 0) {
+#pragma unroll
+                for (int r = 0; r < R; ++r) {
+                    sc.row_m[lrow0 + r] = mx[r];
+                    sc.row_s[lrow0 + r] = sd[r];
+                    sc.row_h[lrow0 + r] = (float)ph[r];
+                }
+            }
+            __syncthreads();
+            // float64 epilogue, one thread per row; new terms go to every block's copy of the tiles
+            unsigned long long term_sum = 0ull;
+            for (int lr = tid; lr < RB; lr += UPD_THREADS) {
+                const int i = b * RB + lr;
+                if (i >= nrows) continue;
+                double pnew, term;
+                row_math(form, leg != LEG_G, lw[lr], sq[lr], leg != LEG_G ? wt[lr] : 0.0, prow[lr], sc.row_m[lr], sc.row_s[lr],
+                         sc.row_h[lr], pnew, term);
+                if (leg != LEG_G) {
+                    if (!isfinite(term)) block_nf = 1;
+                    else term_sum += __double2ull_rn(fmin(term, RSUM_ROW_MAX) * RSUM_SCALE);
+                }
+                if (leg != LEG_V) {
+                    T hi, lo;
+                    split_potential<T>(form, pnew, sq[lr], hi, lo);
+                    T *dst;
+                    if (leg == LEG_F) {
+                        potx[parity ^ 1][lr] = pnew;
+                        dst = colsX + (size_t)(i / TJ) * STX + (DP + 2 * (parity ^ 1)) * TJ + (i % TJ);
+                    } else {
+                        poty[lr] = pnew;
+                        dst = colsY + (size_t)(i / TJ) * STY + DP * TJ + (i % TJ);
+                    }
+                    for (int rk = 0; rk < NC; ++rk) { st_cluster<T>(dst, rk, hi); st_cluster<T>(dst + TJ, rk, lo); }
+                }
+            }
+            if (leg != LEG_G) {
+                block_nf = __syncthreads_or(block_nf);
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) term_sum += __shfl_down_sync(0xffffffffu, term_sum, off);
+                unsigned long long *redu = reinterpret_cast<unsigned long long *>(sc.red);
+                if (lane == 0) redu[warp] = term_sum;
+                __syncthreads();
+                if (tid == 0) for (int w = 0; w < UPD_THREADS / 32; ++w) block_sum += redu[w];
+            }
+        }
+        if (leg != LEG_G && tid == 0) {
+            const int which = leg == LEG_F ? 0 : 1;
+            for (int rk = 0; rk < NC; ++rk) {
+                st_cluster<unsigned long long>(&part[which][b], rk, block_sum);
+                st_cluster<int>(&part_nf[which][b], rk, block_nf);
+            }
+        }
+        cluster_sync_all();
+    };
+
+    int checks = 0, retired_at = 0;
+    int leg = LEG_F, it = 0, nf = 0;
+    double rr = 0.0, rc = 0.0;
+    bool fl = false;
+    for (;;) {                                   // one call site for all three kinds of leg
+        leg_resident(leg, c.parity);
+        if (leg == LEG_G) {
+            if (++it >= cycles) break;
+            leg = LEG_F;
+            continue;
+        }
+        const int k = c.cycle;
+        if (leg == LEG_F) {
+            unsigned long long tot = 0ull;
+            nf = 0;
+            for (int rk = 0; rk < NC; ++rk) { tot += part[0][rk]; nf |= part_nf[0][rk]; }
+            rr = (double)tot * (1.0 / RSUM_SCALE);
+            const bool audited = (k >= 1 && (k % P.audit_every) == 0) || (k == 0 && P.audit_initial);
+            fl = audited && !nf && rr <= P.tol_screen;
+            rc = 0.0;
+            if (fl) { leg = LEG_V; continue; }
+        } else {
+            unsigned long long totc = 0ull;
+            for (int rk = 0; rk < NC; ++rk) { totc += part[1][rk]; nf |= part_nf[1][rk]; }
+            rc = (double)totc * (1.0 / RSUM_SCALE);
+            ++checks;
+        }
+        const bool vd = !nf && fmax(rr, rc) <= P.tol_stop;
+        const bool limit = k >= P.max_iter;
+        int st = LANE_RUNNING;
+        if (nf) st = LANE_NONFINITE;
+        else if (fl && vd) st = LANE_DONE;
+        else if (limit) st = LANE_ITER_LIMIT;
+        if (st != LANE_RUNNING) {
+            for (int lr = tid; lr < RB; lr += UPD_THREADS) {
+                const int i = b * RB + lr;
+                if (i < P.n) P.f_out[(size_t)lane_id * P.n + i] = potx[c.parity][lr] * inv_s;
+                if (i < P.m) P.g_out[(size_t)lane_id * P.m + i] = poty[lr] * inv_s;
+            }
+            if (b == 0 && tid == 0) {
+                P.res_row[lane_id] = rr;
+                P.res_col[lane_id] = fl ? rc : __longlong_as_double(0x7ff8000000000000LL);
+                P.depth[lane_id] = (limit && st != LANE_DONE) ? P.max_iter : k;
+                P.status[lane_id] = st;
+                P.emitted[lane_id] = 1;
+            }
+            retired_at = k + 1;
+            break;
+        }
+        c.cycle = k + 1;
+        c.parity ^= 1;
+        leg = LEG_G;
+    }
+    if (b == 0 && tid == 0) {
+        P.ret_at[slot] = retired_at;
+        P.n_checks[slot] = checks;
+    }
+    if (retired_at) return;
+    // ---- the lane goes back out: this block's rows of the current potentials and per-point terms
+    for (int lr = tid; lr < RB; lr += UPD_THREADS) {
+        const int i = b * RB + lr;
+        if (i < P.n) {
+            const size_t o = (size_t)slot * P.np + i;
+            const T *src = colsX + (size_t)(i / TJ) * STX + (DP + 2 * c.parity) * TJ + (i % TJ);
+            P.phi[c.parity][o] = potx[c.parity][lr];
+            reinterpret_cast<T *>(P.ft[c.parity])[o] = src[0];
+            reinterpret_cast<T *>(P.fl[c.parity])[o] = src[TJ];
+        }
+        if (i < P.m) {
+            const size_t o = (size_t)slot * P.mp + i;
+            const T *src = colsY + (size_t)(i / TJ) * STY + DP * TJ + (i % TJ);
+            P.gam[o] = poty[lr];
+            reinterpret_cast<T *>(P.gt)[o] = src[0];
+            reinterpret_cast<T *>(P.gl)[o] = src[TJ];
+        }
     }
 }
 

@@ -177,7 +177,7 @@ __global__ void __launch_bounds__(UPD_THREADS) update_bigd_kernel(const Dev P, c
         for (int r = 0; r < R; ++r) { row_m[lrow0 + r] = mx[r]; row_s[lrow0 + r] = sd[r]; row_h[lrow0 + r] = 0.f; }
     }
     __syncthreads();
-    finish_rows<T, RB>(P, c, leg, slot, (int)FORM_DOT, row_m, row_s, row_h, red);
+    finish_rows<T, RB>(P, c, leg, slot, (int)FORM_DOT, row_m, row_s, row_h, red, (int)blockIdx.x * RB);
 }
 
 }  // namespace skb

@@ -408,7 +408,7 @@ update_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant_
     if (abort_flag) {
         if (tid == 0) atomicOr(&P.ctl->error, ERR_WAIT);
     }
-    finish_rows<float, TC_BM, TC_THREADS>(P, c, leg, slot, (int)FORM_DOT, row_m, row_s, row_h, red);
+    finish_rows<float, TC_BM, TC_THREADS>(P, c, leg, slot, (int)FORM_DOT, row_m, row_s, row_h, red, (int)blockIdx.x * TC_BM);
 }
 
 // ---------------------------------------------------------------- CTA-pair variant

@@ -132,10 +132,11 @@ def test_early_exit_mask_arm_equals_the_mask_control_bitwise(oracle, case, compu
 
 
 def test_rows_per_thread_follow_the_width_without_changing_bits():
-    # Mixed arithmetic launches four rows per thread while the grid fills the GPU and two rows once the
-    # batch has shrunk; MASKED never shrinks, so it stays on four.  A row's arithmetic does not depend on
-    # the thread that holds it and residual terms are summed as integers, so the two modes must agree
-    # bit for bit at the bench size (1024 lanes, where ACTIVE crosses the switch).
+    # Mixed arithmetic launches four rows per thread while the grid fills the GPU and two rows once it does
+    # not; MASKED never shrinks and stays on the one-launch-per-leg kernels, while ACTIVE runs the 1024
+    # lanes through the multi-cycle cluster kernel (two rows per thread, state in shared memory).  A row's
+    # arithmetic depends neither on the thread that holds it nor on the rows that share its block, and
+    # residual terms are summed as integers, so the two modes must agree bit for bit at full size.
     w = wl.make("sweep")
     ra = run_gpu(w, mode="active", compute="mixed", widths_cap=10)
     rm = run_gpu(w, mode="masked", compute="mixed", widths_cap=10)
@@ -692,3 +693,87 @@ def test_two_batches_interleaved_on_one_stream(oracle):
         np.testing.assert_array_equal(depth.cpu().numpy(), r["depth"])
         np.testing.assert_array_equal(f.cpu().numpy(), r["f"]); np.testing.assert_array_equal(g.cpu().numpy(), r["g"])
         s.close()
+
+
+# ---- audit arms ---------------------------------------------------------------------------------------
+@pytest.mark.parametrize("case", ["tiny", "sensor_ragged", "sweep_small"])
+@pytest.mark.parametrize("every", [1, 4])
+def test_full_check_arm_against_oracle(oracle, case, every):
+    # no screen: every audited lane gets the two-sided check (tol_screen far above any residual); the oracle
+    # runs with the same thresholds and the same audit grid
+    w = _make(case)
+    W = w.shape[0]
+    r = run_gpu(w, mode="active", tol_screen=1e30, audit_every=every)
+    check_against_oracle(oracle, w, r, range(W), pot_tol=POT_TOL_F32, exact_depth=False, tol_screen=1e30,
+                         audit_every=every, floor=MARGIN_AUTO, label=f"full-check arm, every {every}, {case}")
+    assert np.all(r["depth"] % every == 0)
+    # every audit of every lane ran a column check: W*n*m per audit beyond the legs
+    n, m = w.shape[1], w.shape[2]
+    audits = int((r["depth"] // every).sum()) if every > 1 else int(r["depth"].sum())
+    assert r["stats"]["pair_terms"] >= 2 * r["stats"]["slots"] * n * m + audits * n * m
+
+
+def test_last_audit_reports_the_screen_of_the_previous_state(oracle):
+    import torch
+    from paper_2607_24741_b200 import binding as B
+    w = wl.make("sensor", W=6, n=90, m=70)
+    t = lambda v: torch.from_numpy(v).to("cuda:0")
+    sb = B.SinkhornBatch(t(w.x), t(w.y), t(w.a), t(w.b), t(w.eps), 1e-7, mode="masked", compute="f64")
+    sb.step(3)
+    f, g = sb.potentials(f64=True)                       # state after 3 cycles
+    sb.step(1)
+    rr, rc, fl = sb.last_audit()                         # ... whose screen came out of the f-leg of cycle 4
+    fh, gh, rr = f.cpu().numpy(), g.cpu().numpy(), rr.cpu().numpy()
+    for k in range(6):
+        want, _ = oracle.residuals(w.x[k], w.y[k], w.a[k], w.b[k], float(w.eps[k]), fh[k], gh[k])
+        assert abs(rr[k] - want) <= 1e-6 * want
+    assert (fl.cpu().numpy() == 0).all() and np.isnan(rc.cpu().numpy()).all()
+    sb.close()
+    w = wl.make("tiny")                                  # an ACTIVE batch of small lanes runs several cycles per launch
+    act = B.SinkhornBatch(t(w.x), t(w.y), t(w.a), t(w.b), t(w.eps), w.tol, mode="active")
+    act.step(2)
+    with pytest.raises(B.SkbError) as e:
+        act.last_audit()
+    assert e.value.code == 5
+    act.close()
+
+
+# ---- large clouds ---------------------------------------------------------------------------------------
+def test_sixteen_thousand_points_against_oracle_cycles(oracle):
+    # n = m = 16384 (the size of the paper's largest Flash campaigns): the oracle's dense cost matrix is
+    # 2 GB and one cycle takes it tens of seconds, so the comparison is on the state after two cycles
+    w = wl.make("registration", W=1, n=16384)
+    import torch
+    from paper_2607_24741_b200 import binding as B
+    t = lambda v: torch.from_numpy(v).to("cuda:0")
+    sb = B.SinkhornBatch(t(w.x), t(w.y), t(w.a), t(w.b), t(w.eps), w.tol, mode="static")
+    sb.step(2)
+    f, g = sb.potentials(f64=True)
+    sb.close()
+    ref = oracle.solve_lane(w.x[0], w.y[0], w.a[0], w.b[0], float(w.eps[0]), w.tol, fixed_cycles=2)
+    e = pot_err(f.cpu().numpy(), g.cpu().numpy(), ref.f[None], ref.g[None], w.eps.astype(np.float64))
+    assert e.max() <= POT_TOL_F32
+
+
+def test_sixty_five_thousand_points_sampled_marginals():
+    # n = m = 65536: far beyond what the oracle can hold (a 34 GB cost matrix), so the emitted state is
+    # checked on sampled rows and columns, each computed from its definition in float64: after the last
+    # g-leg every column marginal equals b_j (Eq. 4), and the sampled rows' deviations extrapolate to a
+    # row residual below the tolerance the lane stopped at (Eq. 5).
+    w = wl.make("registration", W=1, n=65536)
+    r = run_gpu(w)
+    assert r["status"][0] == 1 and r["r_row"][0] <= w.tol and r["depth"][0] > 50
+    x, y = w.x[0].astype(np.float64), w.y[0].astype(np.float64)
+    a, b, eps = w.a[0].astype(np.float64), w.b[0].astype(np.float64), float(w.eps[0])
+    f, g = r["f"][0], r["g"][0]
+    rng = np.random.default_rng(11)
+    cols = rng.choice(65536, 48, replace=False)
+    for j in cols:
+        c = ((x - y[j]) ** 2).sum(1)
+        assert abs(np.exp((f + g[j] - c) / eps).sum() - b[j]) <= 2e-5 * b[j]
+    rows = rng.choice(65536, 256, replace=False)
+    dev = 0.0
+    for i in rows:
+        c = ((y - x[i]) ** 2).sum(1)
+        dev += abs(np.exp((f[i] + g - c) / eps).sum() - a[i])
+    assert dev * (65536 / 256) <= 1.5 * w.tol          # a 256-row sample of an L1 norm: generous sampling slack
