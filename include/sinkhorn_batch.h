@@ -94,6 +94,13 @@ typedef struct {
     void *stream;          /* cudaStream_t (0 = legacy default stream)                     */
     void *workspace;       /* device, 256-byte aligned                                     */
     size_t workspace_bytes;
+    float guard_band;      /* guard band around the thresholds with float64 escalation     */
+                           /* (Section 5, stress test of near-threshold accept decisions): */
+                           /* a lane whose row screen lies within this RELATIVE distance   */
+                           /* of tau_screen or tau_stop has its row residual re-evaluated  */
+                           /* from the raw inputs in float64 and is decided by that value. */
+                           /* 0 = default (1e-3), negative = off; d <= 32 only (ignored    */
+                           /* for larger d).  Costs a raw copy of x and y in the workspace */
 } skb_config;
 
 /* Bytes of device workspace a batch with this shape, dtype, mode and compute type

@@ -43,7 +43,7 @@ class SkbConfig(ctypes.Structure):
                 ("tol_screen", ctypes.c_float), ("column_split", ctypes.c_int),
                 ("cost_form", ctypes.c_int),
                 ("stream", ctypes.c_void_p), ("workspace", ctypes.c_void_p),
-                ("workspace_bytes", ctypes.c_size_t)]
+                ("workspace_bytes", ctypes.c_size_t), ("guard_band", ctypes.c_float)]
 
 
 class SkbError(RuntimeError):
@@ -113,10 +113,10 @@ def _ptr(t):
 
 
 def make_config(W, n, m, d, *, bf16=False, mode="active", compute="auto", max_iter=5000,
-                audit_every=1, tol_screen=0.0, column_split=0, cost_form=0, stream=0) -> SkbConfig:
+                audit_every=1, tol_screen=0.0, column_split=0, cost_form=0, stream=0, guard_band=0.0) -> SkbConfig:
     return SkbConfig(W, n, m, d, 1 if bf16 else 0, MODES[mode] if isinstance(mode, str) else mode,
                      COMPUTE[compute] if isinstance(compute, str) else compute, max_iter, audit_every,
-                     tol_screen, column_split, cost_form, stream, None, 0)
+                     tol_screen, column_split, cost_form, stream, None, 0, guard_band)
 
 
 # ---- functions with the C names ------------------------------------------------------
@@ -186,7 +186,7 @@ class SinkhornBatch:
     """One batch of W lanes on the current CUDA device (thin wrapper over the C calls)."""
 
     def __init__(self, x, y, a, b, eps, tol, *, mode="active", compute="auto", max_iter=5000,
-                 audit_every=1, tol_screen=0.0, column_split=0, cost_form=0, stream=None):
+                 audit_every=1, tol_screen=0.0, column_split=0, cost_form=0, stream=None, guard_band=0.0):
         if not (x.is_cuda and y.is_cuda and a.is_cuda and b.is_cuda and eps.is_cuda):
             raise ValueError("x, y, a, b, eps must be CUDA tensors")
         if x.dtype not in (torch.float32, torch.bfloat16) or y.dtype != x.dtype:
@@ -204,7 +204,8 @@ class SinkhornBatch:
         self.stream = stream if stream is not None else torch.cuda.current_stream(x.device)
         self.cfg = make_config(W, n, m, d, bf16=x.dtype == torch.bfloat16, mode=mode, compute=compute,
                                max_iter=max_iter, audit_every=audit_every, tol_screen=tol_screen,
-                               column_split=column_split, cost_form=cost_form, stream=self.stream.cuda_stream)
+                               column_split=column_split, cost_form=cost_form, stream=self.stream.cuda_stream,
+                               guard_band=guard_band)
         need = sinkhorn_batch_workspace_bytes(self.cfg)
         if need == 0:
             raise SkbError(2, "configuration rejected (unsupported shape or bad option)")

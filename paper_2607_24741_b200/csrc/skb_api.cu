@@ -98,7 +98,17 @@ static bool config_ok(const skb_config *c, std::string &why)
     if (c->column_split != 0 && c->column_split != 1 && c->column_split != 4 && c->column_split != 32) {
         why = "column_split must be 0, 1, 4 or 32"; return false;
     }
+    if (!(c->guard_band <= 0.5f)) { why = "guard_band must be at most 0.5 (negative: off, 0: default)"; return false; }
     return true;
+}
+
+// Relative half-width of the guard band: the configured value, 1e-3 by default, off when negative
+// and for d > 32 (the float64 re-evaluation walks all pairs of a lane with one thread per row, which
+// is only affordable where a pair is a few dimensions deep).
+static double guard_width(const skb_config *c)
+{
+    if (c->d > 32 || c->guard_band < 0.0f) return 0.0;
+    return c->guard_band > 0.0f ? (double)c->guard_band : 1.0e-3;
 }
 
 // Lays the batch's arrays out in the workspace (base may be null: size query only).
@@ -128,6 +138,7 @@ static size_t carve(const skb_config *c, const Variant *var, bool tensor, char *
     d.state = (int *)take(W * 4); d.flag = (int *)take(W * 4); d.verdict = (int *)take(W * 4);
     d.nonfinite = (int *)take(W * 4);
     d.ret_at = (int *)take(W * 4); d.n_checks = (int *)take(W * 4);
+    d.rsum_row64 = (unsigned long long *)take(W * 8); d.esc = (int *)take(W * 4);
     d.rsum_row = (unsigned long long *)take(W * 8); d.rsum_col = (unsigned long long *)take(W * 8);
     d.depth = (int *)take(W * 4); d.status = (int *)take(W * 4); d.emitted = (int *)take(W * 4);
     d.res_row = (double *)take(W * 8); d.res_col = (double *)take(W * 8);
@@ -157,6 +168,13 @@ static size_t carve(const skb_config *c, const Variant *var, bool tensor, char *
     d.phi[0] = (double *)take(W * np * 8); d.phi[1] = (double *)take(W * np * 8);
     d.gam = (double *)take(W * mp * 8);
     d.f_out = (double *)take(W * n * 8); d.g_out = (double *)take(W * m * 8);
+    // guard band: raw copies of the inputs (the float64 re-evaluation reads nothing but these and the potentials)
+    d.guard = guard_width(c);
+    if (d.guard > 0.0) {
+        const size_t es = c->xy_dtype == SKB_BF16 ? 2 : 4;
+        d.xraw_stride = align_up(n * (size_t)c->d * es, 16); d.yraw_stride = align_up(m * (size_t)c->d * es, 16);
+        d.xraw = take(W * d.xraw_stride); d.yraw = take(W * d.yraw_stride);
+    }
     if (D) { *D = d; D->tol_screen = 0; D->tol_stop = 0; }
     if (zero_end_out) *zero_end_out = zero_end;
     return off;
@@ -298,6 +316,16 @@ extern "C" skb_status sinkhorn_batch_create(const void *x, const void *y, const 
         }
     }
     launch_prep(h->dev, x, y, a, b, h->stream);
+    if (h->dev.guard > 0.0) {
+        const size_t es = cfg->xy_dtype == SKB_BF16 ? 2 : 4;
+        const size_t xb = (size_t)cfg->n * cfg->d * es, yb = (size_t)cfg->m * cfg->d * es;
+        if ((e = cudaMemcpy2DAsync(h->dev.xraw, h->dev.xraw_stride, x, xb, xb, cfg->W, cudaMemcpyDeviceToDevice, h->stream)) != cudaSuccess ||
+            (e = cudaMemcpy2DAsync(h->dev.yraw, h->dev.yraw_stride, y, yb, yb, cfg->W, cudaMemcpyDeviceToDevice, h->stream)) != cudaSuccess) {
+            skb_status st = cuda_fail(nullptr, e, "create (raw input copies)");
+            sinkhorn_batch_destroy(h);
+            return st;
+        }
+    }
     // the pinned block is reused for snapshots: wait until the initial copy has been consumed
     if ((e = cudaEventRecord(h->ev[0], h->stream)) != cudaSuccess || (e = cudaGetLastError()) != cudaSuccess) {
         skb_status st = cuda_fail(nullptr, e, "create");

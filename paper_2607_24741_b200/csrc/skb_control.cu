@@ -20,12 +20,6 @@
 namespace skb {
 
 // ---------------------------------------------------------------- prep
-__device__ __forceinline__ float load_raw(const Dev &P, const void *base, size_t idx)
-{
-    if (P.xy_bf16) return __uint_as_float(((unsigned)reinterpret_cast<const unsigned short *>(base)[idx]) << 16);
-    return reinterpret_cast<const float *>(base)[idx];
-}
-
 // One CTA per lane: joint centroid of the two clouds, the largest scaled squared distance
 // from it, and from that the cost form the lane will use.
 __global__ void __launch_bounds__(256) lane_stats_kernel(const Dev P, const void *xin, const void *yin, const float *eps)
@@ -242,10 +236,10 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_kernel(const Dev P)
         const int fl = lane_flag(P, c, s) ? 1 : 0;
         const int nf = P.nonfinite[s];
         const bool held = (P.mode != MODE_ACTIVE) && P.state[s] != 0;
-        const double rr = (double)P.rsum_row[s] * (1.0 / RSUM_SCALE);
+        const double rr = lane_row_residual(P, s);
         const double rc = (double)P.rsum_col[s] * (1.0 / RSUM_SCALE);
         const int vd = (!nf && fmax(rr, rc) <= P.tol_stop) ? 1 : 0;
-        P.rsum_row[s] = 0ull; P.rsum_col[s] = 0ull;
+        P.rsum_row[s] = 0ull; P.rsum_col[s] = 0ull; P.rsum_row64[s] = 0ull; P.esc[s] = 0;
         P.rrow[s] = rr; P.rcol[s] = rc;
         P.flag[s] = fl; P.verdict[s] = vd;
         int r, st; decide_vals(held, nf, fl, vd, r, st);
@@ -368,6 +362,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_cycles_kernel(const Dev P, 
         if (r > 0) atomicAdd(&left_at[r - 1 - k0], 1);
         nchk += P.n_checks[s];
         P.rsum_row[s] = 0ull; P.rsum_col[s] = 0ull;      // between launches the residual sums are zero
+        P.rsum_row64[s] = 0ull; P.esc[s] = 0;
     }
     for (int off = 16; off > 0; off >>= 1) nchk += __shfl_down_sync(0xffffffffu, nchk, off);
     if ((tid & 31) == 0 && nchk) atomicAdd(&checks_s, nchk);
@@ -473,35 +468,67 @@ __device__ __forceinline__ void emit_move_one(const Dev &P, const Ctl &c, const 
     }
     if (tid == 0 && lane >= 0) P.emitted[lane] = 1;
     if (src < 0) return;
-    // move the survivor in slot `src` into the hole `slot` (16-byte vector copies)
-    auto copy = [&](void *base, size_t bytes_per_lane) {
-        const uint4 *s4 = reinterpret_cast<const uint4 *>((const char *)base + (size_t)src * bytes_per_lane);
-        uint4 *d4 = reinterpret_cast<uint4 *>((char *)base + (size_t)slot * bytes_per_lane);
-        const size_t nv = bytes_per_lane / 16;
-        for (size_t v = tid; v < nv; v += 4 * (size_t)nth) {       // four loads in flight per thread
-            uint4 a[4];
-#pragma unroll
-            for (int u = 0; u < 4; ++u) if (v + (size_t)u * nth < nv) a[u] = s4[v + (size_t)u * nth];
-#pragma unroll
-            for (int u = 0; u < 4; ++u) if (v + (size_t)u * nth < nv) d4[v + (size_t)u * nth] = a[u];
+    // Move the survivor in slot `src` into the hole `slot`: all of its slot-indexed arrays as ONE list
+    // of 16-byte vectors, so that a thread's loads in flight span arrays (array after array, each
+    // with its own loop, cost one DRAM round trip per array: ~15 us for any lane size).
+    __shared__ const uint4 *seg_src[16];
+    __shared__ uint4 *seg_dst[16];
+    __shared__ unsigned seg_end[16];          // running total of vectors up to and including the segment
+    __shared__ int seg_n;
+    __syncthreads();                          // the table may still be in use by this block's previous retiree
+    if (threadIdx.x == 0) {
+        int ns = 0;
+        unsigned run = 0;
+        auto add = [&](void *base, size_t bytes_per_lane) {
+            if (!base || bytes_per_lane == 0) return;
+            seg_src[ns] = reinterpret_cast<const uint4 *>((const char *)base + (size_t)src * bytes_per_lane);
+            seg_dst[ns] = reinterpret_cast<uint4 *>((char *)base + (size_t)slot * bytes_per_lane);
+            run += (unsigned)(bytes_per_lane / 16);
+            seg_end[ns++] = run;
+        };
+        const int np_ = ep ^ 1;   // buffer that holds the survivors' current row potentials
+        if (P.tensor) {
+            add(P.xb, (size_t)((P.n + 127) / 128) * P.d * 256);      // tiled copies: 128-point tiles x d bf16
+            add(P.yb, (size_t)((P.m + 127) / 128) * P.d * 256);
+        } else {
+            add(P.xs, (size_t)P.DP * P.np * sizeof(T));
+            add(P.ys, (size_t)P.DP * P.mp * sizeof(T));
         }
-    };
-    const int np_ = ep ^ 1;   // buffer that holds the survivors' current row potentials
-    if (P.tensor) {
-        copy(P.xb, (size_t)((P.n + 127) / 128) * P.d * 256);      // tiled copies: 128-point tiles x d bf16
-        copy(P.yb, (size_t)((P.m + 127) / 128) * P.d * 256);
-    } else {
-        copy(P.xs, (size_t)P.DP * P.np * sizeof(T));
-        copy(P.ys, (size_t)P.DP * P.mp * sizeof(T));
+        if (P.guard > 0.0) {                                          // raw input copies of the guard band
+            add(P.xraw, P.xraw_stride);
+            add(P.yraw, P.yraw_stride);
+        }
+        add(P.sqx, (size_t)P.np * 8); add(P.sqy, (size_t)P.mp * 8);
+        add(P.la2, (size_t)P.np * 8); add(P.lb2, (size_t)P.mp * 8);
+        add(P.wa, (size_t)P.np * 8); add(P.wb, (size_t)P.mp * 8);
+        add(P.phi[np_], (size_t)P.np * 8);
+        add(P.ft[np_], (size_t)P.np * sizeof(T));
+        add(P.fl[np_], (size_t)P.np * sizeof(T));
+        add(P.gt, (size_t)P.mp * sizeof(T));
+        add(P.gl, (size_t)P.mp * sizeof(T));
+        seg_n = ns;
     }
-    copy(P.sqx, (size_t)P.np * 8); copy(P.sqy, (size_t)P.mp * 8);
-    copy(P.la2, (size_t)P.np * 8); copy(P.lb2, (size_t)P.mp * 8);
-    copy(P.wa, (size_t)P.np * 8); copy(P.wb, (size_t)P.mp * 8);
-    copy(P.phi[np_], (size_t)P.np * 8);
-    copy(P.ft[np_], (size_t)P.np * sizeof(T));
-    copy(P.fl[np_], (size_t)P.np * sizeof(T));
-    copy(P.gt, (size_t)P.mp * sizeof(T));
-    copy(P.gl, (size_t)P.mp * sizeof(T));
+    __syncthreads();
+    const int ns = seg_n;
+    const unsigned total = seg_end[ns - 1];
+    for (unsigned v = tid; v < total; v += 4u * (unsigned)nth) {       // four loads in flight per thread
+        uint4 a[4];
+        uint4 *d[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const unsigned idx = v + (unsigned)u * (unsigned)nth;
+            d[u] = nullptr;
+            if (idx < total) {
+                int sg = 0;
+                while (idx >= seg_end[sg]) ++sg;
+                const unsigned off = idx - (sg ? seg_end[sg - 1] : 0u);
+                a[u] = seg_src[sg][off];
+                d[u] = seg_dst[sg] + off;
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) if (d[u]) *d[u] = a[u];
+    }
 }
 
 // ---------------------------------------------------------------- gather (read-back)
@@ -581,6 +608,7 @@ static size_t lane_state_bytes(const Dev &P)
     const size_t ts = P.compute_f64 ? 8 : 4;
     size_t coords = (size_t)P.DP * (P.np + P.mp) * ts;
     if (P.tensor) coords = ((size_t)((P.n + 127) / 128) + (size_t)((P.m + 127) / 128)) * P.d * 256;
+    if (P.guard > 0.0) coords += P.xraw_stride + P.yraw_stride;
     return coords + (size_t)(P.np + P.mp) * (4 * 8 + 2 * ts + 8);
 }
 // When even the retirement of every lane at once would move little (narrow batches of small

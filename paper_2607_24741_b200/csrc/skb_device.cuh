@@ -81,6 +81,14 @@ struct Dev {
     // multi-cycle launches: cycle count + 1 at which the lane in the slot left inside the launch
     // (0 = still running), and the column checks it ran
     int *ret_at, *n_checks;
+    // guard band (float64 escalation of a near-threshold screen): raw copies of the inputs by slot,
+    // the relative half-width of the band (0 = off), the escalated row residual as a fixed-point
+    // sum and whether it was taken at this audit
+    void *xraw, *yraw;        // [W][n][d], [W][m][d] in the inputs' own type, each slot padded to a multiple of 16 bytes
+    size_t xraw_stride, yraw_stride;   // bytes per slot
+    double guard;
+    unsigned long long *rsum_row64;
+    int *esc;
     double *rrow, *rcol;      // residuals of the audited state
     // marginal residuals of the audited state as fixed-point sums (units of 2^-44): every row block
     // adds its part with one integer atomic, so the total is exact and independent of the order
@@ -103,6 +111,93 @@ struct Dev {
     Ctl *ctl;
 };
 
+// Raw coordinate of the inputs' own storage type (fp32, or bf16 widened exactly).
+__device__ __forceinline__ float load_raw(const Dev &P, const void *base, size_t idx)
+{
+    if (P.xy_bf16) return __uint_as_float(((unsigned)reinterpret_cast<const unsigned short *>(base)[idx]) << 16);
+    return reinterpret_cast<const float *>(base)[idx];
+}
+
+// Guard band around the thresholds (the paper's stress test of near-threshold accept decisions,
+// Section 5: an outward guard with float64 escalation).  A screen value this close to a threshold
+// is within the evaluation error of the fp32 exponentials, so the decision is taken from a float64
+// re-evaluation instead.
+__device__ __forceinline__ bool in_guard_band(const Dev &P, const double rr)
+{
+    return P.guard > 0.0 && (fabs(rr - P.tol_screen) <= P.guard * P.tol_screen || fabs(rr - P.tol_stop) <= P.guard * P.tol_stop);
+}
+
+// One row's term |sum_j pi_ij - a_i| of the row residual (Eq. 5), from the raw inputs and the
+// float64 potentials, float64 throughout (difference-form cost, software exp2): the plain
+// definition, independent of the update kernels' layouts and arithmetic.  One WARP per row: lane l
+// takes the columns l, l + 32, ... with its own running maximum and sum, and the 32 pairs are merged
+// by xor-shuffles (every lane returns the term).  phi: the row's potential (log2 units); the column
+// potentials are read from global memory past L1, because inside a multi-cycle launch other blocks of
+// the cluster have written them.
+__device__ __forceinline__ double direct_row_term_warp(const Dev &P, const int slot, const int i, const double phi)
+{
+    const int lane = threadIdx.x & 31;
+    const double s = P.scale[slot];
+    const double *gam = P.gam + (size_t)slot * P.mp;
+    const void *xl = (const char *)P.xraw + (size_t)slot * P.xraw_stride;
+    const void *yl = (const char *)P.yraw + (size_t)slot * P.yraw_stride;
+    const size_t xb = (size_t)i * P.d;
+    double mx = -1.0e300, sum = 0.0;
+    for (int j = lane; j < P.m; j += 32) {
+        const size_t yb = (size_t)j * P.d;
+        double c = 0.0;
+        for (int k = 0; k < P.d; ++k) {
+            const double t = (double)load_raw(P, xl, xb + k) - (double)load_raw(P, yl, yb + k);
+            c = fma(t, t, c);
+        }
+        const double v = phi + __ldcg(gam + j) - s * c;
+        if (v > mx) { sum *= exp2(mx - v); mx = v; }
+        sum += exp2(v - mx);
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        const double mo = __shfl_xor_sync(0xffffffffu, mx, off);
+        const double so = __shfl_xor_sync(0xffffffffu, sum, off);
+        const double mn = fmax(mx, mo);
+        sum = sum * exp2(mx - mn) + so * exp2(mo - mn);      // a lane without columns carries (-1e300, 0): its factor underflows to 0
+        mx = mn;
+    }
+    return fabs(exp2(mx) * sum - P.wa[(size_t)slot * P.np + i]);
+}
+
+// Rows of a lane for one block of NW warps, one warp per row: warp w takes the rows row_first + w,
+// row_first + w + stride, ... below row_end.  Returns this block's exact fixed-point part of the
+// float64 row residual (valid in thread 0) and whether a term was not finite.  pot[i - pot_first] is
+// row i's potential.
+template <int NW>
+__device__ __forceinline__ unsigned long long direct_rows_block(const Dev &P, const int slot, const int row_first,
+                                                                const int stride, const int row_end, const double *pot,
+                                                                const int pot_first, unsigned long long *red, int *nf)
+{
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    unsigned long long part = 0ull;
+    int bad = 0;
+    for (int i = row_first + warp; i < row_end; i += stride) {
+        const double term = direct_row_term_warp(P, slot, i, pot[i - pot_first]);
+        if (!isfinite(term)) bad = 1;
+        else if (lane == 0) part += __double2ull_rn(fmin(term, RSUM_ROW_MAX) * RSUM_SCALE);
+    }
+    bad = __syncthreads_or(bad);
+    if (lane == 0) red[warp] = part;
+    __syncthreads();
+    unsigned long long sum = 0ull;
+    if (threadIdx.x == 0) for (int w = 0; w < NW; ++w) sum += red[w];
+    __syncthreads();
+    *nf = bad;
+    return sum;
+}
+
+// The row residual a lane's decisions are taken from: the escalated value if one was taken.
+__device__ __forceinline__ double lane_row_residual(const Dev &P, const int slot)
+{
+    return (double)(P.esc[slot] ? P.rsum_row64[slot] : P.rsum_row[slot]) * (1.0 / RSUM_SCALE);
+}
+
 // Screen verdict of a lane from its accumulated row residual: the same predicate for the column
 // check (which lanes to visit) and for the planner (which lanes may retire).
 __device__ __forceinline__ bool lane_flag(const Dev &P, const Ctl &c, const int slot)
@@ -110,7 +205,20 @@ __device__ __forceinline__ bool lane_flag(const Dev &P, const Ctl &c, const int 
     const bool passed = P.state[slot] != 0;                  // MASKED: frozen; STATIC: already passed
     const bool audited = (c.cycle >= 1 && (c.cycle % P.audit_every) == 0) || (c.cycle == 0 && P.audit_initial);
     const bool live = !(passed && (P.mode == MODE_MASKED || P.mode == MODE_STATIC));
-    return audited && live && !P.nonfinite[slot] && (double)P.rsum_row[slot] * (1.0 / RSUM_SCALE) <= P.tol_screen;
+    return audited && live && !P.nonfinite[slot] && lane_row_residual(P, slot) <= P.tol_screen;
+}
+
+// Which lanes the column check visits: the screen-positive ones and, with a guard band, every lane
+// whose screen value lies inside the band - its decision comes from the float64 re-evaluation that
+// other blocks of the same launch are computing, so the column residual is measured in case it passes.
+__device__ __forceinline__ bool lane_needs_column_check(const Dev &P, const Ctl &c, const int slot)
+{
+    if (lane_flag(P, c, slot)) return true;
+    if (!(P.guard > 0.0)) return false;
+    const bool passed = P.state[slot] != 0;
+    const bool audited = (c.cycle >= 1 && (c.cycle % P.audit_every) == 0) || (c.cycle == 0 && P.audit_initial);
+    const bool live = !(passed && (P.mode == MODE_MASKED || P.mode == MODE_STATIC));
+    return audited && live && !P.nonfinite[slot] && in_guard_band(P, (double)P.rsum_row[slot] * (1.0 / RSUM_SCALE));
 }
 
 __device__ __forceinline__ float ex2_fast(float x)

@@ -10,6 +10,12 @@ constexpr size_t RESIDENT_SMEM_LIMIT = 52 * 1024; // shared memory of a block of
 
 constexpr long long NARROW_BLOCKS = 148 * 4;      // below this many blocks some SM has fewer than four
 
+// Grid rows (of `per_row` blocks each) that hold the guard band's pool of about two blocks per SM.
+static int pool_rows(int per_row, bool on)
+{
+    return on ? (2 * 148 + per_row - 1) / per_row : 0;
+}
+
 template <typename T, int DP, int CS, int XF>
 static void launch_update(const Dev &P, int leg, int width, cudaStream_t st)
 {
@@ -21,6 +27,7 @@ static void launch_update(const Dev &P, int leg, int width, cudaStream_t st)
     }
     const int nrows = (leg == LEG_F) ? P.n : P.m;
     const int lanes = width < 1 ? 1 : width;
+    const bool guard_pool = leg == LEG_V && P.guard > 0.0;       // extra grid rows: the guard band's float64 re-evaluation
     if constexpr (sizeof(T) == 8 && XF == 1 && DP <= 8) {
         // Float64 arguments with few dimensions: four rows per thread halve the shared-memory
         // loads per multiply-add (faster when the grid fills the GPU), two rows give twice the
@@ -35,7 +42,7 @@ static void launch_update(const Dev &P, int leg, int width, cudaStream_t st)
         const int rbw = (UPD_THREADS / 32) * RW * (32 / CS);
         const long long ctas = (long long)((nrows + rbw - 1) / rbw) * lanes;
         if (ctas >= 2 * 148 * 4) {
-            launch_pdl(update_kernel<T, DP, CS, XF, RW>, dim3((nrows + rbw - 1) / rbw, lanes), dim3(UPD_THREADS), smem, st, P, leg);
+            launch_pdl(update_kernel<T, DP, CS, XF, RW>, dim3((nrows + rbw - 1) / rbw, lanes + pool_rows((nrows + rbw - 1) / rbw, guard_pool)), dim3(UPD_THREADS), smem, st, P, leg, lanes);
             return;
         }
     }
@@ -50,12 +57,12 @@ static void launch_update(const Dev &P, int leg, int width, cudaStream_t st)
         const int rb2 = (UPD_THREADS / 32) * Tune<T, DP>::R * (32 / CS);
         if ((long long)((nrows + rb2 - 1) / rb2) * lanes < NARROW_BLOCKS) {
             const int rbr = (UPD_THREADS / 32) * 1 * (32 / CS);
-            launch_pdl(update_kernel<T, DP, CS, XF, 1>, dim3((nrows + rbr - 1) / rbr, lanes), dim3(UPD_THREADS), smem, st, P, leg);
+            launch_pdl(update_kernel<T, DP, CS, XF, 1>, dim3((nrows + rbr - 1) / rbr, lanes + pool_rows((nrows + rbr - 1) / rbr, guard_pool)), dim3(UPD_THREADS), smem, st, P, leg, lanes);
             return;
         }
     }
     const int rb = (UPD_THREADS / 32) * Tune<T, DP>::R * (32 / CS);
-    launch_pdl(update_kernel<T, DP, CS, XF>, dim3((nrows + rb - 1) / rb, lanes), dim3(UPD_THREADS), smem, st, P, leg);
+    launch_pdl(update_kernel<T, DP, CS, XF>, dim3((nrows + rb - 1) / rb, lanes + pool_rows((nrows + rb - 1) / rb, guard_pool)), dim3(UPD_THREADS), smem, st, P, leg, lanes);
 }
 
 // Several whole cycles per launch: grid.x = row blocks of the larger cloud = one thread-block

@@ -742,7 +742,7 @@ __device__ __forceinline__ void run_leg(const Dev &P, const Ctl &c, const int le
 // and a row's arithmetic does not depend on which thread holds it, so launches with different RR
 // give the same bits.
 template <typename T, int DP, int CS, int XF, int RR = 0>
-__global__ void __launch_bounds__(UPD_THREADS) update_kernel(const Dev P, const int leg)
+__global__ void __launch_bounds__(UPD_THREADS) update_kernel(const Dev P, const int leg, const int nlanes)
 {
     constexpr int R = RR ? RR : Tune<T, DP>::R;
     constexpr int RB = (UPD_THREADS / 32) * R * (32 / CS);   // rows per CTA
@@ -764,10 +764,53 @@ __global__ void __launch_bounds__(UPD_THREADS) update_kernel(const Dev P, const 
     if (leg == LEG_V) asm volatile("griddepcontrol.wait;" ::: "memory");
     const int slot = blockIdx.y;
     const int row_base = (int)blockIdx.x * RB;
+    if (leg == LEG_V && (int)blockIdx.y >= nlanes) {
+        // Guard band: with it on, a column-check launch carries a pool of extra blocks (grid rows past
+        // the lanes).  The pool looks for lanes whose fused screen came out inside the band and
+        // re-evaluates their row residual from the raw inputs in float64 - one warp per row, all pool
+        // warps sharing a lane's rows, exact integer sum - and the planner decides from that value.
+        if (c.done || c.static_final) return;
+        constexpr int NW = UPD_THREADS / 32;
+        __shared__ int hot[UPD_THREADS];
+        __shared__ int n_hot;
+        const int pool_id = ((int)blockIdx.y - nlanes) * (int)gridDim.x + (int)blockIdx.x;
+        const int pool_warps = ((int)gridDim.y - nlanes) * (int)gridDim.x * NW;
+        const bool audited = (c.cycle >= 1 && (c.cycle % P.audit_every) == 0) || (c.cycle == 0 && P.audit_initial);
+        if (!audited) return;
+        for (int s0 = 0; s0 < c.n_phys; s0 += UPD_THREADS * 4) {
+            if (threadIdx.x == 0) n_hot = 0;
+            __syncthreads();
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int s = s0 + u * UPD_THREADS + (int)threadIdx.x;
+                if (s < c.n_phys && !(P.mode != MODE_ACTIVE && P.state[s] != 0) && !P.nonfinite[s] &&
+                    in_guard_band(P, (double)P.rsum_row[s] * (1.0 / RSUM_SCALE))) {
+                    const int at = atomicAdd(&n_hot, 1);
+                    if (at < UPD_THREADS) hot[at] = s;
+                }
+            }
+            __syncthreads();
+            const int nh = n_hot < UPD_THREADS ? n_hot : UPD_THREADS;   // more than 128 at once: the rest keep their fp32 screen
+            for (int q = 0; q < nh; ++q) {
+                const int s = hot[q];
+                int bad;
+                const unsigned long long mine = direct_rows_block<NW>(P, s, pool_id * NW, pool_warps, P.n,
+                                                                      P.phi[c.parity] + (size_t)s * P.np, 0,
+                                                                      reinterpret_cast<unsigned long long *>(sc.red), &bad);
+                if (threadIdx.x == 0) {
+                    atomicAdd(P.rsum_row64 + s, mine);
+                    if (bad) P.nonfinite[s] = 1;
+                    P.esc[s] = 1;
+                }
+            }
+            __syncthreads();
+        }
+        return;
+    }
     const bool idle = c.done || slot >= c.n_phys
                       || (P.early_exit && P.state[slot] != 0)   // early-exit mask arm: a frozen lane costs a launch slot only
                       || (leg != LEG_V && c.static_final)
-                      || (leg == LEG_V && !(c.static_final || lane_flag(P, c, slot)))
+                      || (leg == LEG_V && !(c.static_final || lane_needs_column_check(P, c, slot)))
                       || row_base >= (leg == LEG_F ? P.n : P.m);
     if (idle) {
         // Every kernel of the chain must wait at least once before it completes: a kernel's wait
@@ -830,7 +873,7 @@ __global__ void __launch_bounds__(UPD_THREADS) lane_cycles_kernel(const Dev P, c
     const int tid = threadIdx.x;
     const int lane_id = P.lane_id[slot];
     const double inv_s = 1.0 / P.scale[slot];
-    unsigned long long seen_row = 0ull, seen_col = 0ull;     // totals already accounted for (the planner clears the sums)
+    unsigned long long seen_row = 0ull, seen_col = 0ull, seen_row64 = 0ull;     // totals already accounted for (the planner clears the sums)
     int checks = 0, retired_at = 0;
 
     // One call site for the three kinds of leg (the leg is a run-time value), so that the streaming
@@ -854,6 +897,23 @@ __global__ void __launch_bounds__(UPD_THREADS) lane_cycles_kernel(const Dev P, c
             seen_row = tot_row;
             nf = ld_cg_s32(P.nonfinite + slot);
             const bool audited = (k >= 1 && (k % P.audit_every) == 0) || (k == 0 && P.audit_initial);
+            if (audited && !nf && in_guard_band(P, rr)) {
+                // guard band: decide from a float64 re-evaluation of the row residual
+                int bad;
+                const double *phi_lane = P.phi[c.parity] + (size_t)slot * P.np;
+                const int r0 = (int)blockIdx.x * RB, r1 = min(r0 + RB, P.n);
+                const unsigned long long mine = direct_rows_block<UPD_THREADS / 32>(
+                    P, slot, r0, UPD_THREADS / 32, r1, phi_lane, 0, reinterpret_cast<unsigned long long *>(sc.red), &bad);
+                if (tid == 0) {
+                    atomicAdd(P.rsum_row64 + slot, mine);
+                    if (bad) P.nonfinite[slot] = 1;
+                }
+                cluster_sync_all();
+                const unsigned long long tot64 = ld_cg_u64(P.rsum_row64 + slot);
+                rr = (double)(tot64 - seen_row64) * (1.0 / RSUM_SCALE);
+                seen_row64 = tot64;
+                nf = ld_cg_s32(P.nonfinite + slot);
+            }
             fl = audited && !nf && rr <= P.tol_screen;
             rc = 0.0;
             if (fl) { leg = LEG_V; continue; }     // two-sided check: the column marginal, genuinely measured
@@ -1141,6 +1201,30 @@ __global__ void __launch_bounds__(UPD_THREADS) lane_resident_kernel(const Dev P,
             for (int rk = 0; rk < NC; ++rk) { tot += part[0][rk]; nf |= part_nf[0][rk]; }
             rr = (double)tot * (1.0 / RSUM_SCALE);
             const bool audited = (k >= 1 && (k % P.audit_every) == 0) || (k == 0 && P.audit_initial);
+            if (audited && !nf && in_guard_band(P, rr)) {
+                // guard band: decide from a float64 re-evaluation of the row residual.  It reads the
+                // column potentials from global memory, so the blocks' rows of g go out first.
+                for (int lr = tid; lr < RB; lr += UPD_THREADS) {
+                    const int i = b * RB + lr;
+                    if (i < P.m) P.gam[(size_t)slot * P.mp + i] = poty[lr];
+                }
+                cluster_sync_all();
+                int bad;
+                const double *pot_own = potx[c.parity];
+                const int r0 = b * RB, r1 = min(r0 + RB, P.n);
+                const unsigned long long mine = direct_rows_block<UPD_THREADS / 32>(
+                    P, slot, r0, UPD_THREADS / 32, r1, pot_own, r0, reinterpret_cast<unsigned long long *>(sc.red), &bad);
+                if (tid == 0) {
+                    for (int rk = 0; rk < NC; ++rk) {
+                        st_cluster<unsigned long long>(&part[0][b], rk, mine);
+                        st_cluster<int>(&part_nf[0][b], rk, bad);
+                    }
+                }
+                cluster_sync_all();
+                tot = 0ull;
+                for (int rk = 0; rk < NC; ++rk) { tot += part[0][rk]; nf |= part_nf[0][rk]; }
+                rr = (double)tot * (1.0 / RSUM_SCALE);
+            }
             fl = audited && !nf && rr <= P.tol_screen;
             rc = 0.0;
             if (fl) { leg = LEG_V; continue; }

@@ -777,3 +777,32 @@ def test_sixty_five_thousand_points_sampled_marginals():
         c = ((y - x[i]) ** 2).sum(1)
         dev += abs(np.exp((f[i] + g - c) / eps).sum() - a[i])
     assert dev * (65536 / 256) <= 1.5 * w.tol          # a 256-row sample of an L1 norm: generous sampling slack
+
+
+# ---- guard band: float64 escalation of near-threshold decisions -------------------------------------------
+@pytest.mark.parametrize("case", ["tiny", "sweep_small", "sensor_ragged", "registration_small"])
+def test_guard_band_decisions_come_from_the_float64_reevaluation(oracle, case):
+    # Section 5's stress test: raw fp32 decisions near the threshold flip; an outward guard with float64
+    # escalation removes the flips.  With a band of 50 % every audit within a factor 1.5 of the threshold is
+    # decided from the float64 re-evaluation of the row residual, so the depths must be the oracle's to
+    # within the acceptance bar's own band of 1e-6, in the multi-cycle kernels (ACTIVE) as in the
+    # one-launch-per-leg path (MASKED), with identical bits.
+    w = _make(case)
+    W = w.shape[0]
+    ra = run_gpu(w, mode="active", guard_band=0.5)
+    rm = run_gpu(w, mode="masked", guard_band=0.5)
+    np.testing.assert_array_equal(ra["depth"], rm["depth"])
+    np.testing.assert_array_equal(ra["f"], rm["f"]); np.testing.assert_array_equal(ra["g"], rm["g"])
+    np.testing.assert_array_equal(ra["r_row"], rm["r_row"])
+    check_against_oracle(oracle, w, ra, range(W), pot_tol=POT_TOL_F32, exact_depth=False, floor=1e-6,
+                         label=f"guard band 0.5, {case}")
+    check_accounting(oracle, ra, W, "active")
+    # the reported row residual of a lane decided by escalation IS the float64 value
+    tol = w.tol
+    for t in range(W):
+        rr, _ = oracle.residuals(w.x[t], w.y[t], w.a[t], w.b[t], float(w.eps[t]), ra["f"][t], ra["g"][t])
+        if ra["status"][t] == 1 and rr >= 0.51 * tol:           # inside the band when it stopped: escalated
+            assert abs(ra["r_row"][t] - rr) <= 2e-7 * rr + 1e-10
+    off = run_gpu(w, mode="active", guard_band=-1.0)              # switched off: still within the usual bar
+    check_against_oracle(oracle, w, off, range(W), pot_tol=POT_TOL_F32, exact_depth=False, floor=MARGIN_AUTO,
+                         label=f"guard band off, {case}")
