@@ -542,6 +542,9 @@ def main():
                          "bytes, time and GB/s (few launches; for profiler captures of the compaction kernel)")
     ap.add_argument("--lanes", type=int, default=0, help="with --move-only / --kernel-only: use the first LANES lanes only")
     ap.add_argument("--unit-rates", action="store_true", help="only run the unit-rate self-test (one JSON line)")
+    ap.add_argument("--refill", action="store_true",
+                    help="stream all lanes of --workload through a batch of a quarter as many slots, new problems replacing "
+                         "finished lanes, against the same lanes as four batches one after the other and as one wide batch")
     ap.add_argument("--shadow-replay", action="store_true",
                     help="replay a solve of the first --lanes lanes (default 256) cycle by cycle and compare, at every audit, "
                          "the fused row screen with the row residual computed directly from the potentials")
@@ -649,6 +652,9 @@ def main():
         return
     if args.shadow_replay:
         print(json.dumps(shadow_replay(R, args)), flush=True)
+        return
+    if args.refill:
+        print(json.dumps(refill_report(R, args)), flush=True)
         return
     if args.kernel_only and args.mode == "active":
         # a few multi-cycle launches of the ACTIVE path (for profiler captures of the cluster kernels)
@@ -786,6 +792,63 @@ def shadow_replay(R, args, max_cycles=4000):
             "missed_ready": missed_ready, "screen_positive_but_direct_above_tol": early_ready,
             "max_abs_screen_minus_direct": worst, "max_rel_screen_minus_direct": worst_rel,
             "paper_in_kind": {"screen_negative": 1488, "missed_ready": 0, "max_discrepancy": 1.86e-7}}
+
+
+def refill_report(R, args):
+    """All W lanes of the workload through S = W/4 slots, three ways: one wide batch (W slots), four batches
+    of S lanes one after the other, and one batch of S slots whose finished lanes are replaced by the next
+    problems whenever at least S/8 slots are free (checked every 16 cycles)."""
+    torch, B, w = R.torch, R.B, R.w
+    W, n, m, d = w.shape
+    S = max(1, W // 4)
+    x, y, a, b, eps = R.x, R.y, R.a, R.b, R.eps
+
+    def timed(fn):
+        best, out = None, None
+        for rep in range(2):
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); out = fn(); e1.record(); torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1)
+            best = ms if best is None or ms < best else best
+        return best, out
+
+    def wide():
+        sb = R.batch("active"); sb.drain(); st = sb.stats(); d_, _ = sb.depths(); sb.close()
+        return st["slots"], st["cycles"], d_
+
+    def quarters():
+        slots = cyc = 0
+        for q in range(0, W, S):
+            sl = slice(q, min(W, q + S))
+            sb = B.SinkhornBatch(x[sl], y[sl], a[sl], b[sl], eps[sl], w.tol, compute=args.compute, max_iter=w.max_iter)
+            sb.drain(); st = sb.stats(); sb.close()
+            slots += st["slots"]; cyc += st["cycles"]
+        return slots, cyc, None
+
+    def refilled():
+        sb = B.SinkhornBatch(x[:S], y[:S], a[:S], b[:S], eps[:S], w.tol, compute=args.compute, max_iter=w.max_iter,
+                             lane_capacity=W)
+        nxt, refills = S, 0
+        while nxt < W:
+            sb.step(16)
+            free = S - sb.active()
+            if free >= max(1, S // 8) or free == S:
+                c = min(free, W - nxt)
+                sl = slice(nxt, nxt + c)
+                sb.refill(x[sl], y[sl], a[sl], b[sl], eps[sl]); nxt += c; refills += 1
+        sb.drain(); st = sb.stats(); d_, _ = sb.depths(); sb.close()
+        return st["slots"], st["cycles"], d_, refills
+
+    ms_w, (sl_w, cy_w, dw) = timed(wide)
+    ms_q, (sl_q, cy_q, _) = timed(quarters)
+    ms_r, (sl_r, cy_r, dr, refills) = timed(refilled)
+    return {"report": "refill", "workload": args.workload, "W": W, "slots_held": S, "n": n, "m": m, "d": d,
+            "one_wide_batch": {"ms": ms_w, "slots": sl_w, "cycles": cy_w},
+            "four_batches_in_turn": {"ms": ms_q, "slots": sl_q, "cycles": cy_q},
+            "refilled_batch": {"ms": ms_r, "slots": sl_r, "cycles": cy_r, "refills": refills,
+                               "depths_equal_to_wide_batch": bool((dw == dr).all().item())},
+            "in_turn_over_refilled": ms_q / ms_r, "refilled_over_wide": ms_r / ms_w}
 
 
 def move_accounting(w, widths, depth, R):

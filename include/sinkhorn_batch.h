@@ -101,6 +101,10 @@ typedef struct {
                            /* from the raw inputs in float64 and is decided by that value. */
                            /* 0 = default (1e-3), negative = off; d <= 32 only (ignored    */
                            /* for larger d).  Costs a raw copy of x and y in the workspace */
+    int lane_capacity;     /* lanes the batch can take in over its life: 0 or W = the W of  */
+                           /* create only; more (ACTIVE mode) lets sinkhorn_batch_refill    */
+                           /* put new problems into the slots finished lanes have freed;    */
+                           /* every per-lane output then has lane_capacity entries          */
 } skb_config;
 
 /* Bytes of device workspace a batch with this shape, dtype, mode and compute type
@@ -144,6 +148,22 @@ skb_status sinkhorn_batch_create(const void *x, const void *y, const float *a, c
  */
 skb_status sinkhorn_batch_warm_start(skb_batch *h, const double *f0, const double *g0, int audit_initial);
 
+/*
+ * Replace finished lanes by new problems (the paper's related work on dynamic batching: completed
+ * problems are replaced so that the width does not collapse; compaction keeps the survivors in a
+ * dense prefix, so the free slots are the ones past the current width).
+ *   x [count, n, d], y [count, m, d], a [count, n], b [count, m], eps [count]   as in create (device)
+ *   first_lane (host out, may be null): the new problems become lanes first_lane .. first_lane+count-1
+ *   in every per-lane output.
+ * ACTIVE mode only; needs count free slots (SKB_ERR_STATE otherwise; the call synchronises the stream
+ * to learn the width) and count unused lanes of cfg->lane_capacity (SKB_ERR_SHAPE).  The new lanes
+ * start cold and run with the arithmetic the batch was created with; their depths count their own
+ * cycles, max_iter applies to each lane's own count, audits stay on the batch's cycle grid.  The
+ * slot identity of Eq. 7 still holds: slots = sum_k A_k = sum of all lanes' depths.
+ */
+skb_status sinkhorn_batch_refill(skb_batch *h, const void *x, const void *y, const float *a, const float *b,
+                                 const float *eps, int count, int *first_lane);
+
 /* Enqueue `cycles` full cycles (both legs of Eq. 3 plus screen, two-sided check and
  * retirement after every audited one).  Never synchronises: each call leaves an asynchronous
  * copy of the device's control block behind and looks, without waiting, whether an earlier
@@ -161,7 +181,7 @@ skb_status sinkhorn_batch_drain(skb_batch *h, int *cycles_run);
 skb_status sinkhorn_batch_active(skb_batch *h, int *n_active);
 
 /* Potentials in the paper's convention pi = exp((f + g - C)/eps), original lane order.
- * f [W, n], g [W, m] device out, either may be null.  Retired lanes give their state at
+ * f [L, n], g [L, m] device out, either may be null (L = lane_capacity, W unless lanes are replaced).  Retired lanes give their state at
  * the completion depth (STATIC: at l_max); running lanes give their current state. */
 skb_status sinkhorn_batch_potentials(skb_batch *h, float *f, float *g);
 skb_status sinkhorn_batch_potentials_f64(skb_batch *h, double *f, double *g);

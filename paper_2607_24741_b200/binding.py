@@ -30,6 +30,7 @@ EXPORTS = (
     "sinkhorn_batch_launch_count", "sinkhorn_batch_profile_update", "sinkhorn_batch_arithmetic",
     "sinkhorn_batch_selftest_bounded_wait", "sinkhorn_batch_warm_start", "sinkhorn_batch_set_profiling",
     "sinkhorn_batch_cycle_trace", "sinkhorn_batch_selftest_unit_rates", "sinkhorn_batch_last_audit",
+    "sinkhorn_batch_refill",
 )
 PHASES = ("create", "f_leg", "column_check", "plan", "emit_move", "g_leg")
 # entry points outside the sinkhorn_batch_* family
@@ -43,7 +44,8 @@ class SkbConfig(ctypes.Structure):
                 ("tol_screen", ctypes.c_float), ("column_split", ctypes.c_int),
                 ("cost_form", ctypes.c_int),
                 ("stream", ctypes.c_void_p), ("workspace", ctypes.c_void_p),
-                ("workspace_bytes", ctypes.c_size_t), ("guard_band", ctypes.c_float)]
+                ("workspace_bytes", ctypes.c_size_t), ("guard_band", ctypes.c_float),
+                ("lane_capacity", ctypes.c_int)]
 
 
 class SkbError(RuntimeError):
@@ -74,6 +76,7 @@ def _load():
                                          vp, ctypes.c_int, ctypes.POINTER(ctypes.c_longlong),
                                          ctypes.POINTER(ctypes.c_float)]
     lib.sinkhorn_batch_last_audit.argtypes = [vp, vp, vp, vp]
+    lib.sinkhorn_batch_refill.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_int, ctypes.POINTER(ctypes.c_int)]
     lib.sinkhorn_batch_warm_start.argtypes = [vp, vp, vp, ctypes.c_int]
     lib.sinkhorn_batch_set_profiling.argtypes = [vp, ctypes.c_int]
     lib.sinkhorn_batch_cycle_trace.argtypes = [vp, vp, ctypes.c_int, ctypes.POINTER(ctypes.c_int)]
@@ -113,10 +116,11 @@ def _ptr(t):
 
 
 def make_config(W, n, m, d, *, bf16=False, mode="active", compute="auto", max_iter=5000,
-                audit_every=1, tol_screen=0.0, column_split=0, cost_form=0, stream=0, guard_band=0.0) -> SkbConfig:
+                audit_every=1, tol_screen=0.0, column_split=0, cost_form=0, stream=0, guard_band=0.0,
+                lane_capacity=0) -> SkbConfig:
     return SkbConfig(W, n, m, d, 1 if bf16 else 0, MODES[mode] if isinstance(mode, str) else mode,
                      COMPUTE[compute] if isinstance(compute, str) else compute, max_iter, audit_every,
-                     tol_screen, column_split, cost_form, stream, None, 0, guard_band)
+                     tol_screen, column_split, cost_form, stream, None, 0, guard_band, lane_capacity)
 
 
 # ---- functions with the C names ------------------------------------------------------
@@ -186,7 +190,8 @@ class SinkhornBatch:
     """One batch of W lanes on the current CUDA device (thin wrapper over the C calls)."""
 
     def __init__(self, x, y, a, b, eps, tol, *, mode="active", compute="auto", max_iter=5000,
-                 audit_every=1, tol_screen=0.0, column_split=0, cost_form=0, stream=None, guard_band=0.0):
+                 audit_every=1, tol_screen=0.0, column_split=0, cost_form=0, stream=None, guard_band=0.0,
+                 lane_capacity=0):
         if not (x.is_cuda and y.is_cuda and a.is_cuda and b.is_cuda and eps.is_cuda):
             raise ValueError("x, y, a, b, eps must be CUDA tensors")
         if x.dtype not in (torch.float32, torch.bfloat16) or y.dtype != x.dtype:
@@ -205,7 +210,8 @@ class SinkhornBatch:
         self.cfg = make_config(W, n, m, d, bf16=x.dtype == torch.bfloat16, mode=mode, compute=compute,
                                max_iter=max_iter, audit_every=audit_every, tol_screen=tol_screen,
                                column_split=column_split, cost_form=cost_form, stream=self.stream.cuda_stream,
-                               guard_band=guard_band)
+                               guard_band=guard_band, lane_capacity=lane_capacity)
+        self.L = max(W, lane_capacity)
         need = sinkhorn_batch_workspace_bytes(self.cfg)
         if need == 0:
             raise SkbError(2, "configuration rejected (unsupported shape or bad option)")
@@ -228,21 +234,21 @@ class SinkhornBatch:
 
     def potentials(self, f64=False):
         dt = torch.float64 if f64 else torch.float32
-        f = torch.zeros(self.W, self.n, dtype=dt, device=self.device)
-        g = torch.zeros(self.W, self.m, dtype=dt, device=self.device)
+        f = torch.zeros(self.L, self.n, dtype=dt, device=self.device)
+        g = torch.zeros(self.L, self.m, dtype=dt, device=self.device)
         fn = lib.sinkhorn_batch_potentials_f64 if f64 else lib.sinkhorn_batch_potentials
         _check(fn(self.h, _ptr(f), _ptr(g)), self.h)
         return f, g
 
     def depths(self):
-        depth = torch.zeros(self.W, dtype=torch.int32, device=self.device)
-        status = torch.zeros(self.W, dtype=torch.int32, device=self.device)
+        depth = torch.zeros(self.L, dtype=torch.int32, device=self.device)
+        status = torch.zeros(self.L, dtype=torch.int32, device=self.device)
         _check(lib.sinkhorn_batch_depths(self.h, _ptr(depth), _ptr(status)), self.h)
         return depth, status
 
     def residuals(self):
-        rr = torch.zeros(self.W, dtype=torch.float32, device=self.device)
-        rc = torch.zeros(self.W, dtype=torch.float32, device=self.device)
+        rr = torch.zeros(self.L, dtype=torch.float32, device=self.device)
+        rc = torch.zeros(self.L, dtype=torch.float32, device=self.device)
         _check(lib.sinkhorn_batch_residuals(self.h, _ptr(rr), _ptr(rc)), self.h)
         return rr, rc
 
@@ -256,11 +262,23 @@ class SinkhornBatch:
 
     def last_audit(self):
         """Row screen value, column residual (NaN where not checked) and screen flag of the most recent audit."""
-        rr = torch.full((self.W,), float("nan"), dtype=torch.float32, device=self.device)
-        rc = torch.full((self.W,), float("nan"), dtype=torch.float32, device=self.device)
-        fl = torch.full((self.W,), -1, dtype=torch.int32, device=self.device)
+        rr = torch.full((self.L,), float("nan"), dtype=torch.float32, device=self.device)
+        rc = torch.full((self.L,), float("nan"), dtype=torch.float32, device=self.device)
+        fl = torch.full((self.L,), -1, dtype=torch.int32, device=self.device)
         _check(lib.sinkhorn_batch_last_audit(self.h, _ptr(rr), _ptr(rc), _ptr(fl)), self.h)
         return rr, rc, fl
+
+    def refill(self, x, y, a, b, eps) -> int:
+        """New problems into the slots finished lanes have freed; returns their first lane number."""
+        x, y, a, b, eps = (t.contiguous() for t in (x, y, a, b, eps))
+        count = x.shape[0]
+        if tuple(x.shape) != (count, self.n, self.d) or tuple(y.shape) != (count, self.m, self.d) or \
+                tuple(a.shape) != (count, self.n) or tuple(b.shape) != (count, self.m) or tuple(eps.shape) != (count,):
+            raise ValueError("shapes must be x[c,n,d] y[c,m,d] a[c,n] b[c,m] eps[c]")
+        first = ctypes.c_int(-1)
+        _check(lib.sinkhorn_batch_refill(self.h, _ptr(x), _ptr(y), _ptr(a), _ptr(b), _ptr(eps), count, ctypes.byref(first)), self.h)
+        self._keep = self._keep + (x, y, a, b, eps)
+        return first.value
 
     def set_profiling(self, on=True):
         _check(lib.sinkhorn_batch_set_profiling(self.h, 1 if on else 0), self.h)

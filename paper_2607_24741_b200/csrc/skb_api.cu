@@ -1,6 +1,7 @@
 // Host side of the C ABI: validation, workspace carving, the cycle enqueue loop and the
 // asynchronous width read-back.  No device memory is allocated here; the only CUDA
-// objects the handle owns are two events and a small pinned host block.
+// objects a handle holds are two events and a small pinned host block borrowed from a pool
+// (plus its own timing events once phase timing has been switched on).
 #include <cmath>
 #include <cstdio>
 #include <cstring>
@@ -31,6 +32,8 @@ struct skb_batch {
     int snap_idx;
     // phase timing (Eq. 11's cost record): off unless sinkhorn_batch_set_profiling turned it on
     bool profiling;
+    int lanes_used;        // lanes the batch has taken in so far (create: W; each refill adds to it)
+    long long enqueued_at_refill;   // cycles enqueued when the last lanes came in (the drain cap counts from there)
     bool no_multi_cycle;   // measurement switch: keep one launch per leg even where several cycles per launch are possible
     std::vector<cudaEvent_t> pev;      // timing events, PHASE_EVENTS_PER_CYCLE per enqueued cycle of a chunk + 1
     int pev_used;                      // events recorded since the last harvest
@@ -39,6 +42,9 @@ struct skb_batch {
     alignas(64) unsigned char maps[2 * 128];   // CUtensorMap of x and of y
     std::string err;
 };
+
+static skb_status poll_snapshot(skb_batch *h, bool wait);
+static skb_status read_ctl(skb_batch *h, Ctl *c);
 
 // Text of the last failed create (or host-buffer solve) of the calling thread.
 static thread_local std::string g_create_err;
@@ -98,6 +104,8 @@ static bool config_ok(const skb_config *c, std::string &why)
     if (c->column_split != 0 && c->column_split != 1 && c->column_split != 4 && c->column_split != 32) {
         why = "column_split must be 0, 1, 4 or 32"; return false;
     }
+    if (c->lane_capacity != 0 && c->lane_capacity < c->W) { why = "lane_capacity must be 0 (= W) or at least W"; return false; }
+    if (c->lane_capacity > c->W && c->mode != SKB_ACTIVE) { why = "finished lanes can only be replaced in ACTIVE mode"; return false; }
     if (!(c->guard_band <= 0.5f)) { why = "guard_band must be at most 0.5 (negative: off, 0: default)"; return false; }
     return true;
 }
@@ -121,10 +129,12 @@ static size_t carve(const skb_config *c, const Variant *var, bool tensor, char *
         return p;
     };
     const size_t W = c->W, n = c->n, m = c->m;
+    const size_t L = c->lane_capacity > c->W ? c->lane_capacity : c->W;      // lanes the result buffers hold
     const size_t np = align_up(n, 4), mp = align_up(m, 4), DP = var->DP ? var->DP : padded_dim(c->d);
     const size_t ts = var->f64 ? 8 : 4;
     Dev d;
     memset(&d, 0, sizeof(d));
+    d.L = (int)L;
     d.W = c->W; d.n = c->n; d.m = c->m; d.d = c->d; d.np = (int)np; d.mp = (int)mp; d.DP = (int)DP;
     d.mode = c->mode == SKB_MASKED_EXIT ? (int)MODE_MASKED : (int)c->mode;
     d.early_exit = c->mode == SKB_MASKED_EXIT;
@@ -140,10 +150,13 @@ static size_t carve(const skb_config *c, const Variant *var, bool tensor, char *
     d.ret_at = (int *)take(W * 4); d.n_checks = (int *)take(W * 4);
     d.rsum_row64 = (unsigned long long *)take(W * 8); d.esc = (int *)take(W * 4);
     d.rsum_row = (unsigned long long *)take(W * 8); d.rsum_col = (unsigned long long *)take(W * 8);
-    d.depth = (int *)take(W * 4); d.status = (int *)take(W * 4); d.emitted = (int *)take(W * 4);
-    d.res_row = (double *)take(W * 8); d.res_col = (double *)take(W * 8);
+    d.depth = (int *)take(L * 4); d.status = (int *)take(L * 4); d.emitted = (int *)take(L * 4);
+    d.res_row = (double *)take(L * 8); d.res_col = (double *)take(L * 8);
+    d.start = (int *)take(W * 4);
     d.rrow = (double *)take(W * 8); d.rcol = (double *)take(W * 8);
-    d.widths = (int *)take(((size_t)c->max_iter + 2) * 4);
+    // widths[k] of every cycle the batch can run: max_iter per generation of lanes
+    d.widths_cap = (int)(((size_t)c->max_iter + 1) * ((L + W - 1) / W) + 1);
+    d.widths = (int *)take((size_t)d.widths_cap * 4);
     const size_t nblk128 = ((n > m ? n : m) + 127) / 128;
     d.tc_cnt = (unsigned *)take(W * nblk128 * 4);     // in every layout, so that the zeroed range is the same for all
     const size_t zero_end = off;
@@ -167,7 +180,7 @@ static size_t carve(const skb_config *c, const Variant *var, bool tensor, char *
     d.wa = (double *)take(W * np * 8); d.wb = (double *)take(W * mp * 8);
     d.phi[0] = (double *)take(W * np * 8); d.phi[1] = (double *)take(W * np * 8);
     d.gam = (double *)take(W * mp * 8);
-    d.f_out = (double *)take(W * n * 8); d.g_out = (double *)take(W * m * 8);
+    d.f_out = (double *)take(L * n * 8); d.g_out = (double *)take(L * m * 8);
     // guard band: raw copies of the inputs (the float64 re-evaluation reads nothing but these and the potentials)
     d.guard = guard_width(c);
     if (d.guard > 0.0) {
@@ -255,6 +268,7 @@ extern "C" skb_status sinkhorn_batch_create(const void *x, const void *y, const 
     h->ev[0] = h->ev[1] = nullptr;
     h->tensor = cfg->compute == SKB_COMPUTE_TENSOR;
     h->snap_pending = false; h->snap_idx = 0; h->profiling = false; h->pev_used = 0; h->no_multi_cycle = false;
+    h->lanes_used = cfg->W; h->enqueued_at_refill = 0;
     for (int i = 0; i < SKB_N_PHASES; ++i) h->phase_ms[i] = 0.f;
     carve(cfg, var, h->tensor, (char *)cfg->workspace, &h->dev);
     h->dev.tol_stop = (double)tol;
@@ -280,7 +294,7 @@ extern "C" skb_status sinkhorn_batch_create(const void *x, const void *y, const 
         sinkhorn_batch_destroy(h);
         return st;
     }
-    launch_lane_stats(h->dev, x, y, eps, nullptr, h->stream);
+    launch_lane_stats(h->dev, x, y, eps, 0, 0, cfg->W, 0, h->stream);
     h->launches += 2;   // lane statistics + layout kernel
     if (automatic) {
         // read the largest scaled radius back and pick the arithmetic for the whole batch
@@ -315,7 +329,7 @@ extern "C" skb_status sinkhorn_batch_create(const void *x, const void *y, const 
             return st;
         }
     }
-    launch_prep(h->dev, x, y, a, b, h->stream);
+    launch_prep(h->dev, x, y, a, b, 0, cfg->W, h->stream);
     if (h->dev.guard > 0.0) {
         const size_t es = cfg->xy_dtype == SKB_BF16 ? 2 : 4;
         const size_t xb = (size_t)cfg->n * cfg->d * es, yb = (size_t)cfg->m * cfg->d * es;
@@ -352,6 +366,58 @@ extern "C" skb_status sinkhorn_batch_warm_start(skb_batch *h, const double *f0, 
     return e == cudaSuccess ? SKB_OK : cuda_fail(h, e, "warm_start");
 }
 
+extern "C" skb_status sinkhorn_batch_refill(skb_batch *h, const void *x, const void *y, const float *a, const float *b,
+                                            const float *eps, int count, int *first_lane)
+{
+    if (!h) return SKB_ERR_NULL;
+    if (!x || !y || !a || !b || !eps) return fail(h, SKB_ERR_NULL, "x, y, a, b and eps are required");
+    if (count < 1) return fail(h, SKB_ERR_VALUE, "count must be >= 1");
+    if (h->cfg.mode != SKB_ACTIVE) return fail(h, SKB_ERR_STATE, "finished lanes can only be replaced in ACTIVE mode");
+    if (h->lanes_used + count > h->dev.L) {
+        char buf[128];
+        snprintf(buf, sizeof(buf), "lane capacity exhausted: %d lanes taken in, %d more asked, capacity %d", h->lanes_used, count, h->dev.L);
+        return fail(h, SKB_ERR_SHAPE, buf);
+    }
+    skb_status st0 = poll_snapshot(h, true);
+    if (st0 != SKB_OK) return st0;
+    Ctl c;
+    st0 = read_ctl(h, &c);                           // synchronises: the free slots are those past the device's width
+    if (st0 != SKB_OK) return st0;
+    const int width = c.n_phys;                      // 0 once everything has finished (ACTIVE: the width is the survivors)
+    if (width + count > h->cfg.W) {
+        char buf[128];
+        snprintf(buf, sizeof(buf), "%d slots are free, %d lanes offered", h->cfg.W - width, count);
+        return fail(h, SKB_ERR_STATE, buf);
+    }
+    const Dev &D = h->dev;
+    const size_t es = h->cfg.xy_dtype == SKB_BF16 ? 2 : 4;
+    launch_lane_stats(D, x, y, eps, width, h->lanes_used, count, c.cycle, h->stream);
+    cudaError_t e = cudaSuccess;
+    if (h->tensor) {
+        const size_t xt = tc_tiled_bytes(1, h->cfg.n, h->cfg.d), yt = tc_tiled_bytes(1, h->cfg.m, h->cfg.d);
+        launch_retile(x, (char *)D.xb + (size_t)width * xt, count, h->cfg.n, h->cfg.d, h->stream);
+        launch_retile(y, (char *)D.yb + (size_t)width * yt, count, h->cfg.m, h->cfg.d, h->stream);
+        h->launches += 2;
+    }
+    launch_prep(D, x, y, a, b, width, count, h->stream);
+    if (D.guard > 0.0) {
+        const size_t xb = (size_t)h->cfg.n * h->cfg.d * es, yb = (size_t)h->cfg.m * h->cfg.d * es;
+        e = cudaMemcpy2DAsync((char *)D.xraw + (size_t)width * D.xraw_stride, D.xraw_stride, x, xb, xb, count, cudaMemcpyDeviceToDevice, h->stream);
+        if (e == cudaSuccess)
+            e = cudaMemcpy2DAsync((char *)D.yraw + (size_t)width * D.yraw_stride, D.yraw_stride, y, yb, yb, count, cudaMemcpyDeviceToDevice, h->stream);
+    }
+    launch_refill_ctl(D, count, h->stream);
+    h->launches += 3;
+    if (e == cudaSuccess) e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(h, e, "refill");
+    if (first_lane) *first_lane = h->lanes_used;
+    h->lanes_used += count;
+    h->known_width = width + count;
+    h->finished = false;
+    h->enqueued_at_refill = h->enqueued;
+    return SKB_OK;
+}
+
 extern "C" skb_status sinkhorn_batch_set_profiling(skb_batch *h, int on)
 {
     if (!h) return SKB_ERR_NULL;
@@ -381,7 +447,13 @@ static bool cycles_in_one_launch(const skb_batch *h)
 {
     if (h->cfg.mode != SKB_ACTIVE || h->tensor || h->profiling || !h->var->launch_cycles || h->no_multi_cycle) return false;
     const int mx = h->cfg.n > h->cfg.m ? h->cfg.n : h->cfg.m;
-    return (mx + h->var->rows_per_cta - 1) / h->var->rows_per_cta <= MAX_CLUSTER_BLOCKS;
+    const int nc = (mx + h->var->rows_per_cta - 1) / h->var->rows_per_cta;
+    if (nc > MAX_CLUSTER_BLOCKS) return false;
+    // Lanes too large for shared memory run the streaming version, which is worth it once the batch is
+    // down to about one wave of blocks (it saves launches, not traffic); a wide batch of such lanes is
+    // better served by one launch per leg (sensor at 256 lanes: 1.12 against 1.20 ms per solve).
+    if (!h->var->lane_fits_shared(h->cfg.n, h->cfg.m) && (long long)h->known_width * nc > 148 * 4) return false;
+    return true;
 }
 
 // `cycles` cycles in one launch (1 <= cycles <= MAX_CYCLES_IN_LAUNCH): lanes that pass inside it write their own
@@ -497,11 +569,11 @@ extern "C" skb_status sinkhorn_batch_drain(skb_batch *h, int *cycles_run)
     }
     int chunk = 2, snap = 0, rounds = 0;
     bool have_prev = false;
-    const bool multi = cycles_in_one_launch(h);
-    const int chunk_max = multi ? 32 : 16;
     // every lane is retired by the audit that follows cycle max_iter; STATIC needs one more pass
     const long long hard_cap = (long long)h->cfg.max_iter + 4;
     while (!h->finished) {
+        const bool multi = cycles_in_one_launch(h);      // may become true as the batch narrows
+        const int chunk_max = multi ? 32 : 16;
         if (multi) enqueue_cycles_launch(h, chunk);
         else for (int i = 0; i < chunk; ++i) enqueue_cycle(h);
         if (h->profiling && (e = harvest_phases(h)) != cudaSuccess) return cuda_fail(h, e, "drain (phase timing)");
@@ -518,7 +590,7 @@ extern "C" skb_status sinkhorn_batch_drain(skb_batch *h, int *cycles_run)
         // grow the chunk every other round: cycles enqueued past completion are empty launches that
         // still have to drain, which matters for batches that finish within a dozen cycles
         if (chunk < chunk_max && (++rounds & 1) == 0) chunk *= 2;
-        if (h->enqueued > hard_cap + 64) break;
+        if (h->enqueued - h->enqueued_at_refill > hard_cap + 64) break;
     }
     if ((e = cudaStreamSynchronize(h->stream)) != cudaSuccess) return cuda_fail(h, e, "drain");
     if ((e = cudaMemcpy(&h->h_ctl[0], h->dev.ctl, sizeof(Ctl), cudaMemcpyDeviceToHost)) != cudaSuccess)
@@ -608,7 +680,7 @@ extern "C" skb_status sinkhorn_batch_stats(skb_batch *h, long long *slots, int *
     if (pair_terms) *pair_terms = c.pair_terms;
     if (widths && widths_cap > 0) {
         int k = c.cycle < widths_cap ? c.cycle : widths_cap;
-        if (k > h->cfg.max_iter + 2) k = h->cfg.max_iter + 2;
+        if (k > h->dev.widths_cap) k = h->dev.widths_cap;
         cudaError_t e = cudaMemcpy(widths, h->dev.widths, (size_t)k * sizeof(int), cudaMemcpyDeviceToHost);
         if (e != cudaSuccess) return cuda_fail(h, e, "stats");
     }

@@ -22,17 +22,20 @@ namespace skb {
 // ---------------------------------------------------------------- prep
 // One CTA per lane: joint centroid of the two clouds, the largest scaled squared distance
 // from it, and from that the cost form the lane will use.
-__global__ void __launch_bounds__(256) lane_stats_kernel(const Dev P, const void *xin, const void *yin, const float *eps)
+// Lanes come in as a block of problems: input problem q goes to slot slot0 + q as lane lane0 + q
+// (create: slot0 = lane0 = 0, all W; a refill: the first free slot, the next unused lane number).
+__global__ void __launch_bounds__(256) lane_stats_kernel(const Dev P, const void *xin, const void *yin, const float *eps,
+                                                         const int slot0, const int lane0, const int cycle0)
 {
     __shared__ double red[256];
     __shared__ double cen[1024];
-    const int slot = blockIdx.x, tid = threadIdx.x;
+    const int q = blockIdx.x, slot = slot0 + q, tid = threadIdx.x;
     const int tot = P.n + P.m;
     for (int k = 0; k < P.d; ++k) {
         double s = 0.0;
         for (int p = tid; p < tot; p += 256) {
             const bool isx = p < P.n;
-            const size_t idx = isx ? ((size_t)slot * P.n + p) * P.d + k : ((size_t)slot * P.m + (p - P.n)) * P.d + k;
+            const size_t idx = isx ? ((size_t)q * P.n + p) * P.d + k : ((size_t)q * P.m + (p - P.n)) * P.d + k;
             s += (double)load_raw(P, isx ? xin : yin, idx);
         }
         red[tid] = s;
@@ -44,7 +47,7 @@ __global__ void __launch_bounds__(256) lane_stats_kernel(const Dev P, const void
     double mxr = 0.0;
     for (int p = tid; p < tot; p += 256) {
         const bool isx = p < P.n;
-        const size_t base = isx ? ((size_t)slot * P.n + p) * P.d : ((size_t)slot * P.m + (p - P.n)) * P.d;
+        const size_t base = isx ? ((size_t)q * P.n + p) * P.d : ((size_t)q * P.m + (p - P.n)) * P.d;
         double r2 = 0.0;
         for (int k = 0; k < P.d; ++k) { const double v = (double)load_raw(P, isx ? xin : yin, base + k) - cen[k]; r2 += v * v; }
         mxr = fmax(mxr, r2);
@@ -54,12 +57,17 @@ __global__ void __launch_bounds__(256) lane_stats_kernel(const Dev P, const void
     for (int off = 128; off > 0; off >>= 1) { if (tid < off) red[tid] = fmax(red[tid], red[tid + off]); __syncthreads(); }
     for (int k = tid; k < P.DP; k += 256) P.center[(size_t)slot * P.DP + k] = k < P.d ? cen[k] : 0.0;
     if (tid == 0) {
-        const double e = (double)eps[slot];
+        const double e = (double)eps[q];
         const bool eps_ok = (e > 0.0) && isfinite(e);
         const double s = eps_ok ? 1.4426950408889634 / e : 1.0;
         if (!eps_ok) atomicOr(&P.ctl->error, ERR_VALUE);
         P.scale[slot] = s;
-        P.lane_id[slot] = slot;
+        P.lane_id[slot] = lane0 + q;
+        P.start[slot] = cycle0;
+        // whatever an earlier lane left in the slot
+        P.nonfinite[slot] = 0; P.state[slot] = 0; P.flag[slot] = 0; P.verdict[slot] = 0;
+        P.rsum_row[slot] = 0ull; P.rsum_col[slot] = 0ull; P.rsum_row64[slot] = 0ull; P.esc[slot] = 0;
+        P.ret_at[slot] = 0; P.n_checks[slot] = 0;
         int form = P.cost_form == 1 ? FORM_DOT : (P.cost_form == 2 ? FORM_DIFF : (s * red[0] > P.form_threshold ? FORM_DIFF : FORM_DOT));
         P.form[slot] = form;
         atomicMax(&P.ctl->max_radius_bits, (unsigned long long)__double_as_longlong(eps_ok ? s * red[0] : 0.0));
@@ -67,9 +75,9 @@ __global__ void __launch_bounds__(256) lane_stats_kernel(const Dev P, const void
 }
 
 template <typename T>
-__global__ void prep_kernel(const Dev P, const void *xin, const void *yin, const float *a, const float *b)
+__global__ void prep_kernel(const Dev P, const void *xin, const void *yin, const float *a, const float *b, const int slot0)
 {
-    const int slot = blockIdx.y;
+    const int q = blockIdx.y, slot = slot0 + q;
     const int side = blockIdx.z;                     // 0: x / a, 1: y / b
     const int npts = side ? P.m : P.n, pp = side ? P.mp : P.np;
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
@@ -89,7 +97,7 @@ __global__ void prep_kernel(const Dev P, const void *xin, const void *yin, const
     } else {
         // tensor-core path: raw coordinates feed the MMA, the scale 2s is applied to its result
         const double sc = P.tensor ? sqrt(2.0 * s) : sqrt(form == FORM_DOT ? 2.0 * s : s);
-        const size_t ibase = ((size_t)slot * npts + i) * P.d;
+        const size_t ibase = ((size_t)q * npts + i) * P.d;
         const double *cen = P.center + (size_t)slot * P.DP;
         double nrm = 0.0;
         bool ok = true;
@@ -105,7 +113,7 @@ __global__ void prep_kernel(const Dev P, const void *xin, const void *yin, const
             nrm += (double)v * (double)v;
         }
         nrm = form == FORM_DOT ? 0.5 * nrm : 0.0;
-        const float w = (side ? b : a)[(size_t)slot * npts + i];
+        const float w = (side ? b : a)[(size_t)q * npts + i];
         ok = ok && (w > 0.0f) && isfinite(w);
         if (!ok) atomicOr(&P.ctl->error, ERR_VALUE);
         sq[o] = nrm;
@@ -189,7 +197,9 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_kernel(const Dev P)
     if (c.done) { if (tid == 0) P.ctl->n_retire = 0; return; }
     const int k = c.cycle;                           // cycles completed by the audited state
     const int A = c.n_phys;
-    const bool limit = k >= P.max_iter;
+    // a lane has used up its cycles when ITS OWN count reaches max_iter (lanes that replaced finished
+    // ones came in later; everywhere else start is 0)
+    auto at_limit = [&](int s) { return k - P.start[s] >= P.max_iter; };
 
     if (P.mode == MODE_STATIC && c.static_final) {   // emit every lane at the common boundary
         for (int s = tid; s < P.W; s += NT) {
@@ -214,7 +224,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_kernel(const Dev P)
     }
 
     // which running lanes leave at this audit
-    auto decide_vals = [&](bool held, int nf, int fl, int vd, int &ret, int &st) {
+    auto decide_vals = [&](bool held, int nf, int fl, int vd, bool limit, int &ret, int &st) {
         ret = 0; st = LANE_RUNNING;
         if (held) return;
         if (nf) { ret = 1; st = LANE_NONFINITE; }
@@ -225,7 +235,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_kernel(const Dev P)
         ret = 0; st = LANE_RUNNING;
         if (s >= A) return;
         const bool held = (P.mode != MODE_ACTIVE) && P.state[s] != 0;   // frozen / already passed
-        decide_vals(held, P.nonfinite[s], P.flag[s], P.verdict[s], ret, st);
+        decide_vals(held, P.nonfinite[s], P.flag[s], P.verdict[s], at_limit(s), ret, st);
     };
 
     // pass 1.  The legs left each lane's residuals as exact fixed-point sums: turn them into the
@@ -242,7 +252,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_kernel(const Dev P)
         P.rsum_row[s] = 0ull; P.rsum_col[s] = 0ull; P.rsum_row64[s] = 0ull; P.esc[s] = 0;
         P.rrow[s] = rr; P.rcol[s] = rc;
         P.flag[s] = fl; P.verdict[s] = vd;
-        int r, st; decide_vals(held, nf, fl, vd, r, st);
+        int r, st; decide_vals(held, nf, fl, vd, at_limit(s), r, st);
         cnt += r;
         nflag += fl;
     }
@@ -276,7 +286,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_kernel(const Dev P)
                 P.res_row[lane] = P.rrow[s];
                 P.res_col[lane] = P.flag[s] ? P.rcol[s] : __longlong_as_double(0x7ff8000000000000LL);
             }
-            P.depth[lane] = limit && st != LANE_DONE ? P.max_iter : k;
+            P.depth[lane] = at_limit(s) && st != LANE_DONE ? P.max_iter : k - P.start[s];
             P.status[lane] = st;
             if (P.mode != MODE_ACTIVE) P.state[s] = 1;
         }
@@ -297,6 +307,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_kernel(const Dev P)
     for (int h = tid; h < nholes; h += NT) {
         const int dst = P.hole_list[h], src = P.fill_list[h];
         P.lane_id[dst] = P.lane_id[src];
+        P.start[dst] = P.start[src];
         P.scale[dst] = P.scale[src];
         P.form[dst] = P.form[src];
         P.nonfinite[dst] = 0;
@@ -325,7 +336,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_kernel(const Dev P)
             g->parity = c.parity ^ 1;
             g->slots += width;
             g->pair_terms += (long long)width * P.n * P.m;     // the g-leg that completes cycle k+1
-            if (k < P.max_iter + 1) P.widths[k] = width;
+            if (k < P.widths_cap) P.widths[k] = width;
         } else if (P.mode != MODE_STATIC) {
             g->done = 1;
         }
@@ -392,6 +403,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_cycles_kernel(const Dev P, 
         const int dst = P.hole_list[h], src = P.fill_list[h];
         P.ret_slot[h] = dst; P.ret_lane[h] = -1; P.ret_src[h] = src; P.ret_scale[h] = 1.0;   // move only
         P.lane_id[dst] = P.lane_id[src];
+        P.start[dst] = P.start[src];
         P.scale[dst] = P.scale[src];
         P.form[dst] = P.form[src];
         P.nonfinite[dst] = 0;
@@ -406,7 +418,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_cycles_kernel(const Dev P, 
             terms += (long long)w * nm;              // the f-leg whose epilogue screened the state after k0 + j cycles
             w -= left_at[j];
             if (w == 0) break;
-            if (k0 + j < P.max_iter + 1) P.widths[k0 + j] = w;      // cycle k0 + j + 1 ran at width w
+            if (k0 + j < P.widths_cap) P.widths[k0 + j] = w;      // cycle k0 + j + 1 ran at width w
             slots += w;
             terms += (long long)w * nm;              // its g-leg
             ++ran;
@@ -538,13 +550,13 @@ __global__ void gather_kernel(const Dev P, O *f, O *g)
     const Ctl c = *P.ctl;
     const int y = blockIdx.y;
     const int tid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
-    if (y < P.W) {                                    // emitted lanes, by lane id
+    if (y < P.L) {                                    // emitted lanes, by lane id
         const int lane = y;
         if (!P.emitted[lane]) return;
         if (f) for (int i = tid; i < P.n; i += nth) f[(size_t)lane * P.n + i] = (O)P.f_out[(size_t)lane * P.n + i];
         if (g) for (int j = tid; j < P.m; j += nth) g[(size_t)lane * P.m + j] = (O)P.g_out[(size_t)lane * P.m + j];
     } else {                                          // lanes still held in a slot
-        const int slot = y - P.W;
+        const int slot = y - P.L;
         if (c.done || slot >= c.n_phys) return;
         if (P.mode == MODE_MASKED && P.state[slot]) return;
         const int lane = P.lane_id[slot];
@@ -560,7 +572,7 @@ __global__ void gather_kernel(const Dev P, O *f, O *g)
 __global__ void gather_small_kernel(const Dev P, int *depth, int *status, float *rrow, float *rcol)
 {
     const int t = blockIdx.x * blockDim.x + threadIdx.x;
-    if (t >= P.W) return;
+    if (t >= P.L) return;
     if (depth) depth[t] = P.depth[t];
     if (status) status[t] = P.status[t];
     if (rrow) rrow[t] = (float)P.res_row[t];
@@ -584,17 +596,25 @@ void launch_gather_audit(const Dev &P, float *rrow, float *rcol, int *flagged, c
 }
 
 // ---------------------------------------------------------------- launchers
-void launch_lane_stats(const Dev &P, const void *x, const void *y, const float *eps, double *, cudaStream_t st)
+void launch_lane_stats(const Dev &P, const void *x, const void *y, const float *eps, int slot0, int lane0, int count,
+                       int cycle0, cudaStream_t st)
 {
-    lane_stats_kernel<<<P.W, 256, 0, st>>>(P, x, y, eps);
+    lane_stats_kernel<<<count, 256, 0, st>>>(P, x, y, eps, slot0, lane0, cycle0);
 }
-void launch_prep(const Dev &P, const void *x, const void *y, const float *a, const float *b, cudaStream_t st)
+void launch_prep(const Dev &P, const void *x, const void *y, const float *a, const float *b, int slot0, int count, cudaStream_t st)
 {
     const int pp = P.np > P.mp ? P.np : P.mp;
-    dim3 grid((pp + 127) / 128, P.W, 2);
-    if (P.compute_f64) prep_kernel<double><<<grid, 128, 0, st>>>(P, x, y, a, b);
-    else prep_kernel<float><<<grid, 128, 0, st>>>(P, x, y, a, b);
+    dim3 grid((pp + 127) / 128, count, 2);
+    if (P.compute_f64) prep_kernel<double><<<grid, 128, 0, st>>>(P, x, y, a, b, slot0);
+    else prep_kernel<float><<<grid, 128, 0, st>>>(P, x, y, a, b, slot0);
 }
+// New lanes have come in: the control block takes them into the width (between cycles, ACTIVE only).
+__global__ void refill_ctl_kernel(const Dev P, const int count)
+{
+    Ctl *g = P.ctl;
+    g->n_phys += count; g->n_running += count; g->done = 0; g->n_retire = 0;
+}
+void launch_refill_ctl(const Dev &P, int count, cudaStream_t st) { refill_ctl_kernel<<<1, 1, 0, st>>>(P, count); }
 void launch_warm(const Dev &P, const double *f0, const double *g0, cudaStream_t st)
 {
     const int pp = P.n > P.m ? P.n : P.m;
@@ -664,13 +684,13 @@ void launch_gather(const Dev &P, void *f, void *g, bool f64, cudaStream_t st)
 {
     const int mx = P.n > P.m ? P.n : P.m;
     int gx = (mx + 1023) / 1024; if (gx > 16) gx = 16;
-    dim3 grid(gx, 2 * P.W);
+    dim3 grid(gx, P.L + P.W);
     if (f64) gather_kernel<double><<<grid, 256, 0, st>>>(P, (double *)f, (double *)g);
     else gather_kernel<float><<<grid, 256, 0, st>>>(P, (float *)f, (float *)g);
 }
 void launch_gather_small(const Dev &P, int *depth, int *status, float *rrow, float *rcol, cudaStream_t st)
 {
-    gather_small_kernel<<<(P.W + 255) / 256, 256, 0, st>>>(P, depth, status, rrow, rcol);
+    gather_small_kernel<<<(P.L + 255) / 256, 256, 0, st>>>(P, depth, status, rrow, rcol);
 }
 
 }  // namespace skb

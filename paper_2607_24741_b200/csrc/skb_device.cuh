@@ -51,7 +51,9 @@ struct Ctl {
 };
 
 struct Dev {
-    int W, n, m, d, np, mp, DP;
+    int W, n, m, d, np, mp, DP;   // W: slots (lanes held at a time)
+    int L;                    // lanes the result buffers hold (> W when finished lanes are replaced by new problems)
+    int widths_cap;           // entries of widths[]
     int mode, max_iter, audit_every, xy_bf16, compute_f64, cost_form, tensor;
     int early_exit;           // MASKED only: CTAs of a frozen lane return at once (an extra arm, not the paper's mask control)
     int dry_run;              // measurement launches: a leg computes everything but stores no potential and adds no residual term
@@ -73,6 +75,7 @@ struct Dev {
     // per-slot scalars
     double *scale;            // s
     int *lane_id;
+    int *start;               // cycle count of the batch when the lane in the slot came in (0 for the first W lanes)
     int *form;                // Form per slot
     int *state;               // MASKED: frozen; STATIC: passed
     int *flag;                // screen-positive at this audit
@@ -192,6 +195,14 @@ __device__ __forceinline__ unsigned long long direct_rows_block(const Dev &P, co
     return sum;
 }
 
+// Is the state of a lane that came in at batch cycle `start` audited when the batch has completed
+// `cycle` cycles?  Audits sit on the BATCH's grid (every audit_every-th cycle) and need at least one
+// cycle of the lane's own; a warm proposal may be audited before its first cycle.
+__device__ __forceinline__ bool lane_audited(const Dev &P, const int cycle, const int start)
+{
+    return (cycle - start >= 1 && (cycle % P.audit_every) == 0) || (cycle == 0 && P.audit_initial);
+}
+
 // The row residual a lane's decisions are taken from: the escalated value if one was taken.
 __device__ __forceinline__ double lane_row_residual(const Dev &P, const int slot)
 {
@@ -203,7 +214,7 @@ __device__ __forceinline__ double lane_row_residual(const Dev &P, const int slot
 __device__ __forceinline__ bool lane_flag(const Dev &P, const Ctl &c, const int slot)
 {
     const bool passed = P.state[slot] != 0;                  // MASKED: frozen; STATIC: already passed
-    const bool audited = (c.cycle >= 1 && (c.cycle % P.audit_every) == 0) || (c.cycle == 0 && P.audit_initial);
+    const bool audited = lane_audited(P, c.cycle, P.start[slot]);
     const bool live = !(passed && (P.mode == MODE_MASKED || P.mode == MODE_STATIC));
     return audited && live && !P.nonfinite[slot] && lane_row_residual(P, slot) <= P.tol_screen;
 }
@@ -216,7 +227,7 @@ __device__ __forceinline__ bool lane_needs_column_check(const Dev &P, const Ctl 
     if (lane_flag(P, c, slot)) return true;
     if (!(P.guard > 0.0)) return false;
     const bool passed = P.state[slot] != 0;
-    const bool audited = (c.cycle >= 1 && (c.cycle % P.audit_every) == 0) || (c.cycle == 0 && P.audit_initial);
+    const bool audited = lane_audited(P, c.cycle, P.start[slot]);
     const bool live = !(passed && (P.mode == MODE_MASKED || P.mode == MODE_STATIC));
     return audited && live && !P.nonfinite[slot] && in_guard_band(P, (double)P.rsum_row[slot] * (1.0 / RSUM_SCALE));
 }

@@ -40,6 +40,8 @@ struct Variant {
     void (*launch)(const Dev &, int leg, int width, cudaStream_t);
     // several whole cycles per launch, one thread-block cluster per lane; null where there is none
     void (*launch_cycles)(const Dev &, int cycles, int width, cudaStream_t);
+    // does a lane of n x m points fit the shared-memory-resident version of the multi-cycle kernel?
+    bool (*lane_fits_shared)(int n, int m);
 };
 constexpr int MAX_CLUSTER_BLOCKS = MAX_CLUSTER_RANKS;   // a lane needs at most this many row blocks
 constexpr int MAX_CYCLES_IN_LAUNCH = 64;    // upper bound on the cycles one multi-cycle launch runs
@@ -48,8 +50,10 @@ constexpr int MAX_CYCLES_IN_LAUNCH = 64;    // upper bound on the cycles one mul
 const Variant *choose_variant(int W, int n, int m, int d, bool f64, bool fast_exp, int force_cs);
 int padded_dim(int d);
 
-void launch_lane_stats(const Dev &P, const void *x, const void *y, const float *eps, double *max_radius, cudaStream_t st);
-void launch_prep(const Dev &P, const void *x, const void *y, const float *a, const float *b, cudaStream_t st);
+void launch_lane_stats(const Dev &P, const void *x, const void *y, const float *eps, int slot0, int lane0, int count,
+                       int cycle0, cudaStream_t st);
+void launch_prep(const Dev &P, const void *x, const void *y, const float *a, const float *b, int slot0, int count, cudaStream_t st);
+void launch_refill_ctl(const Dev &P, int count, cudaStream_t st);
 void launch_warm(const Dev &P, const double *f0, const double *g0, cudaStream_t st);
 int launch_plan(const Dev &P, int width, cudaStream_t st);        // both return the number of kernels launched
 // tensor-core update kernel (bf16 inputs, d a multiple of 64 up to 512)

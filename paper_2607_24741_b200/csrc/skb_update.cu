@@ -102,10 +102,13 @@ static void launch_cycles(const Dev &P, int cycles, int width, cudaStream_t st)
     else cudaLaunchKernelEx(&cfg, lane_cycles_kernel<T, DP, CS, XF>, P, cycles);
 }
 
+template <typename T, int DP, int CS>
+static bool lane_fits_shared(int n, int m) { return ResidentLayout<T, DP, CS>::bytes(n, m) <= RESIDENT_SMEM_LIMIT; }
+
 #define SKB_V(T, F64, XF, DP, CS) \
     { F64, XF, DP, Tune<T, DP>::R, CS, (UPD_THREADS / 32) * Tune<T, DP>::R * (32 / CS), \
       2 * (size_t)(DP + 2) * TileCols<T, DP, CS>::value * sizeof(T), &launch_update<T, DP, CS, XF>, \
-      &launch_cycles<T, DP, CS, XF> }
+      &launch_cycles<T, DP, CS, XF>, &lane_fits_shared<T, DP, CS> }
 #define SKB_ROW(DP) \
     SKB_V(float, 0, 0, DP, 1), SKB_V(float, 0, 0, DP, 4), SKB_V(float, 0, 0, DP, 32), \
     SKB_V(double, 1, 0, DP, 1), SKB_V(double, 1, 0, DP, 4), SKB_V(double, 1, 0, DP, 32), \
@@ -129,9 +132,9 @@ static void launch_bigd(const Dev &P, int leg, int width, cudaStream_t st)
 
 // DP = 0 marks the large-d kernels: the padded dimension is d rounded up to the chunk size
 static const Variant g_bigd[] = {
-    {0, 0, 0, 4, 4, BIGD_RB, 2 * (size_t)BIGD_KC * (BIGD_RB + BIGD_TJ) * 4, &launch_bigd<float, 0>, nullptr},
-    {1, 0, 0, 4, 4, BIGD_RB, 2 * (size_t)BIGD_KC * (BIGD_RB + BIGD_TJ) * 8, &launch_bigd<double, 0>, nullptr},
-    {1, 1, 0, 4, 4, BIGD_RB, 2 * (size_t)BIGD_KC * (BIGD_RB + BIGD_TJ) * 8, &launch_bigd<double, 1>, nullptr},
+    {0, 0, 0, 4, 4, BIGD_RB, 2 * (size_t)BIGD_KC * (BIGD_RB + BIGD_TJ) * 4, &launch_bigd<float, 0>, nullptr, nullptr},
+    {1, 0, 0, 4, 4, BIGD_RB, 2 * (size_t)BIGD_KC * (BIGD_RB + BIGD_TJ) * 8, &launch_bigd<double, 0>, nullptr, nullptr},
+    {1, 1, 0, 4, 4, BIGD_RB, 2 * (size_t)BIGD_KC * (BIGD_RB + BIGD_TJ) * 8, &launch_bigd<double, 1>, nullptr, nullptr},
 };
 
 int padded_dim(int d)

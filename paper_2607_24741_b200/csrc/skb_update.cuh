@@ -738,11 +738,68 @@ __device__ __forceinline__ void run_leg(const Dev &P, const Ctl &c, const int le
     finish_rows<T, RB>(P, c, leg, slot, form, sc.row_m, sc.row_s, sc.row_h, sc.red, row_base);
 }
 
+// Guard band on the one-launch-per-leg path: with it on, a column-check launch carries a pool of extra
+// blocks (grid rows past the lanes).  The pool looks for lanes whose fused screen came out inside the
+// band and re-evaluates their row residual from the raw inputs in float64 - one warp per row, all pool
+// warps sharing a lane's rows, exact integer sum - and the planner decides from that value.
+// (Its float64 exponentials need more registers than the fp32 legs: update_kernel's launch bounds keep
+// the fp32 instances at four blocks per SM, and the surplus spills here, on the rare path.)
+__device__ __forceinline__ void guard_pool(const Dev &P, const Ctl &c, const int nlanes, unsigned long long *red)
+{
+    if (c.done || c.static_final) return;
+    constexpr int NW = UPD_THREADS / 32;
+    __shared__ int hot[UPD_THREADS];
+    __shared__ int n_hot;
+    const int pool_id = ((int)blockIdx.y - nlanes) * (int)gridDim.x + (int)blockIdx.x;
+    const int pool_warps = ((int)gridDim.y - nlanes) * (int)gridDim.x * NW;
+    for (int s0 = 0; s0 < c.n_phys; s0 += UPD_THREADS * 4) {
+        if (threadIdx.x == 0) n_hot = 0;
+        __syncthreads();
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int s = s0 + u * UPD_THREADS + (int)threadIdx.x;
+            if (s < c.n_phys && lane_audited(P, c.cycle, P.start[s]) && !(P.mode != MODE_ACTIVE && P.state[s] != 0) &&
+                !P.nonfinite[s] && in_guard_band(P, (double)P.rsum_row[s] * (1.0 / RSUM_SCALE))) {
+                const int at = atomicAdd(&n_hot, 1);
+                if (at < UPD_THREADS) hot[at] = s;
+            }
+        }
+        __syncthreads();
+        const int nh = n_hot < UPD_THREADS ? n_hot : UPD_THREADS;   // more than 128 at once: the rest keep their fp32 screen
+        for (int q = 0; q < nh; ++q) {
+            const int s = hot[q];
+            int bad;
+            const unsigned long long mine = direct_rows_block<NW>(P, s, pool_id * NW, pool_warps, P.n,
+                                                                  P.phi[c.parity] + (size_t)s * P.np, 0, red, &bad);
+            if (threadIdx.x == 0) {
+                atomicAdd(P.rsum_row64 + s, mine);
+                if (bad) P.nonfinite[s] = 1;
+                P.esc[s] = 1;
+            }
+        }
+        __syncthreads();
+    }
+}
+
+// Blocks per SM the per-leg kernel is held to (register cap): four for fp32 up to 16 dimensions,
+// five / three for float64 arguments with fp32 exponentials at two / four rows per thread - what the
+// legs reach by themselves, so that the guard pool's float64 code, which lives in the same kernel,
+// cannot cost them an occupancy step - and seven for fp32 up to 4 dimensions, where occupancy was
+// measured to pay (registration f-leg at 32 / 8 lanes: 638 / - us at five blocks, 627 / 180 at six,
+// 610 / 174 at seven, 614 / 190 at eight, 615 / 198 at ten).
+#ifndef SKB_BLOCKS_F32_SMALL
+#define SKB_BLOCKS_F32_SMALL 7
+#endif
+template <typename T, int DP, int XF, int RR> struct UpdBlocksPerSM {
+    static constexpr int R = RR ? RR : Tune<T, DP>::R;
+    static constexpr int value = sizeof(T) == 4 ? (DP <= 4 ? SKB_BLOCKS_F32_SMALL : (DP <= 16 ? 4 : 1)) : ((DP <= 8 && XF == 1) ? (R >= 4 ? 3 : 5) : 1);
+};
+
 // One leg as a launch of its own.  RR: rows per thread, 0 = the type's default.  Rows are independent
 // and a row's arithmetic does not depend on which thread holds it, so launches with different RR
 // give the same bits.
 template <typename T, int DP, int CS, int XF, int RR = 0>
-__global__ void __launch_bounds__(UPD_THREADS) update_kernel(const Dev P, const int leg, const int nlanes)
+__global__ void __launch_bounds__(UPD_THREADS, UpdBlocksPerSM<T, DP, XF, RR>::value) update_kernel(const Dev P, const int leg, const int nlanes)
 {
     constexpr int R = RR ? RR : Tune<T, DP>::R;
     constexpr int RB = (UPD_THREADS / 32) * R * (32 / CS);   // rows per CTA
@@ -765,46 +822,7 @@ __global__ void __launch_bounds__(UPD_THREADS) update_kernel(const Dev P, const 
     const int slot = blockIdx.y;
     const int row_base = (int)blockIdx.x * RB;
     if (leg == LEG_V && (int)blockIdx.y >= nlanes) {
-        // Guard band: with it on, a column-check launch carries a pool of extra blocks (grid rows past
-        // the lanes).  The pool looks for lanes whose fused screen came out inside the band and
-        // re-evaluates their row residual from the raw inputs in float64 - one warp per row, all pool
-        // warps sharing a lane's rows, exact integer sum - and the planner decides from that value.
-        if (c.done || c.static_final) return;
-        constexpr int NW = UPD_THREADS / 32;
-        __shared__ int hot[UPD_THREADS];
-        __shared__ int n_hot;
-        const int pool_id = ((int)blockIdx.y - nlanes) * (int)gridDim.x + (int)blockIdx.x;
-        const int pool_warps = ((int)gridDim.y - nlanes) * (int)gridDim.x * NW;
-        const bool audited = (c.cycle >= 1 && (c.cycle % P.audit_every) == 0) || (c.cycle == 0 && P.audit_initial);
-        if (!audited) return;
-        for (int s0 = 0; s0 < c.n_phys; s0 += UPD_THREADS * 4) {
-            if (threadIdx.x == 0) n_hot = 0;
-            __syncthreads();
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int s = s0 + u * UPD_THREADS + (int)threadIdx.x;
-                if (s < c.n_phys && !(P.mode != MODE_ACTIVE && P.state[s] != 0) && !P.nonfinite[s] &&
-                    in_guard_band(P, (double)P.rsum_row[s] * (1.0 / RSUM_SCALE))) {
-                    const int at = atomicAdd(&n_hot, 1);
-                    if (at < UPD_THREADS) hot[at] = s;
-                }
-            }
-            __syncthreads();
-            const int nh = n_hot < UPD_THREADS ? n_hot : UPD_THREADS;   // more than 128 at once: the rest keep their fp32 screen
-            for (int q = 0; q < nh; ++q) {
-                const int s = hot[q];
-                int bad;
-                const unsigned long long mine = direct_rows_block<NW>(P, s, pool_id * NW, pool_warps, P.n,
-                                                                      P.phi[c.parity] + (size_t)s * P.np, 0,
-                                                                      reinterpret_cast<unsigned long long *>(sc.red), &bad);
-                if (threadIdx.x == 0) {
-                    atomicAdd(P.rsum_row64 + s, mine);
-                    if (bad) P.nonfinite[s] = 1;
-                    P.esc[s] = 1;
-                }
-            }
-            __syncthreads();
-        }
+        guard_pool(P, c, nlanes, reinterpret_cast<unsigned long long *>(sc.red));
         return;
     }
     const bool idle = c.done || slot >= c.n_phys
@@ -872,6 +890,7 @@ __global__ void __launch_bounds__(UPD_THREADS) lane_cycles_kernel(const Dev P, c
     if (c.done || slot >= c.n_phys) return;      // the whole cluster takes this exit together
     const int tid = threadIdx.x;
     const int lane_id = P.lane_id[slot];
+    const int start = P.start[slot];             // batch cycle at which this lane came in
     const double inv_s = 1.0 / P.scale[slot];
     unsigned long long seen_row = 0ull, seen_col = 0ull, seen_row64 = 0ull;     // totals already accounted for (the planner clears the sums)
     int checks = 0, retired_at = 0;
@@ -896,7 +915,7 @@ __global__ void __launch_bounds__(UPD_THREADS) lane_cycles_kernel(const Dev P, c
             rr = (double)(tot_row - seen_row) * (1.0 / RSUM_SCALE);
             seen_row = tot_row;
             nf = ld_cg_s32(P.nonfinite + slot);
-            const bool audited = (k >= 1 && (k % P.audit_every) == 0) || (k == 0 && P.audit_initial);
+            const bool audited = lane_audited(P, k, start);
             if (audited && !nf && in_guard_band(P, rr)) {
                 // guard band: decide from a float64 re-evaluation of the row residual
                 int bad;
@@ -925,7 +944,7 @@ __global__ void __launch_bounds__(UPD_THREADS) lane_cycles_kernel(const Dev P, c
             ++checks;
         }
         const bool vd = !nf && fmax(rr, rc) <= P.tol_stop;
-        const bool limit = k >= P.max_iter;
+        const bool limit = k - start >= P.max_iter;
         int st = LANE_RUNNING;
         if (nf) st = LANE_NONFINITE;
         else if (fl && vd) st = LANE_DONE;
@@ -942,7 +961,7 @@ __global__ void __launch_bounds__(UPD_THREADS) lane_cycles_kernel(const Dev P, c
             if (blockIdx.x == 0 && tid == 0) {
                 P.res_row[lane_id] = rr;
                 P.res_col[lane_id] = fl ? rc : __longlong_as_double(0x7ff8000000000000LL);
-                P.depth[lane_id] = (limit && st != LANE_DONE) ? P.max_iter : k;
+                P.depth[lane_id] = (limit && st != LANE_DONE) ? P.max_iter : k - start;
                 P.status[lane_id] = st;
                 P.emitted[lane_id] = 1;
             }
@@ -1063,6 +1082,7 @@ __global__ void __launch_bounds__(UPD_THREADS) lane_resident_kernel(const Dev P,
     cp_async_wait<0>();
     const int form = (sizeof(T) == 8) ? (int)FORM_DOT : P.form[slot];
     const int lane_id = P.lane_id[slot];
+    const int start = P.start[slot];             // batch cycle at which this lane came in
     const double inv_s = 1.0 / P.scale[slot];
     cluster_sync_all();                          // every block's tables exist before anyone writes into them
 
@@ -1200,7 +1220,7 @@ __global__ void __launch_bounds__(UPD_THREADS) lane_resident_kernel(const Dev P,
             nf = 0;
             for (int rk = 0; rk < NC; ++rk) { tot += part[0][rk]; nf |= part_nf[0][rk]; }
             rr = (double)tot * (1.0 / RSUM_SCALE);
-            const bool audited = (k >= 1 && (k % P.audit_every) == 0) || (k == 0 && P.audit_initial);
+            const bool audited = lane_audited(P, k, start);
             if (audited && !nf && in_guard_band(P, rr)) {
                 // guard band: decide from a float64 re-evaluation of the row residual.  It reads the
                 // column potentials from global memory, so the blocks' rows of g go out first.
@@ -1235,7 +1255,7 @@ __global__ void __launch_bounds__(UPD_THREADS) lane_resident_kernel(const Dev P,
             ++checks;
         }
         const bool vd = !nf && fmax(rr, rc) <= P.tol_stop;
-        const bool limit = k >= P.max_iter;
+        const bool limit = k - start >= P.max_iter;
         int st = LANE_RUNNING;
         if (nf) st = LANE_NONFINITE;
         else if (fl && vd) st = LANE_DONE;
@@ -1249,7 +1269,7 @@ __global__ void __launch_bounds__(UPD_THREADS) lane_resident_kernel(const Dev P,
             if (b == 0 && tid == 0) {
                 P.res_row[lane_id] = rr;
                 P.res_col[lane_id] = fl ? rc : __longlong_as_double(0x7ff8000000000000LL);
-                P.depth[lane_id] = (limit && st != LANE_DONE) ? P.max_iter : k;
+                P.depth[lane_id] = (limit && st != LANE_DONE) ? P.max_iter : k - start;
                 P.status[lane_id] = st;
                 P.emitted[lane_id] = 1;
             }

@@ -806,3 +806,72 @@ def test_guard_band_decisions_come_from_the_float64_reevaluation(oracle, case):
     off = run_gpu(w, mode="active", guard_band=-1.0)              # switched off: still within the usual bar
     check_against_oracle(oracle, w, off, range(W), pot_tol=POT_TOL_F32, exact_depth=False, floor=MARGIN_AUTO,
                          label=f"guard band off, {case}")
+
+
+# ---- finished lanes replaced by new problems ------------------------------------------------------------
+@pytest.mark.parametrize("compute", ["f64", "mixed", "f32"])
+def test_refill_keeps_the_width_up_and_every_lane_its_own_result(oracle, compute):
+    # 40 problems through 12 slots: whenever slots are free, the next problems come in.  Lanes are
+    # independent (Eq. 2), so every lane must end exactly as in a one-shot batch of all 40 (same bits:
+    # a lane's arithmetic depends neither on its slot nor on when it came in), depths count the lane's own
+    # cycles, and the slot identity of Eq. 7 holds over the whole run.
+    import torch
+    from paper_2607_24741_b200 import binding as B
+    w = wl.make("sweep", W=40, n=96, m=80, max_iter=3000)
+    S = 12
+    ref = run_gpu(w, compute=compute, guard_band=-1.0 if compute == "f32" else 0.0)
+    dev = torch.device("cuda:0")
+    t = lambda v: torch.from_numpy(v).to(dev)
+    x, y, a, b, eps = t(w.x), t(w.y), t(w.a), t(w.b), t(w.eps)
+    sb = B.SinkhornBatch(x[:S], y[:S], a[:S], b[:S], eps[:S], w.tol, compute=compute, max_iter=w.max_iter,
+                         lane_capacity=40, guard_band=-1.0 if compute == "f32" else 0.0)
+    nxt, refills = S, 0
+    while nxt < 40:
+        sb.step(25)
+        free = S - sb.active()
+        if free > 0:
+            c = min(free, 40 - nxt)
+            first = sb.refill(x[nxt:nxt + c], y[nxt:nxt + c], a[nxt:nxt + c], b[nxt:nxt + c], eps[nxt:nxt + c])
+            assert first == nxt
+            nxt += c; refills += 1
+    assert refills >= 3
+    sb.drain()
+    f, g = sb.potentials(f64=True); depth, status = sb.depths(); rr, rc = sb.residuals()
+    st = sb.stats(widths_cap=100000); left = sb.active()
+    sb.close()
+    depth = depth.cpu().numpy(); assert depth.shape == (40,)
+    np.testing.assert_array_equal(depth, ref["depth"]); np.testing.assert_array_equal(status.cpu().numpy(), ref["status"])
+    np.testing.assert_array_equal(f.cpu().numpy(), ref["f"]); np.testing.assert_array_equal(g.cpu().numpy(), ref["g"])
+    np.testing.assert_array_equal(rr.cpu().numpy(), ref["r_row"])
+    assert left == 0 and st["slots"] == int(depth.sum()) == sum(st["widths"]) and max(st["widths"]) <= S
+    if compute != "f32":            # (pure fp32 on these small-eps lanes has its recorded limits; the bit-identity above stands)
+        lanes = [0, 5, 11, 12, 20, 33, 39]
+        check_against_oracle(oracle, w, dict(ref, depth=depth), lanes, pot_tol=POT_TOL_F64 if compute == "f64" else POT_TOL_F32,
+                             exact_depth=compute == "f64", floor=None if compute == "f64" else MARGIN_AUTO,
+                             label=f"refilled lanes, {compute}")
+
+
+def test_refill_is_refused_where_it_cannot_work():
+    import torch
+    from paper_2607_24741_b200 import binding as B
+    w = wl.make("tiny")
+    t = lambda v: torch.from_numpy(v).to("cuda:0")
+    x, y, a, b, eps = t(w.x), t(w.y), t(w.a), t(w.b), t(w.eps)
+    with pytest.raises(B.SkbError) as e:                          # only ACTIVE batches compact, so only they have free slots
+        B.SinkhornBatch(x, y, a, b, eps, w.tol, mode="masked", lane_capacity=16)
+    assert e.value.code == 2
+    sb = B.SinkhornBatch(x[:4], y[:4], a[:4], b[:4], eps[:4], w.tol, lane_capacity=6)
+    with pytest.raises(B.SkbError) as e:                          # no lane has finished yet
+        sb.refill(x[4:6], y[4:6], a[4:6], b[4:6], eps[4:6])
+    assert e.value.code == 5
+    sb.drain()
+    assert sb.refill(x[4:6], y[4:6], a[4:6], b[4:6], eps[4:6]) == 4
+    with pytest.raises(B.SkbError) as e:                          # capacity of 6 lanes used up
+        sb.refill(x[6:7], y[6:7], a[6:7], b[6:7], eps[6:7])
+    assert e.value.code == 2
+    sb.drain()
+    depth, status = sb.depths()
+    assert depth.shape[0] == 6 and (status.cpu().numpy() == 1).all()
+    ref = run_gpu(w)
+    np.testing.assert_array_equal(depth.cpu().numpy(), ref["depth"][:6])
+    sb.close()
