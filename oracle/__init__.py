@@ -119,6 +119,14 @@ def residuals(x, y, a, b, eps, f, g):
     return float(np.abs(row - _c64(a)).sum()), float(np.abs(col - _c64(b)).sum())
 
 
+def apply_plan(x, y, eps, f, g, v) -> np.ndarray:
+    """The plan of Eq. 3, pi = exp((f + g - C)/eps), applied to values v [m, dv]: pi @ v, written out
+    from the definition with the dense plan (float64)."""
+    C = cost_matrix(x, y)
+    pi = np.exp((_c64(f)[:, None] + _c64(g)[None, :] - C) / float(eps))
+    return pi @ _c64(v)
+
+
 def dual_value(C, f, g, eps, a, b) -> float:
     C, f, g, a, b = _c64(C), _c64(f), _c64(g), _c64(a), _c64(b)
     n, m = C.shape

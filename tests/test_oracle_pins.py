@@ -287,3 +287,22 @@ def test_audit_of_the_proposal_is_eq5_at_the_proposal(oracle):
     # without the initial audit the same call never reports depth 0
     r2 = oracle.solve_lane(x, y, a, b, eps, 2 * max(rr, rc), f0=conv.f, g0=g0)
     assert r2.depth == 1
+
+
+def test_plan_application_against_the_two_by_two_plan_and_the_marginals(oracle):
+    # a=b=(1/2,1/2), C=[[0,c],[c,0]]: the plan after one cycle is [[1,k],[k,1]]/(2+2k) (closed form above)
+    L, eps = 1.3, 0.7
+    x = np.array([[0.0], [L]]); y = np.array([[0.0], [L]])
+    a = b = np.array([0.5, 0.5])
+    r = oracle.solve_lane(x, y, a, b, eps, 1e-12, fixed_cycles=1)
+    kappa = np.exp(-L * L / eps)
+    v = np.array([[2.0, -1.0], [0.5, 3.0]])
+    expect = (np.array([[1, kappa], [kappa, 1]]) / (2 + 2 * kappa)) @ v
+    np.testing.assert_allclose(oracle.apply_plan(x, y, eps, r.f, r.g, v), expect, rtol=1e-13)
+    # applied to ones it is the row marginal; applied to y it is a_i times the barycentric image
+    x, y, a, b = rand_instance(21, 9, 7, 3)
+    s = oracle.solve_lane(x, y, a, b, 0.4, 1e-10)
+    row, _ = oracle.marginals(oracle.cost_matrix(x, y), s.f, s.g, 0.4)
+    np.testing.assert_allclose(oracle.apply_plan(x, y, 0.4, s.f, s.g, np.ones((7, 1)))[:, 0], row, rtol=1e-13)
+    T = oracle.apply_plan(x, y, 0.4, s.f, s.g, y) / a[:, None]
+    assert np.all(T.min(0) >= y.min(0) - 1e-9) and np.all(T.max(0) <= y.max(0) + 1e-9)   # convex combinations of y
