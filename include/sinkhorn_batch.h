@@ -196,6 +196,20 @@ skb_status sinkhorn_batch_depths(skb_batch *h, int *depth, int *lane_status);
 skb_status sinkhorn_batch_residuals(skb_batch *h, float *r_row, float *r_col);
 
 /*
+ * The coupling applied to caller-supplied values (the plan as an output, Section on endpoints:
+ * potentials are the stored result, the plan pi = exp((f + g - C)/eps) of Eq. 3 is implied):
+ *     out[t, i, :] = sum_j pi_ij v[t, j, :]
+ * for every lane t with the potentials it finished with; v = y gives a_i times the barycentric image
+ * of x_i, v = 1 the row marginal.  x, y, eps: the arrays the batch was created from (the batch keeps
+ * no lane-ordered copy of them); v [W, m, dv] fp32, out [W, n, dv] fp32, device; 1 <= dv <= 16.
+ * Valid once every lane has finished (SKB_ERR_STATE before that, and for batches whose lanes were
+ * replaced).  Float64 arithmetic, one pass over all pairs; synchronises to check the state, then
+ * enqueues one kernel.
+ */
+skb_status sinkhorn_batch_apply_plan(skb_batch *h, const void *x, const void *y, const float *eps,
+                                     const float *v, int dv, float *out);
+
+/*
  * What the most recent audit measured, per lane still held in a slot (device outs [W], original
  * lane order, any may be null; entries of lanes that have left are not touched): the fused row
  * screen's value r_row, the column residual r_col of screen-positive lanes (NaN otherwise) and

@@ -30,7 +30,7 @@ EXPORTS = (
     "sinkhorn_batch_launch_count", "sinkhorn_batch_profile_update", "sinkhorn_batch_arithmetic",
     "sinkhorn_batch_selftest_bounded_wait", "sinkhorn_batch_warm_start", "sinkhorn_batch_set_profiling",
     "sinkhorn_batch_cycle_trace", "sinkhorn_batch_selftest_unit_rates", "sinkhorn_batch_last_audit",
-    "sinkhorn_batch_refill",
+    "sinkhorn_batch_refill", "sinkhorn_batch_apply_plan",
 )
 PHASES = ("create", "f_leg", "column_check", "plan", "emit_move", "g_leg")
 # entry points outside the sinkhorn_batch_* family
@@ -76,6 +76,7 @@ def _load():
                                          vp, ctypes.c_int, ctypes.POINTER(ctypes.c_longlong),
                                          ctypes.POINTER(ctypes.c_float)]
     lib.sinkhorn_batch_last_audit.argtypes = [vp, vp, vp, vp]
+    lib.sinkhorn_batch_apply_plan.argtypes = [vp, vp, vp, vp, vp, ctypes.c_int, vp]
     lib.sinkhorn_batch_refill.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_int, ctypes.POINTER(ctypes.c_int)]
     lib.sinkhorn_batch_warm_start.argtypes = [vp, vp, vp, ctypes.c_int]
     lib.sinkhorn_batch_set_profiling.argtypes = [vp, ctypes.c_int]
@@ -279,6 +280,16 @@ class SinkhornBatch:
         _check(lib.sinkhorn_batch_refill(self.h, _ptr(x), _ptr(y), _ptr(a), _ptr(b), _ptr(eps), count, ctypes.byref(first)), self.h)
         self._keep = self._keep + (x, y, a, b, eps)
         return first.value
+
+    def apply_plan(self, v):
+        """out[t, i, :] = sum_j pi_ij v[t, j, :] with the plan of the finished lanes; v [W, m, dv] float32."""
+        x, y, _a, _b, eps = self._keep[:5]
+        v = v.contiguous()
+        if v.dtype != torch.float32 or v.dim() != 3 or tuple(v.shape[:2]) != (self.W, self.m):
+            raise ValueError("v must be float32 [W, m, dv]")
+        out = torch.empty(self.W, self.n, v.shape[2], dtype=torch.float32, device=self.device)
+        _check(lib.sinkhorn_batch_apply_plan(self.h, _ptr(x), _ptr(y), _ptr(eps), _ptr(v), v.shape[2], _ptr(out)), self.h)
+        return out
 
     def set_profiling(self, on=True):
         _check(lib.sinkhorn_batch_set_profiling(self.h, 1 if on else 0), self.h)

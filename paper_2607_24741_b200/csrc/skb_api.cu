@@ -654,6 +654,22 @@ extern "C" skb_status sinkhorn_batch_residuals(skb_batch *h, float *r_row, float
     return e == cudaSuccess ? SKB_OK : cuda_fail(h, e, "residuals");
 }
 
+extern "C" skb_status sinkhorn_batch_apply_plan(skb_batch *h, const void *x, const void *y, const float *eps,
+                                                const float *v, int dv, float *out)
+{
+    if (!h) return SKB_ERR_NULL;
+    if (!x || !y || !eps || !v || !out) return fail(h, SKB_ERR_NULL, "x, y, eps, v and out are required");
+    if (dv < 1 || dv > 16) return fail(h, SKB_ERR_SHAPE, "dv must be between 1 and 16");
+    if (h->lanes_used > h->cfg.W) return fail(h, SKB_ERR_STATE, "not available for batches whose lanes were replaced (the inputs of all lanes are not in one array)");
+    Ctl c;
+    skb_status st = read_ctl(h, &c);
+    if (st != SKB_OK) return st;
+    if (!c.done) return fail(h, SKB_ERR_STATE, "the plan is applied once every lane has finished (drain first)");
+    launch_apply_plan(h->dev, x, y, eps, v, dv, out, h->cfg.W, h->stream);
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? SKB_OK : cuda_fail(h, e, "apply_plan");
+}
+
 extern "C" skb_status sinkhorn_batch_last_audit(skb_batch *h, float *r_row, float *r_col, int *flagged)
 {
     if (!h) return SKB_ERR_NULL;

@@ -595,6 +595,52 @@ void launch_gather_audit(const Dev &P, float *rrow, float *rcol, int *flagged, c
     gather_audit_kernel<<<(P.W + 255) / 256, 256, 0, st>>>(P, rrow, rcol, flagged);
 }
 
+// ---------------------------------------------------------------- plan application
+// out[t, i, :] = sum_j pi_ij v[t, j, :] with pi = exp((f + g - C)/eps) from the potentials the batch
+// holds for lane t (Eq. 3's plan, never stored): the coupling applied to caller-supplied values, e.g.
+// v = y gives a_i times the barycentric image of x_i.  One warp per row, float64 throughout, cost from
+// the caller's raw coordinates.  After a g-leg every pi_ij <= b_j <= 1, so the exponentials need no shift.
+constexpr int APPLY_MAX_DV = 16;
+__global__ void __launch_bounds__(128) apply_plan_kernel(const Dev P, const void *x, const void *y, const float *eps,
+                                                         const float *v, const int dv, float *out)
+{
+    const int lane_t = blockIdx.y, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int i = blockIdx.x * 4 + warp;
+    if (i >= P.n || !P.emitted[lane_t]) return;
+    const double inv_eps = 1.0 / (double)eps[lane_t];
+    const double fi = P.f_out[(size_t)lane_t * P.n + i];
+    const double *g = P.g_out + (size_t)lane_t * P.m;
+    const size_t xb = ((size_t)lane_t * P.n + i) * P.d;
+    double acc[APPLY_MAX_DV];
+#pragma unroll
+    for (int c = 0; c < APPLY_MAX_DV; ++c) acc[c] = 0.0;
+    for (int j = lane; j < P.m; j += 32) {
+        const size_t yb = ((size_t)lane_t * P.m + j) * P.d;
+        double cst = 0.0;
+        for (int k = 0; k < P.d; ++k) {
+            const double t = (double)load_raw(P, x, xb + k) - (double)load_raw(P, y, yb + k);
+            cst = fma(t, t, cst);
+        }
+        const double pij = exp((fi + g[j] - cst) * inv_eps);
+        const float *vj = v + ((size_t)lane_t * P.m + j) * dv;
+#pragma unroll
+        for (int c = 0; c < APPLY_MAX_DV; ++c) if (c < dv) acc[c] = fma(pij, (double)vj[c], acc[c]);
+    }
+#pragma unroll
+    for (int c = 0; c < APPLY_MAX_DV; ++c) {
+        if (c < dv) {
+            double a = acc[c];
+            for (int off = 16; off > 0; off >>= 1) a += __shfl_xor_sync(0xffffffffu, a, off);
+            if (lane == 0) out[((size_t)lane_t * P.n + i) * dv + c] = (float)a;
+        }
+    }
+}
+void launch_apply_plan(const Dev &P, const void *x, const void *y, const float *eps, const float *v, int dv, float *out,
+                       int lanes, cudaStream_t st)
+{
+    apply_plan_kernel<<<dim3((P.n + 3) / 4, lanes), 128, 0, st>>>(P, x, y, eps, v, dv, out);
+}
+
 // ---------------------------------------------------------------- launchers
 void launch_lane_stats(const Dev &P, const void *x, const void *y, const float *eps, int slot0, int lane0, int count,
                        int cycle0, cudaStream_t st)

@@ -67,6 +67,8 @@ int launch_emit_move(const Dev &P, int width, cudaStream_t st);
 int launch_plan_cycles(const Dev &P, int width, int cycles, cudaStream_t st);
 void launch_gather(const Dev &P, void *f, void *g, bool f64, cudaStream_t st);
 void launch_gather_audit(const Dev &P, float *rrow, float *rcol, int *flagged, cudaStream_t st);
+void launch_apply_plan(const Dev &P, const void *x, const void *y, const float *eps, const float *v, int dv, float *out,
+                       int lanes, cudaStream_t st);
 void launch_gather_small(const Dev &P, int *depth, int *status, float *rrow, float *rcol, cudaStream_t st);
 
 }  // namespace skb

@@ -790,9 +790,19 @@ __device__ __forceinline__ void guard_pool(const Dev &P, const Ctl &c, const int
 #ifndef SKB_BLOCKS_F32_SMALL
 #define SKB_BLOCKS_F32_SMALL 7
 #endif
+#ifndef SKB_BLOCKS_F32_MID
+#define SKB_BLOCKS_F32_MID 4
+#endif
+#ifndef SKB_BLOCKS_F64_WIDE
+#define SKB_BLOCKS_F64_WIDE 3
+#endif
+#ifndef SKB_BLOCKS_F64_NARROW
+#define SKB_BLOCKS_F64_NARROW 5
+#endif
 template <typename T, int DP, int XF, int RR> struct UpdBlocksPerSM {
     static constexpr int R = RR ? RR : Tune<T, DP>::R;
-    static constexpr int value = sizeof(T) == 4 ? (DP <= 4 ? SKB_BLOCKS_F32_SMALL : (DP <= 16 ? 4 : 1)) : ((DP <= 8 && XF == 1) ? (R >= 4 ? 3 : 5) : 1);
+    static constexpr int value = sizeof(T) == 4 ? (DP <= 4 ? SKB_BLOCKS_F32_SMALL : (DP <= 16 ? SKB_BLOCKS_F32_MID : 1))
+                                                : ((DP <= 8 && XF == 1) ? (R >= 4 ? SKB_BLOCKS_F64_WIDE : SKB_BLOCKS_F64_NARROW) : 1);
 };
 
 // One leg as a launch of its own.  RR: rows per thread, 0 = the type's default.  Rows are independent

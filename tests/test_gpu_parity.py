@@ -875,3 +875,37 @@ def test_refill_is_refused_where_it_cannot_work():
     ref = run_gpu(w)
     np.testing.assert_array_equal(depth.cpu().numpy(), ref["depth"][:6])
     sb.close()
+
+
+# ---- the plan as an output ------------------------------------------------------------------------------
+@pytest.mark.parametrize("case", ["sensor_ragged", "registration_small", "sweep_small"])
+def test_plan_application_against_the_oracle(oracle, case):
+    import torch
+    from paper_2607_24741_b200 import binding as B
+    w = _make(case)
+    W, n, m, d = w.shape
+    dev = torch.device("cuda:0")
+    t = lambda v: torch.from_numpy(v).to(dev)
+    sb = B.SinkhornBatch(t(w.x), t(w.y), t(w.a), t(w.b), t(w.eps), w.tol, max_iter=w.max_iter)
+    with pytest.raises(B.SkbError) as e:
+        sb.apply_plan(t(w.y))
+    assert e.value.code == 5                                   # lanes still running
+    sb.drain()
+    f, g = sb.potentials(f64=True)
+    out_y = sb.apply_plan(t(w.y)).cpu().numpy()                # a_i times the barycentric image of x_i
+    ones = sb.apply_plan(torch.ones(W, m, 1, device=dev)).cpu().numpy()
+    sb.close()
+    fh, gh = f.cpu().numpy(), g.cpu().numpy()
+    for k in range(W):
+        want = oracle.apply_plan(w.x[k], w.y[k], float(w.eps[k]), fh[k], gh[k], w.y[k])
+        scale = np.abs(want).max()
+        assert np.abs(out_y[k] - want).max() <= 2e-6 * scale           # same potentials: float32 output rounding
+        np.testing.assert_allclose(ones[k, :, 0], want_row(oracle, w, k, fh[k], gh[k]), rtol=2e-6)
+        ref = oracle.solve_lane(w.x[k], w.y[k], w.a[k], w.b[k], float(w.eps[k]), w.tol, max_iter=w.max_iter)
+        mine = oracle.apply_plan(w.x[k], w.y[k], float(w.eps[k]), ref.f, ref.g, w.y[k])
+        assert np.abs(out_y[k] - mine).max() <= 2e-3 * scale           # the oracle's own solve: potentials within 1e-4
+
+
+def want_row(oracle, w, k, f, g):
+    row, _ = oracle.marginals(oracle.cost_matrix(w.x[k], w.y[k]), f, g, float(w.eps[k]))
+    return row
