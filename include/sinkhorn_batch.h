@@ -97,10 +97,11 @@ typedef struct {
     float guard_band;      /* guard band around the thresholds with float64 escalation     */
                            /* (Section 5, stress test of near-threshold accept decisions): */
                            /* a lane whose row screen lies within this RELATIVE distance   */
-                           /* of tau_screen or tau_stop has its row residual re-evaluated  */
-                           /* from the raw inputs in float64 and is decided by that value. */
-                           /* 0 = default (1e-3), negative = off; d <= 32 only (ignored    */
-                           /* for larger d).  Costs a raw copy of x and y in the workspace */
+                           /* of tau_screen or tau_stop (at least 1e-7 absolute) has its   */
+                           /* row residual re-evaluated from the raw inputs in float64 and */
+                           /* is decided by that value.  0 = default (2.5e-4), negative =  */
+                           /* off; d <= 32 only (ignored for larger d).  Costs a raw copy  */
+                           /* of x and y in the workspace                                  */
     int lane_capacity;     /* lanes the batch can take in over its life: 0 or W = the W of  */
                            /* create only; more (ACTIVE mode) lets sinkhorn_batch_refill    */
                            /* put new problems into the slots finished lanes have freed;    */

@@ -110,13 +110,13 @@ static bool config_ok(const skb_config *c, std::string &why)
     return true;
 }
 
-// Relative half-width of the guard band: the configured value, 1e-3 by default, off when negative
+// Relative half-width of the guard band: the configured value, 2.5e-4 by default, off when negative
 // and for d > 32 (the float64 re-evaluation walks all pairs of a lane with one thread per row, which
 // is only affordable where a pair is a few dimensions deep).
 static double guard_width(const skb_config *c)
 {
     if (c->d > 32 || c->guard_band < 0.0f) return 0.0;
-    return c->guard_band > 0.0f ? (double)c->guard_band : 1.0e-3;
+    return c->guard_band > 0.0f ? (double)c->guard_band : 2.5e-4;
 }
 
 // Lays the batch's arrays out in the workspace (base may be null: size query only).

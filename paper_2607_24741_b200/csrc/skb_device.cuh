@@ -125,9 +125,13 @@ __device__ __forceinline__ float load_raw(const Dev &P, const void *base, size_t
 // Section 5: an outward guard with float64 escalation).  A screen value this close to a threshold
 // is within the evaluation error of the fp32 exponentials, so the decision is taken from a float64
 // re-evaluation instead.
+// The band is relative to the threshold with an absolute floor: the fused screen's error is a few 1e-8
+// absolute whatever the tolerance (measured), i.e. 3e-5 of a tolerance of 1e-3 but 3e-4 of 1e-4.
+constexpr double GUARD_ABS_FLOOR = 1.0e-7;
 __device__ __forceinline__ bool in_guard_band(const Dev &P, const double rr)
 {
-    return P.guard > 0.0 && (fabs(rr - P.tol_screen) <= P.guard * P.tol_screen || fabs(rr - P.tol_stop) <= P.guard * P.tol_stop);
+    return P.guard > 0.0 && (fabs(rr - P.tol_screen) <= fmax(P.guard * P.tol_screen, GUARD_ABS_FLOOR) ||
+                             fabs(rr - P.tol_stop) <= fmax(P.guard * P.tol_stop, GUARD_ABS_FLOOR));
 }
 
 // One row's term |sum_j pi_ij - a_i| of the row residual (Eq. 5), from the raw inputs and the

@@ -40,8 +40,7 @@ constexpr int TC_THREADS = TC_EPI_THREADS + 64;            // + producer warp + 
 constexpr int TC_MAX_STAGES = 4;
 constexpr int TC_BM = 128, TC_BK = 64;
 constexpr uint32_t TC_CHUNK = TC_BM * TC_BK * 2;          // 16 KB: 128 points x 64 bf16
-constexpr long long TC_WAIT_CLOCKS = 2000000000LL;        // ~1 s
-__device__ long long g_wait_clocks = TC_WAIT_CLOCKS;      // budget of every bounded wait (a self-test shortens it)
+constexpr long long TC_WAIT_CLOCKS = 2000000000LL;        // ~1 s: budget of every bounded wait of the update kernels
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint32_t a, uint32_t count)
@@ -64,13 +63,16 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t a, uint32_t parity)
     return ok != 0;
 }
 // Bounded wait: false if the budget ran out or another role already gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t a, uint32_t parity, volatile int *abort_flag)
+// The budget is an argument (the update kernels use the constant, the self-test its own short one):
+// a writable global would let a self-test on one stream shorten the waits of a solve on another.
+__device__ __forceinline__ bool mbar_wait(uint32_t a, uint32_t parity, volatile int *abort_flag,
+                                          const long long budget = TC_WAIT_CLOCKS)
 {
     if (mbar_try_wait(a, parity)) return true;          // the common case costs no clock read
     const long long t0 = clock64();
     while (!mbar_try_wait(a, parity)) {
         if (*abort_flag) return false;
-        if (clock64() - t0 > g_wait_clocks) { *abort_flag = 1; return false; }
+        if (clock64() - t0 > budget) { *abort_flag = 1; return false; }
     }
     return true;
 }
@@ -830,14 +832,11 @@ __global__ void wait_probe_kernel(int *out, long long budget)
         mbar_init(smem_u32(&bar), 1);
         abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        const long long saved = g_wait_clocks;
-        g_wait_clocks = budget;
         const long long t0 = clock64();
-        const bool ok = mbar_wait(smem_u32(&bar), 0, &abort_flag);
+        const bool ok = mbar_wait(smem_u32(&bar), 0, &abort_flag, budget);
         out[0] = ok ? 0 : 1;                       // 1: the wait gave up
         out[1] = abort_flag;
         out[2] = (int)((clock64() - t0) >> 10);    // kilo-clocks spent
-        g_wait_clocks = saved;
     }
 }
 
