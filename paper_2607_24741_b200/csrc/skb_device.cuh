@@ -150,16 +150,39 @@ __device__ __forceinline__ double direct_row_term_warp(const Dev &P, const int s
     const void *yl = (const char *)P.yraw + (size_t)slot * P.yraw_stride;
     const size_t xb = (size_t)i * P.d;
     double mx = -1.0e300, sum = 0.0;
-    for (int j = lane; j < P.m; j += 32) {
-        const size_t yb = (size_t)j * P.d;
-        double c = 0.0;
-        for (int k = 0; k < P.d; ++k) {
-            const double t = (double)load_raw(P, xl, xb + k) - (double)load_raw(P, yl, yb + k);
-            c = fma(t, t, c);
+    // four columns per lane and step: their cost chains and exponentials are independent, which is
+    // what keeps the float64 pipe busy at the few warps an escalation runs on
+    constexpr int U = 4;
+    for (int j0 = lane; j0 < P.m; j0 += 32 * U) {
+        size_t yb[U];
+        double c[U], gj[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int j = j0 + 32 * u;
+            const int jc = j < P.m ? j : P.m - 1;          // clamped: loads stay inside the lane, the term is dropped below
+            yb[u] = (size_t)jc * P.d;
+            gj[u] = __ldcg(gam + jc);
+            c[u] = 0.0;
         }
-        const double v = phi + __ldcg(gam + j) - s * c;
-        if (v > mx) { sum *= exp2(mx - v); mx = v; }
-        sum += exp2(v - mx);
+        for (int k = 0; k < P.d; ++k) {
+            const double xk = (double)load_raw(P, xl, xb + k);
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const double t = xk - (double)load_raw(P, yl, yb[u] + k);
+                c[u] = fma(t, t, c[u]);
+            }
+        }
+        double v[U], mn = mx;
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            v[u] = (j0 + 32 * u < P.m) ? phi + gj[u] - s * c[u] : -1.0e300;
+            mn = fmax(mn, v[u]);
+        }
+        double add = 0.0;
+#pragma unroll
+        for (int u = 0; u < U; ++u) add += (j0 + 32 * u < P.m) ? exp2(v[u] - mn) : 0.0;
+        sum = sum * exp2(mx - mn) + add;
+        mx = mn;
     }
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) {

@@ -755,11 +755,24 @@ __device__ __forceinline__ void guard_pool(const Dev &P, const Ctl &c, const int
     for (int s0 = 0; s0 < c.n_phys; s0 += UPD_THREADS * 4) {
         if (threadIdx.x == 0) n_hot = 0;
         __syncthreads();
+        // all loads first (independent, clamped to a valid slot), then the predicates: the scan is on the
+        // launch's critical path and a short-circuit chain would pay one memory latency per term
+        int st_[4], fr_[4], nf_[4];
+        unsigned long long rs_[4];
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
             const int s = s0 + u * UPD_THREADS + (int)threadIdx.x;
-            if (s < c.n_phys && lane_audited(P, c.cycle, P.start[s]) && !(P.mode != MODE_ACTIVE && P.state[s] != 0) &&
-                !P.nonfinite[s] && in_guard_band(P, (double)P.rsum_row[s] * (1.0 / RSUM_SCALE))) {
+            const int sl = s < c.n_phys ? s : 0;
+            st_[u] = P.start[sl];
+            fr_[u] = P.state[sl];
+            nf_[u] = P.nonfinite[sl];
+            rs_[u] = P.rsum_row[sl];
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int s = s0 + u * UPD_THREADS + (int)threadIdx.x;
+            if (s < c.n_phys && lane_audited(P, c.cycle, st_[u]) && !(P.mode != MODE_ACTIVE && fr_[u] != 0) &&
+                !nf_[u] && in_guard_band(P, (double)rs_[u] * (1.0 / RSUM_SCALE))) {
                 const int at = atomicAdd(&n_hot, 1);
                 if (at < UPD_THREADS) hot[at] = s;
             }
@@ -884,8 +897,15 @@ __device__ __forceinline__ int ld_cg_s32(const int *p)
     return v;
 }
 
+// Blocks per SM the multi-cycle kernels are held to.  The launch policy never asks for more than four
+// blocks of them per SM, so up to 128 registers are free and the compiler is told so.  Deep float64
+// variants keep the registers their streaming loops need.
+template <typename T, int DP> struct LaneBlocksPerSM {
+    static constexpr int value = DP <= 8 ? 4 : (DP == 16 ? 3 : (sizeof(T) == 4 ? 4 : 2));
+};
+
 template <typename T, int DP, int CS, int XF, int RR = 0>
-__global__ void __launch_bounds__(UPD_THREADS) lane_cycles_kernel(const Dev P, const int cycles)
+__global__ void __launch_bounds__(UPD_THREADS, LaneBlocksPerSM<T, DP>::value) lane_cycles_kernel(const Dev P, const int cycles)
 {
     constexpr int R = RR ? RR : Tune<T, DP>::R;
     constexpr int RB = (UPD_THREADS / 32) * R * (32 / CS);
@@ -1038,7 +1058,7 @@ struct ResidentLayout {
 };
 
 template <typename T, int DP, int CS, int XF>
-__global__ void __launch_bounds__(UPD_THREADS) lane_resident_kernel(const Dev P, const int cycles)
+__global__ void __launch_bounds__(UPD_THREADS, LaneBlocksPerSM<T, DP>::value) lane_resident_kernel(const Dev P, const int cycles)
 {
     typedef ResidentLayout<T, DP, CS> L;
     constexpr int R = L::R, RB = L::RB, TJ = L::TJ, STY = L::STY, STX = L::STX;
