@@ -272,6 +272,18 @@ skb_status sinkhorn_batch_cycle_trace(skb_batch *h, float *update_ms, int cap, i
 skb_status sinkhorn_batch_arithmetic(skb_batch *h, int *compute);
 
 /*
+ * Integrity check of the caller's workspace (a stand-in for a memory checker: every kernel of
+ * the path writes through index arithmetic into arrays carved out of one allocation).  Every
+ * such array is followed by a guard strip of 256 bytes holding a known pattern, written by
+ * create; this call compares all strips and writes to *first_bad (host) the index, in layout
+ * order, of the first strip that no longer holds its pattern, or -1 if all are intact.  A
+ * damaged strip means a write past the end of the array before it.  May be called at any time
+ * after create; launches one small kernel and synchronises the batch's stream.
+ * Returns SKB_OK whether or not a strip is damaged; SKB_ERR_NULL / SKB_ERR_CUDA otherwise.
+ */
+skb_status sinkhorn_batch_check_guards(skb_batch *h, int *first_bad);
+
+/*
  * Self-test of the kernels' failure detection.  The tensor-core kernel synchronises its
  * warps through mbarriers; every such wait has a clock budget, after which the kernel
  * records an error instead of hanging (the host then reports SKB_ERR_CUDA).  This call runs

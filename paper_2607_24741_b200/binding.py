@@ -30,7 +30,7 @@ EXPORTS = (
     "sinkhorn_batch_launch_count", "sinkhorn_batch_profile_update", "sinkhorn_batch_arithmetic",
     "sinkhorn_batch_selftest_bounded_wait", "sinkhorn_batch_warm_start", "sinkhorn_batch_set_profiling",
     "sinkhorn_batch_cycle_trace", "sinkhorn_batch_selftest_unit_rates", "sinkhorn_batch_last_audit",
-    "sinkhorn_batch_refill", "sinkhorn_batch_apply_plan",
+    "sinkhorn_batch_refill", "sinkhorn_batch_apply_plan", "sinkhorn_batch_check_guards",
 )
 PHASES = ("create", "f_leg", "column_check", "plan", "emit_move", "g_leg")
 # entry points outside the sinkhorn_batch_* family
@@ -82,6 +82,7 @@ def _load():
     lib.sinkhorn_batch_set_profiling.argtypes = [vp, ctypes.c_int]
     lib.sinkhorn_batch_cycle_trace.argtypes = [vp, vp, ctypes.c_int, ctypes.POINTER(ctypes.c_int)]
     lib.sinkhorn_batch_selftest_bounded_wait.argtypes = [vp, ctypes.c_float, vp]
+    lib.sinkhorn_batch_check_guards.argtypes = [vp, ctypes.POINTER(ctypes.c_int)]
     lib.sinkhorn_batch_selftest_unit_rates.argtypes = [ctypes.POINTER(ctypes.c_double), vp, vp]
     lib.sinkhorn_batch_arithmetic.argtypes = [vp, ctypes.POINTER(ctypes.c_int)]
     lib.sinkhorn_batch_launch_count.argtypes = [vp, ctypes.POINTER(ctypes.c_longlong)]
@@ -260,6 +261,12 @@ class SinkhornBatch:
                 raise ValueError("f0 [W,n] and g0 [W,m] must be contiguous float64 CUDA tensors")
         _check(lib.sinkhorn_batch_warm_start(self.h, _ptr(f0), _ptr(g0), 1 if audit_initial else 0), self.h)
         self._warm = (f0, g0)
+
+    def check_guards(self) -> int:
+        """Index of the first damaged guard strip of the workspace, -1 if all are intact (synchronises)."""
+        bad = ctypes.c_int(-2)
+        _check(lib.sinkhorn_batch_check_guards(self.h, ctypes.byref(bad)), self.h)
+        return bad.value
 
     def last_audit(self):
         """Row screen value, column residual (NaN where not checked) and screen flag of the most recent audit."""

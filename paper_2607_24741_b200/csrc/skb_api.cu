@@ -40,6 +40,7 @@ struct skb_batch {
     float phase_ms[SKB_N_PHASES];
     std::vector<float> cycle_update_ms;   // per cycle: f-leg + g-leg
     alignas(64) unsigned char maps[2 * 128];   // CUtensorMap of x and of y
+    GuardList guards;      // guard strips of the workspace in the layout the batch runs in
     std::string err;
 };
 
@@ -120,12 +121,19 @@ static double guard_width(const skb_config *c)
 }
 
 // Lays the batch's arrays out in the workspace (base may be null: size query only).
-static size_t carve(const skb_config *c, const Variant *var, bool tensor, char *base, Dev *D, size_t *zero_end_out = nullptr)
+// Every array is followed by a guard strip (GUARD_STRIP_BYTES of a known pattern, see
+// sinkhorn_batch_check_guards); their offsets are listed in *guards.
+static size_t carve(const skb_config *c, const Variant *var, bool tensor, char *base, Dev *D, size_t *zero_end_out = nullptr,
+                    GuardList *guards = nullptr)
 {
     size_t off = 0;
+    int strips = 0;
     auto take = [&](size_t bytes) -> void * {
         void *p = base ? base + off : nullptr;
         off += align_up(bytes, 256);
+        if (guards && strips < MAX_GUARD_STRIPS) guards->off256[strips] = (unsigned)(off / 256);
+        ++strips;
+        off += GUARD_STRIP_BYTES;
         return p;
     };
     const size_t W = c->W, n = c->n, m = c->m;
@@ -145,6 +153,7 @@ static size_t carve(const skb_config *c, const Variant *var, bool tensor, char *
     d.form_threshold = FORM_DIFF_RADIUS;
     // control block first, then everything that must start at zero, in one contiguous range
     d.ctl = (Ctl *)take(sizeof(Ctl));
+    d.guard_bad = (int *)take(4);
     d.state = (int *)take(W * 4); d.flag = (int *)take(W * 4); d.verdict = (int *)take(W * 4);
     d.nonfinite = (int *)take(W * 4);
     d.ret_at = (int *)take(W * 4); d.n_checks = (int *)take(W * 4);
@@ -190,6 +199,7 @@ static size_t carve(const skb_config *c, const Variant *var, bool tensor, char *
     }
     if (D) { *D = d; D->tol_screen = 0; D->tol_stop = 0; }
     if (zero_end_out) *zero_end_out = zero_end;
+    if (guards) guards->count = strips <= MAX_GUARD_STRIPS ? strips : 0;      // more arrays than the list holds: no strips checked
     return off;
 }
 
@@ -270,7 +280,8 @@ extern "C" skb_status sinkhorn_batch_create(const void *x, const void *y, const 
     h->snap_pending = false; h->snap_idx = 0; h->profiling = false; h->pev_used = 0; h->no_multi_cycle = false;
     h->lanes_used = cfg->W; h->enqueued_at_refill = 0;
     for (int i = 0; i < SKB_N_PHASES; ++i) h->phase_ms[i] = 0.f;
-    carve(cfg, var, h->tensor, (char *)cfg->workspace, &h->dev);
+    h->guards.count = 0;
+    carve(cfg, var, h->tensor, (char *)cfg->workspace, &h->dev, nullptr, &h->guards);
     h->dev.tol_stop = (double)tol;
     h->dev.tol_screen = cfg->tol_screen > 0.0f ? (double)cfg->tol_screen : (double)tol;
     cudaError_t e;
@@ -309,13 +320,15 @@ extern "C" skb_status sinkhorn_batch_create(const void *x, const void *y, const 
         const double ts = h->dev.tol_stop, tsc = h->dev.tol_screen;
         if (radius > MIXED_RADIUS) {
             h->var = var_big;
-            carve(cfg, var_big, false, (char *)cfg->workspace, &h->dev);
+            carve(cfg, var_big, false, (char *)cfg->workspace, &h->dev, nullptr, &h->guards);
         } else if (can_tensor) {
             h->tensor = true;
-            carve(cfg, var, true, (char *)cfg->workspace, &h->dev);
+            carve(cfg, var, true, (char *)cfg->workspace, &h->dev, nullptr, &h->guards);
         }
         h->dev.tol_stop = ts; h->dev.tol_screen = tsc;
     }
+    launch_guard_strips(cfg->workspace, h->guards, true, nullptr, h->stream);      // the layout is final from here on
+    h->launches += 1;
     if (h->tensor) {
         // the MMA operands: tiled copies of x and y that the compaction may permute
         const char *why = nullptr;
@@ -721,6 +734,23 @@ extern "C" skb_status sinkhorn_batch_arithmetic(skb_batch *h, int *compute)
 {
     if (!h || !compute) return SKB_ERR_NULL;
     *compute = h->tensor ? SKB_COMPUTE_TENSOR : (!h->var->f64 ? SKB_COMPUTE_F32 : (h->var->xf ? SKB_COMPUTE_MIXED : SKB_COMPUTE_F64));
+    return SKB_OK;
+}
+
+extern "C" skb_status sinkhorn_batch_check_guards(skb_batch *h, int *first_bad)
+{
+    if (!h || !first_bad) return SKB_ERR_NULL;
+    *first_bad = -1;
+    cudaError_t e = cudaMemsetAsync(h->dev.guard_bad, 0xFF, sizeof(int), h->stream);      // atomicMin target: all ones
+    if (e != cudaSuccess) return cuda_fail(h, e, "check_guards");
+    launch_guard_strips(h->cfg.workspace, h->guards, false, h->dev.guard_bad, h->stream);
+    h->launches += 1;
+    unsigned found = 0xFFFFFFFFu;
+    if ((e = cudaGetLastError()) != cudaSuccess ||
+        (e = cudaMemcpyAsync(&found, h->dev.guard_bad, sizeof(int), cudaMemcpyDeviceToHost, h->stream)) != cudaSuccess ||
+        (e = cudaStreamSynchronize(h->stream)) != cudaSuccess)
+        return cuda_fail(h, e, "check_guards");
+    if (found != 0xFFFFFFFFu) *first_bad = (int)found - 1;
     return SKB_OK;
 }
 

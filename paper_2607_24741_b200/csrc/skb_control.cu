@@ -739,4 +739,21 @@ void launch_gather_small(const Dev &P, int *depth, int *status, float *rrow, flo
     gather_small_kernel<<<(P.L + 255) / 256, 256, 0, st>>>(P, depth, status, rrow, rcol);
 }
 
+// Guard strips: one block per strip, one 32-bit word per thread.  fill = 1 writes the pattern,
+// fill = 0 compares and lowers *bad (all ones on entry) to 1 + the index of a damaged strip.
+__global__ void __launch_bounds__(GUARD_STRIP_BYTES / 4) guard_strips_kernel(unsigned char *base, const GuardList gl, const int fill, unsigned *bad)
+{
+    const int strip = blockIdx.x;
+    if (strip >= gl.count) return;
+    unsigned *w = reinterpret_cast<unsigned *>(base + (size_t)gl.off256[strip] * 256u);
+    const unsigned want = 0xA5C3F00Du ^ ((unsigned)strip * 0x9E3779B9u) ^ threadIdx.x;
+    if (fill) { w[threadIdx.x] = want; return; }
+    if (w[threadIdx.x] != want) atomicMin(bad, (unsigned)strip + 1u);
+}
+void launch_guard_strips(void *base, const GuardList &gl, bool fill, int *bad, cudaStream_t st)
+{
+    if (gl.count < 1) return;
+    guard_strips_kernel<<<gl.count, GUARD_STRIP_BYTES / 4, 0, st>>>((unsigned char *)base, gl, fill ? 1 : 0, (unsigned *)bad);
+}
+
 }  // namespace skb

@@ -111,7 +111,18 @@ struct Dev {
     int *depth, *status, *emitted;
     double *res_row, *res_col;
     int *widths;              // [max_iter + 2]
+    int *guard_bad;           // result word of the guard-strip check
     Ctl *ctl;
+};
+
+// Guard strips of the workspace: 256 bytes of a known pattern after every array the library carves
+// out of the caller's workspace, so that a write past the end of an array is found, on request,
+// instead of silently landing in its neighbour.  Offsets in units of 256 bytes from the workspace.
+constexpr int GUARD_STRIP_BYTES = 256;
+constexpr int MAX_GUARD_STRIPS = 96;
+struct GuardList {
+    int count;
+    unsigned off256[MAX_GUARD_STRIPS];
 };
 
 // Raw coordinate of the inputs' own storage type (fp32, or bf16 widened exactly).

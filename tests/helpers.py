@@ -52,8 +52,11 @@ def run_gpu(w, mode="active", compute="auto", column_split=0, audit_every=1, tol
         stats = sb.stats(widths_cap=widths_cap)
         left = sb.active()
         arith = sb.arithmetic()
+        bad_strip = sb.check_guards()
     finally:
         sb.close()
+    # no kernel of the solve wrote past the end of an array of the workspace (checked in every GPU run)
+    assert bad_strip == -1, f"guard strip {bad_strip} of the workspace was overwritten"
     return dict(f=f.cpu().numpy(), g=g.cpu().numpy(), f32=f32.cpu().numpy(), g32=g32.cpu().numpy(),
                 depth=depth.cpu().numpy(), status=status.cpu().numpy(), r_row=rr.cpu().numpy(),
                 r_col=rc.cpu().numpy(), stats=stats, cycles=cycles, left=left, arith=arith)

@@ -468,6 +468,33 @@ def test_bounded_wait_gives_up_instead_of_hanging():
     assert int(torch.arange(10, device="cuda:0").sum().item()) == 45
 
 
+def test_guard_strips_report_an_overwritten_array_end():
+    # the workspace check itself: intact after a solve, and a write just past the end of the last
+    # array (made here, from the host side of the test) is reported with that strip's index
+    import torch
+    from paper_2607_24741_b200 import binding as B
+    w = wl.make("tiny")
+    dev = torch.device("cuda:0")
+    t = lambda v: torch.from_numpy(v).to(dev)
+    for compute in ("f64", "f32"):                  # explicit arithmetic: the layout ends where the workspace ends
+        sb = B.SinkhornBatch(t(w.x), t(w.y), t(w.a), t(w.b), t(w.eps), w.tol, compute=compute, max_iter=w.max_iter)
+        try:
+            assert sb.check_guards() == -1           # right after create
+            sb.drain()
+            assert sb.check_guards() == -1
+            assert sb.check_guards() == -1           # the check leaves the strips as they are
+            last = sb.workspace.numel() - 1
+            sb.workspace[last] ^= 0x40               # one bit of the last strip's last word
+            bad = sb.check_guards()
+            assert bad >= 40, bad                    # the last of several dozen strips
+            sb.workspace[last] ^= 0x40
+            assert sb.check_guards() == -1
+            sb.workspace[last - 255] ^= 0x01         # first byte of the same strip: same index
+            assert sb.check_guards() == bad
+        finally:
+            sb.close()
+
+
 def test_very_wide_batch_and_rectangular_lanes(oracle):
     # more lanes than the planner has threads: its scans run in several chunks, holes and fillers
     # pair up across chunks
