@@ -2,6 +2,7 @@
 // asynchronous width read-back.  No device memory is allocated here; the only CUDA
 // objects a handle holds are two events and a small pinned host block borrowed from a pool
 // (plus its own timing events once phase timing has been switched on).
+#include <nvtx3/nvToolsExt.h>
 #include <cmath>
 #include <cstdio>
 #include <cstring>
@@ -49,6 +50,15 @@ static skb_status read_ctl(skb_batch *h, Ctl *c);
 
 // Text of the last failed create (or host-buffer solve) of the calling thread.
 static thread_local std::string g_create_err;
+
+// NVTX ranges around the host-side phases (create, step, drain and its chunks, refill): they cost a
+// few nanoseconds when no tool is attached and give a timeline tool the structure of a solve.
+struct NvtxRange {
+    explicit NvtxRange(const char *name) { nvtxRangePushA(name); }
+    ~NvtxRange() { nvtxRangePop(); }
+    NvtxRange(const NvtxRange &) = delete;
+    NvtxRange &operator=(const NvtxRange &) = delete;
+};
 static const int PHASE_EVENTS_PER_CYCLE = 5;     // f-leg | column check | plan | emit/move | g-leg, boundaries shared
 static const int PROFILE_CHUNK = 16;             // cycles between two harvests of the timing events
 
@@ -240,6 +250,7 @@ static skb_status cuda_fail(skb_batch *h, cudaError_t e, const char *where)
 extern "C" skb_status sinkhorn_batch_create(const void *x, const void *y, const float *a, const float *b,
                                             const float *eps, float tol, const skb_config *cfg, skb_batch **out)
 {
+    NvtxRange nvtx_range("skb:create");
     if (!out) return fail(nullptr, SKB_ERR_NULL, "out is null");
     *out = nullptr;
     if (!x || !y || !a || !b || !eps || !cfg) return fail(nullptr, SKB_ERR_NULL, "x, y, a, b, eps and cfg are required");
@@ -382,6 +393,7 @@ extern "C" skb_status sinkhorn_batch_warm_start(skb_batch *h, const double *f0, 
 extern "C" skb_status sinkhorn_batch_refill(skb_batch *h, const void *x, const void *y, const float *a, const float *b,
                                             const float *eps, int count, int *first_lane)
 {
+    NvtxRange nvtx_range("skb:refill");
     if (!h) return SKB_ERR_NULL;
     if (!x || !y || !a || !b || !eps) return fail(h, SKB_ERR_NULL, "x, y, a, b and eps are required");
     if (count < 1) return fail(h, SKB_ERR_VALUE, "count must be >= 1");
@@ -546,6 +558,7 @@ static skb_status poll_snapshot(skb_batch *h, bool wait)
 
 extern "C" skb_status sinkhorn_batch_step(skb_batch *h, int cycles)
 {
+    NvtxRange nvtx_range("skb:step");
     if (!h) return SKB_ERR_NULL;
     if (cycles < 0) return fail(h, SKB_ERR_VALUE, "cycles must be >= 0");
     skb_status st = poll_snapshot(h, false);
@@ -574,6 +587,7 @@ extern "C" skb_status sinkhorn_batch_step(skb_batch *h, int cycles)
 
 extern "C" skb_status sinkhorn_batch_drain(skb_batch *h, int *cycles_run)
 {
+    NvtxRange nvtx_range("skb:drain");
     if (!h) return SKB_ERR_NULL;
     cudaError_t e;
     {
@@ -587,6 +601,7 @@ extern "C" skb_status sinkhorn_batch_drain(skb_batch *h, int *cycles_run)
     while (!h->finished) {
         const bool multi = cycles_in_one_launch(h);      // may become true as the batch narrows
         const int chunk_max = multi ? 32 : 16;
+        NvtxRange nvtx_chunk(multi ? "skb:chunk (cycles in one launch)" : "skb:chunk (launch per leg)");
         if (multi) enqueue_cycles_launch(h, chunk);
         else for (int i = 0; i < chunk; ++i) enqueue_cycle(h);
         if (h->profiling && (e = harvest_phases(h)) != cudaSuccess) return cuda_fail(h, e, "drain (phase timing)");

@@ -15,7 +15,7 @@ import numpy as np
 LEDGER: list[dict] = []
 
 # The band inside which the acceptance bar itself allows a lane to stop one audit away.
-NORTH_STAR_BAND = 1e-6
+ACCEPTANCE_BAND = 1e-6
 
 # |r_col reported by the GPU - float64 column residual of the potentials it emitted|.  After a
 # g-leg the column marginal is current (Eq. 4), so both are pure arithmetic error: the column
@@ -152,7 +152,7 @@ def new_entry(label, w, r, lanes, tol, floor):
 def close_entry(entry, misses, floor):
     for (t, dg, do, margin, decay) in misses:
         entry["misses"].append(dict(lane=int(t), gpu=dg, oracle=do, margin=margin, decay=decay,
-                                    inside_1e6_band=bool(margin <= NORTH_STAR_BAND)))
+                                    inside_1e6_band=bool(margin <= ACCEPTANCE_BAND)))
         if floor is not None:
             assert miss_allowed(margin, decay, floor), \
                 f"{entry['label']} lane {t}: gpu {dg} oracle {do} margin {margin:.2e} decay {decay:.2e}"
