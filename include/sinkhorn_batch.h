@@ -63,7 +63,8 @@ typedef enum { SKB_F32 = 0, SKB_BF16 = 1 } skb_dtype;           /* storage type 
 /* Arithmetic of the pair terms log2 pi_ij and their exponentials. */
 typedef enum {
     SKB_COMPUTE_AUTO = 0,  /* F32 (TENSOR where eligible), or MIXED when some lane's cost/eps  */
-                           /* range is beyond fp32                                             */
+                           /* range is beyond fp32 for the tolerance asked for: scaled squared */
+                           /* radius log2(e)/eps * max|x - centre|^2 above 512 * min(1, tol/1e-3) */
     SKB_COMPUTE_F32 = 1,   /* fp32 exponents and exponentials                                  */
     SKB_COMPUTE_MIXED = 2, /* float64 exponents (half-rate FP64 pipe), fp32 exponentials       */
     SKB_COMPUTE_F64 = 3,   /* float64 throughout, software exp2: the slow validation arithmetic */

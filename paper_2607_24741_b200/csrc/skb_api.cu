@@ -96,10 +96,17 @@ static void host_res_put(const HostRes &r)
 
 // fp32 arithmetic: the expanded cost |x|^2+|y|^2-2x.y carries an error of about one ulp of the
 // scaled squared radius M = s*max|x-c|^2 into every exponent.  Above FORM_DIFF_RADIUS a lane
-// switches to the difference form; above MIXED_RADIUS (any lane) an automatic batch computes
+// switches to the difference form; above mixed_radius(tol) (any lane) an automatic batch computes
 // its exponents in float64 and only the exponentials in fp32.
 static const double FORM_DIFF_RADIUS = 512.0;
 static const double MIXED_RADIUS = 512.0;
+// One ulp of M in the exponent is a relative error of about M * 8e-8 in every plan entry and, where it
+// is systematic, in the residuals: 4 % of a tolerance of 1e-3 at M = 512.  A stricter tolerance lowers
+// the radius in proportion, so that the evaluation error stays the same fraction of the threshold.
+static double mixed_radius(double tol)
+{
+    return MIXED_RADIUS * (tol < 1.0e-3 ? tol / 1.0e-3 : 1.0);
+}
 
 static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
@@ -329,7 +336,7 @@ extern "C" skb_status sinkhorn_batch_create(const void *x, const void *y, const 
         double radius;
         memcpy(&radius, &h->h_ctl[1].max_radius_bits, sizeof(double));
         const double ts = h->dev.tol_stop, tsc = h->dev.tol_screen;
-        if (radius > MIXED_RADIUS) {
+        if (radius > mixed_radius(ts < tsc ? ts : tsc)) {
             h->var = var_big;
             carve(cfg, var_big, false, (char *)cfg->workspace, &h->dev, nullptr, &h->guards);
         } else if (can_tensor) {

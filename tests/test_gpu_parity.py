@@ -204,6 +204,54 @@ def test_degenerate_shapes(oracle):
     check_accounting(oracle, r, 300, "active")
 
 
+@pytest.mark.parametrize("compute", ["auto", "f32", "mixed"])
+def test_degenerate_lanes_in_the_fast_arithmetics(oracle, compute):
+    # the cases the method itself degenerates on, in the arithmetics and kernels a default batch runs
+    # (lanes this small go through the multi-cycle kernels): single points, one point against many,
+    # coincident clouds (zero cost on the diagonal) and a cloud collapsed to one location (all costs
+    # equal: the product coupling is optimal and the first audit passes)
+    rng = np.random.default_rng(11)
+    f32 = np.float32
+
+    def lanes(x, y, a, b, eps, tol=1e-4, max_iter=400, name="degenerate"):
+        return wl.Workload(name, x.astype(f32), y.astype(f32), a.astype(f32), b.astype(f32), eps.astype(f32), tol, max_iter)
+
+    def uniform(W, n):
+        return np.full((W, n), 1.0 / n)
+
+    W = 3
+    cases = []
+    # one point against one point
+    cases.append(lanes(rng.normal(size=(W, 1, 2)), rng.normal(size=(W, 1, 2)), uniform(W, 1), uniform(W, 1),
+                       np.array([0.3, 0.1, 1.0])))
+    # one point against seven, and seven against one
+    wts = rng.uniform(0.5, 1.5, size=(W, 7)); wts /= wts.sum(axis=1, keepdims=True)
+    cases.append(lanes(rng.normal(size=(W, 1, 3)), rng.normal(size=(W, 7, 3)), uniform(W, 1), wts, np.array([0.3, 0.1, 1.0])))
+    cases.append(lanes(rng.normal(size=(W, 7, 3)), rng.normal(size=(W, 1, 3)), wts, uniform(W, 1), np.array([0.3, 0.1, 1.0])))
+    # the same cloud on both sides
+    pts = rng.normal(size=(W, 9, 2))
+    cases.append(lanes(pts, pts.copy(), uniform(W, 9), uniform(W, 9), np.array([0.5, 0.2, 0.1])))
+    # every point of both clouds at one location
+    spot = np.broadcast_to(rng.normal(size=(W, 1, 4)), (W, 6, 4)).copy()
+    cases.append(lanes(spot, spot[:, :5].copy(), uniform(W, 6), uniform(W, 5), np.array([0.5, 0.2, 0.1])))
+    for k, w in enumerate(cases):
+        if compute == "f32":
+            w.tol = 1e-3          # pure fp32 by name: its evaluation error is ~2e-6 absolute here (eps 0.05 .. 1)
+        r = run_gpu(w, compute=compute)
+        if compute == "auto" and k == 3:
+            # the automatic choice follows the tolerance: lane 2 has a scaled squared radius of 60, which
+            # is fp32 territory at a tolerance of 1e-3 (limit 512) and not at 1e-4 (limit 51)
+            assert r["arith"] == "mixed"
+            w.tol = 1e-3
+            assert run_gpu(w, compute="auto")["arith"] == "f32"
+            w.tol = 1e-4
+        assert (r["status"] == 1).all(), (k, r["status"])
+        assert check_against_oracle(oracle, w, r, list(range(W)), pot_tol=POT_TOL_F32, exact_depth=False,
+                                    label=f"degenerate lanes, case {k}, {compute}") == [], k
+    # collapsed clouds: all costs equal, so f = g = const solves the problem after one cycle
+    assert (r["depth"] == 1).all(), r["depth"]
+
+
 def test_step_runs_fixed_cycles_and_running_lanes_are_readable(oracle):
     import torch
     from paper_2607_24741_b200 import binding as B
