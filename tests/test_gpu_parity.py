@@ -361,7 +361,7 @@ class _Stored:
 
 
 def test_full_size_registration_against_stored_oracle(oracle):
-    # One oracle lane at n = m = 8192 takes a quarter of an hour, so the oracle's results for six lanes
+    # One oracle lane at n = m = 8192 takes a quarter of an hour, so the oracle's results for twelve lanes
     # are stored (tests/golden/make_registration_golden.py wrote them, calling the oracle only); the
     # float64 residual evaluation of the emitted state is cheap enough to run here.
     z = np.load(os.path.join(os.path.dirname(__file__), "golden", "registration_n8192.npz"))
