@@ -97,8 +97,10 @@ def miss_allowed(margin, decay, floor):
 
 def compare_lane(oracle, w, r, t, o, *, pot_tol, exact_depth, tol, audit_every=1, report_tol=None, entry=None):
     """One lane of the acceptance bar against an oracle result `o` (anything with depth, status, f, g,
-    f_prev, g_prev, f_next, g_next and the history of max(r_row, r_col) in `hist`).  Returns the miss
-    record of a lane that stopped one audit away, else None."""
+    f_prev, g_prev, f_next, g_next and the history of max(r_row, r_col) in `hist`; an optional
+    `stride` says that its potentials hold every stride-th point only).  Returns the miss record of a
+    lane that stopped one audit away, else None."""
+    st = int(getattr(o, "stride", 1))
     dg = int(r["depth"][t]); do = int(o.depth)
     assert r["status"][t] == o.status, (t, r["status"][t], o.status)
     miss = None
@@ -118,7 +120,7 @@ def compare_lane(oracle, w, r, t, o, *, pot_tol, exact_depth, tol, audit_every=1
             miss = (t, dg, do, float(margin), float(decay))
     e = None
     if dg == do or audit_every == 1:
-        e = pot_err(r["f"][t][None], r["g"][t][None], np.asarray(fo, np.float64)[None],
+        e = pot_err(r["f"][t][None, ::st], r["g"][t][None, ::st], np.asarray(fo, np.float64)[None],
                     np.asarray(go, np.float64)[None], float(w.eps[t]))[0]
         assert e <= pot_tol, f"lane {t}: potential error {e:.3e} > {pot_tol}"
     if o.status == oracle.DONE:

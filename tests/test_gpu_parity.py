@@ -348,22 +348,26 @@ def test_full_size_lanes_against_oracle(oracle, name):
 
 class _Stored:
     """One lane of tests/golden/registration_n8192.npz in the shape compare_lane expects."""
-    def __init__(self, z, i):
-        self.depth = int(z["depth"][i]); self.status = int(z["status"][i])
-        self.f, self.g = z["f"][i], z["g"][i]
-        self.f_prev, self.g_prev = z["f_prev"][i], z["g_prev"][i]
-        self.f_next, self.g_next = z["f_next"][i], z["g_next"][i]
-        tail = z["hist"][i]
+    def __init__(self, z, i, prefix="", stride=1):
+        k_ = lambda name: z[prefix + name][i]
+        self.depth = int(k_("depth")); self.status = int(k_("status"))
+        self.f, self.g = k_("f"), k_("g")
+        self.f_prev, self.g_prev = k_("f_prev"), k_("g_prev")
+        self.f_next, self.g_next = k_("f_next"), k_("g_next")
+        tail = k_("hist")
         self.hist = np.full(self.depth, np.nan)
         k = min(len(tail), self.depth)
         self.hist[self.depth - k:] = tail[len(tail) - k:]
-        self.r_row = float(z["r_row"][i])
+        self.r_row = float(k_("r_row"))
+        self.stride = stride                 # potentials hold every stride-th point
 
 
 def test_full_size_registration_against_stored_oracle(oracle):
-    # One oracle lane at n = m = 8192 takes a quarter of an hour, so the oracle's results for twelve lanes
-    # are stored (tests/golden/make_registration_golden.py wrote them, calling the oracle only); the
-    # float64 residual evaluation of the emitted state is cheap enough to run here.
+    # One oracle lane at n = m = 8192 takes a quarter of an hour, so the oracle's results are stored
+    # (tests/golden/make_registration_golden.py wrote them, calling the oracle only): twelve lanes with
+    # their full potentials, the other twenty with every eighth point.  Every lane of the workload is
+    # held to the oracle's depth; the float64 residual evaluation of the emitted state is cheap enough
+    # to run here.
     z = np.load(os.path.join(os.path.dirname(__file__), "golden", "registration_n8192.npz"))
     w = wl.make("registration")
     W, n, m, d = w.shape
@@ -374,10 +378,13 @@ def test_full_size_registration_against_stored_oracle(oracle):
     assert r["stats"]["slots"] == depth.sum() and r["cycles"] == depth.max()
     np.testing.assert_array_equal(np.array(r["stats"]["widths"]), oracle.survivor_widths(depth))
     lanes = [int(t) for t in z["lanes"]]
-    entry = new_entry("full size, registration (stored oracle)", w, r, lanes, w.tol, MARGIN_AUTO)
+    stored = [(t, _Stored(z, i)) for i, t in enumerate(lanes)]
+    if "light_lanes" in z.files:
+        stored += [(int(t), _Stored(z, i, "light_", int(z["stride"]))) for i, t in enumerate(z["light_lanes"])]
+        assert sorted(t for t, _ in stored) == list(range(W))            # every lane of the workload
+    entry = new_entry("full size, registration (stored oracle)", w, r, [t for t, _ in stored], w.tol, MARGIN_AUTO)
     misses = []
-    for i, t in enumerate(lanes):
-        o = _Stored(z, i)
+    for t, o in stored:
         assert abs(o.r_row - o.hist[-1]) <= 1e-15
         miss = compare_lane(oracle, w, r, t, o, pot_tol=POT_TOL_F32, exact_depth=False, tol=w.tol, entry=entry)
         if miss is not None:
