@@ -24,6 +24,17 @@ ACCEPTANCE_BAND = 1e-6
 # the scaled cost (up to 512, i.e. 2^-15 in the exponent) when the exponents are fp32 too.
 RCOL_ABS = {"f64": 1e-12, "mixed": 5e-7, "f32": 1e-5, "tensor": 3e-5}     # observed: 8.5e-14, 6.1e-8, 1.9e-6, 1.1e-5
 
+# Allowance on "float64 residual of the emitted state <= tol" (as a fraction of tol): the GPU stops a
+# lane when ITS evaluation of the residual passes, so the float64 value may exceed tol by the
+# evaluation error.  fp32 / mixed: observed up to 2e-5 of tol on the workloads, 5e-3 allowed.  Tensor
+# cores: the fp32 accumulation of the 32 k-steps of a d = 512 dot product is the least accurate link
+# (measured on the same inputs: the float64 column residual of an emitted state is 1.0e-5 on every
+# lane, against 6.7e-7 with fp32 FMAs in the SIMT kernel), and the fused screen is off by up to
+# 0.8 % of tol either way, so 1e-2 is allowed there.  The paper's answer to exactly this (Section 5:
+# raw low-precision decisions flip near the threshold; a guard removes them) is the guard arm, which
+# a test runs with NO allowance.
+RESIDUAL_ALLOW = {"f64": 1e-9, "mixed": 5e-3, "f32": 5e-3, "tensor": 1e-2}
+
 
 def run_gpu(w, mode="active", compute="auto", column_split=0, audit_every=1, tol_screen=0.0,
             max_iter=None, tol=None, widths_cap=200000, cost_form=0, warm=None, audit_initial=False,
@@ -130,7 +141,7 @@ def compare_lane(oracle, w, r, t, o, *, pot_tol, exact_depth, tol, audit_every=1
             # guard arm: the solve ran with a stricter threshold, the reported tolerance holds with no slack
             assert max(rr, rc) <= report_tol, (t, rr, rc)
         else:
-            assert max(rr, rc) <= tol * (1 + 5e-3), (t, rr, rc)
+            assert max(rr, rc) <= tol * (1 + RESIDUAL_ALLOW[r["arith"]]), (t, rr, rc)
         assert r["r_row"][t] <= tol
         assert abs(r["r_row"][t] - rr) <= 2e-2 * tol
         # the column half of the two-sided check (Eq. 5) as the GPU measured it
