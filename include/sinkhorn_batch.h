@@ -100,9 +100,12 @@ typedef struct {
                            /* a lane whose row screen lies within this RELATIVE distance   */
                            /* of tau_screen or tau_stop (at least 1e-7 absolute) has its   */
                            /* row residual re-evaluated from the raw inputs in float64 and */
-                           /* is decided by that value.  0 = default (2.5e-4), negative =  */
-                           /* off; d <= 32 only (ignored for larger d).  Costs a raw copy  */
-                           /* of x and y in the workspace                                  */
+                           /* is decided by that value.  Negative = off.  0 = default:     */
+                           /* 2.5e-4 for d <= 32, off for deeper lanes, where one lane's   */
+                           /* re-evaluation is n*m*d float64 multiply-adds in a launch of  */
+                           /* its own per cycle and is only done at a width the caller     */
+                           /* names (the tensor-core path's own evaluation error is up to  */
+                           /* 1 % of tol).  Costs a raw copy of x and y in the workspace   */
     int lane_capacity;     /* lanes the batch can take in over its life: 0 or W = the W of  */
                            /* create only; more (ACTIVE mode) lets sinkhorn_batch_refill    */
                            /* put new problems into the slots finished lanes have freed;    */

@@ -128,13 +128,15 @@ static bool config_ok(const skb_config *c, std::string &why)
     return true;
 }
 
-// Relative half-width of the guard band: the configured value, 2.5e-4 by default, off when negative
-// and for d > 32 (the float64 re-evaluation walks all pairs of a lane with one thread per row, which
-// is only affordable where a pair is a few dimensions deep).
+// Relative half-width of the guard band: the configured value, off when negative; when left at 0 it is
+// 2.5e-4 for d <= 32 and off for deeper lanes, where the float64 re-evaluation of one lane is half a
+// GFLOP (d = 512, n = m = 1024) and the tensor path's own evaluation error would need a band of a
+// per cent: there the caller names the width it is willing to pay for.
 static double guard_width(const skb_config *c)
 {
-    if (c->d > 32 || c->guard_band < 0.0f) return 0.0;
-    return c->guard_band > 0.0f ? (double)c->guard_band : 2.5e-4;
+    if (c->guard_band < 0.0f) return 0.0;
+    if (c->guard_band > 0.0f) return (double)c->guard_band;
+    return c->d > 32 ? 0.0 : 2.5e-4;
 }
 
 // Lays the batch's arrays out in the workspace (base may be null: size query only).
@@ -511,8 +513,14 @@ static void enqueue_cycle(skb_batch *h)
     auto mark = [&]() { if (prof) cudaEventRecord(h->pev[h->pev_used++], h->stream); };
     if (prof && h->pev_used == 0) mark();
     launch_leg(h, LEG_F, w); mark();
-    launch_leg(h, LEG_V, w); mark();
+    launch_leg(h, LEG_V, w);
     int nk = 3;
+    if (h->dev.guard > 0.0 && h->cfg.d > 32) {
+        // deep lanes: their update kernels carry no pool, the guard band's re-evaluation is a launch of its own
+        launch_guard_pool(h->dev, h->stream);
+        ++nk;
+    }
+    mark();
     nk += launch_plan(h->dev, w, h->stream); mark();
     nk += launch_emit_move(h->dev, w, h->stream); mark();
     launch_leg(h, LEG_G, w); mark();

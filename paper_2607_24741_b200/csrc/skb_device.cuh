@@ -175,12 +175,34 @@ __device__ __forceinline__ double direct_row_term_warp(const Dev &P, const int s
             gj[u] = __ldcg(gam + jc);
             c[u] = 0.0;
         }
-        for (int k = 0; k < P.d; ++k) {
-            const double xk = (double)load_raw(P, xl, xb + k);
+        if (P.xy_bf16 && (P.d & 7) == 0) {
+            // deep bf16 lanes: eight dimensions per 16-byte load (same operations in the same order)
+            const unsigned short *x16 = reinterpret_cast<const unsigned short *>(xl);
+            const unsigned short *y16 = reinterpret_cast<const unsigned short *>(yl);
+            for (int k = 0; k < P.d; k += 8) {
+                const uint4 xv = *reinterpret_cast<const uint4 *>(x16 + xb + k);
+                const unsigned xw[4] = {xv.x, xv.y, xv.z, xv.w};
 #pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const double t = xk - (double)load_raw(P, yl, yb[u] + k);
-                c[u] = fma(t, t, c[u]);
+                for (int u = 0; u < U; ++u) {
+                    const uint4 yv = *reinterpret_cast<const uint4 *>(y16 + yb[u] + k);
+                    const unsigned yw[4] = {yv.x, yv.y, yv.z, yv.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const double t0 = (double)__uint_as_float(xw[e] << 16) - (double)__uint_as_float(yw[e] << 16);
+                        c[u] = fma(t0, t0, c[u]);
+                        const double t1 = (double)__uint_as_float(xw[e] & 0xffff0000u) - (double)__uint_as_float(yw[e] & 0xffff0000u);
+                        c[u] = fma(t1, t1, c[u]);
+                    }
+                }
+            }
+        } else {
+            for (int k = 0; k < P.d; ++k) {
+                const double xk = (double)load_raw(P, xl, xb + k);
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const double t = xk - (double)load_raw(P, yl, yb[u] + k);
+                    c[u] = fma(t, t, c[u]);
+                }
             }
         }
         double v[U], mn = mx;

@@ -62,6 +62,7 @@ const char *tc_make_map(void *out_map, void *base, int W, int npts, int d);
 size_t tc_tiled_bytes(int W, int npts, int d);
 void launch_retile(const void *src, void *dst, int W, int npts, int d, cudaStream_t st);
 void launch_wait_probe(int *out, long long budget_clocks, cudaStream_t st);
+void launch_guard_pool(const Dev &P, cudaStream_t st);
 void launch_guard_strips(void *base, const GuardList &gl, bool fill, int *bad, cudaStream_t st);
 void launch_update_tc(const Dev &P, const void *maps, int leg, int width, cudaStream_t st);
 int launch_emit_move(const Dev &P, int width, cudaStream_t st);

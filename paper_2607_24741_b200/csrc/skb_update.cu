@@ -182,4 +182,21 @@ const Variant *choose_variant(int W, int n, int m, int d, bool f64, bool fast_ex
     return nullptr;
 }
 
+// The guard band's float64 re-evaluation as a launch of its own (deep lanes, whose update kernels carry
+// no pool): about two blocks per SM look for lanes whose fused screen lies in the band and share each
+// one's rows.  It sits between the column check and the planner in the chain and, like every kernel of
+// the chain, waits for its predecessor before it reads anything.
+__global__ void __launch_bounds__(UPD_THREADS) guard_pool_kernel(const Dev P)
+{
+    __shared__ unsigned long long red[UPD_THREADS / 32];
+    pdl_enter();
+    const Ctl c = *P.ctl;
+    guard_pool(P, c, 0, red);
+}
+
+void launch_guard_pool(const Dev &P, cudaStream_t st)
+{
+    launch_pdl(guard_pool_kernel, dim3(2 * 148, 1), dim3(UPD_THREADS), 0, st, P);
+}
+
 }  // namespace skb

@@ -47,7 +47,7 @@ __global__ void __launch_bounds__(UPD_THREADS) update_bigd_kernel(const Dev P, c
     if (slot >= c.n_phys) return;
     if (P.early_exit && P.state[slot] != 0) return;     // early-exit mask arm: a frozen lane costs a launch slot only
     if (leg != LEG_V && c.static_final) return;
-    if (leg == LEG_V && !(c.static_final || lane_flag(P, c, slot))) return;
+    if (leg == LEG_V && !(c.static_final || lane_needs_column_check(P, c, slot))) return;
     const bool rows_x = (leg == LEG_F);
     const int nrows = rows_x ? P.n : P.m, rp = rows_x ? P.np : P.mp;
     const int ncols = rows_x ? P.m : P.n, cp = rows_x ? P.mp : P.np;

@@ -260,7 +260,7 @@ update_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant_
     if (slot >= c.n_phys) return;
     if (P.early_exit && P.state[slot] != 0) return;     // early-exit mask arm: a frozen lane costs a launch slot only
     if (leg != LEG_V && c.static_final) return;
-    if (leg == LEG_V && !(c.static_final || lane_flag(P, c, slot))) return;
+    if (leg == LEG_V && !(c.static_final || lane_needs_column_check(P, c, slot))) return;
     const bool rows_x = (leg == LEG_F);
     const int nrows = rows_x ? P.n : P.m;
     const int ncols = rows_x ? P.m : P.n, cp = rows_x ? P.mp : P.np;
@@ -613,7 +613,7 @@ update_tc_pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_cons
     // visits lanes that the screen flagged)
     SegIter it = it0;
     Seg sg;
-#define TC2_SKIP(slot) ((leg == LEG_V && !(c.static_final || lane_flag(P, c, slot))) || (P.early_exit && P.state[slot] != 0))
+#define TC2_SKIP(slot) ((leg == LEG_V && !(c.static_final || lane_needs_column_check(P, c, slot))) || (P.early_exit && P.state[slot] != 0))
 
     if (warp == TC_EPI_WARPS) {
         // ---------------- producer (one per CTA): own row block once per segment, own half of every column tile

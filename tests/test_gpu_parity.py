@@ -32,10 +32,13 @@ CASES = {
     "sweep_small": dict(name="sweep", W=48, n=100, m=77, max_iter=3000),
     "feature_small": dict(name="feature", W=4, n=200, m=333, d=80),      # bf16 inputs, large-d kernels
 }
+DEEP_CASES = {
+    "feature_tensor": dict(name="feature", W=4, n=256, m=320, d=128),    # bf16 inputs on the tensor cores
+}
 
 
 def _make(case):
-    kw = dict(CASES[case]); name = kw.pop("name")
+    kw = dict(CASES[case] if case in CASES else DEEP_CASES[case]); name = kw.pop("name")
     return wl.make(name, **kw)
 
 
@@ -862,7 +865,8 @@ def test_sixty_five_thousand_points_sampled_marginals():
 
 
 # ---- guard band: float64 escalation of near-threshold decisions -------------------------------------------
-@pytest.mark.parametrize("case", ["tiny", "sweep_small", "sensor_ragged", "registration_small"])
+@pytest.mark.parametrize("case", ["tiny", "sweep_small", "sensor_ragged", "registration_small", "feature_small",
+                                  "feature_tensor"])
 def test_guard_band_decisions_come_from_the_float64_reevaluation(oracle, case):
     # Section 5's stress test: raw fp32 decisions near the threshold flip; an outward guard with float64
     # escalation removes the flips.  With a band of 50 % every audit within a factor 1.5 of the threshold is
