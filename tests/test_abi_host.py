@@ -53,6 +53,25 @@ def test_workspace_size_and_config_validation(B):
         assert B.sinkhorn_batch_workspace_bytes(bad) == 0
 
 
+def test_guard_band_and_lane_capacity_show_in_the_workspace(B):
+    # host logic only: what the guard band and the lane capacity cost in workspace
+    W, n, m = 8, 64, 48
+    ws = lambda d, **kw: B.sinkhorn_batch_workspace_bytes(B.make_config(W, n, m, d, compute="f32", **kw))
+    lane = lambda pts, d, es: -(-(pts * d * es) // 16) * 16          # a lane's raw cloud, 16-byte aligned
+    pad = lambda b: -(-b // 256) * 256                                # an array of the workspace
+    # d <= 32: on by default (0), off when negative; the difference is the raw copies of x and y and their two strips
+    on, off = ws(2), ws(2, guard_band=-1.0)
+    assert on == ws(2, guard_band=1e-3)
+    assert on - off == pad(W * lane(n, 2, 4)) + pad(W * lane(m, 2, 4)) + 2 * 256
+    # deeper lanes: off unless the caller names a width
+    assert ws(64) == ws(64, guard_band=-1.0)
+    assert ws(64, guard_band=1e-2) > ws(64)
+    assert B.sinkhorn_batch_workspace_bytes(B.make_config(W, n, m, 2, guard_band=0.75)) == 0      # at most 0.5
+    # per-lane outputs grow with the capacity, per-slot state does not
+    grow = ws(2, lane_capacity=3 * W) - ws(2)
+    assert grow >= 2 * W * (n + m) * 8 and grow < 2 * W * (n + m) * 8 + 64 * 1024
+
+
 def test_create_rejects_bad_arguments_without_touching_the_gpu(B):
     cfg = B.make_config(8, 64, 64, 2)
     h = ctypes.c_void_p()
