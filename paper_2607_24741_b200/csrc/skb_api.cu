@@ -469,10 +469,11 @@ extern "C" skb_status sinkhorn_batch_set_profiling(skb_batch *h, int on)
 
 // one full cycle: f-leg (+ row screen of the previous state), column check of screen-positive
 // lanes, plan, emit/compact, g-leg
-static void launch_leg(skb_batch *h, int leg, int w)
+// Returns 1 if a column-check launch carried the guard band's pool.
+static int launch_leg(skb_batch *h, int leg, int w)
 {
-    if (h->tensor) launch_update_tc(h->dev, h->maps, leg, w, h->stream);
-    else h->var->launch(h->dev, leg, w, h->stream);
+    if (h->tensor) { launch_update_tc(h->dev, h->maps, leg, w, h->stream); return 0; }
+    return h->var->launch(h->dev, leg, w, h->stream);
 }
 
 // ACTIVE batches whose lanes have few row blocks run several whole cycles per launch, one
@@ -513,10 +514,11 @@ static void enqueue_cycle(skb_batch *h)
     auto mark = [&]() { if (prof) cudaEventRecord(h->pev[h->pev_used++], h->stream); };
     if (prof && h->pev_used == 0) mark();
     launch_leg(h, LEG_F, w); mark();
-    launch_leg(h, LEG_V, w);
+    const int pool_rode = launch_leg(h, LEG_V, w);
     int nk = 3;
-    if (h->dev.guard > 0.0 && h->cfg.d > 32) {
-        // deep lanes: their update kernels carry no pool, the guard band's re-evaluation is a launch of its own
+    if (h->dev.guard > 0.0 && !pool_rode) {
+        // deep lanes (their update kernels carry no pool) and batches so wide that the column check's
+        // grid has no rows to spare: the guard band's re-evaluation is a launch of its own
         launch_guard_pool(h->dev, h->stream);
         ++nk;
     }

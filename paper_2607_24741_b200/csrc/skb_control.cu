@@ -548,8 +548,8 @@ template <typename O>
 __global__ void gather_kernel(const Dev P, O *f, O *g)
 {
     const Ctl c = *P.ctl;
-    const int y = blockIdx.y;
-    const int tid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
+    const int y = blockIdx.x;                         // lanes along x: up to twice 65535 of them
+    const int tid = blockIdx.y * blockDim.x + threadIdx.x, nth = gridDim.y * blockDim.x;
     if (y < P.L) {                                    // emitted lanes, by lane id
         const int lane = y;
         if (!P.emitted[lane]) return;
@@ -730,7 +730,7 @@ void launch_gather(const Dev &P, void *f, void *g, bool f64, cudaStream_t st)
 {
     const int mx = P.n > P.m ? P.n : P.m;
     int gx = (mx + 1023) / 1024; if (gx > 16) gx = 16;
-    dim3 grid(gx, P.L + P.W);
+    dim3 grid(P.L + P.W, gx);
     if (f64) gather_kernel<double><<<grid, 256, 0, st>>>(P, (double *)f, (double *)g);
     else gather_kernel<float><<<grid, 256, 0, st>>>(P, (float *)f, (float *)g);
 }

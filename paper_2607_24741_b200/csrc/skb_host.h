@@ -37,7 +37,7 @@ struct Variant {
     int f64, xf, DP, R, CS;   // xf: float64 arguments with fp32 special-function exponentials
     int rows_per_cta;
     size_t smem;
-    void (*launch)(const Dev &, int leg, int width, cudaStream_t);
+    int (*launch)(const Dev &, int leg, int width, cudaStream_t);   // 1: the guard band's pool rode in a column-check launch
     // several whole cycles per launch, one thread-block cluster per lane; null where there is none
     void (*launch_cycles)(const Dev &, int cycles, int width, cudaStream_t);
     // does a lane of n x m points fit the shared-memory-resident version of the multi-cycle kernel?

@@ -11,13 +11,16 @@ constexpr size_t RESIDENT_SMEM_LIMIT = 52 * 1024; // shared memory of a block of
 constexpr long long NARROW_BLOCKS = 148 * 4;      // below this many blocks some SM has fewer than four
 
 // Grid rows (of `per_row` blocks each) that hold the guard band's pool of about two blocks per SM.
-static int pool_rows(int per_row, bool on)
+// None when the launch has no room for them (grid.y is 16 bits): the caller then runs the pool as
+// a launch of its own.
+static int pool_rows(int per_row, bool on, int lanes)
 {
-    return on ? (2 * 148 + per_row - 1) / per_row : 0;
+    const int rows = on ? (2 * 148 + per_row - 1) / per_row : 0;
+    return lanes + rows <= 65535 ? rows : 0;
 }
 
 template <typename T, int DP, int CS, int XF>
-static void launch_update(const Dev &P, int leg, int width, cudaStream_t st)
+static int launch_update(const Dev &P, int leg, int width, cudaStream_t st)   // returns 1 if the guard band's pool rode in the launch
 {
     static bool attr_set = false;
     const size_t smem = 2 * (size_t)(DP + 2) * TileCols<T, DP, CS>::value * sizeof(T);
@@ -42,8 +45,9 @@ static void launch_update(const Dev &P, int leg, int width, cudaStream_t st)
         const int rbw = (UPD_THREADS / 32) * RW * (32 / CS);
         const long long ctas = (long long)((nrows + rbw - 1) / rbw) * lanes;
         if (ctas >= 2 * 148 * 4) {
-            launch_pdl(update_kernel<T, DP, CS, XF, RW>, dim3((nrows + rbw - 1) / rbw, lanes + pool_rows((nrows + rbw - 1) / rbw, guard_pool)), dim3(UPD_THREADS), smem, st, P, leg, lanes);
-            return;
+            const int pool = pool_rows((nrows + rbw - 1) / rbw, guard_pool, lanes);
+            launch_pdl(update_kernel<T, DP, CS, XF, RW>, dim3((nrows + rbw - 1) / rbw, lanes + pool), dim3(UPD_THREADS), smem, st, P, leg, lanes);
+            return pool > 0;
         }
     }
     if constexpr (sizeof(T) == 4 && DP <= 4 && CS == 4) {
@@ -57,12 +61,15 @@ static void launch_update(const Dev &P, int leg, int width, cudaStream_t st)
         const int rb2 = (UPD_THREADS / 32) * Tune<T, DP>::R * (32 / CS);
         if ((long long)((nrows + rb2 - 1) / rb2) * lanes < NARROW_BLOCKS) {
             const int rbr = (UPD_THREADS / 32) * 1 * (32 / CS);
-            launch_pdl(update_kernel<T, DP, CS, XF, 1>, dim3((nrows + rbr - 1) / rbr, lanes + pool_rows((nrows + rbr - 1) / rbr, guard_pool)), dim3(UPD_THREADS), smem, st, P, leg, lanes);
-            return;
+            const int pool = pool_rows((nrows + rbr - 1) / rbr, guard_pool, lanes);
+            launch_pdl(update_kernel<T, DP, CS, XF, 1>, dim3((nrows + rbr - 1) / rbr, lanes + pool), dim3(UPD_THREADS), smem, st, P, leg, lanes);
+            return pool > 0;
         }
     }
     const int rb = (UPD_THREADS / 32) * Tune<T, DP>::R * (32 / CS);
-    launch_pdl(update_kernel<T, DP, CS, XF>, dim3((nrows + rb - 1) / rb, lanes + pool_rows((nrows + rb - 1) / rb, guard_pool)), dim3(UPD_THREADS), smem, st, P, leg, lanes);
+    const int pool = pool_rows((nrows + rb - 1) / rb, guard_pool, lanes);
+    launch_pdl(update_kernel<T, DP, CS, XF>, dim3((nrows + rb - 1) / rb, lanes + pool), dim3(UPD_THREADS), smem, st, P, leg, lanes);
+    return pool > 0;
 }
 
 // Several whole cycles per launch: grid.x = row blocks of the larger cloud = one thread-block
@@ -117,7 +124,7 @@ static bool lane_fits_shared(int n, int m) { return ResidentLayout<T, DP, CS>::b
 static const Variant g_variants[] = {SKB_ROW(2), SKB_ROW(3), SKB_ROW(4), SKB_ROW(8), SKB_ROW(16), SKB_ROW(32)};
 
 template <typename T, int XF>
-static void launch_bigd(const Dev &P, int leg, int width, cudaStream_t st)
+static int launch_bigd(const Dev &P, int leg, int width, cudaStream_t st)
 {
     static bool attr_set = false;
     const size_t smem = 2 * (size_t)BIGD_KC * (BIGD_RB + BIGD_TJ) * sizeof(T);
@@ -128,6 +135,7 @@ static void launch_bigd(const Dev &P, int leg, int width, cudaStream_t st)
     const int nrows = (leg == LEG_F) ? P.n : P.m;
     dim3 grid((nrows + BIGD_RB - 1) / BIGD_RB, width < 1 ? 1 : width);
     launch_pdl(update_bigd_kernel<T, XF>, grid, dim3(UPD_THREADS), smem, st, P, leg);
+    return 0;                       // no pool in this kernel
 }
 
 // DP = 0 marks the large-d kernels: the padded dimension is d rounded up to the chunk size

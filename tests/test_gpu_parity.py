@@ -573,6 +573,29 @@ def test_very_wide_batch_and_rectangular_lanes(oracle):
             assert misses == []
 
 
+def test_widest_batch_the_interface_takes(oracle):
+    # W = 65535 lanes (the interface's limit: one grid row per lane) of four points against five, in the
+    # default arithmetic: the planner's scans run over 64 chunks, retirements and moves happen in every
+    # cycle, and the widths shrink from 65535 to 1.  Depths of a sample of lanes against the oracle,
+    # accounting identities (Eq. 6-8) over all of them.
+    W = 65535
+    w = wl.make("sweep", W=W, n=4, m=5, max_iter=20000)
+    r = run_gpu(w, mode="active", widths_cap=30000)
+    depth = r["depth"].astype(np.int64)
+    assert np.all(r["status"] == 1) and r["left"] == 0
+    assert r["stats"]["slots"] == int(depth.sum()) and r["cycles"] == int(depth.max())
+    np.testing.assert_array_equal(np.array(r["stats"]["widths"]), oracle.survivor_widths(depth))
+    lanes = [0, 1, 1023, 1024, 32767, 32768, 65534] + list(range(500, W, 4099))
+    check_against_oracle(oracle, w, r, lanes, pot_tol=POT_TOL_F32, exact_depth=False, floor=MARGIN_AUTO, max_iter=20000,
+                         label="widest batch, W = 65535")
+    # the one-launch-per-leg path at this width: the column check's grid has no rows left for the guard
+    # band's pool, which then runs as a launch of its own - same bits as ACTIVE
+    rm = run_gpu(w, mode="masked", max_iter=20000, widths_cap=30000)
+    np.testing.assert_array_equal(rm["depth"], r["depth"]); np.testing.assert_array_equal(rm["f"], r["f"])
+    with pytest.raises(Exception):
+        run_gpu(wl.make("sweep", W=W + 1, n=4, m=5, max_iter=10))       # one lane more is refused, not mis-launched
+
+
 def test_mixed_arithmetic_with_a_useless_reference_estimate(oracle):
     # Clouds ten units apart at a small eps: starting from zero potentials, the first legs move
     # every potential by thousands of log2 units, so a reference point estimated from the old
