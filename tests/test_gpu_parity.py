@@ -863,6 +863,52 @@ def test_sixteen_thousand_points_against_oracle_cycles(oracle):
     assert e.max() <= POT_TOL_F32
 
 
+def test_limits_of_dimension_size_and_iteration_count(oracle):
+    import torch
+    from paper_2607_24741_b200 import binding as B
+    t = lambda v: torch.from_numpy(v).to("cuda:0")
+    # every padded dimension of the SIMT kernels (1 -> 2, 5 -> 8, 17 -> 32, 32), the first and the last
+    # dimension of the large-d kernels (33, 1024), in the default arithmetic, against the oracle
+    for d in (1, 5, 17, 32, 33, 100, 1024):
+        w = wl.make("sensor", W=3, n=40, m=50, d=d)
+        r = run_gpu(w)
+        assert check_against_oracle(oracle, w, r, range(3), pot_tol=POT_TOL_F32, exact_depth=False, floor=MARGIN_AUTO,
+                                    label=f"dimension limits, d = {d}") == [], d
+    w = wl.make("sensor", W=3, n=40, m=50, d=1024)
+    bad = B.make_config(3, 40, 50, 1025)
+    assert B.sinkhorn_batch_workspace_bytes(bad) == 0                      # one dimension more is refused
+    # bf16 inputs just past the tensor-core range (d = 576 > 512) fall back to the large-d SIMT kernels
+    w = wl.make("feature", W=2, n=96, m=130, d=576)
+    r = run_gpu(w)
+    assert r["arith"] != "tensor"
+    assert check_against_oracle(oracle, w, r, range(2), pot_tol=POT_TOL_F32, exact_depth=False, floor=MARGIN_AUTO,
+                                label="bf16, d = 576") == []
+    # the largest cloud the interface takes (262143 points, fixed-point residual sums) against three points
+    n_max = 262143
+    w = wl.make("sweep", W=1, n=n_max, m=3, d=2, max_iter=10)
+    sb = B.SinkhornBatch(t(w.x), t(w.y), t(w.a), t(w.b), t(w.eps), w.tol, mode="static", max_iter=10)
+    sb.step(2)
+    f, g = sb.potentials(f64=True)
+    assert sb.check_guards() == -1
+    sb.close()
+    ref = oracle.solve_lane(w.x[0], w.y[0], w.a[0], w.b[0], float(w.eps[0]), w.tol, fixed_cycles=2)
+    assert pot_err(f.cpu().numpy(), g.cpu().numpy(), ref.f[None], ref.g[None], w.eps.astype(np.float64)).max() <= POT_TOL_F32
+    assert B.sinkhorn_batch_workspace_bytes(B.make_config(1, n_max + 1, 3, 2)) > 0          # sized ...
+    with pytest.raises(B.SkbError):                                                          # ... but refused at create
+        w1 = wl.make("sweep", W=1, n=n_max + 1, m=3, d=2, max_iter=10)
+        B.SinkhornBatch(t(w1.x), t(w1.y), t(w1.a), t(w1.b), t(w1.eps), w1.tol)
+    # one cycle allowed: every lane either passes its first audit or stops at the limit with depth 1
+    w = wl.make("tiny", max_iter=1)
+    r = run_gpu(w)
+    ref = oracle.solve_batch(w.x, w.y, w.a, w.b, w.eps, w.tol, max_iter=1)
+    np.testing.assert_array_equal(r["depth"], ref.depth); np.testing.assert_array_equal(r["status"], ref.status)
+    assert (r["depth"] == 1).all() and r["stats"]["slots"] == 8
+    # a tolerance nothing can miss (the L1 residual of unit-mass marginals is at most 2): depth 1 everywhere
+    w = wl.make("sensor", W=5, n=30, m=20, tol=2.5)
+    r = run_gpu(w)
+    assert (r["depth"] == 1).all() and (r["status"] == 1).all()
+
+
 def test_sixty_five_thousand_points_sampled_marginals():
     # n = m = 65536: far beyond what the oracle can hold (a 34 GB cost matrix), so the emitted state is
     # checked on sampled rows and columns, each computed from its definition in float64: after the last
