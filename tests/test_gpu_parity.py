@@ -883,6 +883,13 @@ def test_limits_of_dimension_size_and_iteration_count(oracle):
     assert r["arith"] != "tensor"
     assert check_against_oracle(oracle, w, r, range(2), pot_tol=POT_TOL_F32, exact_depth=False, floor=MARGIN_AUTO,
                                 label="bf16, d = 576") == []
+    # bf16 storage on the small-d kernels, with every near-threshold audit escalated (the float64
+    # re-evaluation reads the raw bf16 copies: vector loads where d is a multiple of 8, scalar otherwise)
+    for d in (2, 12, 16):
+        w = wl.make("feature", W=3, n=70, m=90, d=d)
+        r = run_gpu(w, guard_band=0.5)
+        assert check_against_oracle(oracle, w, r, range(3), pot_tol=POT_TOL_F32, exact_depth=False, floor=1e-6,
+                                    label=f"bf16 inputs, d = {d}, guard band 0.5") == [], d
     # the largest cloud the interface takes (262143 points, fixed-point residual sums) against three points
     n_max = 262143
     w = wl.make("sweep", W=1, n=n_max, m=3, d=2, max_iter=10)
