@@ -192,11 +192,11 @@ skb_status sinkhorn_batch_potentials(skb_batch *h, float *f, float *g);
 skb_status sinkhorn_batch_potentials_f64(skb_batch *h, double *f, double *g);
 
 /* Completion depth l_t (first audited cycle at which the lane passed; Eq. 6) and
- * skb_lane_status per lane, device out [W], original lane order; either may be null. */
+ * skb_lane_status per lane, device out [L] (L as above), original lane order; either may be null. */
 skb_status sinkhorn_batch_depths(skb_batch *h, int *depth, int *lane_status);
 
 /* Residuals of Eq. 5 measured at the state that was emitted: r_row = |pi 1 - a|_1,
- * r_col = |pi^T 1 - b|_1, device out [W] fp32.  r_col is NaN for a lane that was never
+ * r_col = |pi^T 1 - b|_1, device out [L] fp32.  r_col is NaN for a lane that was never
  * sent to the two-sided check (iteration limit without a screen pass). */
 skb_status sinkhorn_batch_residuals(skb_batch *h, float *r_row, float *r_col);
 
