@@ -1013,6 +1013,48 @@ def test_refill_keeps_the_width_up_and_every_lane_its_own_result(oracle, compute
                              label=f"refilled lanes, {compute}")
 
 
+@pytest.mark.parametrize("options", [dict(guard_band=0.5), dict(audit_every=4, guard_band=0.5), dict(profiling=True),
+                                     dict(compute="mixed", audit_every=3, guard_band=0.5)],
+                         ids=["guard", "grid4_guard", "profiled", "mixed_grid3_guard"])
+def test_refill_combined_with_the_other_options(options):
+    # refill together with an audit grid (new lanes come in on the grid), a guard band wide enough that
+    # most audits escalate, and phase timing: every lane ends with the bits of a one-shot batch
+    import torch
+    from paper_2607_24741_b200 import binding as B
+    dev = torch.device("cuda:0")
+    t = lambda v: torch.from_numpy(v).to(dev)
+    profiling = options.get("profiling", False)
+    kw = {k: v for k, v in options.items() if k != "profiling"}
+    every = kw.get("audit_every", 1)
+    for name, shape, S in (("sweep", dict(W=40, n=96, m=80, max_iter=3000), 7), ("tiny", dict(W=24), 5)):
+        w = wl.make(name, **shape)
+        N = w.shape[0]
+        ref = run_gpu(w, **kw)
+        x, y, a, b, eps = t(w.x), t(w.y), t(w.a), t(w.b), t(w.eps)
+        sb = B.SinkhornBatch(x[:S], y[:S], a[:S], b[:S], eps[:S], w.tol, max_iter=w.max_iter, lane_capacity=N, **kw)
+        try:
+            if profiling:
+                sb.set_profiling(True)
+            nxt = S
+            while nxt < N:
+                sb.step(12 * every)
+                free = S - sb.active()
+                if free > 0:
+                    c = min(free, N - nxt)
+                    sb.refill(x[nxt:nxt + c], y[nxt:nxt + c], a[nxt:nxt + c], b[nxt:nxt + c], eps[nxt:nxt + c])
+                    nxt += c
+            sb.drain()
+            f, g = sb.potentials(f64=True); depth, status = sb.depths(); rr, _ = sb.residuals()
+            slots = sb.stats(widths_cap=200000)["slots"]
+            assert sb.check_guards() == -1
+        finally:
+            sb.close()
+        np.testing.assert_array_equal(depth.cpu().numpy(), ref["depth"])
+        np.testing.assert_array_equal(f.cpu().numpy(), ref["f"]); np.testing.assert_array_equal(g.cpu().numpy(), ref["g"])
+        np.testing.assert_array_equal(rr.cpu().numpy(), ref["r_row"])
+        assert slots == int(ref["depth"].sum())
+
+
 def test_refill_is_refused_where_it_cannot_work():
     import torch
     from paper_2607_24741_b200 import binding as B
