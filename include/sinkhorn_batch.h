@@ -162,7 +162,9 @@ skb_status sinkhorn_batch_warm_start(skb_batch *h, const double *f0, const doubl
  *   in every per-lane output.
  * ACTIVE mode only; needs count free slots (SKB_ERR_STATE otherwise; the call synchronises the stream
  * to learn the width) and count unused lanes of cfg->lane_capacity (SKB_ERR_SHAPE).  The new lanes
- * start cold and run with the arithmetic the batch was created with; their depths count their own
+ * start cold and run with the arithmetic the batch was created with (SKB_COMPUTE_AUTO chose it from
+ * the first lanes' cost range: name the arithmetic where later problems may have a smaller eps or a
+ * wider cloud); their depths count their own
  * cycles, max_iter applies to each lane's own count, audits stay on the batch's cycle grid.  The
  * slot identity of Eq. 7 still holds: slots = sum_k A_k = sum of all lanes' depths.
  */
