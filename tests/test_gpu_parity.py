@@ -402,6 +402,39 @@ def test_full_size_registration_against_stored_oracle(oracle):
     assert np.abs(row - w.a[t]).sum() < rr0
 
 
+def test_four_batches_running_on_four_streams():
+    # one batch per stream, four arithmetics / kernel families, stepped in turn without any
+    # synchronisation in between: every batch ends with the bits it has when it runs alone
+    import torch
+    from paper_2607_24741_b200 import binding as B
+    dev = torch.device("cuda:0")
+    t = lambda v: torch.from_numpy(v).to(dev)
+    cases = [wl.make("tiny"), _make("sensor_ragged"), _make("sweep_small"), _make("feature_tensor")]
+    alone = [run_gpu(w) for w in cases]
+    batches = []
+    try:
+        for w in cases:
+            x, y = t(w.x), t(w.y)
+            if w.xy_dtype == "bf16":
+                x, y = x.bfloat16(), y.bfloat16()
+            torch.cuda.synchronize()
+            batches.append(B.SinkhornBatch(x, y, t(w.a), t(w.b), t(w.eps), w.tol, max_iter=w.max_iter,
+                                           stream=torch.cuda.Stream(dev)))
+        for _ in range(450):
+            for sb in batches:
+                sb.step(7)
+        for sb, ref in zip(batches, alone):
+            sb.drain()
+            f, g = sb.potentials(f64=True)
+            depth, _ = sb.depths()
+            np.testing.assert_array_equal(depth.cpu().numpy(), ref["depth"])
+            np.testing.assert_array_equal(f.cpu().numpy(), ref["f"]); np.testing.assert_array_equal(g.cpu().numpy(), ref["g"])
+            assert sb.check_guards() == -1
+    finally:
+        for sb in batches:
+            sb.close()
+
+
 # ---- the paper's guard: a stricter threshold inside, the reported tolerance outside ----------------
 @pytest.mark.parametrize("case", list(CASES))
 def test_guarded_thresholds_meet_the_reported_tolerance_without_slack(oracle, case):
