@@ -152,6 +152,7 @@ __device__ __forceinline__ bool in_guard_band(const Dev &P, const double rr)
 // by xor-shuffles (every lane returns the term).  phi: the row's potential (log2 units); the column
 // potentials are read from global memory past L1, because inside a multi-cycle launch other blocks of
 // the cluster have written them.
+template <bool VEC = false>
 __device__ __forceinline__ double direct_row_term_warp(const Dev &P, const int slot, const int i, const double phi)
 {
     const int lane = threadIdx.x & 31;
@@ -175,7 +176,7 @@ __device__ __forceinline__ double direct_row_term_warp(const Dev &P, const int s
             gj[u] = __ldcg(gam + jc);
             c[u] = 0.0;
         }
-        if (P.xy_bf16 && (P.d & 7) == 0) {
+        if (VEC && P.xy_bf16 && (P.d & 7) == 0) {       // VEC: only the stand-alone pool kernel carries this path
             // deep bf16 lanes: eight dimensions per 16-byte load (same operations in the same order)
             const unsigned short *x16 = reinterpret_cast<const unsigned short *>(xl);
             const unsigned short *y16 = reinterpret_cast<const unsigned short *>(yl);
@@ -232,7 +233,7 @@ __device__ __forceinline__ double direct_row_term_warp(const Dev &P, const int s
 // row_first + w + stride, ... below row_end.  Returns this block's exact fixed-point part of the
 // float64 row residual (valid in thread 0) and whether a term was not finite.  pot[i - pot_first] is
 // row i's potential.
-template <int NW>
+template <int NW, bool VEC = false>
 __device__ __forceinline__ unsigned long long direct_rows_block(const Dev &P, const int slot, const int row_first,
                                                                 const int stride, const int row_end, const double *pot,
                                                                 const int pot_first, unsigned long long *red, int *nf)
@@ -241,7 +242,7 @@ __device__ __forceinline__ unsigned long long direct_rows_block(const Dev &P, co
     unsigned long long part = 0ull;
     int bad = 0;
     for (int i = row_first + warp; i < row_end; i += stride) {
-        const double term = direct_row_term_warp(P, slot, i, pot[i - pot_first]);
+        const double term = direct_row_term_warp<VEC>(P, slot, i, pot[i - pot_first]);
         if (!isfinite(term)) bad = 1;
         else if (lane == 0) part += __double2ull_rn(fmin(term, RSUM_ROW_MAX) * RSUM_SCALE);
     }

@@ -199,7 +199,7 @@ __global__ void __launch_bounds__(UPD_THREADS) guard_pool_kernel(const Dev P)
     __shared__ unsigned long long red[UPD_THREADS / 32];
     pdl_enter();
     const Ctl c = *P.ctl;
-    guard_pool(P, c, 0, red);
+    guard_pool<true>(P, c, 0, red);        // with the 16-byte loads for deep bf16 lanes
 }
 
 void launch_guard_pool(const Dev &P, cudaStream_t st)

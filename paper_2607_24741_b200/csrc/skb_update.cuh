@@ -744,6 +744,7 @@ __device__ __forceinline__ void run_leg(const Dev &P, const Ctl &c, const int le
 // warps sharing a lane's rows, exact integer sum - and the planner decides from that value.
 // (Its float64 exponentials need more registers than the fp32 legs: update_kernel's launch bounds keep
 // the fp32 instances at four blocks per SM, and the surplus spills here, on the rare path.)
+template <bool VEC = false>
 __device__ __forceinline__ void guard_pool(const Dev &P, const Ctl &c, const int nlanes, unsigned long long *red)
 {
     if (c.done || c.static_final) return;
@@ -782,7 +783,7 @@ __device__ __forceinline__ void guard_pool(const Dev &P, const Ctl &c, const int
         for (int q = 0; q < nh; ++q) {
             const int s = hot[q];
             int bad;
-            const unsigned long long mine = direct_rows_block<NW>(P, s, pool_id * NW, pool_warps, P.n,
+            const unsigned long long mine = direct_rows_block<NW, VEC>(P, s, pool_id * NW, pool_warps, P.n,
                                                                   P.phi[c.parity] + (size_t)s * P.np, 0, red, &bad);
             if (threadIdx.x == 0) {
                 atomicAdd(P.rsum_row64 + s, mine);
