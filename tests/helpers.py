@@ -22,7 +22,9 @@ ACCEPTANCE_BAND = 1e-6
 # check repeats the g-leg's sums in the GPU's arithmetic and finds (almost) nothing, while the
 # float64 evaluation sees the g-leg's own error: 2^-22 per fp32 exponential, plus half an ulp of
 # the scaled cost (up to 512, i.e. 2^-15 in the exponent) when the exponents are fp32 too.
-RCOL_ABS = {"f64": 1e-12, "mixed": 5e-7, "f32": 1e-5, "tensor": 3e-5}     # observed: 8.5e-14, 6.1e-8, 1.9e-6, 1.1e-5
+# Float64: one ulp of an exponent of size C/eps (up to ~5e3 for eps = 0.01 at d = 40: 9e-13) in every
+# plan entry, i.e. ~1e-12 in the column sums; ten times that is allowed.
+RCOL_ABS = {"f64": 1e-11, "mixed": 5e-7, "f32": 1e-5, "tensor": 3e-5}     # observed: 1.6e-12, 8.9e-8, 1.9e-6, 1.1e-5
 
 # Allowance on "float64 residual of the emitted state <= tol" (as a fraction of tol): the GPU stops a
 # lane when ITS evaluation of the residual passes, so the float64 value may exceed tol by the

@@ -402,6 +402,45 @@ def test_full_size_registration_against_stored_oracle(oracle):
     assert np.abs(row - w.a[t]).sum() < rr0
 
 
+@pytest.mark.parametrize("seed", [2, 3])
+def test_random_configurations(oracle, seed):
+    # sixty random combinations of law, shape (down to one point, ragged, d = 1 .. 40), mode, audit
+    # grid, column split, cost form, screen threshold and guard band, in float64 (exact depths, exact
+    # accounting) and mixed arithmetic (the usual bar)
+    rng = np.random.default_rng(seed)
+    for it in range(60):
+        name = str(rng.choice(["sensor", "sweep", "tiny", "registration"]))
+        W = int(rng.choice([1, 2, 3, 7, 16, 33]))
+        kw = dict(W=W, n=int(rng.choice([1, 2, 5, 31, 64, 100, 129, 300])), max_iter=int(rng.choice([50, 400, 1500])))
+        if name != "registration":
+            kw["m"] = int(rng.choice([1, 3, 8, 33, 64, 77, 128, 257]))
+        if name in ("sensor", "sweep"):
+            kw["d"] = int(rng.choice([1, 2, 3, 4, 6, 8, 15, 16, 24, 32, 40]))
+        w = wl.make(name, **kw)
+        mode = str(rng.choice(["active", "masked", "static", "masked_exit"]))
+        compute = str(rng.choice(["f64", "mixed"]))
+        opts = dict(mode=mode, compute=compute, audit_every=int(rng.choice([1, 1, 2, 5])),
+                    column_split=int(rng.choice([0, 0, 1, 4, 32])), cost_form=int(rng.choice([0, 0, 1, 2])),
+                    guard_band=float(rng.choice([0.0, -1.0, 0.5])))
+        if rng.random() < 0.3:
+            opts["tol_screen"] = float(w.tol * rng.choice([0.5, 2.0]))
+        what = f"random configuration {seed}/{it}: {name} {kw} {opts}"
+        r = run_gpu(w, **opts)
+        exact = compute == "f64"
+        if mode == "static":
+            ref = oracle.solve_batch(w.x, w.y, w.a, w.b, w.eps, w.tol, fixed_cycles=r["cycles"])
+            err = pot_err(r["f"], r["g"], ref.f, ref.g, w.eps.astype(np.float64)).max()
+            assert err <= (POT_TOL_F64 if exact else POT_TOL_F32), (what, err)
+            assert r["stats"]["slots"] == r["cycles"] * W, what
+        else:
+            misses = check_against_oracle(oracle, w, r, range(W), pot_tol=POT_TOL_F64 if exact else POT_TOL_F32,
+                                          exact_depth=exact, floor=None if exact else MARGIN_AUTO, max_iter=kw["max_iter"],
+                                          audit_every=opts["audit_every"], tol_screen=opts.get("tol_screen", 0.0), label=what)
+            assert not exact or misses == [], what
+            if exact:
+                check_accounting(oracle, r, W, "active" if mode == "masked_exit" else mode)
+
+
 def test_four_batches_running_on_four_streams():
     # one batch per stream, four arithmetics / kernel families, stepped in turn without any
     # synchronisation in between: every batch ends with the bits it has when it runs alone
